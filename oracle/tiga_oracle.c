@@ -1,0 +1,498 @@
+/*
+ * CPU ORACLE -- TEST INFRASTRUCTURE, NOT PART OF THE PRODUCT PATH.
+ *
+ * Plain, slow, fp64 restatement of what the gf.apply hot path computes, written from the
+ * paper's definitions.  It shares no code, header, table or helper with the CUDA library;
+ * only tests, the smoke check and the benchmark's cpu_baseline leg may call it.
+ *
+ * What is written out here, with the passage each function follows:
+ *   - gather / message / reduce over a destination-oriented CSR relation
+ *     (Section 3.1: m_e = f(x_s(e), a_e), y_i = finalize(combine over e with d(e)=i);
+ *      Section 4.3: row_ptr gives edge ranges, the edge position indexes the weight,
+ *      col_idx[e] supplies the source id; empty row -> reducer identity then finalize)
+ *   - the weighted-sum adjoint (Section 5: xbar_j = sum_{e:s(e)=j} w_e ybar_d(e),
+ *     wbar_e = x_s(e) . ybar_d(e); repeated sources accumulate)
+ *   - the radius relation N(i) = { j != i : |p_j - p_i| <= r } (Appendix A) consumed by a
+ *     message and a sum reducer without ever being stored (Section 4.9), by brute force
+ *     over all ordered pairs, and its reverse mode with membership frozen (Section 5,
+ *     Appendix A: the position derivative acts through the displacement of selected edges)
+ *   - a cell directory (Section 4.9) used only to restrict candidates; the exact distance
+ *     predicate is unchanged.
+ * Readings where the paper is silent (max reducer: empty row finalizes to 0 with arg -1,
+ * ties go to the lowest edge position; periodic boxes use the minimum image; Gaussian and
+ * Lennard-Jones messages; the cell-grid constants) are the build's own and are listed in
+ * the design notes.
+ *
+ * Precision: every floating-point input is converted exactly to double; sums run in edge
+ * order / index order with no blocking, no fusion, no reordering.
+ * Compile with -ffp-contract=off so that no multiply-add is contracted.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { DT_F32 = 0, DT_F16 = 1, DT_F64 = 2 };
+enum { RED_SUM = 0, RED_MAX = 1 };
+enum { MSG_GAUSS = 2, MSG_DIST = 3, MSG_LJ = 4 };
+
+static double half_to_double(uint16_t h) {
+    int s = (h >> 15) & 1, e = (h >> 10) & 31, m = h & 1023;
+    double v;
+    if (e == 0) v = ldexp((double)m, -24);
+    else if (e == 31) v = m ? NAN : INFINITY;
+    else v = ldexp((double)(m + 1024), e - 25);
+    return s ? -v : v;
+}
+
+static inline double ld(const void* p, int dt, int64_t i) {
+    if (dt == DT_F32) return (double)((const float*)p)[i];
+    if (dt == DT_F64) return ((const double*)p)[i];
+    return half_to_double(((const uint16_t*)p)[i]);
+}
+
+/* ------------------------------------------------------------------ CSR forward
+ * Section 3.1 / 4.3.  message m = w[e] * x[col[e], f]  (w == NULL means weight 1).
+ * sum : y = sum of m in edge order, A = sum of |m|.
+ * max : y = largest m, arg = lowest edge position attaining it (strict '>' while
+ *       scanning in edge order); empty row -> y = 0, arg = -1.  A = |y|.
+ */
+int oracle_csr_forward(const int64_t* rowptr, const int32_t* col, int64_t n_dst,
+                       const void* w, int w_dt, const void* x, int x_dt, int F, int reducer,
+                       double* y, double* A, int64_t* arg) {
+#pragma omp parallel for schedule(dynamic, 256)
+    for (int64_t i = 0; i < n_dst; ++i) {
+        for (int f = 0; f < F; ++f) {
+            double acc = 0.0, absacc = 0.0;
+            int64_t best = -1;
+            for (int64_t e = rowptr[i]; e < rowptr[i + 1]; ++e) {
+                double we = w ? ld(w, w_dt, e) : 1.0;
+                double m = we * ld(x, x_dt, (int64_t)col[e] * F + f);
+                if (reducer == RED_SUM) {
+                    acc += m;
+                    absacc += fabs(m);
+                } else if (best < 0 || m > acc) {
+                    acc = m;
+                    best = e;
+                }
+            }
+            y[i * F + f] = acc;
+            if (A) A[i * F + f] = (reducer == RED_SUM) ? absacc : fabs(acc);
+            if (arg) arg[i * F + f] = best;
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ CSR backward, sum
+ * Section 5: wbar_e = sum_f x[col[e],f] * ybar[row(e),f];
+ *            xbar_j = sum over edges e with col[e] = j of w_e * ybar[row(e),:].
+ * Aw / Ax hold the sums of absolute contributions.  Any output pointer may be NULL.
+ * The scatter into xbar is applied in edge order; threads own disjoint source ranges.
+ */
+int oracle_csr_backward_sum(const int64_t* rowptr, const int32_t* col, int64_t n_dst, int64_t n_src,
+                            const void* w, int w_dt, const void* x, int x_dt, int F,
+                            const void* gy, int gy_dt,
+                            double* gw, double* Aw, double* gx, double* Ax) {
+    if (gw) {
+#pragma omp parallel for schedule(dynamic, 256)
+        for (int64_t i = 0; i < n_dst; ++i)
+            for (int64_t e = rowptr[i]; e < rowptr[i + 1]; ++e) {
+                double s = 0.0, a = 0.0;
+                for (int f = 0; f < F; ++f) {
+                    double t = ld(x, x_dt, (int64_t)col[e] * F + f) * ld(gy, gy_dt, i * F + f);
+                    s += t;
+                    a += fabs(t);
+                }
+                gw[e] = s;
+                if (Aw) Aw[e] = a;
+            }
+    }
+    if (gx) {
+        memset(gx, 0, sizeof(double) * (size_t)n_src * F);
+        if (Ax) memset(Ax, 0, sizeof(double) * (size_t)n_src * F);
+        int nparts = 64;
+#pragma omp parallel for schedule(dynamic, 1)
+        for (int p = 0; p < nparts; ++p) {
+            int64_t lo = n_src * p / nparts, hi = n_src * (p + 1) / nparts;
+            for (int64_t i = 0; i < n_dst; ++i)
+                for (int64_t e = rowptr[i]; e < rowptr[i + 1]; ++e) {
+                    int64_t j = col[e];
+                    if (j < lo || j >= hi) continue;
+                    double we = w ? ld(w, w_dt, e) : 1.0;
+                    for (int f = 0; f < F; ++f) {
+                        double t = we * ld(gy, gy_dt, i * F + f);
+                        gx[j * F + f] += t;
+                        if (Ax) Ax[j * F + f] += fabs(t);
+                    }
+                }
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ CSR backward, max
+ * The cotangent of (i,f) flows only through the selected edge e* = arg[i,f] >= 0:
+ *   wbar[e*] += x[col[e*],f] * ybar[i,f];  xbar[col[e*],f] += w[e*] * ybar[i,f].
+ * Serial on purpose (scatter in (i,f) order).
+ */
+int oracle_csr_backward_max(const int32_t* col, int64_t n_dst, int64_t n_src, int64_t n_edges,
+                            const void* w, int w_dt, const void* x, int x_dt, int F,
+                            const void* gy, int gy_dt, const int64_t* arg,
+                            double* gw, double* Aw, double* gx, double* Ax) {
+    if (gw) memset(gw, 0, sizeof(double) * (size_t)n_edges);
+    if (Aw) memset(Aw, 0, sizeof(double) * (size_t)n_edges);
+    if (gx) memset(gx, 0, sizeof(double) * (size_t)n_src * F);
+    if (Ax) memset(Ax, 0, sizeof(double) * (size_t)n_src * F);
+    for (int64_t i = 0; i < n_dst; ++i)
+        for (int f = 0; f < F; ++f) {
+            int64_t e = arg[i * F + f];
+            if (e < 0) continue;
+            int64_t j = col[e];
+            double g = ld(gy, gy_dt, i * F + f);
+            double we = w ? ld(w, w_dt, e) : 1.0;
+            double tw = ld(x, x_dt, j * F + f) * g, tx = we * g;
+            if (gw) gw[e] += tw;
+            if (Aw) Aw[e] += fabs(tw);
+            if (gx) gx[j * F + f] += tx;
+            if (Ax) Ax[j * F + f] += fabs(tx);
+        }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ degree histogram
+ * deg_i = rowptr[i+1]-rowptr[i]; hist[d] counts rows of degree d for d < nbins-1, the
+ * last bin counts deg >= nbins-1.
+ */
+int oracle_degree_histogram(const int64_t* rowptr, int64_t n, int64_t nbins, int64_t* hist,
+                            int64_t* max_degree) {
+    int64_t mx = 0;
+    for (int64_t b = 0; b < nbins; ++b) hist[b] = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        int64_t d = rowptr[i + 1] - rowptr[i];
+        if (d > mx) mx = d;
+        hist[d < nbins - 1 ? d : nbins - 1] += 1;
+    }
+    *max_degree = mx;
+    return 0;
+}
+
+/* ------------------------------------------------------------------ cell directory
+ * Grid constants (the build's reading; the paper only says "a cell directory restricts
+ * candidate traversal to nearby spatial cells", Section 4.9):
+ *   n_d = clamp(floor(len_d / (r (1 + 2^-10))), 1, min(1024, icbrt(8 n)))  in double,
+ *   periodic dimensions with n_d < 3 use n_d = 1,  invh_d = (float)(n_d / len_d).
+ * Cell of a point: c_d = min(n_d - 1, (int)floorf(p_d * invh_d)) with ONE fp32 multiply;
+ * linear id (c_z n_y + c_y) n_x + c_x.
+ */
+static int64_t icbrt64(int64_t v) {
+    int64_t c = 0;
+    while ((c + 1) * (c + 1) * (c + 1) <= v) ++c;
+    return c;
+}
+
+int oracle_cell_grid(int64_t n, float r, const float* len, const int32_t* periodic,
+                     int32_t* ncell, float* invh) {
+    int64_t cap = icbrt64(8 * (n > 0 ? n : 1));
+    if (cap > 1024) cap = 1024;
+    if (cap < 1) cap = 1;
+    for (int d = 0; d < 3; ++d) {
+        double q = floor((double)len[d] / ((double)r * (1.0 + 1.0 / 1024.0)));
+        int64_t nd = q < 1.0 ? 1 : (q > (double)cap ? cap : (int64_t)q);
+        if (periodic[d] && nd < 3) nd = 1;
+        ncell[d] = (int32_t)nd;
+        invh[d] = (float)((double)nd / (double)len[d]);
+    }
+    return 0;
+}
+
+/* stable counting sort of the points by cell id (ties by original index) */
+int oracle_bin(const float* pos, int64_t n, const int32_t* ncell, const float* invh,
+               int32_t* cell, int32_t* cell_start, int32_t* order) {
+    int64_t nc = (int64_t)ncell[0] * ncell[1] * ncell[2];
+    for (int64_t c = 0; c <= nc; ++c) cell_start[c] = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        int32_t c[3];
+        for (int d = 0; d < 3; ++d) {
+            volatile float t = pos[3 * i + d] * invh[d];   /* one rounded fp32 product */
+            int32_t k = (int32_t)floorf(t);
+            if (k > ncell[d] - 1) k = ncell[d] - 1;
+            if (k < 0) k = 0;
+            c[d] = k;
+        }
+        cell[i] = (c[2] * ncell[1] + c[1]) * ncell[0] + c[0];
+        cell_start[cell[i] + 1] += 1;
+    }
+    for (int64_t c = 0; c < nc; ++c) cell_start[c + 1] += cell_start[c];
+    int32_t* fill = (int32_t*)malloc(sizeof(int32_t) * (size_t)(nc > 0 ? nc : 1));
+    if (!fill) return 1;
+    memcpy(fill, cell_start, sizeof(int32_t) * (size_t)nc);
+    for (int64_t i = 0; i < n; ++i) order[fill[cell[i]]++] = (int32_t)i;
+    free(fill);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ radius relation
+ * Displacement of the ordered pair (i, j): D = p_i - p_j, minimum image in periodic
+ * dimensions (D -= L rint(D / L)), d2 = Dx^2 + Dy^2 + Dz^2 summed left to right,
+ * j is a neighbour of i iff j != i and d2 <= r*r (inclusive, Appendix A).
+ */
+typedef struct {
+    const double* pos;
+    int64_t n;
+    double r2;
+    double len[3];
+    int periodic[3];
+} rel_t;
+
+static inline int pair_d2(const rel_t* R, int64_t i, int64_t j, double D[3], double* d2) {
+    for (int d = 0; d < 3; ++d) {
+        double t = R->pos[3 * i + d] - R->pos[3 * j + d];
+        if (R->periodic[d]) t -= R->len[d] * rint(t / R->len[d]);
+        D[d] = t;
+    }
+    *d2 = D[0] * D[0] + D[1] * D[1] + D[2] * D[2];
+    return *d2 <= R->r2;
+}
+
+/* Optional candidate restriction: an fp64 cell directory of the oracle's own
+ * (cell edge >= r, 27-cell stencil, wrapped or clipped).  It changes which pairs are
+ * tested, never the predicate; the tests check it against the all-pairs loop. */
+typedef struct {
+    int nc[3];
+    int64_t* start;   /* [ncells+1] */
+    int64_t* items;   /* point ids grouped by cell, ascending inside a cell */
+} grid_t;
+
+static void cell_of(const rel_t* R, const grid_t* G, int64_t i, int c[3]) {
+    for (int d = 0; d < 3; ++d) {
+        int k = (int)floor(R->pos[3 * i + d] / R->len[d] * G->nc[d]);
+        if (k < 0) k = 0;
+        if (k > G->nc[d] - 1) k = G->nc[d] - 1;
+        c[d] = k;
+    }
+}
+
+static int grid_build(const rel_t* R, double r, grid_t* G) {
+    int64_t total = 1;
+    for (int d = 0; d < 3; ++d) {
+        double q = floor(R->len[d] / r);
+        int k = q < 1.0 ? 1 : (q > 512.0 ? 512 : (int)q);
+        if (k < 3) k = 1;
+        G->nc[d] = k;
+        total *= k;
+    }
+    G->start = (int64_t*)calloc((size_t)total + 1, sizeof(int64_t));
+    G->items = (int64_t*)malloc(sizeof(int64_t) * (size_t)(R->n > 0 ? R->n : 1));
+    if (!G->start || !G->items) return 1;
+    for (int64_t i = 0; i < R->n; ++i) {
+        int c[3];
+        cell_of(R, G, i, c);
+        G->start[((int64_t)c[2] * G->nc[1] + c[1]) * G->nc[0] + c[0] + 1] += 1;
+    }
+    for (int64_t c = 0; c < total; ++c) G->start[c + 1] += G->start[c];
+    int64_t* fill = (int64_t*)malloc(sizeof(int64_t) * (size_t)total);
+    if (!fill) return 1;
+    memcpy(fill, G->start, sizeof(int64_t) * (size_t)total);
+    for (int64_t i = 0; i < R->n; ++i) {
+        int c[3];
+        cell_of(R, G, i, c);
+        G->items[fill[((int64_t)c[2] * G->nc[1] + c[1]) * G->nc[0] + c[0]]++] = i;
+    }
+    free(fill);
+    return 0;
+}
+
+/* candidate list of point i into buf (ascending ids are NOT guaranteed; callers that need
+ * index order sort it).  Returns the number of candidates. */
+static int cmp_i64(const void* a, const void* b) {
+    int64_t x = *(const int64_t*)a, y = *(const int64_t*)b;
+    return (x > y) - (x < y);
+}
+
+static int64_t candidates(const rel_t* R, const grid_t* G, int64_t i, int64_t** buf, int64_t* cap) {
+    int c[3];
+    cell_of(R, G, i, c);
+    int64_t m = 0;
+    int lo[3], hi[3];
+    for (int d = 0; d < 3; ++d) {
+        if (G->nc[d] == 1) { lo[d] = 0; hi[d] = 0; }
+        else { lo[d] = -1; hi[d] = 1; }
+    }
+    for (int dz = lo[2]; dz <= hi[2]; ++dz)
+        for (int dy = lo[1]; dy <= hi[1]; ++dy)
+            for (int dx = lo[0]; dx <= hi[0]; ++dx) {
+                int q[3] = { c[0] + dx, c[1] + dy, c[2] + dz };
+                int ok = 1;
+                for (int d = 0; d < 3; ++d) {
+                    if (q[d] < 0 || q[d] >= G->nc[d]) {
+                        if (R->periodic[d]) q[d] = (q[d] + G->nc[d]) % G->nc[d];
+                        else ok = 0;
+                    }
+                }
+                if (!ok) continue;
+                int64_t id = ((int64_t)q[2] * G->nc[1] + q[1]) * G->nc[0] + q[0];
+                for (int64_t t = G->start[id]; t < G->start[id + 1]; ++t) {
+                    if (m == *cap) {
+                        *cap = *cap ? *cap * 2 : 256;
+                        *buf = (int64_t*)realloc(*buf, sizeof(int64_t) * (size_t)*cap);
+                    }
+                    (*buf)[m++] = G->items[t];
+                }
+            }
+    qsort(*buf, (size_t)m, sizeof(int64_t), cmp_i64);
+    return m;
+}
+
+static void rel_init(rel_t* R, const double* pos, int64_t n, double r, const double* len,
+                     const int32_t* periodic) {
+    R->pos = pos;
+    R->n = n;
+    R->r2 = r * r;
+    for (int d = 0; d < 3; ++d) { R->len[d] = len[d]; R->periodic[d] = periodic[d]; }
+}
+
+/* ------------------------------------------------------------------ fused radius forward
+ * For each requested row i (rows == NULL: all rows) and every neighbour j in index order:
+ *   GAUSS : y_i += exp(-d2 / (2 p0^2)) x_j                       (Fout = F)
+ *   DIST  : y_i += sqrt(d2) x_j                                  (Fout = F)
+ *   LJ    : q = p1^2/d2, q3 = q^3, (Fx,Fy,Fz) += 24 p0 (2 q3^2 - q3)/d2 * D,
+ *           e += (1/2) 4 p0 (q3^2 - q3)                          (Fout = 4, feat unused)
+ * A receives the sums of absolute contributions, count the number of neighbours.
+ * No neighbours -> zero vector (Appendix A).
+ */
+int oracle_radius_forward(const double* pos, const double* feat, int64_t n, int F,
+                          double r, const double* len, const int32_t* periodic,
+                          int kind, double p0, double p1,
+                          const int64_t* rows, int64_t n_rows, int use_cells,
+                          double* y, double* A, int32_t* count) {
+    rel_t R;
+    rel_init(&R, pos, n, r, len, periodic);
+    grid_t G = { {0, 0, 0}, NULL, NULL };
+    if (use_cells && grid_build(&R, r, &G)) return 1;
+    const int Fo = (kind == MSG_LJ) ? 4 : F;
+    if (!rows) n_rows = n;
+#pragma omp parallel
+    {
+        int64_t* buf = NULL;
+        int64_t cap = 0;
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t t = 0; t < n_rows; ++t) {
+            int64_t i = rows ? rows[t] : t;
+            double* yi = y + t * Fo;
+            double* Ai = A ? A + t * Fo : NULL;
+            for (int f = 0; f < Fo; ++f) { yi[f] = 0.0; if (Ai) Ai[f] = 0.0; }
+            int32_t cnt = 0;
+            int64_t m = use_cells ? candidates(&R, &G, i, &buf, &cap) : n;
+            for (int64_t u = 0; u < m; ++u) {
+                int64_t j = use_cells ? buf[u] : u;
+                if (j == i) continue;
+                double D[3], d2;
+                if (!pair_d2(&R, i, j, D, &d2)) continue;
+                ++cnt;
+                if (kind == MSG_LJ) {
+                    double q = p1 * p1 / d2, q3 = q * q * q;
+                    double fs = 24.0 * p0 * (2.0 * q3 * q3 - q3) / d2;
+                    double e = 0.5 * 4.0 * p0 * (q3 * q3 - q3);
+                    for (int d = 0; d < 3; ++d) {
+                        yi[d] += fs * D[d];
+                        if (Ai) Ai[d] += fabs(fs * D[d]);
+                    }
+                    yi[3] += e;
+                    if (Ai) Ai[3] += fabs(e);
+                } else {
+                    double g = (kind == MSG_GAUSS) ? exp(-d2 / (2.0 * p0 * p0)) : sqrt(d2);
+                    for (int f = 0; f < F; ++f) {
+                        double c = g * feat[j * F + f];
+                        yi[f] += c;
+                        if (Ai) Ai[f] += fabs(c);
+                    }
+                }
+            }
+            if (count) count[t] = cnt;
+        }
+        free(buf);
+    }
+    free(G.start);
+    free(G.items);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ fused radius backward
+ * Gaussian message, membership frozen (Section 5).  With L = sum_i ybar_i . y_i
+ *   = sum over ordered pairs (i, j in N(i)) of g_ij (ybar_i . x_j),  g_ij = exp(-|D_ij|^2/(2 s^2)),
+ * the plain chain rule gives, for output row k,
+ *   xbar_k  = sum over i with k in N(i) of g_ik ybar_i
+ *   pbar_k  = sum over j in N(k)        of (-g_kj / s^2) D_kj (ybar_k . x_j)     [k is the query]
+ *           + sum over i with k in N(i) of (+g_ik / s^2) D_ik (ybar_i . x_k)     [k is the source]
+ * Both sums are evaluated separately, each pair from its own displacement.
+ */
+int oracle_radius_backward_gauss(const double* pos, const double* feat, const double* gy,
+                                 int64_t n, int F, double r, const double* len,
+                                 const int32_t* periodic, double sigma,
+                                 const int64_t* rows, int64_t n_rows, int use_cells,
+                                 double* gx, double* Agx, double* gp, double* Agp) {
+    rel_t R;
+    rel_init(&R, pos, n, r, len, periodic);
+    grid_t G = { {0, 0, 0}, NULL, NULL };
+    if (use_cells && grid_build(&R, r, &G)) return 1;
+    if (!rows) n_rows = n;
+    const double is2 = 1.0 / (sigma * sigma);
+#pragma omp parallel
+    {
+        int64_t* buf = NULL;
+        int64_t cap = 0;
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t t = 0; t < n_rows; ++t) {
+            int64_t k = rows ? rows[t] : t;
+            if (gx) for (int f = 0; f < F; ++f) { gx[t * F + f] = 0.0; if (Agx) Agx[t * F + f] = 0.0; }
+            if (gp) for (int d = 0; d < 3; ++d) { gp[t * 3 + d] = 0.0; if (Agp) Agp[t * 3 + d] = 0.0; }
+            int64_t m = use_cells ? candidates(&R, &G, k, &buf, &cap) : n;
+            for (int64_t u = 0; u < m; ++u) {
+                int64_t o = use_cells ? buf[u] : u;
+                if (o == k) continue;
+                double D[3], d2;
+                /* k as the query, o as its neighbour j */
+                if (pair_d2(&R, k, o, D, &d2)) {
+                    double g = exp(-d2 / (2.0 * sigma * sigma));
+                    double dot = 0.0;
+                    for (int f = 0; f < F; ++f) dot += gy[k * F + f] * feat[o * F + f];
+                    if (gp) for (int d = 0; d < 3; ++d) {
+                        double c = (-g * is2) * D[d] * dot;
+                        gp[t * 3 + d] += c;
+                        if (Agp) Agp[t * 3 + d] += fabs(c);
+                    }
+                }
+                /* o as the query i, k as its neighbour (the source) */
+                if (pair_d2(&R, o, k, D, &d2)) {
+                    double g = exp(-d2 / (2.0 * sigma * sigma));
+                    double dot = 0.0;
+                    for (int f = 0; f < F; ++f) dot += gy[o * F + f] * feat[k * F + f];
+                    if (gp) for (int d = 0; d < 3; ++d) {
+                        double c = (g * is2) * D[d] * dot;
+                        gp[t * 3 + d] += c;
+                        if (Agp) Agp[t * 3 + d] += fabs(c);
+                    }
+                    if (gx) for (int f = 0; f < F; ++f) {
+                        double c = g * gy[o * F + f];
+                        gx[t * F + f] += c;
+                        if (Agx) Agx[t * F + f] += fabs(c);
+                    }
+                }
+            }
+        }
+        free(buf);
+    }
+    free(G.start);
+    free(G.items);
+    return 0;
+}
+
+int oracle_num_threads(void) {
+    int n = 1;
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    n = omp_get_max_threads();
+#endif
+    return n;
+}
