@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the gf.apply hot path on B200: interactions/s and roofline fractions.
+
+One *step* is one pass of the whole hot path over one batch of seeded synthetic input:
+  CSR relation   (R-MAT scale 20, 16.8M directed edges, F=64 fp32): sum forward, sum backward
+                 (grad x, grad w), max forward, max backward, degree histogram;
+  radius relation (1M uniform points, periodic unit cube, 32 expected neighbours, F=32):
+                 cell binning + fused Gaussian forward, backward (grad x, grad positions);
+  Lennard-Jones   (160^3 jittered lattice, cutoff 2.5): cell binning + fused force/energy.
+One interaction = one directed edge / one ordered accepted pair visited by one traversal.
+
+`python bench.py --gpus N --steps K --warmup W` prints ONE JSON line (rank 0).  Under
+torchrun every rank runs an independent replica of the step on its own GPU (the path has no
+exchange step); the time is the max over ranks and `value` the sum of all ranks' work.
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workloads.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import gen  # noqa: E402
+
+METRIC = "interactions/sec fwd and fwd+bwd for gf.apply"
+UNIT = "interactions/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return float(d["hbm_gbs"]), float(d.get("sm_max_mhz", 1965.0)), "measured"
+    return 6650.0, 1965.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index = index
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self.stop_flag = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self.stop_flag.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def summary(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons)}
+
+
+def physical_gpu_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ------------------------------------------------------------------------------ workloads
+def make_workloads(seed):
+    t0 = time.time()
+    w = {"csr": gen.config("cfg1", seed), "rad": gen.config("cfg2", seed), "lj": gen.config("cfg3", seed)}
+    w["gen_seconds"] = time.time() - t0
+    return w
+
+
+def roofline_models(w, counts, hbm_gbs, clock_mhz):
+    """Algorithmic work per launch of every row of the hot path.
+
+    CSR: cache-oblivious gather model, bytes = E (col + w + one source row) + N (rowptr + one
+    output row); backward adds the cotangent row, the atomic read-modify-write of the
+    source-gradient row and the edge gradient.  Radius: fp32 lane operations (FMA = 1),
+    7 per candidate pair (27-cell stencil) plus F+3 (Gaussian forward), 3F+12 (Gaussian
+    backward) or 14 (Lennard-Jones) per accepted pair.
+    """
+    c = w["csr"]
+    E, N, F = c["E"], c["n"], c["F"]
+    fb = 4 * F
+    m = {}
+    m["csr_sum_fwd"] = dict(bound="hbm", work=E * (8 + fb) + N * (4 + fb), inter=E)
+    m["csr_max_fwd"] = dict(bound="hbm", work=E * (8 + fb) + N * (4 + 2 * fb), inter=E)
+    m["csr_sum_bwd"] = dict(bound="hbm", work=E * (8 + fb + 4 + 2 * fb) + N * (4 + fb) + N * fb, inter=E)
+    m["csr_max_bwd"] = dict(bound="hbm", work=N * F * (4 + 4 + 4 + 4 + 4 + 8 + 8), inter=E)
+    m["csr_hist"] = dict(bound="hbm", work=4 * (N + 1), inter=0)
+    alu_peak = 148 * 128 * clock_mhz * 1e6      # fp32 lane operations per second
+    for key, cfg, acc in (("rad", w["rad"], counts["rad_pairs"]), ("lj", w["lj"], counts["lj_pairs"])):
+        n = cfg["n"]
+        ncell = counts[key + "_ncell"]
+        cand = 27.0 * n * n / ncell             # candidate pairs tested by a 27-cell stencil
+        if key == "rad":
+            Fr = cfg["F"]
+            m["radius_gauss_fwd"] = dict(bound="alu", work=7 * cand + (Fr + 3) * acc, inter=acc)
+            m["radius_gauss_bwd"] = dict(bound="alu", work=7 * cand + (3 * Fr + 12) * acc, inter=acc)
+        else:
+            m["radius_lj_fwd"] = dict(bound="alu", work=7 * cand + 14 * acc, inter=acc)
+    for k, v in m.items():
+        v["peak"] = hbm_gbs * 1e9 if v["bound"] == "hbm" else alu_peak
+    return m
+
+
+# ------------------------------------------------------------------------------ our arm
+def run_ours(args, rank, world, local_rank):
+    import torch
+    from paper_2609_24802_b200 import api as T
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    hbm_gbs, sm_max, peak_kind = measured_peaks()
+    w = make_workloads(args.seed + rank)
+    c, r, lj = w["csr"], w["rad"], w["lj"]
+
+    def pin(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+
+    # pinned host copies (for the end-to-end leg) and device-resident inputs
+    h = {"rowptr": pin(c["rowptr"]), "col": pin(c["col"]), "w": pin(c["w"]), "x": pin(c["x"]), "gy": pin(c["gy"]),
+         "rpos": pin(r["pos"]), "rx": pin(r["x"]), "rgy": pin(r["gy"]), "ljpos": pin(lj["pos"])}
+    d = {k: v.to(dev) for k, v in h.items()}
+    g = T.CsrRelation(d["rowptr"], d["col"], c["n"])
+    N, E, F = c["n"], c["E"], c["F"]
+    n2, F2 = r["n"], r["F"]
+    n3 = lj["n"]
+
+    out_sum = torch.empty((N, F), device=dev); out_max = torch.empty((N, F), device=dev)
+    arg = torch.empty((N, F), dtype=torch.int32, device=dev)
+    gx = torch.empty((N, F), device=dev); gw = torch.empty(E, device=dev)
+    gxm = torch.empty((N, F), device=dev); gwm = torch.empty(E, device=dev)
+    ws_csr = torch.empty(T.tiga_csr_workspace_bytes(g, F, T.F32, T.MAX), dtype=torch.uint8, device=dev)
+    rout = torch.empty((n2, F2), device=dev); rcount = torch.empty(n2, dtype=torch.int32, device=dev)
+    rgx = torch.empty((n2, F2), device=dev); rgp = torch.empty((n2, 3), device=dev)
+    ws_rad = torch.empty(T.tiga_radius_workspace_bytes(n2, F2, r["r"], r["box"], r["periodic"]), dtype=torch.uint8, device=dev)
+    ljout = torch.empty((n3, 4), device=dev); ljcount = torch.empty(n3, dtype=torch.int32, device=dev)
+    ws_lj = torch.empty(T.tiga_radius_workspace_bytes(n3, 4, lj["r"], lj["box"], lj["periodic"]), dtype=torch.uint8, device=dev)
+
+    rows = ["csr_sum_fwd", "csr_sum_bwd", "csr_max_fwd", "csr_max_bwd", "csr_hist",
+            "radius_gauss_fwd", "radius_gauss_bwd", "radius_lj_fwd"]
+    stream = torch.cuda.current_stream()
+
+    def step(ev=None):
+        def mark(i):
+            if ev is not None:
+                ev[i].record(stream)
+        mark(0)
+        T.tiga_apply_csr(g, d["x"], d["w"], T.SUM, out=out_sum, ws=ws_csr); mark(1)
+        T.tiga_apply_csr_backward(g, d["x"], d["w"], d["gy"], T.SUM, grad_x=gx, grad_w=gw); mark(2)
+        T.tiga_apply_csr(g, d["x"], d["w"], T.MAX, out=out_max, argmax=arg, ws=ws_csr); mark(3)
+        T.tiga_apply_csr_backward(g, d["x"], d["w"], d["gy"], T.MAX, argmax=arg, grad_x=gxm, grad_w=gwm); mark(4)
+        hist, mx = T.tiga_csr_degree_histogram(g, 4096); mark(5)
+        T.tiga_apply_radius(d["rpos"], d["rx"], r["r"], r["box"], r["periodic"], T.MSG_GAUSS, p0=r["sigma"],
+                            out=rout, count=rcount, ws=ws_rad); mark(6)
+        T.tiga_apply_radius_backward(d["rpos"], d["rx"], d["rgy"], r["r"], r["box"], r["periodic"], r["sigma"],
+                                     ws=ws_rad, reuse_plan=True, grad_feat=rgx, grad_pos=rgp); mark(7)
+        T.tiga_apply_radius(d["ljpos"], None, lj["r"], lj["box"], lj["periodic"], T.MSG_LJ, p0=lj["eps"], p1=lj["s"],
+                            out=ljout, count=ljcount, ws=ws_lj); mark(8)
+        return hist, mx
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sync_all()
+    counts = {"rad_pairs": int(rcount.sum().item()), "lj_pairs": int(ljcount.sum().item()),
+              "rad_ncell": int(np.prod(T.tiga_radius_grid(n2, r["r"], r["box"], r["periodic"])[0])),
+              "lj_ncell": int(np.prod(T.tiga_radius_grid(n3, lj["r"], lj["box"], lj["periodic"])[0]))}
+    inter_step = 4 * E + 2 * counts["rad_pairs"] + counts["lj_pairs"]
+
+    # ---- timed region: device-resident inputs
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(9)] for _ in range(args.steps)]
+    l0 = T.launch_count()
+    sync_all()
+    sampler.start()
+    t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for k in range(args.steps):
+        step(evs[k])
+    t_end.record(stream)
+    sync_all()
+    sampler.stop_flag.set()
+    launches = T.launch_count() - l0
+    total_ms = t_start.elapsed_time(t_end)
+    per_row_ms = [statistics.mean(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps)) for i in range(8)]
+    clocks = sampler.summary()
+
+    # ---- end-to-end leg: inputs start in pinned host memory, results end in pinned host memory
+    res_h = {"out_sum": torch.empty((N, F)).pin_memory(), "gx": torch.empty((N, F)).pin_memory(),
+             "gw": torch.empty(E).pin_memory(), "out_max": torch.empty((N, F)).pin_memory(),
+             "gxm": torch.empty((N, F)).pin_memory(), "gwm": torch.empty(E).pin_memory(),
+             "hist": torch.empty(4096, dtype=torch.int64).pin_memory(),
+             "rout": torch.empty((n2, F2)).pin_memory(), "rgx": torch.empty((n2, F2)).pin_memory(),
+             "rgp": torch.empty((n2, 3)).pin_memory(), "ljout": torch.empty((n3, 4)).pin_memory()}
+    h2d = sum(v.numel() * v.element_size() for v in h.values())
+    d2h = sum(v.numel() * v.element_size() for v in res_h.values())
+
+    def e2e_step():
+        for k, v in h.items():
+            d[k].copy_(v, non_blocking=True)
+        hist, _ = step()
+        for k, src in (("out_sum", out_sum), ("gx", gx), ("gw", gw), ("out_max", out_max), ("gxm", gxm), ("gwm", gwm),
+                       ("hist", hist), ("rout", rout), ("rgx", rgx), ("rgp", rgp), ("ljout", ljout)):
+            res_h[k].copy_(src, non_blocking=True)
+
+    e2e_step()
+    sync_all()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record(stream)
+    sync_all()
+    e2e_ms = e0.elapsed_time(e1)
+
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = t.tolist()
+        tot = torch.tensor([inter_step], device=dev, dtype=torch.float64)
+        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
+        inter_all = tot.item()
+    else:
+        inter_all = float(inter_step)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = total_ms / args.steps
+    value = inter_all / (ms_per_step * 1e-3)
+    clock_for_alu = clocks["sm_mhz"] or sm_max
+    models = roofline_models(w, counts, hbm_gbs, clock_for_alu)
+    row_report = {}
+    for name, ms in zip(rows, per_row_ms):
+        mdl = models[name]
+        ach = mdl["work"] / (ms * 1e-3)
+        row_report[name] = {"ms": round(ms, 4), "interactions_per_s": (mdl["inter"] / (ms * 1e-3)) if mdl["inter"] else None,
+                            "bound": mdl["bound"],
+                            "achieved": ach / (1e9 if mdl["bound"] == "hbm" else 1e12),
+                            "peak": mdl["peak"] / (1e9 if mdl["bound"] == "hbm" else 1e12),
+                            "unit": "GB/s" if mdl["bound"] == "hbm" else "Tlaneop/s", "frac": ach / mdl["peak"]}
+    dom = max(rows, key=lambda k: row_report[k]["ms"])
+    dr = row_report[dom]
+    fwd = {"csr_sum": E / (per_row_ms[0] * 1e-3), "csr_max": E / (per_row_ms[2] * 1e-3),
+           "radius_gauss": counts["rad_pairs"] / (per_row_ms[5] * 1e-3), "radius_lj": counts["lj_pairs"] / (per_row_ms[7] * 1e-3)}
+    fwd_bwd = {"csr_sum": E / ((per_row_ms[0] + per_row_ms[1]) * 1e-3), "csr_max": E / ((per_row_ms[2] + per_row_ms[3]) * 1e-3),
+               "radius_gauss": counts["rad_pairs"] / ((per_row_ms[5] + per_row_ms[6]) * 1e-3)}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "cfg1 CSR R-MAT scale 20 E=16,777,216 F=64 fp32 (sum fwd+bwd, max fwd+bwd, degree histogram) "
+                               "+ cfg2 radius N=1,000,000 periodic F=32 Gaussian (bin+fwd, bwd) "
+                               "+ cfg3 Lennard-Jones N=4,096,000 (bin+fwd)",
+                   "seed": args.seed, "l2": "inputs larger than L2 (644 MB CSR inputs; each kernel streams >126 MB between repeats)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "interactions_per_step": inter_step, "radius_pairs": counts["rad_pairs"], "lj_pairs": counts["lj_pairs"]},
+        "fwd_interactions_per_s": fwd, "fwd_bwd_interactions_per_s": fwd_bwd, "rows": row_report,
+        "roofline": {"kernel": dom, "bound": dr["bound"], "achieved": dr["achieved"], "peak": dr["peak"], "unit": dr["unit"],
+                     "frac": dr["frac"], "traffic": None, "peak_source": peak_kind + (" hbm copy" if dr["bound"] == "hbm" else
+                                                                                     " 148 SM x 128 lanes x sampled SM clock")},
+        "e2e": {"value": inter_all / (e2e_ms / args.steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches, "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world >= 1:
+        line["cpu_baseline"] = cpu_baseline(w, seconds_hint=20)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------ CPU oracle arms
+def cpu_baseline(w, seconds_hint=20):
+    """The fp64 oracle, as it stands, on a bounded sample of the step's workloads."""
+    import oracle
+    c = w["csr"]
+    rows = 1 << 18                                  # first quarter of the destination rows
+    rp = c["rowptr"][: rows + 1].astype(np.int64)
+    e = int(rp[-1])
+    col = c["col"][:e]; wt = c["w"][:e]; gy = c["gy"][:rows]
+    t0 = time.time()
+    oracle.csr_forward(rp, col, c["x"], wt, oracle.SUM)
+    oracle.csr_backward_sum(rp, col, c["x"], wt, gy)
+    t_csr = time.time() - t0
+    rr = gen.config("cfg2", n=131_072)
+    t0 = time.time()
+    _, _, cnt = oracle.radius_forward(rr["pos"], rr["x"], rr["r"], rr["box"], rr["periodic"], oracle.MSG_GAUSS,
+                                      p0=rr["sigma"], use_cells=True)
+    oracle.radius_backward_gauss(rr["pos"], rr["x"], rr["gy"], rr["r"], rr["box"], rr["periodic"], rr["sigma"], use_cells=True)
+    t_rad = time.time() - t0
+    inter = 2 * e + 2 * int(cnt.sum())
+    return {"value": inter / (t_csr + t_rad), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"CSR sum fwd+bwd on the first {rows} rows of cfg1 ({e} edges, {t_csr:.2f} s) + radius Gaussian fwd+bwd "
+                      f"(cell directory) on a 131,072-point replica of cfg2 ({int(cnt.sum())} pairs, {t_rad:.2f} s)"}
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    import oracle
+    w = {"csr": gen.config("cfg1", args.seed, scale=16)}
+    c = w["csr"]
+    rr = gen.config("cfg2", args.seed, n=32_768)
+    lj = gen.config("cfg3", args.seed, m=20)
+
+    def step():
+        inter = 0
+        for red in (oracle.SUM, oracle.MAX):
+            y, A, arg = oracle.csr_forward(c["rowptr"], c["col"], c["x"], c["w"], red)
+            if red == oracle.SUM:
+                oracle.csr_backward_sum(c["rowptr"], c["col"], c["x"], c["w"], c["gy"])
+            else:
+                oracle.csr_backward_max(c["rowptr"], c["col"], c["x"], c["w"], c["gy"], arg)
+            inter += 2 * c["E"]
+        oracle.degree_histogram(c["rowptr"], 4096)
+        _, _, cnt = oracle.radius_forward(rr["pos"], rr["x"], rr["r"], rr["box"], rr["periodic"], oracle.MSG_GAUSS,
+                                          p0=rr["sigma"], use_cells=True)
+        oracle.radius_backward_gauss(rr["pos"], rr["x"], rr["gy"], rr["r"], rr["box"], rr["periodic"], rr["sigma"], use_cells=True)
+        inter += 2 * int(cnt.sum())
+        _, _, cnt = oracle.radius_forward(lj["pos"], None, lj["r"], lj["box"], lj["periodic"], oracle.MSG_LJ, 1.0, 1.0, use_cells=True)
+        inter += int(cnt.sum())
+        return inter
+
+    for _ in range(min(args.warmup, 1)):
+        step()
+    t0 = time.time()
+    inter = 0
+    for _ in range(args.steps):
+        inter += step()
+    dt = time.time() - t0
+    value = inter / dt
+    sample = ("every row of the step on scaled-down replicas: R-MAT scale 16 (1,048,576 edges, F=64), "
+              "32,768-point periodic Gaussian radius, 8,000-particle Lennard-Jones")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "bounded sample of: cfg1 CSR + cfg2 radius + cfg3 Lennard-Jones (" + sample + ")", "seed": args.seed},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--seed", type=int, default=gen.DEFAULT_SEED)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

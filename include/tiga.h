@@ -1,0 +1,186 @@
+/*
+ * tiga.h -- C ABI of libtiga: the gf.apply gather / message / reduce hot path of
+ * "Tiga: Compiling Graph Message Passing at Scale" as hand-written CUDA for sm_100a.
+ *
+ * Two traversals of the same operation (paper Section 3.1):
+ *     m_e = f(x_s(e), a_e),     y_i = finalize( combine_{e : d(e) = i} lift(m_e) )
+ *   1. a stored destination-oriented CSR relation with a sum or max segment reduce
+ *      (Sections 3.1 and 4.3) and its reverse mode (Section 5);
+ *   2. a generated radius relation N(i) = { j != i : |p_j - p_i| <= r } (Appendix A) that is
+ *      produced on the fly through a cell directory and consumed by the message and a sum
+ *      reducer without storing edges or messages (Section 4.9), and its reverse mode with
+ *      the membership frozen (Section 5).
+ *
+ * Conventions for every entry point
+ *   - All array arguments are DEVICE pointers (global memory of the current device) unless
+ *     the comment says "host".  The small structs (tiga_csr, tiga_box, tiga_msg) are passed
+ *     by HOST pointer and read before the call returns; no struct crosses the ABI by value.
+ *   - The caller owns every buffer.  The library allocates nothing and keeps no state
+ *     between calls except what it writes into the caller's workspace `ws`.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = the default
+ *     stream) and return without synchronising unless stated otherwise.
+ *   - Outputs are overwritten in full (empty rows and points without neighbours included);
+ *     gradients are overwritten, not accumulated.  Rows of every output are in the
+ *     caller's original row / point order.
+ *   - Base pointers must be 16-byte aligned.  Feature rows are dense, row major.
+ *   - Return value: TIGA_OK, or the first error found on the host.  Nothing is launched
+ *     when an error is returned.  Errors never raise a device fault.
+ */
+#ifndef TIGA_H
+#define TIGA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TIGA_OK = 0,
+    TIGA_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, negative size, bad enum, bad box */
+    TIGA_ERR_UNSUPPORTED = 2,   /* a combination this build has no kernel for */
+    TIGA_ERR_WORKSPACE = 3,     /* ws is NULL or smaller than *_workspace_bytes() */
+    TIGA_ERR_CUDA = 4,          /* a CUDA runtime call failed */
+    TIGA_ERR_INVALID_GRAPH = 5  /* tiga_validate_csr found a malformed relation */
+} tiga_status;
+
+typedef enum { TIGA_F32 = 0, TIGA_F16 = 1 } tiga_dtype;   /* feature storage; accumulation is fp32 */
+typedef enum { TIGA_I32 = 0, TIGA_I64 = 1 } tiga_itype;   /* rowptr storage; col is always int32 */
+typedef enum { TIGA_SUM = 0, TIGA_MAX = 1 } tiga_reducer;
+
+typedef enum {
+    TIGA_MSG_COPY = 0,      /* CSR: m = x_j                         (w must be NULL)           */
+    TIGA_MSG_WEIGHTED = 1,  /* CSR: m = w_e * x_j                   (Section 3.1 example)      */
+    TIGA_MSG_GAUSS = 2,     /* radius: m = exp(-d^2 / (2 p0^2)) * x_j,  p0 = sigma             */
+    TIGA_MSG_DIST = 3,      /* radius: m = d * x_j  (the paper's distance-weighted sum, Sec. 7) */
+    TIGA_MSG_LJ = 4         /* radius: Lennard-Jones pair force and energy, p0 = eps, p1 = s   */
+} tiga_msg_kind;
+
+typedef struct {
+    int32_t kind;           /* tiga_msg_kind */
+    float p0, p1;
+} tiga_msg;
+
+/* Destination-oriented CSR relation (Section 3.1): rows enumerate destinations, col[e] is
+ * the source of edge e, the edge position e indexes edge fields.  Duplicate edges are
+ * separate messages, a self edge is ordinary, there is no implicit reverse edge. */
+typedef struct {
+    const void* rowptr;     /* device, int32 or int64 [n_dst + 1], rowptr[0] = 0, rowptr[n_dst] = n_edges */
+    int32_t rowptr_type;    /* tiga_itype */
+    const int32_t* col;     /* device, int32 [n_edges], values in [0, n_src) */
+    int64_t n_dst, n_src, n_edges;
+} tiga_csr;
+
+/* Axis-aligned box with its origin at 0.  Points must lie in [0, len[d]] in every dimension.
+ * periodic[d] != 0 selects the minimum image in that dimension and requires r < len[d] / 2. */
+typedef struct {
+    float len[3];
+    int32_t periodic[3];
+} tiga_box;
+
+const char* tiga_status_string(tiga_status s);
+
+/* ------------------------------------------------------------------------------------ CSR */
+
+/* Bytes of workspace tiga_apply_csr (backward = 0) or tiga_apply_csr_backward (backward = 1)
+ * needs for this relation, feature width and reducer.  Host only, launches nothing. */
+size_t tiga_csr_workspace_bytes(const tiga_csr* g, int32_t F, tiga_dtype x_dtype,
+                                tiga_reducer reducer, int backward);
+
+/* Full validation (Section 6, "Validation and trust boundaries": monotone row pointers,
+ * endpoints, source-index bounds) when level = 1; metadata only when level = 0.
+ * ws: at least 16 bytes of device memory.  level 1 launches a scan and SYNCHRONISES the
+ * stream.  Returns TIGA_ERR_INVALID_GRAPH when a check fails. */
+tiga_status tiga_validate_csr(const tiga_csr* g, int level, void* ws, size_t ws_bytes, void* stream);
+
+/* Fused gather-message-reduce over a stored relation (Sections 3.1, 4.2, 4.3):
+ *   sum : out[i,f] = sum over e in [rowptr[i], rowptr[i+1]) of w[e] * x[col[e], f]
+ *   max : out[i,f] = max over the same edges; argmax[i,f] = the lowest edge position that
+ *         attains it.  An empty row gives 0 (and argmax = -1).
+ * No E x F message array is formed.
+ *   x      : [n_src, F], x_dtype.  F must be a multiple of 4 (fp32) or 8 (fp16).
+ *   w      : fp32 [n_edges] or NULL for unit weights (msg.kind = TIGA_MSG_COPY).
+ *   out    : fp32 [n_dst, F].
+ *   argmax : int32 [n_dst, F]; required for TIGA_MAX (needs n_edges < 2^31), ignored for TIGA_SUM.
+ *   ws     : tiga_csr_workspace_bytes(g, F, x_dtype, reducer, 0) bytes; contents are scratch.
+ * Rows longer than one tile are split and their partial states merged in edge order, so
+ * results are reproducible from run to run. */
+tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
+                           const float* w, const tiga_msg* msg, tiga_reducer reducer,
+                           float* out, int32_t* argmax, void* ws, size_t ws_bytes, void* stream);
+
+/* Reverse mode of tiga_apply_csr for fixed relation indices (Section 5):
+ *   sum : grad_w[e] = sum_f x[col[e],f] * grad_out[row(e),f]
+ *         grad_x[j,:] = sum over edges e with col[e] = j of w[e] * grad_out[row(e),:]
+ *   max : the cotangent of (i,f) flows only through edge argmax[i,f] (nothing if it is -1).
+ *   grad_out : fp32 [n_dst, F];  argmax : the forward's output (TIGA_MAX only).
+ *   grad_x   : fp32 [n_src, F] or NULL to skip;  grad_w : fp32 [n_edges] or NULL to skip.
+ * x must be fp32.  Repeated sources accumulate with floating-point atomics, so grad_x (and
+ * grad_w for TIGA_MAX) may differ in the last bits between runs. */
+tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
+                                    const float* w, const tiga_msg* msg, tiga_reducer reducer,
+                                    const float* grad_out, const int32_t* argmax,
+                                    float* grad_x, float* grad_w,
+                                    void* ws, size_t ws_bytes, void* stream);
+
+/* Degree histogram: deg_i = rowptr[i+1] - rowptr[i]; hist[d] = number of rows of degree d for
+ * d < nbins - 1, hist[nbins-1] = number of rows with deg >= nbins - 1; *max_degree = max deg.
+ *   hist : device int64 [nbins], 1 <= nbins <= 8192;  max_degree : device int64 [1]. */
+tiga_status tiga_csr_degree_histogram(const tiga_csr* g, int64_t* hist, int64_t nbins,
+                                      int64_t* max_degree, void* stream);
+
+/* --------------------------------------------------------------------------------- radius */
+
+/* Cell directory constants for n points, cutoff r and this box (host only):
+ *   ncell[d] = clamp(floor(len[d] / (r (1 + 2^-10))), 1, min(1024, floor(cbrt(8 n)))),
+ *   periodic dimensions with fewer than 3 cells use one cell,  invh[d] = (float)(ncell[d] / len[d]).
+ * A point's cell is min(ncell[d]-1, (int)floorf(p[d] * invh[d])) with one fp32 multiply;
+ * linear id = (c_z ncell[1] + c_y) ncell[0] + c_x.  Either output may be NULL. */
+tiga_status tiga_radius_grid(int64_t n, float r, const tiga_box* box, int32_t ncell[3], float invh[3]);
+
+/* Workspace bytes for tiga_radius_bin / tiga_apply_radius / tiga_apply_radius_backward. */
+size_t tiga_radius_workspace_bytes(int64_t n, int32_t F, float r, const tiga_box* box, int backward);
+
+/* Cell binning pass of the generated relation (Section 4.9): per-cell counts, exclusive scan,
+ * stable scatter into cell order.
+ *   pos        : fp32 [n, 3]
+ *   cell       : int32 [n]            cell id of every point                 (NULL to skip)
+ *   cell_start : int32 [ncells + 1]   exclusive scan of the per-cell counts  (NULL to skip)
+ *   order      : int32 [n]            point ids sorted by (cell id, point id) (NULL to skip)
+ * The same plan is left in ws for the apply calls. */
+tiga_status tiga_radius_bin(const float* pos, int64_t n, float r, const tiga_box* box,
+                            int32_t* cell, int32_t* cell_start, int32_t* order,
+                            void* ws, size_t ws_bytes, void* stream);
+
+/* Fused generated-relation apply (Section 4.9, Appendix A): bins the points, then for every
+ * point i accumulates the messages of all j != i with |p_i - p_j| <= r (minimum image in
+ * periodic dimensions; the predicate is decided exactly as in double precision) straight
+ * into the sum reducer.  Neither an edge list nor per-edge messages are written.
+ *   GAUSS / DIST : feat fp32 [n, F] (F multiple of 4, <= 128), out fp32 [n, F]
+ *   LJ           : feat ignored, F ignored, out fp32 [n, 4] = (Fx, Fy, Fz, e_i) with
+ *                  F_i = sum_j 24 eps (2 (s/d)^12 - (s/d)^6) (p_i - p_j) / d^2 and
+ *                  e_i = (1/2) sum_j 4 eps ((s/d)^12 - (s/d)^6)
+ *   count        : int32 [n] number of neighbours of every point, or NULL
+ * A point without neighbours gets the zero vector. */
+tiga_status tiga_apply_radius(const float* pos, const float* feat, int64_t n, int32_t F,
+                              float r, const tiga_box* box, const tiga_msg* msg,
+                              float* out, int32_t* count, void* ws, size_t ws_bytes, void* stream);
+
+/* Reverse mode of tiga_apply_radius for TIGA_MSG_GAUSS with the membership frozen
+ * (Section 5; Appendix A: positions enter through the displacement of selected edges):
+ *   grad_feat[j,:] = sum over i with j in N(i) of g_ij grad_out[i,:]
+ *   grad_pos[k,:]  = -(1/sigma^2) sum over j in N(k) of g_kj (p_k - p_j)
+ *                                  (grad_out[k].feat[j] + grad_out[j].feat[k])
+ *   grad_feat : fp32 [n, F] or NULL;  grad_pos : fp32 [n, 3] or NULL.
+ *   reuse_plan != 0: ws still holds the bins of this very position snapshot (left there by
+ *   tiga_apply_radius or tiga_radius_bin with the same n, r, box); otherwise it is rebuilt. */
+tiga_status tiga_apply_radius_backward(const float* pos, const float* feat, int64_t n, int32_t F,
+                                       float r, const tiga_box* box, const tiga_msg* msg,
+                                       const float* grad_out, float* grad_feat, float* grad_pos,
+                                       void* ws, size_t ws_bytes, int reuse_plan, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TIGA_H */

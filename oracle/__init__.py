@@ -66,7 +66,10 @@ def _i32(a):
 
 # ------------------------------------------------------------------------------ CSR
 def csr_forward(rowptr, col, x, w=None, reducer=SUM):
-    """Returns (y fp64 [n_dst,F], A fp64 [n_dst,F], arg int64 [n_dst,F] or None)."""
+    """Returns (y fp64 [n_dst,F], A fp64 [n_dst,F], arg int64 [n_dst,F] or None).
+
+    For the max reducer with fp32 / fp16 features each message is rounded once to fp32
+    before the comparison (the precision the messages exist in); fp64 features compare in fp64."""
     lib = _load()
     rowptr = _i64(rowptr); col = _i32(col)
     x, xdt = _field(x); w, wdt = _field(w)
@@ -76,7 +79,8 @@ def csr_forward(rowptr, col, x, w=None, reducer=SUM):
     A = np.empty((n, F), np.float64)
     arg = np.empty((n, F), np.int64) if reducer == MAX else None
     rc = lib.oracle_csr_forward(_p(rowptr), _p(col), ctypes.c_int64(n), _p(w), wdt, _p(x), xdt,
-                                ctypes.c_int(F), ctypes.c_int(reducer), _p(y), _p(A), _p(arg))
+                                ctypes.c_int(F), ctypes.c_int(reducer), ctypes.c_int(int(xdt != 2)),
+                                _p(y), _p(A), _p(arg))
     assert rc == 0
     return y, A, arg
 

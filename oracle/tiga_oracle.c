@@ -56,10 +56,14 @@ static inline double ld(const void* p, int dt, int64_t i) {
  * sum : y = sum of m in edge order, A = sum of |m|.
  * max : y = largest m, arg = lowest edge position attaining it (strict '>' while
  *       scanning in edge order); empty row -> y = 0, arg = -1.  A = |y|.
+ *       The selection is an integer decided by floating point, so it is taken in the
+ *       precision the messages exist in: with fp32 / fp16 inputs (decide_fp32 != 0) every
+ *       message is the fp64 product rounded once to fp32 before it is compared; two
+ *       products that round to the same fp32 value are a tie and the earlier edge wins.
  */
 int oracle_csr_forward(const int64_t* rowptr, const int32_t* col, int64_t n_dst,
                        const void* w, int w_dt, const void* x, int x_dt, int F, int reducer,
-                       double* y, double* A, int64_t* arg) {
+                       int decide_fp32, double* y, double* A, int64_t* arg) {
 #pragma omp parallel for schedule(dynamic, 256)
     for (int64_t i = 0; i < n_dst; ++i) {
         for (int f = 0; f < F; ++f) {
@@ -68,6 +72,7 @@ int oracle_csr_forward(const int64_t* rowptr, const int32_t* col, int64_t n_dst,
             for (int64_t e = rowptr[i]; e < rowptr[i + 1]; ++e) {
                 double we = w ? ld(w, w_dt, e) : 1.0;
                 double m = we * ld(x, x_dt, (int64_t)col[e] * F + f);
+                if (reducer == RED_MAX && decide_fp32) m = (double)(float)m;
                 if (reducer == RED_SUM) {
                     acc += m;
                     absacc += fabs(m);

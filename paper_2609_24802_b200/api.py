@@ -1,0 +1,295 @@
+"""ctypes binding of libtiga.so -- argument marshalling only.
+
+Every function has the name of the C entry point it calls (see ``include/tiga.h``) and takes
+torch CUDA tensors for the device arrays.  Nothing is computed here; when the library is
+missing the import fails, there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+__all__ = [
+    "TigaError", "load_library", "EXPORTS", "SUM", "MAX", "F32", "F16",
+    "MSG_COPY", "MSG_WEIGHTED", "MSG_GAUSS", "MSG_DIST", "MSG_LJ",
+    "CsrRelation", "tiga_status_string", "tiga_csr_workspace_bytes", "tiga_validate_csr",
+    "tiga_apply_csr", "tiga_apply_csr_backward", "tiga_csr_degree_histogram",
+    "tiga_radius_grid", "tiga_radius_workspace_bytes", "tiga_radius_bin",
+    "tiga_apply_radius", "tiga_apply_radius_backward", "launch_count",
+]
+
+SUM, MAX = 0, 1
+F32, F16 = 0, 1
+I32, I64 = 0, 1
+MSG_COPY, MSG_WEIGHTED, MSG_GAUSS, MSG_DIST, MSG_LJ = 0, 1, 2, 3, 4
+
+EXPORTS = [
+    "tiga_status_string", "tiga_csr_workspace_bytes", "tiga_validate_csr", "tiga_apply_csr",
+    "tiga_apply_csr_backward", "tiga_csr_degree_histogram", "tiga_radius_grid",
+    "tiga_radius_workspace_bytes", "tiga_radius_bin", "tiga_apply_radius",
+    "tiga_apply_radius_backward",
+]
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtiga.so")
+
+
+class TigaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {tiga_status_string(status)} (status {status})")
+
+
+class _Msg(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int32), ("p0", ctypes.c_float), ("p1", ctypes.c_float)]
+
+
+class _Csr(ctypes.Structure):
+    _fields_ = [("rowptr", ctypes.c_void_p), ("rowptr_type", ctypes.c_int32), ("col", ctypes.c_void_p),
+                ("n_dst", ctypes.c_int64), ("n_src", ctypes.c_int64), ("n_edges", ctypes.c_int64)]
+
+
+class _Box(ctypes.Structure):
+    _fields_ = [("len", ctypes.c_float * 3), ("periodic", ctypes.c_int32 * 3)]
+
+
+_lib = None
+_launches = 0     # kernels launched by the library through this binding (for benchmarks)
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libtiga.so; raises ImportError when it has not been built (no fallback)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with "
+                          "`python -m paper_2609_24802_b200.build` (nvcc, sm_100a)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, sz, f = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t, ctypes.c_float
+    lib.tiga_status_string.restype = ctypes.c_char_p
+    lib.tiga_status_string.argtypes = [ctypes.c_int]
+    lib.tiga_csr_workspace_bytes.restype = sz
+    lib.tiga_csr_workspace_bytes.argtypes = [ctypes.POINTER(_Csr), i32, ctypes.c_int, ctypes.c_int, ctypes.c_int]
+    lib.tiga_validate_csr.restype = ctypes.c_int
+    lib.tiga_validate_csr.argtypes = [ctypes.POINTER(_Csr), ctypes.c_int, vp, sz, vp]
+    lib.tiga_apply_csr.restype = ctypes.c_int
+    lib.tiga_apply_csr.argtypes = [ctypes.POINTER(_Csr), vp, ctypes.c_int, i32, vp, ctypes.POINTER(_Msg), ctypes.c_int,
+                                   vp, vp, vp, sz, vp]
+    lib.tiga_apply_csr_backward.restype = ctypes.c_int
+    lib.tiga_apply_csr_backward.argtypes = [ctypes.POINTER(_Csr), vp, ctypes.c_int, i32, vp, ctypes.POINTER(_Msg), ctypes.c_int,
+                                            vp, vp, vp, vp, vp, sz, vp]
+    lib.tiga_csr_degree_histogram.restype = ctypes.c_int
+    lib.tiga_csr_degree_histogram.argtypes = [ctypes.POINTER(_Csr), vp, i64, vp, vp]
+    lib.tiga_radius_grid.restype = ctypes.c_int
+    lib.tiga_radius_grid.argtypes = [i64, f, ctypes.POINTER(_Box), ctypes.POINTER(i32), ctypes.POINTER(f)]
+    lib.tiga_radius_workspace_bytes.restype = sz
+    lib.tiga_radius_workspace_bytes.argtypes = [i64, i32, f, ctypes.POINTER(_Box), ctypes.c_int]
+    lib.tiga_radius_bin.restype = ctypes.c_int
+    lib.tiga_radius_bin.argtypes = [vp, i64, f, ctypes.POINTER(_Box), vp, vp, vp, vp, sz, vp]
+    lib.tiga_apply_radius.restype = ctypes.c_int
+    lib.tiga_apply_radius.argtypes = [vp, vp, i64, i32, f, ctypes.POINTER(_Box), ctypes.POINTER(_Msg), vp, vp, vp, sz, vp]
+    lib.tiga_apply_radius_backward.restype = ctypes.c_int
+    lib.tiga_apply_radius_backward.argtypes = [vp, vp, i64, i32, f, ctypes.POINTER(_Box), ctypes.POINTER(_Msg), vp, vp, vp,
+                                               vp, sz, ctypes.c_int, vp]
+    _lib = lib
+    return lib
+
+
+load_library()      # fail at import time, loudly, when the CUDA library is not there
+
+
+def launch_count() -> int:
+    return _launches
+
+
+def _ptr(t):
+    if t is None:
+        return ctypes.c_void_p(0)
+    assert t.is_cuda and t.is_contiguous(), "device arrays must be contiguous CUDA tensors"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _ok(st, where):
+    if st != 0:
+        raise TigaError(st, where)
+
+
+def _ws(nbytes, like):
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=like.device)
+
+
+def _dt(t):
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.float16:
+        return F16
+    raise TypeError("features must be float32 or float16")
+
+
+def tiga_status_string(status: int) -> str:
+    return load_library().tiga_status_string(int(status)).decode()
+
+
+class CsrRelation:
+    """Host-side descriptor (the C struct ``tiga_csr``) of device CSR arrays."""
+
+    def __init__(self, rowptr: torch.Tensor, col: torch.Tensor, n_src: int):
+        assert rowptr.dtype in (torch.int32, torch.int64) and col.dtype == torch.int32
+        self.rowptr, self.col = rowptr, col
+        self.n_dst = rowptr.numel() - 1
+        self.n_src = int(n_src)
+        self.n_edges = col.numel()
+        self.c = _Csr(rowptr.data_ptr(), I32 if rowptr.dtype == torch.int32 else I64,
+                      col.data_ptr() if col.numel() else 0, self.n_dst, self.n_src, self.n_edges)
+
+    @property
+    def ref(self):
+        return ctypes.byref(self.c)
+
+
+def tiga_csr_workspace_bytes(g: CsrRelation, F: int, x_dtype: int = F32, reducer: int = SUM,
+                             backward: bool = False) -> int:
+    return int(load_library().tiga_csr_workspace_bytes(g.ref, F, x_dtype, reducer, int(backward)))
+
+
+def tiga_validate_csr(g: CsrRelation, level: int = 1, stream=None) -> None:
+    ws = _ws(256, g.rowptr)
+    _ok(load_library().tiga_validate_csr(g.ref, level, _ptr(ws), ws.numel(), _stream(stream)), "tiga_validate_csr")
+
+
+def tiga_apply_csr(g: CsrRelation, x, w=None, reducer: int = SUM, out=None, argmax=None, ws=None, stream=None):
+    """out[i,:] = reduce over the row's edges of w[e] * x[col[e],:].  Returns (out, argmax)."""
+    global _launches
+    F = x.shape[1]
+    if out is None:
+        out = torch.empty((g.n_dst, F), dtype=torch.float32, device=x.device)
+    if reducer == MAX and argmax is None:
+        argmax = torch.empty((g.n_dst, F), dtype=torch.int32, device=x.device)
+    if ws is None:
+        ws = _ws(tiga_csr_workspace_bytes(g, F, _dt(x), reducer, False), x)
+    msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)
+    _ok(load_library().tiga_apply_csr(g.ref, _ptr(x), _dt(x), F, _ptr(w), ctypes.byref(msg), reducer, _ptr(out),
+                                      _ptr(argmax), _ptr(ws), ws.numel(), _stream(stream)), "tiga_apply_csr")
+    _launches += 2
+    return out, argmax
+
+
+def tiga_apply_csr_backward(g: CsrRelation, x, w, grad_out, reducer: int = SUM, argmax=None,
+                            grad_x=None, grad_w=None, want_x=True, want_w=True, ws=None, stream=None):
+    """Returns (grad_x, grad_w); either is None when not requested."""
+    global _launches
+    F = x.shape[1]
+    if want_x and grad_x is None:
+        grad_x = torch.empty((g.n_src, F), dtype=torch.float32, device=x.device)
+    if want_w and grad_w is None:
+        grad_w = torch.empty((g.n_edges,), dtype=torch.float32, device=x.device)
+    if ws is None:
+        ws = _ws(tiga_csr_workspace_bytes(g, F, _dt(x), reducer, True), x)
+    msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)
+    _ok(load_library().tiga_apply_csr_backward(g.ref, _ptr(x), _dt(x), F, _ptr(w), ctypes.byref(msg), reducer, _ptr(grad_out),
+                                               _ptr(argmax), _ptr(grad_x), _ptr(grad_w), _ptr(ws), ws.numel(),
+                                               _stream(stream)), "tiga_apply_csr_backward")
+    _launches += 1
+    return grad_x, grad_w
+
+
+def tiga_csr_degree_histogram(g: CsrRelation, nbins: int = 4096, stream=None):
+    """Returns (hist int64[nbins], max_degree int64[1]) as device tensors."""
+    global _launches
+    hist = torch.empty(nbins, dtype=torch.int64, device=g.rowptr.device)
+    mx = torch.empty(1, dtype=torch.int64, device=g.rowptr.device)
+    _ok(load_library().tiga_csr_degree_histogram(g.ref, _ptr(hist), nbins, _ptr(mx), _stream(stream)),
+        "tiga_csr_degree_histogram")
+    _launches += 1
+    return hist, mx
+
+
+def _box(box, periodic):
+    b = _Box()
+    for d in range(3):
+        b.len[d] = float(box[d])
+        b.periodic[d] = int(periodic[d])
+    return b
+
+
+def tiga_radius_grid(n: int, r: float, box, periodic):
+    """Returns (ncell list[3], invh list[3]) -- host only."""
+    b = _box(box, periodic)
+    nc = (ctypes.c_int32 * 3)()
+    ih = (ctypes.c_float * 3)()
+    _ok(load_library().tiga_radius_grid(n, float(r), ctypes.byref(b), nc, ih), "tiga_radius_grid")
+    return list(nc), list(ih)
+
+
+def tiga_radius_workspace_bytes(n: int, F: int, r: float, box, periodic, backward: bool = False) -> int:
+    b = _box(box, periodic)
+    return int(load_library().tiga_radius_workspace_bytes(n, F, float(r), ctypes.byref(b), int(backward)))
+
+
+def tiga_radius_bin(pos, r: float, box, periodic, ws=None, stream=None):
+    """Returns dict(cell, cell_start, order, ncell, ws)."""
+    global _launches
+    n = pos.shape[0]
+    b = _box(box, periodic)
+    ncell, _ = tiga_radius_grid(n, r, box, periodic)
+    nc = ncell[0] * ncell[1] * ncell[2]
+    cell = torch.empty(n, dtype=torch.int32, device=pos.device)
+    start = torch.empty(nc + 1, dtype=torch.int32, device=pos.device)
+    order = torch.empty(n, dtype=torch.int32, device=pos.device)
+    if ws is None:
+        ws = _ws(tiga_radius_workspace_bytes(n, 0, r, box, periodic), pos)
+    _ok(load_library().tiga_radius_bin(_ptr(pos), n, float(r), ctypes.byref(b), _ptr(cell), _ptr(start),
+                                       _ptr(order), _ptr(ws), ws.numel(), _stream(stream)), "tiga_radius_bin")
+    _launches += 6
+    return dict(cell=cell, cell_start=start, order=order, ncell=ncell, ws=ws)
+
+
+def tiga_apply_radius(pos, feat, r: float, box, periodic, kind: int = MSG_GAUSS, p0: float = 1.0,
+                      p1: float = 1.0, out=None, count=None, want_count=False, ws=None, stream=None):
+    """Fused bin + traverse + message + sum.  Returns (out, count, ws)."""
+    global _launches
+    n = pos.shape[0]
+    F = 4 if kind == MSG_LJ else feat.shape[1]
+    b = _box(box, periodic)
+    if out is None:
+        out = torch.empty((n, F), dtype=torch.float32, device=pos.device)
+    if want_count and count is None:
+        count = torch.empty(n, dtype=torch.int32, device=pos.device)
+    if ws is None:
+        ws = _ws(tiga_radius_workspace_bytes(n, F, r, box, periodic), pos)
+    _ok(load_library().tiga_apply_radius(_ptr(pos), _ptr(feat), n, F, float(r), ctypes.byref(b),
+                                         ctypes.byref(_Msg(kind, float(p0), float(p1))), _ptr(out), _ptr(count), _ptr(ws),
+                                         ws.numel(), _stream(stream)), "tiga_apply_radius")
+    _launches += 7
+    return out, count, ws
+
+
+def tiga_apply_radius_backward(pos, feat, grad_out, r: float, box, periodic, sigma: float, ws=None,
+                               reuse_plan=False, grad_feat=None, grad_pos=None, want_feat=True, want_pos=True,
+                               stream=None):
+    """Reverse mode of the Gaussian message.  Returns (grad_feat, grad_pos)."""
+    global _launches
+    n, F = feat.shape
+    b = _box(box, periodic)
+    if want_feat and grad_feat is None:
+        grad_feat = torch.empty((n, F), dtype=torch.float32, device=pos.device)
+    if want_pos and grad_pos is None:
+        grad_pos = torch.empty((n, 3), dtype=torch.float32, device=pos.device)
+    if ws is None:
+        assert not reuse_plan
+        ws = _ws(tiga_radius_workspace_bytes(n, F, r, box, periodic, True), pos)
+    _ok(load_library().tiga_apply_radius_backward(_ptr(pos), _ptr(feat), n, F, float(r), ctypes.byref(b),
+                                                  ctypes.byref(_Msg(MSG_GAUSS, float(sigma), 0.0)), _ptr(grad_out),
+                                                  _ptr(grad_feat), _ptr(grad_pos), _ptr(ws), ws.numel(),
+                                                  int(bool(reuse_plan)), _stream(stream)),
+        "tiga_apply_radius_backward")
+    _launches += 1 if reuse_plan else 7
+    return grad_feat, grad_pos

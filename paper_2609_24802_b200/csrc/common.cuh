@@ -1,0 +1,43 @@
+// Shared host/device helpers of libtiga (CUDA side only; the CPU oracle shares nothing with this).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include "tiga.h"
+
+namespace tiga {
+
+#define TIGA_CUDA_TRY(expr)                                   \
+    do {                                                      \
+        cudaError_t _e = (expr);                              \
+        if (_e != cudaSuccess) return TIGA_ERR_CUDA;          \
+    } while (0)
+
+// Peek (do not clear sticky errors of other users of the context) after a launch.
+static inline tiga_status launch_status() {
+    return cudaPeekAtLastError() == cudaSuccess ? TIGA_OK : TIGA_ERR_CUDA;
+}
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// A bump allocator over the caller's workspace (256-byte granules).
+struct Carver {
+    char* base;
+    size_t off;
+    explicit Carver(void* p) : base(static_cast<char*>(p)), off(0) {}
+    template <typename T>
+    T* take(size_t count) {
+        T* r = reinterpret_cast<T*>(base + off);
+        off += align_up(count * sizeof(T), 256);
+        return r;
+    }
+};
+
+// streaming (read-once) loads and write-once stores keep L2 for the gathered rows
+template <typename T>
+__device__ __forceinline__ T ld_stream(const T* p) { return __ldcs(p); }
+template <typename T>
+__device__ __forceinline__ void st_stream(T* p, T v) { __stcs(p, v); }
+
+}  // namespace tiga

@@ -1,0 +1,762 @@
+// Stored-relation gf.apply for sm_100a: gather / message / reduce over a destination-
+// oriented CSR (paper Sections 3.1, 4.2, 4.3) and its reverse mode (Section 5).
+//
+// Schedule (ours, not the paper's bounded-ragged Triton tile of Section 4.4):
+//   * The merged sequence "row ends + edges" (N + E items) is cut into equal tiles, one CTA
+//     per tile, so neither a 69k-edge row nor a run of a million empty rows unbalances a CTA
+//     (Section 4.4: "a high-degree split requires explicit partial states and a legal merge").
+//   * A CTA stages its slice of rowptr, col and w in shared memory with coalesced streaming
+//     loads, then splits its edges evenly over "workers" of G lanes.  A worker walks its edge
+//     span in order; each lane owns 16 bytes of the feature row, so one gathered source row
+//     is one fully coalesced 128-bit-per-lane request.  Several gathers are kept in flight
+//     per lane.  The reducer state lives in registers.
+//   * Rows wholly inside one worker's span are stored straight to global memory.  Partial
+//     states (head / tail of a span) go to shared memory and are merged in edge order; the
+//     CTA's trailing unfinished row becomes one carry-out in the workspace, which a small
+//     fix-up kernel folds into the row, again in edge order.  No atomics in the forward, so
+//     results are reproducible.
+#include "common.cuh"
+
+namespace tiga {
+
+constexpr int CSR_THREADS = 256;
+constexpr int CSR_TILE = 2048;     // merge-path items per CTA
+
+template <typename XT> struct XTraits;
+template <> struct XTraits<float> {
+    static constexpr int VW = 4;   // floats per 16-byte vector
+    __device__ static __forceinline__ void unpack(const uint4& v, float* f) {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    }
+};
+template <> struct XTraits<__half> {
+    static constexpr int VW = 8;
+    __device__ static __forceinline__ void unpack(const uint4& v, float* f) {
+        const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            float2 t = __half22float2(h[k]);
+            f[2 * k] = t.x; f[2 * k + 1] = t.y;
+        }
+    }
+};
+
+struct CsrParams {
+    const void* rowptr;
+    const int32_t* col;
+    const float* w;          // may be null (unit weights)
+    const void* x;
+    float* out;
+    int32_t* arg;
+    long long n_dst, n_edges;
+    int F;                   // features per row
+    int nvec;                // 16-byte vectors per feature row
+    // workspace
+    int32_t* carry_row;      // [ntiles]  row of the tile's trailing partial state, or -1
+    float* carry_val;        // [ntiles, F]
+    int32_t* carry_arg;      // [ntiles, F] (max only)
+    long long ntiles;
+    // backward
+    const float* gy;
+    float* gx;
+    float* gw;
+};
+
+// Number of rows whose row-end item lies before merge diagonal d:
+//   #{ i : rowptr[i+1] + i + 1 <= d }   (strictly increasing in i -> 32-ary search by one warp)
+template <typename IT>
+__device__ long long rows_done(const IT* __restrict__ rowptr, long long n, long long d) {
+    long long lo = 0, hi = n;
+    const int lane = threadIdx.x & 31;
+    while (lo < hi) {
+        const long long step = (hi - lo + 31) / 32;
+        const long long q = lo + (long long)(lane + 1) * step;
+        bool pred = false;
+        if (q <= hi) pred = ((long long)rowptr[q] + q <= d);
+        const int c = __popc(__ballot_sync(0xffffffffu, pred));
+        const long long nhi = lo + (long long)(c + 1) * step - 1;
+        lo = lo + (long long)c * step;
+        hi = nhi < hi ? nhi : hi;
+        if (lo > hi) lo = hi;
+    }
+    return lo;
+}
+
+struct Tile {
+    long long i0, e0;   // first row / first edge of the tile
+    int nfin;           // rows whose row-end item is in the tile: [i0, i0 + nfin)
+    int nrows;          // rows staged: nfin (+1 when a trailing partial row exists)
+    int ne;             // edges in the tile
+};
+
+// Stage the tile: s_ptr[k] = clamp(rowptr[i0+k] - e0, -1, ne+1) for k = 0..nrows, col and w.
+template <typename IT>
+__device__ Tile stage_tile(const CsrParams& p, int* s_ptr, int* s_col, float* s_w, long long* s_coord) {
+    const IT* rowptr = static_cast<const IT*>(p.rowptr);
+    const long long total = p.n_dst + p.n_edges;
+    const long long d0 = (long long)blockIdx.x * CSR_TILE;
+    const long long d1 = (d0 + CSR_TILE < total) ? d0 + CSR_TILE : total;
+    const int warp = threadIdx.x >> 5;
+    if (warp == 0) {
+        long long i = rows_done(rowptr, p.n_dst, d0);
+        if ((threadIdx.x & 31) == 0) s_coord[0] = i;
+    } else if (warp == 1) {
+        long long i = rows_done(rowptr, p.n_dst, d1);
+        if ((threadIdx.x & 31) == 0) s_coord[1] = i;
+    }
+    __syncthreads();
+    Tile t;
+    t.i0 = s_coord[0];
+    const long long i1 = s_coord[1];
+    t.e0 = d0 - t.i0;
+    const long long e1 = d1 - i1;
+    t.ne = (int)(e1 - t.e0);
+    t.nfin = (int)(i1 - t.i0);
+    t.nrows = t.nfin + (i1 < p.n_dst ? 1 : 0);
+    for (int k = threadIdx.x; k <= t.nrows; k += CSR_THREADS) {
+        long long v = (long long)rowptr[t.i0 + k] - t.e0;
+        if (v < -1) v = -1;
+        if (v > t.ne + 1) v = t.ne + 1;
+        // a trailing partial row never ends inside this tile, whatever rowptr says
+        if (k == t.nrows && t.nrows > t.nfin) v = t.ne + 1;
+        s_ptr[k] = (int)v;
+    }
+    for (int k = threadIdx.x; k < t.ne; k += CSR_THREADS) {
+        s_col[k] = ld_stream(p.col + t.e0 + k);
+        if (p.w) s_w[k] = ld_stream(p.w + t.e0 + k);
+    }
+    __syncthreads();
+    return t;
+}
+
+// last k in [0, nrows] with s_ptr[k] <= a   (s_ptr[0] <= 0 <= a always)
+__device__ __forceinline__ int row_of_edge(const int* s_ptr, int nrows, int a) {
+    int lo = 0, hi = nrows;          // invariant: s_ptr[lo] <= a
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (s_ptr[mid] <= a) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// --------------------------------------------------------------------------------------------
+// Forward.  G lanes per worker, VPL 16-byte vectors per lane, RED = 0 sum / 1 max.
+// --------------------------------------------------------------------------------------------
+template <int RED, int VPL, int VW>
+struct State {
+    float v[VPL][VW];
+    int a[RED ? VPL : 1][RED ? VW : 1];
+    __device__ __forceinline__ void reset() {
+#pragma unroll
+        for (int i = 0; i < VPL; ++i)
+#pragma unroll
+            for (int k = 0; k < VW; ++k) {
+                v[i][k] = 0.f;
+                if constexpr (RED != 0) a[i][k] = -1;
+            }
+    }
+    // fold a message that comes later in edge order
+    __device__ __forceinline__ void message(int i, int k, float wgt, float xv, int e) {
+        if constexpr (RED == 0) {
+            v[i][k] = fmaf(wgt, xv, v[i][k]);
+        } else {
+            const float m = __fmul_rn(wgt, xv);        // one rounding, never contracted
+            if (a[i][k] < 0 || m > v[i][k]) { v[i][k] = m; a[i][k] = e; }
+        }
+    }
+    // fold a partial state that comes later in edge order
+    __device__ __forceinline__ void merge(int i, int k, float ov, int oa) {
+        if constexpr (RED == 0) {
+            v[i][k] += ov;
+        } else {
+            if (oa >= 0 && (a[i][k] < 0 || ov > v[i][k])) { v[i][k] = ov; a[i][k] = oa; }
+        }
+    }
+};
+
+template <typename XT, int G, int VPL, int RED, typename IT>
+__global__ void __launch_bounds__(CSR_THREADS) csr_forward_kernel(const CsrParams p) {
+    constexpr int VW = XTraits<XT>::VW;
+    constexpr int NW = CSR_THREADS / G;          // workers per CTA
+    constexpr int LV = G * VPL * VW;             // floats of one partial state
+    constexpr int U = (VPL == 1) ? 4 : (VPL == 2 ? 2 : 1);   // gathers in flight per lane
+
+    __shared__ int s_ptr[CSR_TILE + 2];
+    __shared__ int s_col[CSR_TILE];
+    __shared__ float s_w[CSR_TILE];
+    __shared__ long long s_coord[2];
+    __shared__ int s_tag[2 * NW];                // local row of head (even) / tail (odd) partial, -1 = none
+    __shared__ unsigned char s_first[NW];        // tail partial starts its chain
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    float* s_pv = reinterpret_cast<float*>(s_dyn);              // [2*NW][LV]
+    int* s_pa = reinterpret_cast<int*>(s_pv + 2 * NW * LV);     // [2*NW][LV] (max only)
+
+    const Tile t = stage_tile<IT>(p, s_ptr, s_col, s_w, s_coord);
+    const int wk = threadIdx.x / G;
+    const int ln = threadIdx.x % G;
+    const bool has_w = p.w != nullptr;
+    const uint4* __restrict__ xbase = static_cast<const uint4*>(p.x);
+    const long long e0 = t.e0;
+
+    bool act[VPL];
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) act[i] = (i * G + ln) < p.nvec;
+
+    auto store_row = [&](long long row, const State<RED, VPL, VW>& s) {
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) {
+            if (!act[i]) continue;
+            float* o = p.out + row * p.F + (size_t)(i * G + ln) * VW;
+#pragma unroll
+            for (int k = 0; k < VW; k += 4)
+                st_stream(reinterpret_cast<float4*>(o + k), make_float4(s.v[i][k], s.v[i][k + 1], s.v[i][k + 2], s.v[i][k + 3]));
+            if constexpr (RED != 0) {
+                int* ao = p.arg + row * p.F + (size_t)(i * G + ln) * VW;
+#pragma unroll
+                for (int k = 0; k < VW; k += 4)
+                    st_stream(reinterpret_cast<int4*>(ao + k), make_int4(s.a[i][k], s.a[i][k + 1], s.a[i][k + 2], s.a[i][k + 3]));
+            }
+        }
+    };
+    auto store_partial = [&](int entry, const State<RED, VPL, VW>& s) {
+#pragma unroll
+        for (int i = 0; i < VPL; ++i)
+#pragma unroll
+            for (int k = 0; k < VW; ++k) {
+                s_pv[entry * LV + (i * G + ln) * VW + k] = s.v[i][k];
+                if constexpr (RED != 0) s_pa[entry * LV + (i * G + ln) * VW + k] = s.a[i][k];
+            }
+    };
+    auto merge_partial = [&](int entry, State<RED, VPL, VW>& s) {
+#pragma unroll
+        for (int i = 0; i < VPL; ++i)
+#pragma unroll
+            for (int k = 0; k < VW; ++k)
+                s.merge(i, k, s_pv[entry * LV + (i * G + ln) * VW + k],
+                        RED ? s_pa[entry * LV + (i * G + ln) * VW + k] : 0);
+    };
+
+    // rows that end in this tile without an edge in it: the reducer identity (finalised to 0)
+    {
+        State<RED, VPL, VW> idn;
+        idn.reset();
+        for (int k = wk; k < t.nfin; k += NW) {
+            const int ls = s_ptr[k] < 0 ? 0 : s_ptr[k];
+            if (s_ptr[k + 1] == ls) store_row(t.i0 + k, idn);
+        }
+    }
+
+    if (ln == 0) { s_tag[2 * wk] = -1; s_tag[2 * wk + 1] = -1; s_first[wk] = 0; }
+    if (threadIdx.x == 0) p.carry_row[blockIdx.x] = -1;
+
+    const int chunk = (t.ne + NW - 1) / NW;
+    const int a = wk * chunk;
+    const int b = (a + chunk < t.ne) ? a + chunk : t.ne;
+
+    State<RED, VPL, VW> st;
+    st.reset();
+    int r = 0;
+    bool tail_valid = false, tail_first = false;
+    if (a < b) {
+        r = row_of_edge(s_ptr, t.nrows, a);
+        int cur_end = s_ptr[r + 1];
+        bool head = (s_ptr[r] < 0 ? 0 : s_ptr[r]) < a;   // the row began in an earlier span of this tile
+        for (int e = a; e < b; e += U) {
+            uint4 xv[U][VPL];
+            float wv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int ee = (e + u < b) ? e + u : b - 1;
+                const long long c = s_col[ee];
+                wv[u] = has_w ? s_w[ee] : 1.f;
+                const uint4* src = xbase + c * p.nvec;
+#pragma unroll
+                for (int i = 0; i < VPL; ++i)
+                    xv[u][i] = act[i] ? __ldg(src + i * G + ln) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (e + u < b) {
+                    if (e + u >= cur_end) {
+                        // the current row is complete inside this span
+                        if (head) { store_partial(2 * wk, st); if (ln == 0) s_tag[2 * wk] = r; }
+                        else store_row(t.i0 + r, st);
+                        st.reset();
+                        head = false;
+                        do { ++r; cur_end = s_ptr[r + 1]; } while (e + u >= cur_end);   // skip empty rows
+                    }
+                    float xf[VW];
+#pragma unroll
+                    for (int i = 0; i < VPL; ++i) {
+                        XTraits<XT>::unpack(xv[u][i], xf);
+#pragma unroll
+                        for (int k = 0; k < VW; ++k) st.message(i, k, wv[u], xf[k], (int)(e0 + e + u));
+                    }
+                }
+            }
+        }
+        if (cur_end <= b) {
+            if (head) { store_partial(2 * wk, st); if (ln == 0) s_tag[2 * wk] = r; }
+            else store_row(t.i0 + r, st);
+        } else {
+            // the row continues past this span: tail partial
+            tail_valid = true;
+            tail_first = !head;
+            store_partial(2 * wk + 1, st);
+            if (ln == 0) { s_tag[2 * wk + 1] = r; s_first[wk] = tail_first ? 1 : 0; }
+        }
+    }
+    __syncthreads();
+
+    // merge chains of partial states in edge order; the worker that opens a chain owns it
+    if (tail_valid && tail_first) {
+        bool finished = false;
+        for (int w2 = wk + 1; w2 < NW; ++w2) {
+            if (s_tag[2 * w2] == r) { merge_partial(2 * w2, st); finished = true; break; }
+            if (s_tag[2 * w2 + 1] == r && !s_first[w2]) merge_partial(2 * w2 + 1, st);
+            else break;
+        }
+        if (finished) {
+            store_row(t.i0 + r, st);
+        } else {
+            // trailing unfinished row of the tile -> carry-out
+            if (ln == 0) p.carry_row[blockIdx.x] = (int32_t)(t.i0 + r);
+#pragma unroll
+            for (int i = 0; i < VPL; ++i) {
+                if (!act[i]) continue;
+                const size_t o = (size_t)blockIdx.x * p.F + (size_t)(i * G + ln) * VW;
+#pragma unroll
+                for (int k = 0; k < VW; ++k) {
+                    p.carry_val[o + k] = st.v[i][k];
+                    if constexpr (RED != 0) p.carry_arg[o + k] = st.a[i][k];
+                }
+            }
+        }
+    }
+}
+
+// Fold the carry-outs of consecutive tiles that belong to one row into that row, in edge
+// order.  One thread per (tile, feature); only the first tile of a run does the work.
+template <int RED>
+__global__ void csr_fixup_kernel(const CsrParams p) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long tile = idx / p.F;
+    const int f = (int)(idx % p.F);
+    if (tile >= p.ntiles) return;
+    const int row = p.carry_row[tile];
+    if (row < 0) return;
+    if (tile > 0 && p.carry_row[tile - 1] == row) return;
+    float v = p.carry_val[tile * p.F + f];
+    int a = RED ? p.carry_arg[tile * p.F + f] : 0;
+    for (long long u = tile + 1; u < p.ntiles && p.carry_row[u] == row; ++u) {
+        const float ov = p.carry_val[u * p.F + f];
+        if (RED == 0) v += ov;
+        else {
+            const int oa = p.carry_arg[u * p.F + f];
+            if (oa >= 0 && (a < 0 || ov > v)) { v = ov; a = oa; }
+        }
+    }
+    const size_t o = (size_t)row * p.F + f;
+    if (RED == 0) {
+        p.out[o] = v + p.out[o];
+    } else {
+        const float ov = p.out[o];
+        const int oa = p.arg[o];
+        if (oa >= 0 && (a < 0 || ov > v)) { v = ov; a = oa; }
+        p.out[o] = v;
+        p.arg[o] = a;
+    }
+}
+
+// --------------------------------------------------------------------------------------------
+// Backward, sum reducer (Section 5).  Same tiles and workers; every edge is independent:
+//   gw[e] = x[col[e],:] . gy[row,:]            (edge gradients retain edge identity)
+//   gx[col[e],:] += w[e] * gy[row,:]           (reverse incidence: vector atomics)
+// --------------------------------------------------------------------------------------------
+template <int G, int VPL, typename IT>
+__global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const CsrParams p) {
+    constexpr int VW = 4;
+    constexpr int NW = CSR_THREADS / G;
+    constexpr int U = (VPL == 1) ? 4 : (VPL == 2 ? 2 : 1);
+    __shared__ int s_ptr[CSR_TILE + 2];
+    __shared__ int s_col[CSR_TILE];
+    __shared__ float s_w[CSR_TILE];
+    __shared__ float s_gw[CSR_TILE];
+    __shared__ long long s_coord[2];
+
+    const Tile t = stage_tile<IT>(p, s_ptr, s_col, s_w, s_coord);
+    const int wk = threadIdx.x / G;
+    const int ln = threadIdx.x % G;
+    const bool has_w = p.w != nullptr;
+    // lanes of one worker stay converged; workers of one warp do not
+    const unsigned wmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) & ~(G - 1)));
+    const float4* __restrict__ xbase = static_cast<const float4*>(p.x);
+    const float4* __restrict__ gybase = reinterpret_cast<const float4*>(p.gy);
+    float4* gxbase = reinterpret_cast<float4*>(p.gx);
+
+    bool act[VPL];
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) act[i] = (i * G + ln) < p.nvec;
+
+    const int chunk = (t.ne + NW - 1) / NW;
+    const int a = wk * chunk;
+    const int b = (a + chunk < t.ne) ? a + chunk : t.ne;
+    if (a < b) {
+        int r = row_of_edge(s_ptr, t.nrows, a);
+        int cur_end = s_ptr[r + 1];
+        float4 g[VPL];
+        auto load_gy = [&](int rr) {
+#pragma unroll
+            for (int i = 0; i < VPL; ++i)
+                g[i] = act[i] ? __ldg(gybase + (t.i0 + rr) * p.nvec + i * G + ln) : make_float4(0.f, 0.f, 0.f, 0.f);
+        };
+        load_gy(r);
+        for (int e = a; e < b; e += U) {
+            float4 xv[U][VPL];
+            int cv[U];
+            float wv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int ee = (e + u < b) ? e + u : b - 1;
+                cv[u] = s_col[ee];
+                wv[u] = has_w ? s_w[ee] : 1.f;
+                if (p.gw) {
+#pragma unroll
+                    for (int i = 0; i < VPL; ++i)
+                        xv[u][i] = act[i] ? __ldg(xbase + (long long)cv[u] * p.nvec + i * G + ln) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (e + u < b) {           // uniform inside a worker
+                    if (e + u >= cur_end) {
+                        do { ++r; cur_end = s_ptr[r + 1]; } while (e + u >= cur_end);
+                        load_gy(r);
+                    }
+                    if (p.gw) {
+                        float d = 0.f;
+#pragma unroll
+                        for (int i = 0; i < VPL; ++i) {
+                            d = fmaf(xv[u][i].x, g[i].x, d); d = fmaf(xv[u][i].y, g[i].y, d);
+                            d = fmaf(xv[u][i].z, g[i].z, d); d = fmaf(xv[u][i].w, g[i].w, d);
+                        }
+#pragma unroll
+                        for (int o = G / 2; o > 0; o >>= 1) d += __shfl_xor_sync(wmask, d, o, G);
+                        if (ln == 0) s_gw[e + u] = d;
+                    }
+                    if (p.gx) {
+#pragma unroll
+                        for (int i = 0; i < VPL; ++i)
+                            if (act[i])
+                                atomicAdd(gxbase + (long long)cv[u] * p.nvec + i * G + ln,
+                                          make_float4(wv[u] * g[i].x, wv[u] * g[i].y, wv[u] * g[i].z, wv[u] * g[i].w));
+                    }
+                }
+            }
+        }
+    }
+    if (p.gw) {
+        __syncthreads();
+        for (int k = threadIdx.x; k < t.ne; k += CSR_THREADS) st_stream(p.gw + t.e0 + k, s_gw[k]);
+    }
+}
+
+// Backward, max reducer: the cotangent of (i, f) goes through the selected edge only.
+__global__ void csr_backward_max_kernel(const CsrParams p) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= p.n_dst * p.F) return;
+    const int e = p.arg[idx];
+    if (e < 0) return;
+    const int f = (int)(idx % p.F);
+    const long long j = p.col[e];
+    const float g = p.gy[idx];
+    if (p.gw) atomicAdd(p.gw + e, static_cast<const float*>(p.x)[j * p.F + f] * g);
+    if (p.gx) atomicAdd(p.gx + j * p.F + f, (p.w ? p.w[e] : 1.f) * g);
+}
+
+// --------------------------------------------------------------------------------------------
+// Degree histogram and validation
+// --------------------------------------------------------------------------------------------
+template <typename IT>
+__global__ void degree_hist_kernel(const IT* __restrict__ rowptr, long long n, int nbins,
+                                   unsigned long long* hist, unsigned long long* maxdeg) {
+    extern __shared__ unsigned int s_hist[];
+    for (int k = threadIdx.x; k < nbins; k += blockDim.x) s_hist[k] = 0;
+    __syncthreads();
+    long long mx = 0;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const long long d = (long long)rowptr[i + 1] - (long long)rowptr[i];
+        mx = d > mx ? d : mx;
+        atomicAdd(&s_hist[d < nbins - 1 ? (int)d : nbins - 1], 1u);
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const long long other = __shfl_xor_sync(0xffffffffu, mx, o);
+        mx = other > mx ? other : mx;
+    }
+    if ((threadIdx.x & 31) == 0 && mx > 0) atomicMax(maxdeg, (unsigned long long)mx);
+    __syncthreads();
+    for (int k = threadIdx.x; k < nbins; k += blockDim.x)
+        if (s_hist[k]) atomicAdd(hist + k, (unsigned long long)s_hist[k]);
+}
+
+template <typename IT>
+__global__ void validate_kernel(const IT* __restrict__ rowptr, const int32_t* __restrict__ col,
+                                long long n_dst, long long n_src, long long n_edges, int* flags) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const long long t0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    int bad = 0;
+    if (t0 == 0) {
+        if ((long long)rowptr[0] != 0) bad |= 1;
+        if ((long long)rowptr[n_dst] != n_edges) bad |= 2;
+    }
+    for (long long i = t0; i < n_dst; i += stride)
+        if ((long long)rowptr[i + 1] < (long long)rowptr[i]) bad |= 4;
+    for (long long e = t0; e < n_edges; e += stride) {
+        const int c = col[e];
+        if (c < 0 || (long long)c >= n_src) bad |= 8;
+    }
+    if (bad) atomicOr(flags, bad);
+}
+
+// --------------------------------------------------------------------------------------------
+// Host side
+// --------------------------------------------------------------------------------------------
+static bool pick_shape(int nvec, int* G, int* VPL) {
+    if (nvec <= 0) return false;
+    if (nvec <= 32) {
+        int g = 1;
+        while (g < nvec) g <<= 1;
+        *G = g; *VPL = 1;
+        return true;
+    }
+    *G = 32;
+    const int v = (nvec + 31) / 32;
+    if (v <= 2) *VPL = 2; else if (v <= 4) *VPL = 4; else return false;
+    return true;
+}
+
+static long long num_tiles(const tiga_csr* g) { return (g->n_dst + g->n_edges + CSR_TILE - 1) / CSR_TILE; }
+
+template <typename XT, int G, int VPL, int RED, typename IT>
+static tiga_status launch_fwd_t(const CsrParams& p, cudaStream_t s) {
+    constexpr int VW = XTraits<XT>::VW;
+    constexpr int NW = CSR_THREADS / G;
+    const size_t dyn = (size_t)2 * NW * G * VPL * VW * sizeof(float) * (RED ? 2 : 1);
+    auto kern = csr_forward_kernel<XT, G, VPL, RED, IT>;
+    if (dyn > 16 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
+    kern<<<(unsigned)p.ntiles, CSR_THREADS, dyn, s>>>(p);
+    return launch_status();
+}
+
+template <typename XT, int RED, typename IT>
+static tiga_status launch_fwd_g(const CsrParams& p, int G, int VPL, cudaStream_t s) {
+    switch (G) {
+        case 1: return launch_fwd_t<XT, 1, 1, RED, IT>(p, s);
+        case 2: return launch_fwd_t<XT, 2, 1, RED, IT>(p, s);
+        case 4: return launch_fwd_t<XT, 4, 1, RED, IT>(p, s);
+        case 8: return launch_fwd_t<XT, 8, 1, RED, IT>(p, s);
+        case 16: return launch_fwd_t<XT, 16, 1, RED, IT>(p, s);
+        default:
+            if (VPL == 1) return launch_fwd_t<XT, 32, 1, RED, IT>(p, s);
+            if (VPL == 2) return launch_fwd_t<XT, 32, 2, RED, IT>(p, s);
+            return launch_fwd_t<XT, 32, 4, RED, IT>(p, s);
+    }
+}
+
+template <typename IT>
+static tiga_status launch_bwd_g(const CsrParams& p, int G, int VPL, cudaStream_t s) {
+#define TIGA_BWD(GG, VV) csr_backward_sum_kernel<GG, VV, IT><<<(unsigned)p.ntiles, CSR_THREADS, 0, s>>>(p); break
+    switch (G) {
+        case 1: TIGA_BWD(1, 1);
+        case 2: TIGA_BWD(2, 1);
+        case 4: TIGA_BWD(4, 1);
+        case 8: TIGA_BWD(8, 1);
+        case 16: TIGA_BWD(16, 1);
+        default:
+            if (VPL == 1) { TIGA_BWD(32, 1); }
+            if (VPL == 2) { TIGA_BWD(32, 2); }
+            TIGA_BWD(32, 4);
+    }
+#undef TIGA_BWD
+    return launch_status();
+}
+
+static tiga_status check_csr(const tiga_csr* g) {
+    if (!g) return TIGA_ERR_INVALID_ARG;
+    if (g->n_dst < 0 || g->n_src < 0 || g->n_edges < 0) return TIGA_ERR_INVALID_ARG;
+    if (g->rowptr_type != TIGA_I32 && g->rowptr_type != TIGA_I64) return TIGA_ERR_INVALID_ARG;
+    if (!g->rowptr || !aligned16(g->rowptr)) return TIGA_ERR_INVALID_ARG;
+    if (g->n_edges > 0 && (!g->col || !aligned16(g->col))) return TIGA_ERR_INVALID_ARG;
+    if (g->rowptr_type == TIGA_I32 && g->n_edges > 0x7fffffffLL) return TIGA_ERR_INVALID_ARG;
+    if (g->n_dst > 0x7fffffffLL || g->n_src > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;
+    if (num_tiles(g) > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;
+    return TIGA_OK;
+}
+
+static tiga_status check_features(int32_t F, tiga_dtype dt, int* nvec, int* G, int* VPL) {
+    if (F <= 0) return TIGA_ERR_INVALID_ARG;
+    if (dt != TIGA_F32 && dt != TIGA_F16) return TIGA_ERR_INVALID_ARG;
+    const int vw = dt == TIGA_F32 ? 4 : 8;
+    if (F % vw) return TIGA_ERR_UNSUPPORTED;
+    *nvec = F / vw;
+    return pick_shape(*nvec, G, VPL) ? TIGA_OK : TIGA_ERR_UNSUPPORTED;
+}
+
+}  // namespace tiga
+
+using namespace tiga;
+
+extern "C" size_t tiga_csr_workspace_bytes(const tiga_csr* g, int32_t F, tiga_dtype, tiga_reducer reducer, int backward) {
+    if (!g || F <= 0 || g->n_dst < 0 || g->n_edges < 0) return 0;
+    if (backward) return 256;
+    const size_t nt = (size_t)num_tiles(g) + 1;
+    size_t b = align_up(nt * sizeof(int32_t), 256) + align_up(nt * F * sizeof(float), 256);
+    if (reducer == TIGA_MAX) b += align_up(nt * F * sizeof(int32_t), 256);
+    return b + 256;
+}
+
+extern "C" tiga_status tiga_validate_csr(const tiga_csr* g, int level, void* ws, size_t ws_bytes, void* stream) {
+    tiga_status st = check_csr(g);
+    if (st != TIGA_OK) return st;
+    if (level == 0) return TIGA_OK;
+    if (!ws || ws_bytes < 16) return TIGA_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int* flags = static_cast<int*>(ws);
+    TIGA_CUDA_TRY(cudaMemsetAsync(flags, 0, sizeof(int), s));
+    const long long work = g->n_dst > g->n_edges ? g->n_dst : g->n_edges;
+    long long blocks = (work + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks < 1) blocks = 1;
+    if (g->rowptr_type == TIGA_I32)
+        validate_kernel<int32_t><<<(unsigned)blocks, 256, 0, s>>>(static_cast<const int32_t*>(g->rowptr), g->col, g->n_dst, g->n_src, g->n_edges, flags);
+    else
+        validate_kernel<int64_t><<<(unsigned)blocks, 256, 0, s>>>(static_cast<const int64_t*>(g->rowptr), g->col, g->n_dst, g->n_src, g->n_edges, flags);
+    if (launch_status() != TIGA_OK) return TIGA_ERR_CUDA;
+    int h = 0;
+    TIGA_CUDA_TRY(cudaMemcpyAsync(&h, flags, sizeof(int), cudaMemcpyDeviceToHost, s));
+    TIGA_CUDA_TRY(cudaStreamSynchronize(s));
+    return h ? TIGA_ERR_INVALID_GRAPH : TIGA_OK;
+}
+
+extern "C" tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
+                                      const float* w, const tiga_msg* msg, tiga_reducer reducer,
+                                      float* out, int32_t* argmax, void* ws, size_t ws_bytes, void* stream) {
+    tiga_status st = check_csr(g);
+    if (st != TIGA_OK) return st;
+    int nvec, G, VPL;
+    st = check_features(F, x_dtype, &nvec, &G, &VPL);
+    if (st != TIGA_OK) return st;
+    if (reducer != TIGA_SUM && reducer != TIGA_MAX) return TIGA_ERR_INVALID_ARG;
+    if (!msg) return TIGA_ERR_INVALID_ARG;
+    if (msg->kind == TIGA_MSG_COPY) { if (w) return TIGA_ERR_INVALID_ARG; }
+    else if (msg->kind == TIGA_MSG_WEIGHTED) { if (!w && g->n_edges > 0) return TIGA_ERR_INVALID_ARG; }
+    else return TIGA_ERR_UNSUPPORTED;
+    if (g->n_dst == 0) return TIGA_OK;
+    if (!out || !aligned16(out) || (g->n_src > 0 && (!x || !aligned16(x)))) return TIGA_ERR_INVALID_ARG;
+    if (w && !aligned16(w)) return TIGA_ERR_INVALID_ARG;
+    if (reducer == TIGA_MAX) {
+        if (!argmax || !aligned16(argmax)) return TIGA_ERR_INVALID_ARG;
+        if (g->n_edges > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;
+    }
+    if (!ws || !aligned16(ws) || ws_bytes < tiga_csr_workspace_bytes(g, F, x_dtype, reducer, 0)) return TIGA_ERR_WORKSPACE;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CsrParams p{};
+    p.rowptr = g->rowptr; p.col = g->col; p.w = w; p.x = x; p.out = out; p.arg = argmax;
+    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.F = F; p.nvec = nvec;
+    p.ntiles = num_tiles(g);
+    Carver cv(ws);
+    p.carry_row = cv.take<int32_t>((size_t)p.ntiles + 1);
+    p.carry_val = cv.take<float>(((size_t)p.ntiles + 1) * F);
+    p.carry_arg = reducer == TIGA_MAX ? cv.take<int32_t>(((size_t)p.ntiles + 1) * F) : nullptr;
+
+    const bool i64 = g->rowptr_type == TIGA_I64;
+    if (x_dtype == TIGA_F32) {
+        if (reducer == TIGA_SUM) st = i64 ? launch_fwd_g<float, 0, int64_t>(p, G, VPL, s) : launch_fwd_g<float, 0, int32_t>(p, G, VPL, s);
+        else st = i64 ? launch_fwd_g<float, 1, int64_t>(p, G, VPL, s) : launch_fwd_g<float, 1, int32_t>(p, G, VPL, s);
+    } else {
+        if (reducer == TIGA_SUM) st = i64 ? launch_fwd_g<__half, 0, int64_t>(p, G, VPL, s) : launch_fwd_g<__half, 0, int32_t>(p, G, VPL, s);
+        else st = i64 ? launch_fwd_g<__half, 1, int64_t>(p, G, VPL, s) : launch_fwd_g<__half, 1, int32_t>(p, G, VPL, s);
+    }
+    if (st != TIGA_OK) return st;
+    const long long work = p.ntiles * F;
+    if (reducer == TIGA_SUM) csr_fixup_kernel<0><<<(unsigned)((work + 255) / 256), 256, 0, s>>>(p);
+    else csr_fixup_kernel<1><<<(unsigned)((work + 255) / 256), 256, 0, s>>>(p);
+    return launch_status();
+}
+
+extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
+                                               const float* w, const tiga_msg* msg, tiga_reducer reducer,
+                                               const float* grad_out, const int32_t* argmax,
+                                               float* grad_x, float* grad_w,
+                                               void* ws, size_t ws_bytes, void* stream) {
+    (void)ws; (void)ws_bytes;
+    tiga_status st = check_csr(g);
+    if (st != TIGA_OK) return st;
+    if (x_dtype != TIGA_F32) return TIGA_ERR_UNSUPPORTED;
+    int nvec, G, VPL;
+    st = check_features(F, x_dtype, &nvec, &G, &VPL);
+    if (st != TIGA_OK) return st;
+    if (reducer != TIGA_SUM && reducer != TIGA_MAX) return TIGA_ERR_INVALID_ARG;
+    if (!msg) return TIGA_ERR_INVALID_ARG;
+    if (msg->kind == TIGA_MSG_COPY) { if (w) return TIGA_ERR_INVALID_ARG; }
+    else if (msg->kind == TIGA_MSG_WEIGHTED) { if (!w && g->n_edges > 0) return TIGA_ERR_INVALID_ARG; }
+    else return TIGA_ERR_UNSUPPORTED;
+    if (g->n_dst > 0 && (!grad_out || !aligned16(grad_out))) return TIGA_ERR_INVALID_ARG;
+    if (g->n_src > 0 && (!x || !aligned16(x))) return TIGA_ERR_INVALID_ARG;
+    if ((grad_x && !aligned16(grad_x)) || (grad_w && !aligned16(grad_w)) || (w && !aligned16(w))) return TIGA_ERR_INVALID_ARG;
+    if (reducer == TIGA_MAX) {
+        if (g->n_dst > 0 && (!argmax || !aligned16(argmax))) return TIGA_ERR_INVALID_ARG;
+        if (g->n_edges > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (grad_x && g->n_src > 0) TIGA_CUDA_TRY(cudaMemsetAsync(grad_x, 0, (size_t)g->n_src * F * sizeof(float), s));
+    if (reducer == TIGA_MAX && grad_w && g->n_edges > 0) TIGA_CUDA_TRY(cudaMemsetAsync(grad_w, 0, (size_t)g->n_edges * sizeof(float), s));
+    if (g->n_dst == 0 || g->n_edges == 0 || (!grad_x && !grad_w)) return TIGA_OK;
+
+    CsrParams p{};
+    p.rowptr = g->rowptr; p.col = g->col; p.w = w; p.x = x; p.arg = const_cast<int32_t*>(argmax);
+    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.F = F; p.nvec = nvec;
+    p.ntiles = num_tiles(g);
+    p.gy = grad_out; p.gx = grad_x; p.gw = grad_w;
+    if (reducer == TIGA_SUM) {
+        return g->rowptr_type == TIGA_I64 ? launch_bwd_g<int64_t>(p, G, VPL, s) : launch_bwd_g<int32_t>(p, G, VPL, s);
+    }
+    const long long work = g->n_dst * F;
+    csr_backward_max_kernel<<<(unsigned)((work + 255) / 256), 256, 0, s>>>(p);
+    return launch_status();
+}
+
+extern "C" tiga_status tiga_csr_degree_histogram(const tiga_csr* g, int64_t* hist, int64_t nbins,
+                                                 int64_t* max_degree, void* stream) {
+    tiga_status st = check_csr(g);
+    if (st != TIGA_OK) return st;
+    if (!hist || !max_degree || nbins < 1 || nbins > 8192) return TIGA_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    TIGA_CUDA_TRY(cudaMemsetAsync(hist, 0, (size_t)nbins * sizeof(int64_t), s));
+    TIGA_CUDA_TRY(cudaMemsetAsync(max_degree, 0, sizeof(int64_t), s));
+    if (g->n_dst == 0) return TIGA_OK;
+    long long blocks = (g->n_dst + 1023) / 1024;
+    if (blocks > 148 * 4) blocks = 148 * 4;
+    const size_t sm = (size_t)nbins * sizeof(unsigned int);
+    if (g->rowptr_type == TIGA_I32)
+        degree_hist_kernel<int32_t><<<(unsigned)blocks, 256, sm, s>>>(static_cast<const int32_t*>(g->rowptr), g->n_dst, (int)nbins,
+                                                                   reinterpret_cast<unsigned long long*>(hist), reinterpret_cast<unsigned long long*>(max_degree));
+    else
+        degree_hist_kernel<int64_t><<<(unsigned)blocks, 256, sm, s>>>(static_cast<const int64_t*>(g->rowptr), g->n_dst, (int)nbins,
+                                                                   reinterpret_cast<unsigned long long*>(hist), reinterpret_cast<unsigned long long*>(max_degree));
+    return launch_status();
+}
+
+extern "C" const char* tiga_status_string(tiga_status s) {
+    switch (s) {
+        case TIGA_OK: return "ok";
+        case TIGA_ERR_INVALID_ARG: return "invalid argument";
+        case TIGA_ERR_UNSUPPORTED: return "unsupported combination";
+        case TIGA_ERR_WORKSPACE: return "workspace missing or too small";
+        case TIGA_ERR_CUDA: return "CUDA runtime error";
+        case TIGA_ERR_INVALID_GRAPH: return "malformed CSR relation";
+    }
+    return "unknown status";
+}

@@ -1,0 +1,76 @@
+"""CPU-only checks of the C ABI: the library builds, loads, exports every symbol the header
+declares, and rejects bad arguments on the host before touching a device."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import gen
+import oracle
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2609_24802_b200 import build
+    build.build_library()
+    from paper_2609_24802_b200 import api
+    return api
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "tiga.h")).read()
+    declared = set(re.findall(r"\b(tiga_[a-z_0-9]+)\s*\(", header))
+    assert declared == set(lib.EXPORTS)
+    cdll = lib.load_library()
+    for name in declared:
+        assert getattr(cdll, name) is not None
+
+
+def test_status_strings(lib):
+    assert lib.tiga_status_string(0) == "ok"
+    assert len({lib.tiga_status_string(s) for s in range(6)}) == 6
+
+
+def test_grid_matches_the_oracle_reading(lib):
+    cases = [(4096, 0.06, [1, 1, 1], [0, 0, 0]), (1_000_000, float(gen.radius_for_expected_neighbours(1_000_000, 32)), [1, 1, 1], [1, 1, 1]),
+             (160 ** 3, 2.5, [172.3548] * 3, [1, 1, 1]), (128, 0.35, [1, 1, 1], [1, 0, 1]),
+             (10, 0.001, [1, 1, 1], [0, 0, 0]), (5000, 0.07, [1.0, 2.5, 0.3], [1, 0, 0]), (1, 0.1, [1, 1, 1], [0, 0, 0])]
+    for n, r, box, per in cases:
+        nc, ih = lib.tiga_radius_grid(n, np.float32(r), np.float32(box), per)
+        onc, oih = oracle.cell_grid(n, np.float32(r), np.float32(box), per)
+        assert nc == onc.tolist() and np.array_equal(np.float32(ih), oih)
+
+
+def test_host_side_argument_errors(lib):
+    cdll = lib.load_library()
+    from paper_2609_24802_b200.api import _Box, _Csr, _Msg
+    b = _Box()
+    for d in range(3):
+        b.len[d] = 1.0
+        b.periodic[d] = 1
+    nc = (ctypes.c_int32 * 3)()
+    # periodic box needs r < len/2; r must be positive
+    assert cdll.tiga_radius_grid(100, ctypes.c_float(0.6), ctypes.byref(b), nc, None) == 1
+    assert cdll.tiga_radius_grid(100, ctypes.c_float(-1.0), ctypes.byref(b), nc, None) == 1
+    assert cdll.tiga_radius_grid(100, ctypes.c_float(0.1), None, nc, None) == 1
+    assert cdll.tiga_radius_workspace_bytes(100, 4, ctypes.c_float(0.6), ctypes.byref(b), 0) == 0
+    # CSR: null / misaligned pointers, negative sizes, unsupported widths
+    g = _Csr(0, 0, 0, 4, 4, 0)
+    msg = _Msg(0, 0.0, 0.0)
+    assert cdll.tiga_apply_csr(ctypes.byref(g), None, 0, 4, None, ctypes.byref(msg), 0, None, None, None, 0, None) == 1
+    g = _Csr(256, 0, 256, -1, 4, 0)
+    assert cdll.tiga_apply_csr(ctypes.byref(g), None, 0, 4, None, ctypes.byref(msg), 0, None, None, None, 0, None) == 1
+    g = _Csr(260, 0, 256, 4, 4, 8)            # rowptr not 16-byte aligned
+    assert cdll.tiga_apply_csr(ctypes.byref(g), 256, 0, 4, None, ctypes.byref(msg), 0, 256, None, 256, 1 << 20, None) == 1
+    g = _Csr(256, 0, 256, 4, 4, 8)
+    assert cdll.tiga_apply_csr(ctypes.byref(g), 256, 0, 6, None, ctypes.byref(msg), 0, 256, None, 256, 1 << 20, None) == 2   # F % 4
+    assert cdll.tiga_apply_csr(ctypes.byref(g), 256, 0, 4, None, ctypes.byref(msg), 0, 256, None, 256, 8, None) == 3        # workspace
+    assert cdll.tiga_apply_csr(ctypes.byref(g), 256, 0, 4, None, ctypes.byref(msg), 1, 256, None, 256, 1 << 20, None) == 1  # max needs argmax
+    assert cdll.tiga_apply_csr(ctypes.byref(g), 256, 0, 4, 256, ctypes.byref(msg), 0, 256, None, 256, 1 << 20, None) == 1   # COPY with weights
+    assert cdll.tiga_csr_workspace_bytes(ctypes.byref(g), 64, 0, 0, 0) >= 2 * 64 * 4
+    assert cdll.tiga_csr_degree_histogram(ctypes.byref(g), 256, 0, 256, None) == 1                          # nbins < 1
+    assert cdll.tiga_validate_csr(ctypes.byref(g), 0, None, 0, None) == 0                                   # metadata only

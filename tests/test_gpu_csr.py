@@ -1,0 +1,216 @@
+"""GPU parity: the CUDA CSR traversal (through the C ABI) against the fp64 CPU oracle, element
+by element on the same seeded inputs.  Integers and max outputs must match bit-exactly, sums
+within 1e-5 and gradients within 1e-4 of the sum of absolute contributions."""
+import numpy as np
+import pytest
+
+import gen
+import oracle
+from conftest import read_golden
+from parity import GRAD_TOL, SUM_TOL, dev, host, rel_err
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tiga():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2609_24802_b200 import api
+    return api
+
+
+def _relation(tiga, rowptr, col, n_src, index64=False):
+    rp = dev(rowptr.astype(np.int64 if index64 else np.int32), torch)
+    return tiga.CsrRelation(rp, dev(col.astype(np.int32), torch), n_src)
+
+
+def _check_forward(tiga, rowptr, col, x, w, index64=False, reducers=(0, 1)):
+    g = _relation(tiga, rowptr, col, x.shape[0], index64)
+    xd = dev(x, torch)
+    wd = None if w is None else dev(w, torch)
+    res = {}
+    for red in reducers:
+        y, A, arg = oracle.csr_forward(rowptr, col, x, w, red)
+        out, am = tiga.tiga_apply_csr(g, xd, wd, red)
+        out2, am2 = tiga.tiga_apply_csr(g, xd, wd, red)
+        torch.cuda.synchronize()
+        assert torch.equal(out, out2), "forward must be reproducible run to run"
+        if red == tiga.SUM:
+            assert rel_err(host(out), y, A) <= SUM_TOL
+        else:
+            assert np.array_equal(host(out), y.astype(np.float32)), "max outputs must be bit exact"
+            assert np.array_equal(host(am).astype(np.int64), arg), "argmax must be bit exact"
+            assert torch.equal(am, am2)
+        res[red] = (out, am)
+    return g, xd, wd, res
+
+
+def _check_backward(tiga, rowptr, col, x, w, gy, g, xd, wd, res):
+    gyd = dev(gy, torch)
+    ref = oracle.csr_backward_sum(rowptr, col, x, w, gy)
+    gx, gw = tiga.tiga_apply_csr_backward(g, xd, wd, gyd, tiga.SUM)
+    assert rel_err(host(gx), ref["gx"], ref["Ax"]) <= GRAD_TOL
+    assert rel_err(host(gw), ref["gw"], ref["Aw"]) <= GRAD_TOL
+    only_x, none_w = tiga.tiga_apply_csr_backward(g, xd, wd, gyd, tiga.SUM, want_w=False)
+    assert none_w is None and rel_err(host(only_x), ref["gx"], ref["Ax"]) <= GRAD_TOL
+    if 1 in res:
+        am = res[1][1]
+        _, _, arg = oracle.csr_forward(rowptr, col, x, w, oracle.MAX)
+        refm = oracle.csr_backward_max(rowptr, col, x, w, gy, arg)
+        gx, gw = tiga.tiga_apply_csr_backward(g, xd, wd, gyd, tiga.MAX, argmax=am)
+        assert rel_err(host(gx), refm["gx"], refm["Ax"]) <= GRAD_TOL
+        assert rel_err(host(gw), refm["gw"], refm["Aw"]) <= GRAD_TOL
+
+
+def _random_graph(seed, n_dst, n_src, max_deg, F, p_empty=0.3):
+    g = gen.rng(seed, 700)
+    deg = g.integers(0, max_deg + 1, size=n_dst)
+    deg[g.random(n_dst) < p_empty] = 0
+    rowptr = np.concatenate([[0], np.cumsum(deg)]).astype(np.int64)
+    E = int(rowptr[-1])
+    col = g.integers(0, n_src, size=E).astype(np.int32)
+    x = g.standard_normal((n_src, F)).astype(np.float32)
+    w = ((g.integers(0, 2**24 - 1, size=E) + 1) * 2.0**-24).astype(np.float32)
+    gy = g.standard_normal((n_dst, F)).astype(np.float32)
+    return rowptr, col, x, w, gy
+
+
+def test_printed_worked_example(tiga):
+    gd = read_golden("csr_worked_example.txt")
+    rowptr = np.array(gd["rowptr"], np.int64)
+    col = np.array(gd["col"], np.int32)
+    x = np.repeat(np.array(gd["x"], np.float32)[:, None], 4, axis=1)
+    w = np.array(gd["w"], np.float32)
+    g, xd, wd, res = _check_forward(tiga, rowptr, col, x, w)
+    assert host(res[0][0])[:, 0].tolist() == gd["y"]
+    gx, gw = tiga.tiga_apply_csr_backward(g, xd, wd, torch.ones((3, 4), device="cuda"), tiga.SUM)
+    assert host(gx)[:, 0].tolist() == gd["dx"]
+    assert host(gw).tolist() == [4 * v for v in gd["dw"]]      # four identical feature columns
+
+
+@pytest.mark.parametrize("F", [4, 8, 12, 16, 32, 64, 100, 128, 160, 256, 512])
+def test_random_graphs_all_widths(tiga, F):
+    rowptr, col, x, w, gy = _random_graph(F, n_dst=3000, n_src=1000, max_deg=40, F=F)
+    g, xd, wd, res = _check_forward(tiga, rowptr, col, x, w)
+    _check_backward(tiga, rowptr, col, x, w, gy, g, xd, wd, res)
+
+
+def test_unit_weights_and_duplicates(tiga):
+    rowptr, col, x, _, gy = _random_graph(77, n_dst=500, n_src=5, max_deg=30, F=16)   # 5 sources: many duplicates and ties
+    g, xd, wd, res = _check_forward(tiga, rowptr, col, x, None)
+    _check_backward(tiga, rowptr, col, x, None, gy, g, xd, wd, res)
+    # integer-valued features make ties frequent: the lowest edge position must win
+    xi = gen.small_int_features(5, 16, 3)
+    _check_forward(tiga, rowptr, col, xi, None)
+
+
+def test_degenerate_shapes(tiga):
+    F = 8
+    x = gen.normal_features(7, F, 1)
+    # no edges at all; one row; one huge row between empty ones; last row heavy
+    for rowptr in ([0, 0, 0, 0, 0], [0, 0], [0, 3], [0, 0, 30000, 30000], [0, 5, 5, 9000]):
+        rowptr = np.array(rowptr, np.int64)
+        E = int(rowptr[-1])
+        col = gen.rng(E, 5).integers(0, 7, size=E).astype(np.int32)
+        w = gen.edge_weights(E, 2) if E else np.zeros(0, np.float32)
+        g, xd, wd, res = _check_forward(tiga, rowptr, col, x, w if E else None)
+        gy = gen.normal_features(len(rowptr) - 1, F, 2, 32)
+        _check_backward(tiga, rowptr, col, x, w if E else None, gy, g, xd, wd, res)
+    # a long run of empty rows (more rows than one tile holds) around a few edges
+    rowptr = np.zeros(10001, np.int64)
+    rowptr[5000:] = 3
+    rowptr[9000:] = 7
+    col = np.array([0, 1, 2, 3, 4, 5, 6], np.int32)
+    _check_forward(tiga, rowptr, col, x, gen.edge_weights(7, 3))
+
+
+def test_heavy_rows_span_many_tiles(tiga):
+    rowptr, col = gen.rmat_csr(14, 16 << 14, seed=3)
+    n = 1 << 14
+    assert np.diff(rowptr).max() > 2 * 2048
+    x = gen.normal_features(n, 64, 3)
+    w = gen.edge_weights(16 << 14, 3)
+    gy = gen.normal_features(n, 64, 3, 32)
+    g, xd, wd, res = _check_forward(tiga, rowptr, col, x, w)
+    _check_backward(tiga, rowptr, col, x, w, gy, g, xd, wd, res)
+
+
+def test_hex_mesh_degrees(tiga):
+    L = 24
+    rowptr, col = gen.hex_mesh_csr(L)
+    ones = np.ones((L ** 3, 16), np.float32)
+    g = _relation(tiga, rowptr, col, L ** 3)
+    out, _ = tiga.tiga_apply_csr(g, dev(ones, torch), None, tiga.SUM)
+    deg = np.diff(rowptr).astype(np.float32)
+    assert np.array_equal(host(out), np.repeat(deg[:, None], 16, axis=1))
+    assert deg.max() == read_golden("hex_mesh_counts.txt")["interior_degree"][0]
+
+
+def test_periodic_closed_form_is_bit_exact(tiga):
+    n, F = 1 << 16, 32
+    offs = [1, 2, 3, 5, 8, 13, 21, 34, -1, -2, -3, -5, -8, -13, -21, -34]
+    rowptr, col = gen.periodic_offset_csr(n, offs)
+    x = gen.small_int_features(n, F, 4)
+    w = gen.small_int_weights(16 * n, 4)
+    g = _relation(tiga, rowptr, col, n)
+    out, _ = tiga.tiga_apply_csr(g, dev(x, torch), dev(w, torch), tiga.SUM)
+    ref = np.zeros((n, F))
+    for k, o in enumerate(offs):
+        ref += w[k::16, None].astype(np.float64) * np.roll(x.astype(np.float64), -o, axis=0)
+    assert np.array_equal(host(out).astype(np.float64), ref)
+
+
+def test_fp16_features_int64_rowptr(tiga):
+    c = gen.config("cfg4", scale=15)
+    assert c["x"].dtype == np.float16 and c["rowptr"].dtype == np.int64
+    _check_forward(tiga, c["rowptr"], c["col"], c["x"], None, index64=True)
+    for F in (16, 64, 264):
+        x = gen.normal_features(1 << 15, F, 8, dtype=np.float16)
+        w = gen.edge_weights(c["E"], 8)
+        _check_forward(tiga, c["rowptr"], c["col"], x, w, index64=True)
+
+
+def test_degree_histogram_is_bit_exact(tiga):
+    for scale, index64 in ((12, False), (16, True)):
+        rowptr, col = gen.rmat_csr(scale, 16 << scale, seed=9)
+        g = _relation(tiga, rowptr, col, 1 << scale, index64)
+        for nbins in (4096, 8, 1):
+            hist, mx = tiga.tiga_csr_degree_histogram(g, nbins)
+            ref, rmx = oracle.degree_histogram(rowptr, nbins)
+            assert np.array_equal(host(hist), ref) and int(host(mx)[0]) == rmx
+        hist, _ = tiga.tiga_csr_degree_histogram(g, 8192)
+        h = host(hist)
+        if h[-1] == 0:
+            assert int(np.sum(np.arange(8192) * h)) == int(rowptr[-1])     # degree sums equal E
+
+
+def test_full_validation_finds_malformed_relations(tiga):
+    rowptr, col = gen.rmat_csr(10, 16 << 10, seed=1)
+    n = 1 << 10
+    tiga.tiga_validate_csr(_relation(tiga, rowptr, col, n), 1)
+    bad = rowptr.copy(); bad[100], bad[101] = bad[101] + 5, bad[100]          # not monotone
+    cases = [(bad, col, n)]
+    bad = rowptr.copy(); bad[0] = 1
+    cases.append((bad, col, n))                                                # does not start at 0
+    bad = rowptr.copy(); bad[-1] -= 1
+    cases.append((bad, col, n))                                                # endpoint != E
+    badc = col.copy(); badc[17] = n
+    cases.append((rowptr, badc, n))                                            # source out of range
+    badc = col.copy(); badc[5] = -1
+    cases.append((rowptr, badc, n))
+    for rp, cc, ns in cases:
+        with pytest.raises(tiga.TigaError) as ei:
+            tiga.tiga_validate_csr(_relation(tiga, rp, cc, ns), 1)
+        assert ei.value.status == 5
+    torch.cuda.synchronize()
+
+
+def test_cfg1_full_size(tiga):
+    """R-MAT scale 20, 16.8M edges, F=64: every output element against the oracle."""
+    c = gen.config("cfg1")
+    g, xd, wd, res = _check_forward(tiga, c["rowptr"], c["col"], c["x"], c["w"])
+    _check_backward(tiga, c["rowptr"], c["col"], c["x"], c["w"], c["gy"], g, xd, wd, res)
+    hist, mx = tiga.tiga_csr_degree_histogram(g, 4096)
+    ref, rmx = oracle.degree_histogram(c["rowptr"], 4096)
+    assert np.array_equal(host(hist), ref) and int(host(mx)[0]) == rmx

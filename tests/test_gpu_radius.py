@@ -1,0 +1,199 @@
+"""GPU parity: cell binning and the fused radius traversal (through the C ABI) against the
+fp64 CPU oracle.  Cells, offsets, order and neighbour counts must match bit-exactly; sums
+within 1e-5 and gradients within 1e-4 of the sum of absolute contributions."""
+import numpy as np
+import pytest
+
+import gen
+import oracle
+from parity import GRAD_TOL, SUM_TOL, dev, host, rel_err
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tiga():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2609_24802_b200 import api
+    return api
+
+
+def _check_bin(tiga, pos, r, box, per):
+    ref = oracle.bin_points(pos, r, box, per)
+    got = tiga.tiga_radius_bin(dev(pos, torch), r, box, per)
+    assert got["ncell"] == ref["ncell"].tolist()
+    assert np.array_equal(host(got["cell"]), ref["cell"])
+    assert np.array_equal(host(got["cell_start"]), ref["cell_start"])
+    assert np.array_equal(host(got["order"]), ref["order"])
+
+
+def _check_gauss(tiga, pos, x, gy, r, box, per, sigma, kind=None, use_cells=False, backward=True):
+    kind = tiga.MSG_GAUSS if kind is None else kind
+    y, A, cnt = oracle.radius_forward(pos, x, r, box, per, kind, p0=sigma, use_cells=use_cells)
+    pd, xd = dev(pos, torch), dev(x, torch)
+    out, count, ws = tiga.tiga_apply_radius(pd, xd, r, box, per, kind, p0=sigma, want_count=True)
+    assert np.array_equal(host(count), cnt), "neighbour counts must be bit exact"
+    assert rel_err(host(out), y, A) <= SUM_TOL
+    if backward and kind == tiga.MSG_GAUSS:
+        ref = oracle.radius_backward_gauss(pos, x, gy, r, box, per, sigma, use_cells=use_cells)
+        gyd = dev(gy, torch)
+        gx, gp = tiga.tiga_apply_radius_backward(pd, xd, gyd, r, box, per, sigma, ws=ws, reuse_plan=True)
+        assert rel_err(host(gx), ref["gx"], ref["Agx"]) <= GRAD_TOL
+        assert rel_err(host(gp), ref["gp"], ref["Agp"]) <= GRAD_TOL
+        gx2, gp2 = tiga.tiga_apply_radius_backward(pd, xd, gyd, r, box, per, sigma)      # rebuilds the bins
+        assert torch.equal(gx, gx2) and torch.equal(gp, gp2)
+    return out, count
+
+
+# ------------------------------------------------------------------------------ binning
+def test_binning_is_bit_exact(tiga):
+    ones = np.ones(3, np.float32)
+    for n, r, per, seed in [(4096, 0.06, [0, 0, 0], 1), (50_000, 0.05, [1, 1, 1], 2), (128, 0.35, [0, 0, 0], 7),
+                            (3000, 0.3, [1, 0, 1], 3), (1000, 0.45, [1, 1, 1], 4), (7, 0.2, [0, 0, 0], 5),
+                            (200_000, 0.004, [1, 1, 1], 6)]:
+        pos = gen.uniform_points(n, seed)
+        pos[0] = 0.0
+        pos[-1] = 1.0                     # on the upper faces: clamped into the last cell
+        _check_bin(tiga, pos, np.float32(r), ones, per)
+    # everything in one cell; clustered points (a few very full cells)
+    _check_bin(tiga, gen.uniform_points(500, 9) * np.float32(0.01), np.float32(0.1), ones, [0, 0, 0])
+    p = gen.uniform_points(20_000, 10)
+    p[:15_000] = p[:15_000] * np.float32(0.02) + np.float32(0.5)
+    _check_bin(tiga, p, np.float32(0.05), ones, [1, 1, 1])
+    # anisotropic box
+    box = np.array([1.0, 2.5, 0.3], np.float32)
+    _check_bin(tiga, gen.uniform_points(5000, 11) * box[None, :], np.float32(0.07), box, [1, 0, 0])
+    c = gen.config("cfg3", m=20)
+    _check_bin(tiga, c["pos"], c["r"], c["box"], c["periodic"])
+
+
+# ------------------------------------------------------------------------------ Gaussian
+def test_cfg0_tiny_forward_and_backward(tiga):
+    c = gen.config("cfg0")
+    _check_gauss(tiga, c["pos"], c["x"], c["gy"], c["r"], c["box"], c["periodic"], c["sigma"])
+
+
+@pytest.mark.parametrize("periodic", [0, 1])
+@pytest.mark.parametrize("F", [4, 16, 32, 64, 128])
+def test_gaussian_small(tiga, periodic, F):
+    n = 6000
+    pos = gen.uniform_points(n, 20 + F)
+    x = gen.normal_features(n, F, 20 + F, 31)
+    gy = gen.normal_features(n, F, 20 + F, 32)
+    r = gen.radius_for_expected_neighbours(n, 24.0)
+    _check_gauss(tiga, pos, x, gy, r, np.ones(3, np.float32), [periodic] * 3, np.float32(float(r) / 2))
+
+
+def test_few_cells_mixed_periodicity_and_anisotropic_box(tiga):
+    # the paper's tiny radius shape: 128 points, cutoff 0.35 (two cells per dimension)
+    pos = gen.uniform_points(128, 7)
+    x = gen.normal_features(128, 8, 7); gy = gen.normal_features(128, 8, 7, 32)
+    ones = np.ones(3, np.float32)
+    _check_gauss(tiga, pos, x, gy, np.float32(0.35), ones, [0, 0, 0], np.float32(0.2))
+    _check_gauss(tiga, pos, x, gy, np.float32(0.35), ones, [1, 1, 1], np.float32(0.2))   # one cell, minimum image
+    _check_gauss(tiga, pos, x, gy, np.float32(0.3), ones, [1, 0, 1], np.float32(0.2))    # three cells where periodic
+    box = np.array([1.0, 2.5, 0.3], np.float32)
+    n = 4000
+    pos = gen.uniform_points(n, 12) * box[None, :]
+    x = gen.normal_features(n, 16, 12); gy = gen.normal_features(n, 16, 12, 32)
+    _check_gauss(tiga, pos, x, gy, np.float32(0.09), box, [1, 0, 1], np.float32(0.05))
+    # the paper's own message: distance-weighted sum
+    _check_gauss(tiga, pos, x, gy, np.float32(0.09), box, [1, 0, 1], np.float32(0.05), kind=tiga.MSG_DIST)
+
+
+def test_pairs_exactly_on_the_cutoff_are_neighbours(tiga):
+    # binary-grid coordinates: many pairs at distance exactly r (inclusive predicate)
+    k = np.arange(16, dtype=np.float32) / 16
+    X, Y, Z = np.meshgrid(k, k, k, indexing="ij")
+    pos = np.stack([X.ravel(), Y.ravel(), Z.ravel()], 1).astype(np.float32)
+    n = pos.shape[0]
+    x = gen.normal_features(n, 8, 5); gy = gen.normal_features(n, 8, 5, 32)
+    for per in ([0, 0, 0], [1, 1, 1]):
+        out, count = _check_gauss(tiga, pos, x, gy, np.float32(3.0 / 16), np.ones(3, np.float32), per, np.float32(0.1))
+        if per[0]:
+            # |v| <= 3 on the integer lattice: 123 points minus the origin
+            assert np.all(host(count) == 122)
+
+
+def test_no_neighbours_and_coincident_points(tiga):
+    pos = np.array([[0.1, 0.1, 0.1], [0.9, 0.9, 0.9], [0.5, 0.5, 0.5], [0.5, 0.5, 0.5], [0.5, 0.5, 0.5]], np.float32)
+    x = gen.normal_features(5, 4, 1); gy = gen.normal_features(5, 4, 1, 32)
+    out, count = _check_gauss(tiga, pos, x, gy, np.float32(0.05), np.ones(3, np.float32), [0, 0, 0], np.float32(0.02))
+    assert host(count).tolist() == [0, 0, 2, 2, 2]
+    assert np.all(host(out)[:2] == 0.0)
+
+
+def test_clustered_points_overflow_the_pair_list(tiga):
+    n = 3000
+    pos = gen.uniform_points(n, 15) * np.float32(0.1) + np.float32(0.3)       # ~500 neighbours each
+    x = gen.normal_features(n, 32, 15); gy = gen.normal_features(n, 32, 15, 32)
+    _check_gauss(tiga, pos, x, gy, np.float32(0.05), np.ones(3, np.float32), [0, 0, 0], np.float32(0.03))
+
+
+def test_gaussian_mid_replica(tiga):
+    """A 131,072-point replica of the 1M-point periodic workload (32 expected neighbours, F=32),
+    every row against the oracle's cell-directory variant (itself pinned to all pairs)."""
+    c = gen.config("cfg2", n=131_072)
+    _check_gauss(tiga, c["pos"], c["x"], c["gy"], c["r"], c["box"], c["periodic"], c["sigma"], use_cells=True)
+
+
+# ------------------------------------------------------------------------------ Lennard-Jones
+def _check_lj(tiga, pos, r, box, per, eps=1.0, s=1.0, use_cells=False):
+    y, A, cnt = oracle.radius_forward(pos, None, r, box, per, oracle.MSG_LJ, eps, s, use_cells=use_cells)
+    out, count, _ = tiga.tiga_apply_radius(dev(pos, torch), None, r, box, per, tiga.MSG_LJ, p0=eps, p1=s, want_count=True)
+    assert np.array_equal(host(count), cnt)
+    assert rel_err(host(out), y, A) <= SUM_TOL
+    return host(out), A
+
+
+def test_lennard_jones_lattices(tiga):
+    c = gen.config("cfg3", m=12)
+    out, A = _check_lj(tiga, c["pos"], c["r"], c["box"], c["periodic"])
+    assert np.max(np.abs(out[:, :3].astype(np.float64).sum(0))) < 1e-6 * A[:, :3].sum()   # Newton's third law
+    # perfect lattice: 56 neighbours, zero force, closed-form energy per particle
+    pos, L = gen.jittered_lattice(10, 0.8, 0.0)
+    out, A = _check_lj(tiga, pos, np.float32(2.5), np.full(3, L, np.float32), [1, 1, 1])
+    assert np.max(np.abs(out[:, 3] - (-5.264771118950892))) < 2e-4
+    # other eps / s, non-periodic
+    pos = gen.uniform_points(2000, 3) * np.float32(12.0)
+    keep = np.ones(len(pos), bool)
+    d = np.linalg.norm(pos[:, None, :].astype(np.float64) - pos[None, :, :], axis=2) + np.eye(len(pos)) * 9
+    keep[np.unique(np.nonzero(d < 0.7)[0])] = False          # no overlapping particles
+    _check_lj(tiga, pos[keep], np.float32(2.0), np.full(3, 12.0, np.float32), [0, 0, 0], eps=1.5, s=0.8)
+
+
+def test_lennard_jones_replica(tiga):
+    c = gen.config("cfg3", m=40)          # 64,000 particles
+    out, A = _check_lj(tiga, c["pos"], c["r"], c["box"], c["periodic"], use_cells=True)
+    assert np.max(np.abs(out[:, :3].astype(np.float64).sum(0))) < 1e-6 * A[:, :3].sum()
+
+
+# ------------------------------------------------------------------------------ full size
+def test_cfg2_full_size_sampled_rows(tiga):
+    """1M points, periodic, F=32: 4096 sampled rows against all-pairs brute force, all rows
+    against the oracle's cell-directory variant, plus global invariants."""
+    c = gen.config("cfg2")
+    n = c["n"]
+    pd, xd, gyd = dev(c["pos"], torch), dev(c["x"], torch), dev(c["gy"], torch)
+    out, count, ws = tiga.tiga_apply_radius(pd, xd, c["r"], c["box"], c["periodic"], tiga.MSG_GAUSS,
+                                            p0=c["sigma"], want_count=True)
+    gx, gp = tiga.tiga_apply_radius_backward(pd, xd, gyd, c["r"], c["box"], c["periodic"], c["sigma"], ws=ws, reuse_plan=True)
+    out, count, gx, gp = host(out), host(count), host(gx), host(gp)
+    rows = np.sort(gen.rng(1, 77).choice(n, 4096, replace=False))
+    y, A, cnt = oracle.radius_forward(c["pos"], c["x"], c["r"], c["box"], c["periodic"], oracle.MSG_GAUSS,
+                                      p0=c["sigma"], rows=rows)
+    assert np.array_equal(count[rows], cnt)
+    assert rel_err(out[rows], y, A) <= SUM_TOL
+    b = oracle.radius_backward_gauss(c["pos"], c["x"], c["gy"], c["r"], c["box"], c["periodic"], c["sigma"], rows=rows)
+    assert rel_err(gx[rows], b["gx"], b["Agx"]) <= GRAD_TOL
+    assert rel_err(gp[rows], b["gp"], b["Agp"]) <= GRAD_TOL
+    y, A, cnt = oracle.radius_forward(c["pos"], c["x"], c["r"], c["box"], c["periodic"], oracle.MSG_GAUSS,
+                                      p0=c["sigma"], use_cells=True)
+    assert np.array_equal(count, cnt) and count.sum() % 2 == 0
+    assert rel_err(out, y, A) <= SUM_TOL
+    assert abs(count.mean() - 32.0) < 0.1
+    b = oracle.radius_backward_gauss(c["pos"], c["x"], c["gy"], c["r"], c["box"], c["periodic"], c["sigma"], use_cells=True)
+    assert rel_err(gx, b["gx"], b["Agx"]) <= GRAD_TOL
+    assert rel_err(gp, b["gp"], b["Agp"]) <= GRAD_TOL
+    assert np.max(np.abs(gp.astype(np.float64).sum(0))) < 1e-5 * b["Agp"].sum()     # translation invariance

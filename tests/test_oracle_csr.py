@@ -57,6 +57,8 @@ def _brute_forward(rowptr, col, x, w, reducer):
                     s += m
                 y[i, f] = s
             else:
+                # fp32 inputs: the selection compares messages rounded once to fp32
+                msgs = [(float(np.float32(m)), e) for m, e in msgs]
                 best = max(m for m, _ in msgs)
                 y[i, f] = best
                 arg[i, f] = min(e for m, e in msgs if m == best)
@@ -93,7 +95,7 @@ def test_max_values_match_torch_scatter_reduce():
     ref = torch.full((len(rowptr) - 1, 4), float("-inf"), dtype=torch.float64)
     ref = ref.scatter_reduce(0, torch.from_numpy(rows)[:, None].expand(-1, 4), msg, "amax")
     ref[torch.isinf(ref)] = 0.0
-    assert np.array_equal(y, ref.numpy())
+    assert np.array_equal(y, ref.numpy().astype(np.float32).astype(np.float64))   # rounding is monotone
 
 
 # ------------------------------------------------------------------ library special case
@@ -245,3 +247,18 @@ def test_max_backward_matches_central_differences_away_from_ties():
     sel = np.unique(arg[arg >= 0])
     mask = np.ones(len(w), bool); mask[sel] = False
     assert np.all(b["gw"][mask] == 0.0)
+
+
+def test_max_selection_is_taken_in_message_precision():
+    # two products that differ in fp64 but round to the same fp32 value are a tie:
+    # the earlier edge wins and the output is that fp32 value
+    x = np.array([[1.0 + 2 * 2.0 ** -23], [1.0]], np.float32)
+    w = np.array([1.0 - 2 * 2.0 ** -24, 1.0 + 2.0 ** -23], np.float32)
+    p0 = float(w[0]) * float(x[0, 0]); p1 = float(w[1]) * float(x[1, 0])
+    assert p0 != p1 and np.float32(p0) == np.float32(p1) and p1 > p0
+    y, _, arg = oracle.csr_forward(np.array([0, 2]), np.array([0, 1], np.int32), x, w, oracle.MAX)
+    assert arg[0, 0] == 0 and y[0, 0] == float(np.float32(p0))
+    # the same data in fp64 is no tie
+    y, _, arg = oracle.csr_forward(np.array([0, 2]), np.array([0, 1], np.int32),
+                                   x.astype(np.float64), w.astype(np.float64), oracle.MAX)
+    assert arg[0, 0] == 1 and y[0, 0] == p1
