@@ -402,6 +402,58 @@ def run_reference(args, rank, world):
     }))
 
 
+def run_case(args):
+    """One traversal on a reduced replica of its workload, a few launches, for profiler
+    captures of a single kernel (`--case csr|radius_gauss|radius_lj --size S`)."""
+    import torch
+    from paper_2609_24802_b200 import api as T
+    dev = torch.device("cuda", 0)
+    to = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    ev0 = torch.cuda.Event(enable_timing=True); ev1 = torch.cuda.Event(enable_timing=True)
+    if args.case == "csr":
+        c = gen.config("cfg1", args.seed, scale=args.size or 18)
+        g = T.CsrRelation(to(c["rowptr"]), to(c["col"]), c["n"])
+        x, w, gy = to(c["x"]), to(c["w"]), to(c["gy"])
+        def run():
+            out, arg = T.tiga_apply_csr(g, x, w, T.SUM)
+            T.tiga_apply_csr_backward(g, x, w, gy, T.SUM)
+            om, am = T.tiga_apply_csr(g, x, w, T.MAX)
+            T.tiga_apply_csr_backward(g, x, w, gy, T.MAX, argmax=am)
+        units = c["E"]
+    elif args.case == "csr_large":
+        c = gen.config("cfg4", args.seed, scale=args.size or 26)
+        g = T.CsrRelation(to(c["rowptr"]), to(c["col"]), c["n"])
+        x = to(c["x"])
+        out = torch.empty((c["n"], c["F"]), device=dev)
+        ws = torch.empty(T.tiga_csr_workspace_bytes(g, c["F"], T.F16, T.SUM), dtype=torch.uint8, device=dev)
+        def run():
+            T.tiga_apply_csr(g, x, None, T.SUM, out=out, ws=ws)
+        units = c["E"]
+    elif args.case == "radius_gauss":
+        c = gen.config("cfg2", args.seed, n=args.size or 300_000)
+        pos, x, gy = to(c["pos"]), to(c["x"]), to(c["gy"])
+        def run():
+            out, cnt, ws = T.tiga_apply_radius(pos, x, c["r"], c["box"], c["periodic"], T.MSG_GAUSS, p0=c["sigma"])
+            T.tiga_apply_radius_backward(pos, x, gy, c["r"], c["box"], c["periodic"], c["sigma"], ws=ws, reuse_plan=True)
+        units = c["n"]
+    else:
+        c = gen.config("cfg3", args.seed, m=args.size or 100)
+        pos = to(c["pos"])
+        def run():
+            T.tiga_apply_radius(pos, None, c["r"], c["box"], c["periodic"], T.MSG_LJ, p0=1.0, p1=1.0)
+        units = c["n"]
+    for _ in range(max(args.warmup, 1)):
+        run()
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(args.steps):
+        run()
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    print(json.dumps({"case": args.case, "units": units, "ms_per_step": ms, "units_per_s": units / (ms * 1e-3)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -410,11 +462,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--seed", type=int, default=gen.DEFAULT_SEED)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--case", default=None, choices=["csr", "csr_large", "radius_gauss", "radius_lj"],
+                    help="run one traversal on a reduced replica (for profiler captures) instead of the benchmark")
+    ap.add_argument("--size", type=int, default=0, help="--case size: R-MAT scale, number of points, or lattice side")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.impl == "reference":
+    if args.case:
+        run_case(args)
+    elif args.impl == "reference":
         run_reference(args, rank, world)
     else:
         run_ours(args, rank, world, local_rank)

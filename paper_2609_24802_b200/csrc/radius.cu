@@ -9,9 +9,10 @@
 //      inter-CTA waiting), scatter into cell order, per-cell rank sort by point id (which
 //      makes the scatter stable and therefore unique), sorted copy of the positions;
 //   2. traversal: one warp per query cell walks the 27 neighbouring cells (wrapped or
-//      clipped).  Lanes test candidates; accepted (source, weight) pairs are compacted
-//      through shared memory and consumed with lanes across the feature axis, so every
-//      gathered feature row is one coalesced request.
+//      clipped) as contiguous candidate ranges.  The lanes of a query split its candidates;
+//      accepted (source, weight) pairs go to lane-private lists in shared memory and are
+//      consumed with groups of lanes across the feature axis, so every gathered feature
+//      row is one coalesced 128-bit-per-lane request.
 //
 // Exact membership: the fp32 squared distance is only a filter.  A pair whose fp32 value
 // falls within a few ulps of r^2 is re-decided in fp64 with the defining formula
@@ -25,8 +26,6 @@
 namespace tiga {
 
 constexpr int RAD_THREADS = 256;
-constexpr int RAD_WARPS = RAD_THREADS / 32;
-constexpr int LIST_CAP = 64;
 constexpr int SCAN_BLOCK = 2048;   // elements per CTA in the scan passes
 
 struct RadiusParams {
@@ -47,6 +46,7 @@ struct RadiusParams {
     int periodic[3];
     int nc[3];
     float invh[3];
+    float hcell[3];           // cell edge, len / nc
     int ncells;
     float p0, p1;             // message parameters
     // plan (workspace)
@@ -195,8 +195,11 @@ __global__ void bin_sort_kernel(const RadiusParams p) {
 }
 
 // ------------------------------------------------------------------------------ traversal
+constexpr int TRAV_WARPS = 4;
+constexpr int TRAV_THREADS = TRAV_WARPS * 32;
+
 // The defining predicate in double precision (same operations as the plain definition).
-__device__ __noinline__ bool exact_within(const RadiusParams& p, const float4& a, const float4& b) {
+__device__ __noinline__ bool exact_within(const RadiusParams& p, const float4 a, const float4 b) {
     const float pa[3] = {a.x, a.y, a.z}, pb[3] = {b.x, b.y, b.z};
     double d2 = 0.0;
 #pragma unroll
@@ -212,199 +215,356 @@ __device__ __noinline__ bool exact_within(const RadiusParams& p, const float4& a
     return d2 <= p.r2_exact;
 }
 
-struct CellWalk {
-    int cs, ce;          // candidate slots [cs, ce)
-    float qs[3];         // subtract from the query coordinate (box length where the neighbour cell wrapped upwards)
-    float js[3];         // subtract from the candidate coordinate (where it wrapped downwards)
+__device__ __forceinline__ float fast_rcp(float x) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+// One warp per query cell.
+//   staging : the candidates of the 27-cell stencil (contiguous ranges of the cell-sorted
+//             positions) are copied once into shared memory in coordinates relative to the
+//             query cell's corner, periodic images already applied.  All subtractions involved
+//             are exact or act on numbers of the size of a cell, so the fp32 displacement is
+//             accurate to a few ulps of the cell size on both sides of a periodic face.
+//   phase A : every lane keeps one staged candidate in registers and tests it against the
+//             queries of the cell, eight queries per batch (their coordinates are broadcast
+//             from shared memory).  Accepted pairs are compacted with a warp ballot into one
+//             contiguous list per query: (source, weight) for the forward messages,
+//             (staged slot, d^2 or weight) where the displacement is needed again.
+//   phase B : MODE 0 (Gaussian / distance forward) and MODE 2 (Gaussian backward): LF lanes
+//             span one feature row with 128-bit accesses and 32 / LF queries advance together,
+//             four gathered rows in flight per lane; MODE 1 (Lennard-Jones): four lanes share
+//             a query's list and evaluate the pair forces.
+// Lists hold QCAP entries per query and the stage STAGE_CAP candidates; when either fills up
+// the warp drains / processes and goes on, so any density works.
+constexpr int STAGE_PAD = 32;           // sentinels behind the staged candidates: no bounds checks
+constexpr int QB = 8;                   // queries per batch
+constexpr float FAR_AWAY = 1.0e18f;
+
+template <int MODE> struct TravSmem {
+    // sized for the workloads' densities (about 216 / 351 candidates, 32 / 54 neighbours);
+    // denser inputs only mean more chunks and drains
+    static constexpr int STAGE_CAP = (MODE == 1) ? 384 : 256;      // candidates staged per chunk
+    static constexpr int QCAP = (MODE == 1) ? 96 : 80;             // list entries per query
+    static constexpr int QSTRIDE = QCAP + 1;                       // odd stride: the lists of different queries fall in different banks
+    static constexpr int STAGE_BYTES = (STAGE_CAP + STAGE_PAD) * 16;
+    static constexpr int LIST_BYTES = (QB * QSTRIDE * 8 + 15) / 16 * 16;
+    static constexpr int MISC_BYTES = QB * 16 + QB * 4 * 2;          // query coordinates, counts, totals
+    static constexpr int PER_WARP = STAGE_BYTES + LIST_BYTES + MISC_BYTES;
 };
 
-// neighbour cell `k` (0..26) of cell (cx,cy,cz); returns false when it does not exist
-__device__ __forceinline__ bool neighbour_cell(const RadiusParams& p, const int c[3], int k, CellWalk* w) {
-    const int off[3] = {k % 3 - 1, (k / 3) % 3 - 1, k / 9 - 1};
-    int q[3];
-#pragma unroll
-    for (int d = 0; d < 3; ++d) {
-        w->qs[d] = 0.f; w->js[d] = 0.f;
-        if (p.nc[d] == 1) {
-            if (off[d] != 0) return false;
-            q[d] = 0;
-            continue;
-        }
-        int v = c[d] + off[d];
-        if (v < 0) {
-            if (!p.periodic[d]) return false;
-            v += p.nc[d]; w->js[d] = p.len[d];
-        } else if (v >= p.nc[d]) {
-            if (!p.periodic[d]) return false;
-            v -= p.nc[d]; w->qs[d] = p.len[d];
-        }
-        q[d] = v;
-    }
-    const int id = (q[2] * p.nc[1] + q[1]) * p.nc[0] + q[0];
-    w->cs = p.cell_start[id];
-    w->ce = p.cell_start[id + 1];
-    return true;
+// exact predicate for the pair of original point ids (a, b)
+__device__ __noinline__ bool exact_pair(const RadiusParams& p, int a, int b) {
+    const float4 pa = make_float4(p.pos[3 * (size_t)a], p.pos[3 * (size_t)a + 1], p.pos[3 * (size_t)a + 2], 0.f);
+    const float4 pb = make_float4(p.pos[3 * (size_t)b], p.pos[3 * (size_t)b + 1], p.pos[3 * (size_t)b + 2], 0.f);
+    return exact_within(p, pa, pb);
 }
 
-// fp32 displacement p_q - p_j (minimum image) and squared distance
-__device__ __forceinline__ float displacement(const RadiusParams& p, const float qsh[3], const float4& pj,
-                                              const CellWalk& w, float D[3]) {
-    const float pjv[3] = {pj.x, pj.y, pj.z};
-#pragma unroll
-    for (int d = 0; d < 3; ++d) {
-        float t = qsh[d] - (pjv[d] - w.js[d]);
-        if (p.periodic[d] && p.nc[d] == 1) t -= p.len[d] * rintf(t * p.inv_len[d]);
-        D[d] = t;
-    }
-    return fmaf(D[2], D[2], fmaf(D[1], D[1], D[0] * D[0]));
-}
-
-// MODE 0: GAUSS/DIST forward   1: LJ forward   2: GAUSS backward
-template <int MODE>
-__global__ void __launch_bounds__(RAD_THREADS) radius_kernel(const RadiusParams p, int kind) {
-    __shared__ int s_id[RAD_WARPS][LIST_CAP];
-    __shared__ float s_g[RAD_WARPS][LIST_CAP];
-    __shared__ float s_d[MODE == 2 ? RAD_WARPS : 1][3][LIST_CAP];
+// MODE 0: Gaussian (DIST = false) or distance-weighted (DIST = true) forward; 1: Lennard-Jones;
+// 2: Gaussian backward.  MI: some periodic dimension has a single cell (explicit minimum image).
+template <int MODE, int LF, bool DIST, bool MI>
+__global__ void __launch_bounds__(TRAV_THREADS) radius_traverse_kernel(const __grid_constant__ RadiusParams p) {
+    using SM = TravSmem<MODE>;
+    constexpr int STAGE_CAP = SM::STAGE_CAP, QCAP = SM::QCAP, QSTRIDE = SM::QSTRIDE;
+    constexpr unsigned FULL = 0xffffffffu;
+    extern __shared__ __align__(16) unsigned char s_raw[];
 
     const int lane = threadIdx.x & 31;
     const int wib = threadIdx.x >> 5;
-    const int cellid = blockIdx.x * RAD_WARPS + wib;
+    const int cellid = blockIdx.x * TRAV_WARPS + wib;
     if (cellid >= p.ncells) return;
-    const int qs = p.cell_start[cellid], qe = p.cell_start[cellid + 1];
-    if (qs == qe) return;
+    const int qs0 = p.cell_start[cellid], qe0 = p.cell_start[cellid + 1];
+    if (qs0 == qe0) return;
+
+    unsigned char* base = s_raw + (size_t)wib * SM::PER_WARP;
+    float4* stage = reinterpret_cast<float4*>(base);
+    float2* list = reinterpret_cast<float2*>(base + SM::STAGE_BYTES);
+    float4* s_q = reinterpret_cast<float4*>(base + SM::STAGE_BYTES + SM::LIST_BYTES);   // local x, y, z, point id
+    int* s_n = reinterpret_cast<int*>(s_q + QB);                                        // list lengths of the drain in progress
+    int* s_tot = s_n + QB;                                                              // neighbours found so far in this chunk
+
     const int c[3] = {cellid % p.nc[0], (cellid / p.nc[0]) % p.nc[1], cellid / (p.nc[0] * p.nc[1])};
+    const float org[3] = {(float)c[0] * p.hcell[0], (float)c[1] * p.hcell[1], (float)c[2] * p.hcell[2]};
     const int F = p.F;
-    const float inv2s2 = (MODE != 1 && kind == TIGA_MSG_GAUSS) ? 1.f / (2.f * p.p0 * p.p0) : 0.f;
-    const float inv_s2 = (MODE == 2) ? 1.f / (p.p0 * p.p0) : 0.f;
+    const float inv2s2 = (MODE != 1 && !DIST) ? 1.f / (2.f * p.p0 * p.p0) : 0.f;
+    const int fl = lane % LF, grp = lane / LF;
+    const bool mi0 = MI && p.periodic[0] && p.nc[0] == 1, mi1 = MI && p.periodic[1] && p.nc[1] == 1, mi2 = MI && p.periodic[2] && p.nc[2] == 1;
+    constexpr int QP = 32 / LF;
+    const bool fvalid = fl * 4 < F;
+    const unsigned lt_mask = (1u << lane) - 1u;
 
-    for (int q = qs; q < qe; ++q) {
-        const float4 pq = p.spos[q];
-        const int oq = __float_as_int(pq.w);
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};     // MODE 0: features lane+32k; MODE 1: Fx,Fy,Fz,e; MODE 2: grad_feat
-        float gp[3] = {0.f, 0.f, 0.f};           // MODE 2: per-lane share of grad_pos
-        float xk[4] = {0.f, 0.f, 0.f, 0.f}, gk[4] = {0.f, 0.f, 0.f, 0.f};
-        if (MODE == 2) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (lane + 32 * k < F) {
-                    xk[k] = p.feat[(size_t)oq * F + lane + 32 * k];
-                    gk[k] = p.gy[(size_t)oq * F + lane + 32 * k];
-                }
+    auto fold = [&](float& dx, float& dy, float& dz) {
+        if (MI) {          // periodic dimension folded into a single cell: explicit minimum image
+            if (mi0) dx -= p.len[0] * rintf(dx * p.inv_len[0]);
+            if (mi1) dy -= p.len[1] * rintf(dy * p.inv_len[1]);
+            if (mi2) dz -= p.len[2] * rintf(dz * p.inv_len[2]);
         }
-        int nacc = 0;      // neighbours found (warp uniform)
-        int fill = 0;      // entries waiting in the list (warp uniform)
+    };
 
-        auto consume = [&]() {
+    // ---- all queries of the cell against the ns candidates currently staged
+    auto process_chunk = [&](const int ns, const bool first_chunk) {
+        if (lane < STAGE_PAD) stage[ns + lane] = make_float4(FAR_AWAY, FAR_AWAY, FAR_AWAY, __int_as_float(-1));
+        for (int qb0 = qs0; qb0 < qe0; qb0 += QB) {
+            const int nq = (qe0 - qb0 < QB) ? qe0 - qb0 : QB;
             __syncwarp();
-            if (MODE == 0) {
-                for (int t = 0; t < fill; ++t) {
-                    const size_t row = (size_t)s_id[wib][t] * F;
-                    const float g = s_g[wib][t];
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (lane + 32 * k < F) acc[k] = fmaf(g, __ldg(p.feat + row + lane + 32 * k), acc[k]);
-                }
-            } else if (MODE == 2) {
-                for (int t = 0; t < fill; ++t) {
-                    const size_t row = (size_t)s_id[wib][t] * F;
-                    const float g = s_g[wib][t];
-                    float part = 0.f;
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (lane + 32 * k < F) {
-                            const float xj = __ldg(p.feat + row + lane + 32 * k);
-                            const float gj = __ldg(p.gy + row + lane + 32 * k);
-                            acc[k] = fmaf(g, gj, acc[k]);
-                            part = fmaf(gk[k], xj, part);
-                            part = fmaf(gj, xk[k], part);
-                        }
-                    const float gpart = g * part;
-#pragma unroll
-                    for (int d = 0; d < 3; ++d) gp[d] = fmaf(gpart, s_d[MODE == 2 ? wib : 0][d][t], gp[d]);
-                }
+            if (lane < nq) {
+                const float4 pq = p.spos[qb0 + lane];
+                s_q[lane] = make_float4(pq.x - org[0], pq.y - org[1], pq.z - org[2], pq.w);
+                s_tot[lane] = 0;
             }
-            fill = 0;
             __syncwarp();
-        };
+            unsigned cnt_lo = 0, cnt_hi = 0;      // eight list lengths, one byte each (never above QCAP < 256)
+            bool first = first_chunk;
 
-        for (int k27 = 0; k27 < 27; ++k27) {
-            CellWalk w;
-            if (!neighbour_cell(p, c, k27, &w)) continue;
-            const float qsh[3] = {pq.x - w.qs[0], pq.y - w.qs[1], pq.z - w.qs[2]};
-            for (int base = w.cs; base < w.ce; base += 32) {
-                const int j = base + lane;
-                bool ok = false;
-                float D[3] = {0.f, 0.f, 0.f};
-                float d2 = 0.f;
-                float4 pj = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (j < w.ce && j != q) {
-                    pj = p.spos[j];
-                    d2 = displacement(p, qsh, pj, w, D);
-                    if (d2 <= p.r2_hi) {
-                        ok = true;
-                        if (d2 > p.r2_lo) ok = exact_within(p, pq, pj);
-                    }
+            auto drain = [&]() {
+                __syncwarp();
+                if (lane < QB) {
+                    const int n = (int)(((lane < 4 ? cnt_lo : cnt_hi) >> (8 * (lane & 3))) & 0xffu);
+                    s_n[lane] = n;
+                    s_tot[lane] += n;
                 }
+                __syncwarp();
                 if (MODE == 1) {
-                    if (ok) {
-                        const float inv = 1.f / d2;
-                        const float qq = p.p1 * p.p1 * inv;
-                        const float q3 = qq * qq * qq;
-                        const float fs = 24.f * p.p0 * (2.f * q3 * q3 - q3) * inv;
-                        acc[0] = fmaf(fs, D[0], acc[0]);
-                        acc[1] = fmaf(fs, D[1], acc[1]);
-                        acc[2] = fmaf(fs, D[2], acc[2]);
-                        acc[3] += 2.f * p.p0 * (q3 * q3 - q3);
-                    }
-                    nacc += __popc(__ballot_sync(0xffffffffu, ok));
-                } else {
-                    const unsigned m = __ballot_sync(0xffffffffu, ok);
-                    if (ok) {
-                        const int slot = fill + __popc(m & ((1u << lane) - 1u));
-                        s_id[wib][slot] = __float_as_int(pj.w);
-                        s_g[wib][slot] = (kind == TIGA_MSG_GAUSS) ? __expf(-d2 * inv2s2) : sqrtf(d2);
-                        if (MODE == 2) {
-                            s_d[MODE == 2 ? wib : 0][0][slot] = D[0];
-                            s_d[MODE == 2 ? wib : 0][1][slot] = D[1];
-                            s_d[MODE == 2 ? wib : 0][2][slot] = D[2];
+                    // four lanes per query
+                    const int q = lane >> 2, sub = lane & 3;
+                    float fx = 0.f, fy = 0.f, fz = 0.f, en = 0.f;
+                    if (q < nq) {
+                        const float4 qv = s_q[q];
+                        const int n = s_n[q];
+                        const float s2 = p.p1 * p.p1, e24 = 24.f * p.p0, e2x = 2.f * p.p0;
+                        const float2* lq = list + q * QSTRIDE;
+                        for (int t = sub; t < n; t += 8) {
+                            float2 e[2];
+                            float4 pj[2];
+#pragma unroll
+                            for (int u = 0; u < 2; ++u) {
+                                e[u] = lq[t + 4 * u < n ? t + 4 * u : t];
+                                pj[u] = stage[__float_as_int(e[u].x)];
+                            }
+#pragma unroll
+                            for (int u = 0; u < 2; ++u) {
+                                const float inv = (t + 4 * u < n) ? fast_rcp(e[u].y) : 0.f;      // 0 switches the pair off
+                                const float qq = s2 * inv;
+                                const float q3 = qq * qq * qq;
+                                const float fs = e24 * (2.f * q3 * q3 - q3) * inv;
+                                float dx = qv.x - pj[u].x, dy = qv.y - pj[u].y, dz = qv.z - pj[u].z;
+                                fold(dx, dy, dz);
+                                fx = fmaf(fs, dx, fx); fy = fmaf(fs, dy, fy); fz = fmaf(fs, dz, fz);
+                                en = fmaf(e2x, q3 * q3 - q3, en);
+                            }
                         }
                     }
-                    const int add = __popc(m);
-                    fill += add;
-                    nacc += add;
-                    if (fill > LIST_CAP - 32) consume();
+#pragma unroll
+                    for (int o = 1; o <= 2; o <<= 1) {
+                        fx += __shfl_xor_sync(FULL, fx, o); fy += __shfl_xor_sync(FULL, fy, o);
+                        fz += __shfl_xor_sync(FULL, fz, o); en += __shfl_xor_sync(FULL, en, o);
+                    }
+                    if (q < nq && sub == 0) {
+                        float4* o = reinterpret_cast<float4*>(p.out) + __float_as_int(s_q[q].w);
+                        float4 a = make_float4(fx, fy, fz, en);
+                        if (!first) { const float4 old = *o; a.x += old.x; a.y += old.y; a.z += old.z; a.w += old.w; }
+                        *o = a;
+                    }
+                } else {
+                    for (int pass = 0; pass * QP < nq; ++pass) {
+                        const int qq = pass * QP + grp;
+                        const bool valid = qq < nq && fvalid;
+                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        float px = 0.f, py = 0.f, pz = 0.f;
+                        int oqq = 0;
+                        if (valid) {
+                            const float4 qv = s_q[qq];
+                            oqq = __float_as_int(qv.w);
+                            const int n = s_n[qq];
+                            const float2* lq = list + qq * QSTRIDE;
+                            if (MODE == 0) {
+                                for (int t = 0; t < n; t += 4) {
+                                    float2 e[4];
+                                    float4 x[4];
+#pragma unroll
+                                    for (int u = 0; u < 4; ++u) {      // four gathered rows in flight
+                                        e[u] = lq[t + u < n ? t + u : t];
+                                        if (t + u >= n) e[u].y = 0.f;
+                                        x[u] = __ldg(reinterpret_cast<const float4*>(p.feat + (size_t)__float_as_int(e[u].x) * F) + fl);
+                                    }
+#pragma unroll
+                                    for (int u = 0; u < 4; ++u) {
+                                        acc.x = fmaf(e[u].y, x[u].x, acc.x); acc.y = fmaf(e[u].y, x[u].y, acc.y);
+                                        acc.z = fmaf(e[u].y, x[u].z, acc.z); acc.w = fmaf(e[u].y, x[u].w, acc.w);
+                                    }
+                                }
+                            } else {
+                                const float4 xk = __ldg(reinterpret_cast<const float4*>(p.feat + (size_t)oqq * F) + fl);
+                                const float4 gk = __ldg(reinterpret_cast<const float4*>(p.gy + (size_t)oqq * F) + fl);
+                                for (int t = 0; t < n; t += 2) {
+                                    float4 e[2], xj[2], gj[2];
+                                    float g[2];
+#pragma unroll
+                                    for (int u = 0; u < 2; ++u) {
+                                        const float2 en2 = lq[t + u < n ? t + u : t];
+                                        g[u] = (t + u < n) ? en2.y : 0.f;
+                                        const float4 pj = stage[__float_as_int(en2.x)];
+                                        float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
+                                        fold(dx, dy, dz);
+                                        e[u] = make_float4(dx, dy, dz, 0.f);
+                                        const size_t row = (size_t)__float_as_int(pj.w) * F;
+                                        xj[u] = __ldg(reinterpret_cast<const float4*>(p.feat + row) + fl);
+                                        gj[u] = __ldg(reinterpret_cast<const float4*>(p.gy + row) + fl);
+                                    }
+#pragma unroll
+                                    for (int u = 0; u < 2; ++u) {
+                                        acc.x = fmaf(g[u], gj[u].x, acc.x); acc.y = fmaf(g[u], gj[u].y, acc.y);
+                                        acc.z = fmaf(g[u], gj[u].z, acc.z); acc.w = fmaf(g[u], gj[u].w, acc.w);
+                                        float part = gk.x * xj[u].x;
+                                        part = fmaf(gk.y, xj[u].y, part); part = fmaf(gk.z, xj[u].z, part); part = fmaf(gk.w, xj[u].w, part);
+                                        part = fmaf(gj[u].x, xk.x, part); part = fmaf(gj[u].y, xk.y, part);
+                                        part = fmaf(gj[u].z, xk.z, part); part = fmaf(gj[u].w, xk.w, part);
+                                        const float gpart = g[u] * part;
+                                        px = fmaf(gpart, e[u].x, px); py = fmaf(gpart, e[u].y, py); pz = fmaf(gpart, e[u].z, pz);
+                                    }
+                                }
+                            }
+                            float* orow = (MODE == 0 ? p.out : p.gfeat);
+                            if (orow) {
+                                float4* o = reinterpret_cast<float4*>(orow + (size_t)oqq * F) + fl;
+                                if (!first) { const float4 old = *o; acc.x += old.x; acc.y += old.y; acc.z += old.z; acc.w += old.w; }
+                                *o = acc;
+                            }
+                        }
+                        if (MODE == 2) {
+#pragma unroll
+                            for (int o = LF / 2; o > 0; o >>= 1) {
+                                px += __shfl_xor_sync(FULL, px, o);
+                                py += __shfl_xor_sync(FULL, py, o);
+                                pz += __shfl_xor_sync(FULL, pz, o);
+                            }
+                            if (p.gpos && qq < nq && fl == 0) {
+                                const float sc = -1.f / (p.p0 * p.p0);
+                                float* o = p.gpos + 3 * (size_t)oqq;
+                                if (first) { o[0] = sc * px; o[1] = sc * py; o[2] = sc * pz; }
+                                else { o[0] += sc * px; o[1] += sc * py; o[2] += sc * pz; }
+                            }
+                        }
+                    }
                 }
-            }
-        }
-        if (MODE != 1 && fill > 0) consume();
+                cnt_lo = 0; cnt_hi = 0;
+                first = false;
+                __syncwarp();
+            };
 
-        if (MODE == 0) {
+            // ---- phase A: one staged candidate per lane against the queries of the batch
+            constexpr unsigned DRAIN_AT = (unsigned)(QCAP - 32) * 0x01010101u;
+            for (int cbase = 0; cbase < ns; cbase += 32) {
+                const float4 pj = stage[cbase + lane];
+                const int idj = __float_as_int(pj.w);
+                float d2q[QB];
+                bool suspect = false;
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (lane + 32 * k < F) p.out[(size_t)oq * F + lane + 32 * k] = acc[k];
-        } else if (MODE == 1) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], o);
-            if (lane == 0) reinterpret_cast<float4*>(p.out)[oq] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-        } else {
-            if (p.gfeat) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    if (lane + 32 * k < F) p.gfeat[(size_t)oq * F + lane + 32 * k] = acc[k];
-            }
-            if (p.gpos) {
-#pragma unroll
-                for (int d = 0; d < 3; ++d) {
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) gp[d] += __shfl_xor_sync(0xffffffffu, gp[d], o);
+                for (int q = 0; q < QB; ++q) {
+                    if (q >= nq) break;
+                    const float4 qv = s_q[q];
+                    float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
+                    fold(dx, dy, dz);
+                    float d2 = fmaf(dz, dz, fmaf(dy, dy, dx * dx));
+                    if (idj == __float_as_int(qv.w) || (MI && idj < 0)) d2 = FAR_AWAY;     // self (by index); folded sentinels
+                    suspect = suspect || (d2 > p.r2_lo && d2 <= p.r2_hi);
+                    d2q[q] = d2;
                 }
-                if (lane < 3) p.gpos[3 * (size_t)oq + lane] = -inv_s2 * (lane == 0 ? gp[0] : (lane == 1 ? gp[1] : gp[2]));
+                unsigned fix = 0;     // pairs inside the fp32 band that the fp64 predicate accepts
+                if (__any_sync(FULL, suspect)) {
+#pragma unroll
+                    for (int q = 0; q < QB; ++q) {
+                        if (q >= nq) break;
+                        if (d2q[q] > p.r2_lo && d2q[q] <= p.r2_hi && exact_pair(p, __float_as_int(s_q[q].w), idj)) fix |= 1u << q;
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < QB; ++q) {
+                    if (q >= nq) break;
+                    const bool ok = d2q[q] <= p.r2_lo || ((fix >> q) & 1u);
+                    const unsigned m = __ballot_sync(FULL, ok);
+                    float val;
+                    if (MODE == 1) val = d2q[q];
+                    else val = DIST ? sqrtf(d2q[q]) : __expf(-d2q[q] * inv2s2);
+                    const unsigned have = ((q < 4 ? cnt_lo : cnt_hi) >> (8 * (q & 3))) & 0xffu;
+                    float2* dst = list + q * QSTRIDE + have + __popc(m & lt_mask);
+                    if (ok) *dst = make_float2(MODE == 0 ? pj.w : __int_as_float(cbase + lane), val);
+                    if (q < 4) cnt_lo += (unsigned)__popc(m) << (8 * (q & 3));
+                    else cnt_hi += (unsigned)__popc(m) << (8 * (q & 3));
+                }
+                if ((__vcmpgtu4(cnt_lo, DRAIN_AT) | __vcmpgtu4(cnt_hi, DRAIN_AT)) != 0u) drain();
+            }
+            drain();      // on the first chunk this also writes the zero vector of a query without neighbours
+            if (p.count && lane < nq) {
+                const int oq = __float_as_int(s_q[lane].w);
+                p.count[oq] = first_chunk ? s_tot[lane] : p.count[oq] + s_tot[lane];
             }
         }
-        if (p.count && lane == 0) p.count[oq] = nacc;
+        __syncwarp();
+    };
+
+    // ---- the 27-cell stencil as candidate ranges: lane r < 27 resolves neighbour offset r
+    int r_cs = 0, r_ce = 0;
+    float r_off[3] = {0.f, 0.f, 0.f};
+    {
+        const int off[3] = {lane % 3 - 1, (lane / 3) % 3 - 1, lane / 9 - 1};
+        bool ok = lane < 27;
+        int q[3] = {0, 0, 0};
+        bool merged = false;
+#pragma unroll
+        for (int d = 0; d < 3; ++d) {
+            if (p.nc[d] == 1) { ok = ok && off[d] == 0; r_off[d] = org[d]; continue; }
+            if (d == 0 && c[0] >= 1 && c[0] <= p.nc[0] - 2) {
+                // away from the x faces the three x-adjacent cells are one contiguous range
+                merged = true; ok = ok && off[0] == 0; q[0] = c[0] - 1; r_off[0] = org[0];
+                continue;
+            }
+            int v = c[d] + off[d];
+            r_off[d] = org[d];
+            if (v < 0) {
+                if (p.periodic[d]) { v += p.nc[d]; r_off[d] = org[d] + p.len[d]; }     // org is 0 here: exact
+                else ok = false;
+            } else if (v >= p.nc[d]) {
+                if (p.periodic[d]) { v -= p.nc[d]; r_off[d] = org[d] - p.len[d]; }     // exact (Sterbenz)
+                else ok = false;
+            }
+            q[d] = v;
+        }
+        if (ok) {
+            const int id = (q[2] * p.nc[1] + q[1]) * p.nc[0] + q[0];
+            r_cs = p.cell_start[id];
+            r_ce = p.cell_start[id + (merged ? 3 : 1)];
+        }
     }
+    unsigned live = __ballot_sync(FULL, r_ce > r_cs);
+    int ns = 0;
+    bool first_chunk = true;
+    while (live) {
+        const int r = __ffs(live) - 1;
+        live &= live - 1;
+        const int cs = __shfl_sync(FULL, r_cs, r), ce = __shfl_sync(FULL, r_ce, r);
+        const float ox = __shfl_sync(FULL, r_off[0], r), oy = __shfl_sync(FULL, r_off[1], r), oz = __shfl_sync(FULL, r_off[2], r);
+        int pos = cs;
+        while (pos < ce) {
+            int take = ce - pos;
+            take = take < STAGE_CAP - ns ? take : STAGE_CAP - ns;
+            for (int k = lane; k < take; k += 32) {
+                const float4 v = __ldg(p.spos + pos + k);
+                stage[ns + k] = make_float4(v.x - ox, v.y - oy, v.z - oz, v.w);
+            }
+            ns += take;
+            pos += take;
+            if (ns == STAGE_CAP) {
+                __syncwarp();
+                process_chunk(ns, first_chunk);
+                first_chunk = false;
+                ns = 0;
+            }
+        }
+    }
+    __syncwarp();
+    if (ns > 0 || first_chunk) process_chunk(ns, first_chunk);
 }
 
 // ------------------------------------------------------------------------------ host side
@@ -464,12 +624,13 @@ static tiga_status fill_params(RadiusParams* p, long long n, float r, const tiga
     for (int d = 0; d < 3; ++d) {
         p->nc[d] = nc[d]; p->invh[d] = invh[d];
         p->len[d] = box->len[d]; p->inv_len[d] = 1.f / box->len[d];
+        p->hcell[d] = box->len[d] / (float)nc[d];
         p->periodic[d] = box->periodic[d] ? 1 : 0;
         if (p->periodic[d] && nc[d] == 1) single_periodic = true;
     }
     p->ncells = nc[0] * nc[1] * nc[2];
     const float r2 = r * r;
-    const float beta = (single_periodic ? 64.f : 16.f) * 5.9604645e-8f;
+    const float beta = (single_periodic ? 96.f : 32.f) * 5.9604645e-8f;
     p->r2_lo = r2 * (1.f - beta);
     p->r2_hi = r2 * (1.f + beta);
     p->r2_exact = (double)r * (double)r;
@@ -487,6 +648,41 @@ static tiga_status run_binning(RadiusParams& p, int32_t* fill, int nblocks, cuda
     bin_scatter_kernel<<<pb, 256, 0, s>>>(p, fill);
     bin_sort_kernel<<<(unsigned)(((size_t)p.ncells * 32 + 255) / 256), 256, 0, s>>>(p);
     return launch_status();
+}
+
+static int feature_lanes(int F) {
+    int lf = 1;
+    while (lf * 4 < F) lf <<= 1;
+    return lf;
+}
+
+template <int MODE, int LF, bool DIST, bool MI>
+static tiga_status launch_traverse_t(const RadiusParams& p, cudaStream_t s) {
+    const unsigned blocks = (unsigned)((p.ncells + TRAV_WARPS - 1) / TRAV_WARPS);
+    constexpr int smem = TravSmem<MODE>::PER_WARP * TRAV_WARPS;
+    auto kern = radius_traverse_kernel<MODE, LF, DIST, MI>;
+    if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    kern<<<blocks, TRAV_THREADS, smem, s>>>(p);
+    return launch_status();
+}
+
+template <int MODE, bool DIST, bool MI>
+static tiga_status launch_traverse_lf(const RadiusParams& p, cudaStream_t s) {
+    switch (MODE == 1 ? 1 : feature_lanes(p.F)) {
+        case 1: return launch_traverse_t<MODE, 1, DIST, MI>(p, s);
+        case 2: return launch_traverse_t<MODE, 2, DIST, MI>(p, s);
+        case 4: return launch_traverse_t<MODE, 4, DIST, MI>(p, s);
+        case 8: return launch_traverse_t<MODE, 8, DIST, MI>(p, s);
+        case 16: return launch_traverse_t<MODE, 16, DIST, MI>(p, s);
+        default: return launch_traverse_t<MODE, 32, DIST, MI>(p, s);
+    }
+}
+
+template <int MODE, bool DIST>
+static tiga_status launch_traverse(const RadiusParams& p, cudaStream_t s) {
+    bool mi = false;
+    for (int d = 0; d < 3; ++d) mi = mi || (p.periodic[d] && p.nc[d] == 1);
+    return mi ? launch_traverse_lf<MODE, DIST, true>(p, s) : launch_traverse_lf<MODE, DIST, false>(p, s);
 }
 
 }  // namespace tiga
@@ -571,10 +767,9 @@ extern "C" tiga_status tiga_apply_radius(const float* pos, const float* feat, in
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     st = run_binning(p, fill, lay.nblocks, s);
     if (st != TIGA_OK) return st;
-    const unsigned blocks = (unsigned)((p.ncells + RAD_WARPS - 1) / RAD_WARPS);
-    if (msg->kind == TIGA_MSG_LJ) radius_kernel<1><<<blocks, RAD_THREADS, 0, s>>>(p, msg->kind);
-    else radius_kernel<0><<<blocks, RAD_THREADS, 0, s>>>(p, msg->kind);
-    return launch_status();
+    if (msg->kind == TIGA_MSG_LJ) return launch_traverse<1, false>(p, s);
+    if (msg->kind == TIGA_MSG_DIST) return launch_traverse<0, true>(p, s);
+    return launch_traverse<0, false>(p, s);
 }
 
 extern "C" tiga_status tiga_apply_radius_backward(const float* pos, const float* feat, int64_t n, int32_t F,
@@ -597,7 +792,5 @@ extern "C" tiga_status tiga_apply_radius_backward(const float* pos, const float*
         st = run_binning(p, fill, lay.nblocks, s);
         if (st != TIGA_OK) return st;
     }
-    const unsigned blocks = (unsigned)((p.ncells + RAD_WARPS - 1) / RAD_WARPS);
-    radius_kernel<2><<<blocks, RAD_THREADS, 0, s>>>(p, msg->kind);
-    return launch_status();
+    return launch_traverse<2, false>(p, s);
 }

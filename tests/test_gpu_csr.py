@@ -214,3 +214,20 @@ def test_cfg1_full_size(tiga):
     hist, mx = tiga.tiga_csr_degree_histogram(g, 4096)
     ref, rmx = oracle.degree_histogram(c["rowptr"], 4096)
     assert np.array_equal(host(hist), ref) and int(host(mx)[0]) == rmx
+
+
+def test_cfg4_full_size(tiga):
+    """R-MAT scale 26, 2^30 edges, int64 rowptr, F=8 fp16 features, unit weights, fp32 output:
+    every output element against the oracle, and the degree histogram bit-exactly."""
+    c = gen.config("cfg4")
+    assert c["E"] == 1 << 30 and c["rowptr"].dtype == np.int64
+    g = _relation(tiga, c["rowptr"], c["col"], c["n"], index64=True)
+    xd = dev(c["x"], torch)
+    out, _ = tiga.tiga_apply_csr(g, xd, None, tiga.SUM)
+    hist, mx = tiga.tiga_csr_degree_histogram(g, 4096)
+    torch.cuda.synchronize()
+    out = host(out)
+    ref, rmx = oracle.degree_histogram(c["rowptr"], 4096)
+    assert np.array_equal(host(hist), ref) and int(host(mx)[0]) == rmx
+    y, A, _ = oracle.csr_forward(c["rowptr"], c["col"], c["x"], None, oracle.SUM)
+    assert rel_err(out, y, A) <= SUM_TOL
