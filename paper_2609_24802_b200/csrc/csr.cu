@@ -91,7 +91,10 @@ struct Tile {
 };
 
 // Stage the tile: s_ptr[k] = clamp(rowptr[i0+k] - e0, -1, ne+1) for k = 0..nrows, col and w.
-template <typename IT>
+// index with one pad word per 32: threads that read consecutive runs of 8 stay conflict free
+__device__ __forceinline__ int pad32(int i) { return i + (i >> 5); }
+
+template <typename IT, bool PADDED = false>
 __device__ Tile stage_tile(const CsrParams& p, int* s_ptr, int* s_col, float* s_w, long long* s_coord) {
     const IT* rowptr = static_cast<const IT*>(p.rowptr);
     const long long total = p.n_dst + p.n_edges;
@@ -123,8 +126,9 @@ __device__ Tile stage_tile(const CsrParams& p, int* s_ptr, int* s_col, float* s_
         s_ptr[k] = (int)v;
     }
     for (int k = threadIdx.x; k < t.ne; k += CSR_THREADS) {
-        s_col[k] = ld_stream(p.col + t.e0 + k);
-        if (p.w) s_w[k] = ld_stream(p.w + t.e0 + k);
+        const int kk = PADDED ? pad32(k) : k;
+        s_col[kk] = ld_stream(p.col + t.e0 + k);
+        if (p.w) s_w[kk] = ld_stream(p.w + t.e0 + k);
     }
     __syncthreads();
     return t;
@@ -332,6 +336,209 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_forward_kernel(const CsrParam
                     if constexpr (RED != 0) p.carry_arg[o + k] = st.a[i][k];
                 }
             }
+        }
+    }
+}
+
+// --------------------------------------------------------------------------------------------
+// Forward for narrow rows (one or two 16-byte vectors per feature row, e.g. F = 8 fp16).
+// A worker of G lanes would leave most of a warp idle here, so every THREAD owns IPT
+// consecutive items of the tile's merged "row ends + edges" sequence and walks them in order
+// with its reducer state in registers (all its gathers are issued up front).  Rows wholly
+// inside a thread's items are stored directly; the state of the row that is open at the end
+// of a thread's items is combined across threads by a segmented scan (warp shuffles, then the
+// eight warp totals), which hands every thread the partial state of the row that was already
+// open when its items began.  Merging stays in edge order, so results are reproducible.
+// --------------------------------------------------------------------------------------------
+constexpr int NARROW_IPT = CSR_TILE / CSR_THREADS;
+
+template <typename XT, int NV, int RED, typename IT>
+__global__ void __launch_bounds__(CSR_THREADS) csr_forward_narrow_kernel(const CsrParams p) {
+    constexpr int VW = XTraits<XT>::VW;
+    constexpr int IPT = NARROW_IPT;
+    constexpr int U = IPT / NV;                  // gathers in flight per thread
+    constexpr int NWARP = CSR_THREADS / 32;
+    constexpr unsigned FULL = 0xffffffffu;
+    using St = State<RED, NV, VW>;
+
+    __shared__ int s_ptr[CSR_TILE + 2];
+    __shared__ int s_col[CSR_TILE + CSR_TILE / 32 + 1];
+    __shared__ float s_w[CSR_TILE + CSR_TILE / 32 + 1];
+    __shared__ long long s_coord[2];
+    __shared__ int s_start[CSR_THREADS + 1];
+    __shared__ float s_tv[2][NWARP][NV * VW];     // [0] inclusive warp totals, [1] exclusive prefixes over warps
+    __shared__ int s_ta[2][NWARP][RED ? NV * VW : 1];
+    __shared__ int s_tf[2][NWARP];
+
+    const Tile t = stage_tile<IT, true>(p, s_ptr, s_col, s_w, s_coord);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool has_w = p.w != nullptr;
+    const uint4* __restrict__ xbase = static_cast<const uint4*>(p.x);
+    const int total = t.nfin + t.ne;
+
+    // merge coordinates of this thread's first item: rows finished before diagonal d
+    const int d0 = tid * IPT < total ? tid * IPT : total;
+    const int d1 = (tid + 1) * IPT < total ? (tid + 1) * IPT : total;
+    {
+        int lo = 0, hi = t.nfin;
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (s_ptr[mid + 1] + mid + 1 <= d0) lo = mid + 1; else hi = mid;
+        }
+        s_start[tid] = lo;
+        if (tid == 0) s_start[CSR_THREADS] = t.nfin;
+    }
+    __syncthreads();
+    const int r0 = s_start[tid], r1 = s_start[tid + 1];
+    const int ea = d0 - r0, eb = d1 - r1;         // this thread's edges [ea, eb), rows to finish [r0, r1)
+
+    auto store_row = [&](long long row, const St& s) {
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            float* o = p.out + row * p.F + (size_t)i * VW;
+#pragma unroll
+            for (int k = 0; k < VW; k += 4)
+                st_stream(reinterpret_cast<float4*>(o + k), make_float4(s.v[i][k], s.v[i][k + 1], s.v[i][k + 2], s.v[i][k + 3]));
+            if constexpr (RED != 0) {
+                int* ao = p.arg + row * p.F + (size_t)i * VW;
+#pragma unroll
+                for (int k = 0; k < VW; k += 4)
+                    st_stream(reinterpret_cast<int4*>(ao + k), make_int4(s.a[i][k], s.a[i][k + 1], s.a[i][k + 2], s.a[i][k + 3]));
+            }
+        }
+    };
+    // fold a partial state that comes EARLIER in edge order into s
+    auto merge_earlier = [&](St& s, int i, int k, float ov, int oa) {
+        if constexpr (RED == 0) {
+            s.v[i][k] = ov + s.v[i][k];
+        } else {
+            if (oa >= 0 && (s.a[i][k] < 0 || !(s.v[i][k] > ov))) { s.v[i][k] = ov; s.a[i][k] = oa; }
+        }
+    };
+
+    St st, head;
+    st.reset();
+    head.reset();
+    int row = r0, hrow = -1;
+    bool head_open = false;
+    if (ea < eb || r0 < r1) {
+        int cur_end = row < t.nrows ? s_ptr[row + 1] : 0x7fffffff;
+        head_open = (s_ptr[row] < 0 ? 0 : s_ptr[row]) < ea;
+        auto finish_row = [&]() {
+            if (head_open) { head = st; hrow = row; head_open = false; }
+            else store_row(t.i0 + row, st);
+            st.reset();
+            ++row;
+            cur_end = row < t.nrows ? s_ptr[row + 1] : 0x7fffffff;
+        };
+#pragma unroll
+        for (int ub = 0; ub < IPT; ub += U) {
+            uint4 xv[U][NV];
+            float wv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int e = ea + ub + u < eb ? ea + ub + u : (eb > ea ? eb - 1 : 0);
+                const long long c = (ea < eb) ? s_col[pad32(e)] : 0;
+                wv[u] = (has_w && ea < eb) ? s_w[pad32(e)] : 1.f;
+#pragma unroll
+                for (int i = 0; i < NV; ++i) xv[u][i] = (ea + ub + u < eb) ? __ldg(xbase + c * p.nvec + i) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int e = ea + ub + u;
+                if (e < eb) {
+                    while (e >= cur_end) finish_row();
+                    float xf[VW];
+#pragma unroll
+                    for (int i = 0; i < NV; ++i) {
+                        XTraits<XT>::unpack(xv[u][i], xf);
+#pragma unroll
+                        for (int k = 0; k < VW; ++k) st.message(i, k, wv[u], xf[k], (int)(t.e0 + e));
+                    }
+                }
+            }
+        }
+        while (row < r1) finish_row();
+    }
+    // st is now the state of the row that is open after this thread's items (identity if none);
+    // it restarts the scan unless the thread lies wholly inside a row that began before it
+    int flag = head_open ? 0 : ((ea < eb || r0 < r1) ? 1 : 0);
+    St inc = st;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int of = __shfl_up_sync(FULL, flag, o);
+#pragma unroll
+        for (int i = 0; i < NV; ++i)
+#pragma unroll
+            for (int k = 0; k < VW; ++k) {
+                const float ov = __shfl_up_sync(FULL, inc.v[i][k], o);
+                int oa = 0;
+                if constexpr (RED != 0) oa = __shfl_up_sync(FULL, inc.a[i][k], o);
+                if (lane >= o && !flag) merge_earlier(inc, i, k, ov, oa);
+            }
+        if (lane >= o) flag |= of;
+    }
+    if (lane == 31) {
+#pragma unroll
+        for (int i = 0; i < NV; ++i)
+#pragma unroll
+            for (int k = 0; k < VW; ++k) {
+                s_tv[0][warp][i * VW + k] = inc.v[i][k];
+                if constexpr (RED != 0) s_ta[0][warp][i * VW + k] = inc.a[i][k];
+            }
+        s_tf[0][warp] = flag;
+    }
+    __syncthreads();
+    if (tid < NV * VW) {
+        // exclusive scan over the eight warp totals, one feature per thread
+        float v = 0.f;
+        int a = -1;
+        for (int w2 = 0; w2 < NWARP; ++w2) {
+            s_tv[1][w2][tid] = v;
+            if constexpr (RED != 0) s_ta[1][w2][tid] = a;
+            const float tv = s_tv[0][w2][tid];
+            const int ta = RED ? s_ta[0][w2][RED ? tid : 0] : 0;
+            if (s_tf[0][w2]) { v = tv; a = ta; }
+            else if constexpr (RED == 0) v = v + tv;
+            else { if (ta >= 0 && (a < 0 || tv > v)) { v = tv; a = ta; } }
+        }
+    }
+    __syncthreads();
+    // exclusive prefix of this thread: the open row's state contributed by earlier threads
+    St pre;
+    const int ef = __shfl_up_sync(FULL, flag, 1);
+#pragma unroll
+    for (int i = 0; i < NV; ++i)
+#pragma unroll
+        for (int k = 0; k < VW; ++k) {
+            float ev = __shfl_up_sync(FULL, inc.v[i][k], 1);
+            int ea2 = -1;
+            if constexpr (RED != 0) ea2 = __shfl_up_sync(FULL, inc.a[i][k], 1);
+            if (lane == 0) { ev = 0.f; ea2 = -1; }
+            pre.v[i][k] = ev;
+            if constexpr (RED != 0) pre.a[i][k] = ea2;
+            if (lane == 0 || !ef) merge_earlier(pre, i, k, s_tv[1][warp][i * VW + k], RED ? s_ta[1][warp][RED ? i * VW + k : 0] : 0);
+        }
+    if (hrow >= 0) {
+#pragma unroll
+        for (int i = 0; i < NV; ++i)
+#pragma unroll
+            for (int k = 0; k < VW; ++k) merge_earlier(head, i, k, pre.v[i][k], RED ? pre.a[RED ? i : 0][RED ? k : 0] : 0);
+        store_row(t.i0 + hrow, head);
+    }
+    if (tid == CSR_THREADS - 1) {
+        // trailing unfinished row of the tile -> carry-out (inclusive value at the last thread)
+        const bool open = t.nrows > t.nfin && t.ne > (s_ptr[t.nfin] < 0 ? 0 : s_ptr[t.nfin]);
+        p.carry_row[blockIdx.x] = open ? (int32_t)(t.i0 + t.nfin) : -1;
+        if (open) {
+#pragma unroll
+            for (int i = 0; i < NV; ++i)
+#pragma unroll
+                for (int k = 0; k < VW; ++k) {
+                    if (!flag) merge_earlier(inc, i, k, s_tv[1][warp][i * VW + k], RED ? s_ta[1][warp][RED ? i * VW + k : 0] : 0);
+                    p.carry_val[(size_t)blockIdx.x * p.F + i * VW + k] = inc.v[i][k];
+                    if constexpr (RED != 0) p.carry_arg[(size_t)blockIdx.x * p.F + i * VW + k] = inc.a[i][k];
+                }
         }
     }
 }
@@ -551,6 +758,8 @@ static tiga_status launch_fwd_t(const CsrParams& p, cudaStream_t s) {
 
 template <typename XT, int RED, typename IT>
 static tiga_status launch_fwd_g(const CsrParams& p, int G, int VPL, cudaStream_t s) {
+    if (p.nvec == 1) { csr_forward_narrow_kernel<XT, 1, RED, IT><<<(unsigned)p.ntiles, CSR_THREADS, 0, s>>>(p); return launch_status(); }
+    if (p.nvec == 2) { csr_forward_narrow_kernel<XT, 2, RED, IT><<<(unsigned)p.ntiles, CSR_THREADS, 0, s>>>(p); return launch_status(); }
     switch (G) {
         case 1: return launch_fwd_t<XT, 1, 1, RED, IT>(p, s);
         case 2: return launch_fwd_t<XT, 2, 1, RED, IT>(p, s);
