@@ -22,6 +22,7 @@
 // face, which is exact in fp32, so wrapped pairs are as accurate as interior ones.
 #include "common.cuh"
 #include <math.h>
+#include <type_traits>
 
 namespace tiga {
 
@@ -40,6 +41,7 @@ struct RadiusParams {
     int F;
     float r;
     float r2_lo, r2_hi;       // fp32 filter band around r^2
+    float r2_mid, r2_band;    // its centre and half width
     double r2_exact;          // (double)r * (double)r
     float len[3];
     float inv_len[3];
@@ -215,6 +217,12 @@ __device__ __noinline__ bool exact_within(const RadiusParams& p, const float4 a,
     return d2 <= p.r2_exact;
 }
 
+__device__ __forceinline__ float fast_exp2(float x) {
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
 __device__ __forceinline__ float fast_rcp(float x) {
     float r;
     asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
@@ -287,7 +295,7 @@ __global__ void __launch_bounds__(TRAV_THREADS) radius_traverse_kernel(const __g
     const int c[3] = {cellid % p.nc[0], (cellid / p.nc[0]) % p.nc[1], cellid / (p.nc[0] * p.nc[1])};
     const float org[3] = {(float)c[0] * p.hcell[0], (float)c[1] * p.hcell[1], (float)c[2] * p.hcell[2]};
     const int F = p.F;
-    const float inv2s2 = (MODE != 1 && !DIST) ? 1.f / (2.f * p.p0 * p.p0) : 0.f;
+    const float neg_c2 = (MODE != 1 && !DIST) ? -1.4426950408889634f / (2.f * p.p0 * p.p0) : 0.f;   // exp(-d2/(2 s^2)) = 2^(d2 * neg_c2)
     const int fl = lane % LF, grp = lane / LF;
     const bool mi0 = MI && p.periodic[0] && p.nc[0] == 1, mi1 = MI && p.periodic[1] && p.nc[1] == 1, mi2 = MI && p.periodic[2] && p.nc[2] == 1;
     constexpr int QP = 32 / LF;
@@ -314,15 +322,16 @@ __global__ void __launch_bounds__(TRAV_THREADS) radius_traverse_kernel(const __g
                 s_tot[lane] = 0;
             }
             __syncwarp();
-            unsigned cnt_lo = 0, cnt_hi = 0;      // eight list lengths, one byte each (never above QCAP < 256)
+            int qcnt[QB];                         // list lengths (warp uniform, kept in registers)
+#pragma unroll
+            for (int q = 0; q < QB; ++q) qcnt[q] = 0;
             bool first = first_chunk;
 
             auto drain = [&]() {
                 __syncwarp();
-                if (lane < QB) {
-                    const int n = (int)(((lane < 4 ? cnt_lo : cnt_hi) >> (8 * (lane & 3))) & 0xffu);
-                    s_n[lane] = n;
-                    s_tot[lane] += n;
+                if (lane == 0) {
+#pragma unroll
+                    for (int q = 0; q < QB; ++q) { s_n[q] = qcnt[q]; s_tot[q] += qcnt[q]; }
                 }
                 __syncwarp();
                 if (MODE == 1) {
@@ -448,54 +457,65 @@ __global__ void __launch_bounds__(TRAV_THREADS) radius_traverse_kernel(const __g
                         }
                     }
                 }
-                cnt_lo = 0; cnt_hi = 0;
+#pragma unroll
+                for (int q = 0; q < QB; ++q) qcnt[q] = 0;
                 first = false;
                 __syncwarp();
             };
 
             // ---- phase A: one staged candidate per lane against the queries of the batch
-            constexpr unsigned DRAIN_AT = (unsigned)(QCAP - 32) * 0x01010101u;
-            for (int cbase = 0; cbase < ns; cbase += 32) {
+            auto phase_a = [&](const int cbase, auto full_batch) -> bool {
+                constexpr bool FULLB = decltype(full_batch)::value;     // all QB queries present: no trip tests
                 const float4 pj = stage[cbase + lane];
                 const int idj = __float_as_int(pj.w);
                 float d2q[QB];
-                bool suspect = false;
+                float nearest = FAR_AWAY;       // smallest |d2 - r^2| seen by this lane
 #pragma unroll
                 for (int q = 0; q < QB; ++q) {
-                    if (q >= nq) break;
+                    if (!FULLB && q >= nq) break;
                     const float4 qv = s_q[q];
                     float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
                     fold(dx, dy, dz);
                     float d2 = fmaf(dz, dz, fmaf(dy, dy, dx * dx));
                     if (idj == __float_as_int(qv.w) || (MI && idj < 0)) d2 = FAR_AWAY;     // self (by index); folded sentinels
-                    suspect = suspect || (d2 > p.r2_lo && d2 <= p.r2_hi);
+                    nearest = fminf(nearest, fabsf(d2 - p.r2_mid));
                     d2q[q] = d2;
                 }
-                unsigned fix = 0;     // pairs inside the fp32 band that the fp64 predicate accepts
-                if (__any_sync(FULL, suspect)) {
+                if (__any_sync(FULL, nearest <= p.r2_band)) {
+                    // some pair lies within the fp32 error band of the cutoff: decide it in fp64 and
+                    // move it clear of the band (the change of d2 is below the fp32 error itself)
 #pragma unroll
                     for (int q = 0; q < QB; ++q) {
-                        if (q >= nq) break;
-                        if (d2q[q] > p.r2_lo && d2q[q] <= p.r2_hi && exact_pair(p, __float_as_int(s_q[q].w), idj)) fix |= 1u << q;
+                        if (!FULLB && q >= nq) break;
+                        if (fabsf(d2q[q] - p.r2_mid) <= p.r2_band)
+                            d2q[q] = exact_pair(p, __float_as_int(s_q[q].w), idj) ? fminf(d2q[q], p.r2_lo) : FAR_AWAY;
                     }
                 }
+                int mx = 0;
 #pragma unroll
                 for (int q = 0; q < QB; ++q) {
-                    if (q >= nq) break;
-                    const bool ok = d2q[q] <= p.r2_lo || ((fix >> q) & 1u);
+                    if (!FULLB && q >= nq) break;
+                    const bool ok = d2q[q] <= p.r2_lo;
                     const unsigned m = __ballot_sync(FULL, ok);
                     float val;
                     if (MODE == 1) val = d2q[q];
-                    else val = DIST ? sqrtf(d2q[q]) : __expf(-d2q[q] * inv2s2);
-                    const unsigned have = ((q < 4 ? cnt_lo : cnt_hi) >> (8 * (q & 3))) & 0xffu;
-                    float2* dst = list + q * QSTRIDE + have + __popc(m & lt_mask);
+                    else val = DIST ? sqrtf(d2q[q]) : fast_exp2(d2q[q] * neg_c2);
+                    float2* dst = list + q * QSTRIDE + qcnt[q] + __popc(m & lt_mask);
                     if (ok) *dst = make_float2(MODE == 0 ? pj.w : __int_as_float(cbase + lane), val);
-                    if (q < 4) cnt_lo += (unsigned)__popc(m) << (8 * (q & 3));
-                    else cnt_hi += (unsigned)__popc(m) << (8 * (q & 3));
+                    qcnt[q] += __popc(m);
+                    mx = qcnt[q] > mx ? qcnt[q] : mx;
                 }
-                if ((__vcmpgtu4(cnt_lo, DRAIN_AT) | __vcmpgtu4(cnt_hi, DRAIN_AT)) != 0u) drain();
+                return mx > QCAP - 32;
+            };
+            // one drain site: it runs when a list may overflow on the next trip and once at the end
+            // (on the first chunk the final drain also writes the zero vector of a query without neighbours)
+            bool need = false;
+            for (int cbase = 0;; cbase += 32) {
+                const bool done = cbase >= ns;
+                if (done || need) drain();
+                if (done) break;
+                need = (nq == QB) ? phase_a(cbase, std::true_type{}) : phase_a(cbase, std::false_type{});
             }
-            drain();      // on the first chunk this also writes the zero vector of a query without neighbours
             if (p.count && lane < nq) {
                 const int oq = __float_as_int(s_q[lane].w);
                 p.count[oq] = first_chunk ? s_tot[lane] : p.count[oq] + s_tot[lane];
@@ -537,34 +557,38 @@ __global__ void __launch_bounds__(TRAV_THREADS) radius_traverse_kernel(const __g
             r_ce = p.cell_start[id + (merged ? 3 : 1)];
         }
     }
-    unsigned live = __ballot_sync(FULL, r_ce > r_cs);
-    int ns = 0;
+    // flat copy: staged slot v belongs to the range whose inclusive prefix of lengths first exceeds v
+    const int r_len = r_ce - r_cs;
+    int r_incl = r_len;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(FULL, r_incl, o);
+        if (lane >= o) r_incl += t;
+    }
+    const int total = __shfl_sync(FULL, r_incl, 31);
     bool first_chunk = true;
-    while (live) {
-        const int r = __ffs(live) - 1;
-        live &= live - 1;
-        const int cs = __shfl_sync(FULL, r_cs, r), ce = __shfl_sync(FULL, r_ce, r);
-        const float ox = __shfl_sync(FULL, r_off[0], r), oy = __shfl_sync(FULL, r_off[1], r), oz = __shfl_sync(FULL, r_off[2], r);
-        int pos = cs;
-        while (pos < ce) {
-            int take = ce - pos;
-            take = take < STAGE_CAP - ns ? take : STAGE_CAP - ns;
-            for (int k = lane; k < take; k += 32) {
-                const float4 v = __ldg(p.spos + pos + k);
-                stage[ns + k] = make_float4(v.x - ox, v.y - oy, v.z - oz, v.w);
+    for (int lo = 0; lo < total || first_chunk; lo += STAGE_CAP) {
+        const int ns = total - lo < STAGE_CAP ? total - lo : STAGE_CAP;
+        for (int k = lane; k < ns + (32 - (ns & 31)) % 32; k += 32) {        // whole warp trips: shuffles inside
+            const int v = lo + k;
+            int r = 0;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const int probe = __shfl_sync(FULL, r_incl, r + o - 1);
+                if (probe <= v) r += o;
             }
-            ns += take;
-            pos += take;
-            if (ns == STAGE_CAP) {
-                __syncwarp();
-                process_chunk(ns, first_chunk);
-                first_chunk = false;
-                ns = 0;
+            r = r > 31 ? 31 : r;
+            const int src = __shfl_sync(FULL, r_cs, r) + (v - (__shfl_sync(FULL, r_incl, r) - __shfl_sync(FULL, r_len, r)));
+            const float ox = __shfl_sync(FULL, r_off[0], r), oy = __shfl_sync(FULL, r_off[1], r), oz = __shfl_sync(FULL, r_off[2], r);
+            if (k < ns) {
+                const float4 c4 = __ldg(p.spos + src);
+                stage[k] = make_float4(c4.x - ox, c4.y - oy, c4.z - oz, c4.w);
             }
         }
+        __syncwarp();
+        process_chunk(ns, first_chunk);
+        first_chunk = false;
     }
-    __syncwarp();
-    if (ns > 0 || first_chunk) process_chunk(ns, first_chunk);
 }
 
 // ------------------------------------------------------------------------------ host side
@@ -633,6 +657,8 @@ static tiga_status fill_params(RadiusParams* p, long long n, float r, const tiga
     const float beta = (single_periodic ? 96.f : 32.f) * 5.9604645e-8f;
     p->r2_lo = r2 * (1.f - beta);
     p->r2_hi = r2 * (1.f + beta);
+    p->r2_mid = r2;
+    p->r2_band = r2 * beta * 1.25f;      // a little wider than [r2_lo, r2_hi]: nothing near the cutoff escapes the exact test
     p->r2_exact = (double)r * (double)r;
     return TIGA_OK;
 }
