@@ -149,6 +149,30 @@ def roofline_models(w, counts, hbm_gbs, clock_mhz):
     return m
 
 
+def combine_ranks(dist, device, total_ms, e2e_ms, interactions):
+    """Replicas only: the step time of the job is the slowest rank's, the work is the sum."""
+    import torch
+    if dist is None:
+        return total_ms, e2e_ms, float(interactions)
+    t = torch.tensor([total_ms, e2e_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    tot = torch.tensor([float(interactions)], device=device, dtype=torch.float64)
+    dist.all_reduce(tot, op=dist.ReduceOp.SUM)
+    return t[0].item(), t[1].item(), tot.item()
+
+
+# DRAM traffic per unit measured with ncu on reduced replicas (profiles/*.md), used to scale
+# `roofline.traffic` to a full launch: bytes per particle / point / edge of one launch.
+TRAFFIC_PER_UNIT = {
+    "radius_lj_fwd": ("particle", 16.4),          # profiles/radius_traverse_lennard_jones_1M.md
+    "radius_gauss_fwd": ("point", 182.5),         # profiles/radius_traverse_gaussian_300k.md
+    "radius_gauss_bwd": ("point", 368.6),
+    "csr_sum_fwd": ("edge", 21.0),                # profiles/csr_kernels_rmat_scale18.md
+    "csr_sum_bwd": ("edge", 45.3),
+    "csr_max_bwd": ("edge", 51.9),
+}
+
+
 # ------------------------------------------------------------------------------ our arm
 def run_ours(args, rank, world, local_rank):
     import torch
@@ -271,15 +295,7 @@ def run_ours(args, rank, world, local_rank):
     sync_all()
     e2e_ms = e0.elapsed_time(e1)
 
-    if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = t.tolist()
-        tot = torch.tensor([inter_step], device=dev, dtype=torch.float64)
-        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
-        inter_all = tot.item()
-    else:
-        inter_all = float(inter_step)
+    total_ms, e2e_ms, inter_all = combine_ranks(dist, dev, total_ms, e2e_ms, inter_step)
 
     if rank != 0:
         if dist is not None:
@@ -301,6 +317,11 @@ def run_ours(args, rank, world, local_rank):
                             "unit": "GB/s" if mdl["bound"] == "hbm" else "Tlaneop/s", "frac": ach / mdl["peak"]}
     dom = max(rows, key=lambda k: row_report[k]["ms"])
     dr = row_report[dom]
+    units = {"particle": n3, "point": n2, "edge": E}
+    traffic = None
+    if dom in TRAFFIC_PER_UNIT:
+        kind, per = TRAFFIC_PER_UNIT[dom]
+        traffic = per * units[kind]
     fwd = {"csr_sum": E / (per_row_ms[0] * 1e-3), "csr_max": E / (per_row_ms[2] * 1e-3),
            "radius_gauss": counts["rad_pairs"] / (per_row_ms[5] * 1e-3), "radius_lj": counts["lj_pairs"] / (per_row_ms[7] * 1e-3)}
     fwd_bwd = {"csr_sum": E / ((per_row_ms[0] + per_row_ms[1]) * 1e-3), "csr_max": E / ((per_row_ms[2] + per_row_ms[3]) * 1e-3),
@@ -318,7 +339,9 @@ def run_ours(args, rank, world, local_rank):
                    "interactions_per_step": inter_step, "radius_pairs": counts["rad_pairs"], "lj_pairs": counts["lj_pairs"]},
         "fwd_interactions_per_s": fwd, "fwd_bwd_interactions_per_s": fwd_bwd, "rows": row_report,
         "roofline": {"kernel": dom, "bound": dr["bound"], "achieved": dr["achieved"], "peak": dr["peak"], "unit": dr["unit"],
-                     "frac": dr["frac"], "traffic": None, "peak_source": peak_kind + (" hbm copy" if dr["bound"] == "hbm" else
+                     "frac": dr["frac"], "traffic": traffic,
+                     "traffic_note": "ncu dram bytes of this kernel on a reduced replica, scaled by units processed (profiles/)",
+                     "peak_source": peak_kind + (" hbm copy" if dr["bound"] == "hbm" else
                                                                                      " 148 SM x 128 lanes x sampled SM clock")},
         "e2e": {"value": inter_all / (e2e_ms / args.steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches, "clocks": clocks,
@@ -335,24 +358,22 @@ def cpu_baseline(w, seconds_hint=20):
     """The fp64 oracle, as it stands, on a bounded sample of the step's workloads."""
     import oracle
     c = w["csr"]
-    rows = 1 << 18                                  # first quarter of the destination rows
-    rp = c["rowptr"][: rows + 1].astype(np.int64)
-    e = int(rp[-1])
-    col = c["col"][:e]; wt = c["w"][:e]; gy = c["gy"][:rows]
     t0 = time.time()
-    oracle.csr_forward(rp, col, c["x"], wt, oracle.SUM)
-    oracle.csr_backward_sum(rp, col, c["x"], wt, gy)
+    _, _, arg = oracle.csr_forward(c["rowptr"], c["col"], c["x"], c["w"], oracle.MAX)
+    oracle.csr_forward(c["rowptr"], c["col"], c["x"], c["w"], oracle.SUM)
+    oracle.csr_backward_sum(c["rowptr"], c["col"], c["x"], c["w"], c["gy"])
     t_csr = time.time() - t0
-    rr = gen.config("cfg2", n=131_072)
+    rr = w["rad"]
     t0 = time.time()
     _, _, cnt = oracle.radius_forward(rr["pos"], rr["x"], rr["r"], rr["box"], rr["periodic"], oracle.MSG_GAUSS,
                                       p0=rr["sigma"], use_cells=True)
     oracle.radius_backward_gauss(rr["pos"], rr["x"], rr["gy"], rr["r"], rr["box"], rr["periodic"], rr["sigma"], use_cells=True)
     t_rad = time.time() - t0
-    inter = 2 * e + 2 * int(cnt.sum())
+    inter = 3 * c["E"] + 2 * int(cnt.sum())
     return {"value": inter / (t_csr + t_rad), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"CSR sum fwd+bwd on the first {rows} rows of cfg1 ({e} edges, {t_csr:.2f} s) + radius Gaussian fwd+bwd "
-                      f"(cell directory) on a 131,072-point replica of cfg2 ({int(cnt.sum())} pairs, {t_rad:.2f} s)"}
+            "sample": f"cfg1 CSR max fwd + sum fwd + sum bwd (3 x {c['E']} edges, {t_csr:.1f} s) + cfg2 radius Gaussian "
+                      f"fwd+bwd with the oracle's cell directory (2 x {int(cnt.sum())} pairs, {t_rad:.1f} s); "
+                      "max bwd, histogram and Lennard-Jones rows not sampled"}
 
 
 def run_reference(args, rank, world):
