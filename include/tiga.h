@@ -42,7 +42,8 @@ typedef enum {
     TIGA_ERR_UNSUPPORTED = 2,   /* a combination this build has no kernel for */
     TIGA_ERR_WORKSPACE = 3,     /* ws is NULL or smaller than *_workspace_bytes() */
     TIGA_ERR_CUDA = 4,          /* a CUDA runtime call failed */
-    TIGA_ERR_INVALID_GRAPH = 5  /* tiga_validate_csr found a malformed relation */
+    TIGA_ERR_INVALID_GRAPH = 5, /* tiga_validate_csr found a malformed relation */
+    TIGA_ERR_TOO_LARGE = 6      /* the problem needs more scratch than the library's built-in array holds */
 } tiga_status;
 
 typedef enum { TIGA_F32 = 0, TIGA_F16 = 1 } tiga_dtype;   /* feature storage; accumulation is fp32 */
@@ -109,6 +110,36 @@ tiga_status tiga_validate_csr(const tiga_csr* g, int level, void* ws, size_t ws_
 tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
                            const float* w, const tiga_msg* msg, tiga_reducer reducer,
                            float* out, int32_t* argmax, void* ws, size_t ws_bytes, void* stream);
+
+/* tiga_apply_csr for callers that cannot hand over a workspace.  (The paper has no counterpart;
+ * this entry point exists for integration reasons only.)
+ *
+ * Who needs it: code that is given nothing but its input and output buffers and must not call
+ * cudaMalloc -- a plug-in inside a host framework that owns the device allocator, a step
+ * inside a latency-critical loop where an allocation would stall the device, a process whose
+ * memory budget was fixed at start-up.  Such a caller cannot size and allocate the `ws` that
+ * tiga_apply_csr wants, so here the scratch (one carry-out slot per tile) lives in a fixed
+ * array inside the library's own device image: TIGA_BUILTIN_WS_BYTES (8 MiB) on every GPU that
+ * loads the library, for as long as the process lives.
+ *
+ * Same arguments and results as tiga_apply_csr, minus ws / ws_bytes.  Differences:
+ *   - Capacity: the call is refused with TIGA_ERR_TOO_LARGE, before anything is launched, when
+ *     tiga_csr_workspace_bytes(g, F, x_dtype, reducer, 0) exceeds TIGA_BUILTIN_WS_BYTES
+ *     (roughly (n_dst + n_edges) / 2048 * (4 F + 4) bytes, twice the F term for TIGA_MAX;
+ *     e.g. 16.8M edges at F = 64 need 2.2 MiB).
+ *   - It never calls cudaMalloc, cudaFree or any other allocating routine.
+ *   - The first call on each device looks up the array's device address (a host-side lookup,
+ *     done with that device current and cached per device).  Make that first call before any
+ *     stream capture begins.
+ *   - All calls on one device share the one array, and it keeps whatever the previous call
+ *     left in it.  Nothing in it has to start at zero: every tile writes its own slot before
+ *     the fix-up pass reads it.  Two calls that overlap on the GPU (different streams, or
+ *     different host threads) race on the array and corrupt each other's results; serialise
+ *     them, or use tiga_apply_csr with separate workspaces. */
+#define TIGA_BUILTIN_WS_BYTES (8u << 20)
+tiga_status tiga_apply_csr_builtin_ws(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
+                                      const float* w, const tiga_msg* msg, tiga_reducer reducer,
+                                      float* out, int32_t* argmax, void* stream);
 
 /* Reverse mode of tiga_apply_csr for fixed relation indices (Section 5):
  *   sum : grad_w[e] = sum_f x[col[e],f] * grad_out[row(e),f]

@@ -15,7 +15,7 @@ __all__ = [
     "TigaError", "load_library", "EXPORTS", "SUM", "MAX", "F32", "F16",
     "MSG_COPY", "MSG_WEIGHTED", "MSG_GAUSS", "MSG_DIST", "MSG_LJ",
     "CsrRelation", "tiga_status_string", "tiga_csr_workspace_bytes", "tiga_validate_csr",
-    "tiga_apply_csr", "tiga_apply_csr_backward", "tiga_csr_degree_histogram",
+    "tiga_apply_csr", "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram",
     "tiga_radius_grid", "tiga_radius_workspace_bytes", "tiga_radius_bin",
     "tiga_apply_radius", "tiga_apply_radius_backward", "launch_count",
 ]
@@ -27,7 +27,7 @@ MSG_COPY, MSG_WEIGHTED, MSG_GAUSS, MSG_DIST, MSG_LJ = 0, 1, 2, 3, 4
 
 EXPORTS = [
     "tiga_status_string", "tiga_csr_workspace_bytes", "tiga_validate_csr", "tiga_apply_csr",
-    "tiga_apply_csr_backward", "tiga_csr_degree_histogram", "tiga_radius_grid",
+    "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram", "tiga_radius_grid",
     "tiga_radius_workspace_bytes", "tiga_radius_bin", "tiga_apply_radius",
     "tiga_apply_radius_backward",
 ]
@@ -78,6 +78,9 @@ def load_library() -> ctypes.CDLL:
     lib.tiga_apply_csr.restype = ctypes.c_int
     lib.tiga_apply_csr.argtypes = [ctypes.POINTER(_Csr), vp, ctypes.c_int, i32, vp, ctypes.POINTER(_Msg), ctypes.c_int,
                                    vp, vp, vp, sz, vp]
+    lib.tiga_apply_csr_builtin_ws.restype = ctypes.c_int
+    lib.tiga_apply_csr_builtin_ws.argtypes = [ctypes.POINTER(_Csr), vp, ctypes.c_int, i32, vp, ctypes.POINTER(_Msg),
+                                              ctypes.c_int, vp, vp, vp]
     lib.tiga_apply_csr_backward.restype = ctypes.c_int
     lib.tiga_apply_csr_backward.argtypes = [ctypes.POINTER(_Csr), vp, ctypes.c_int, i32, vp, ctypes.POINTER(_Msg), ctypes.c_int,
                                             vp, vp, vp, vp, vp, sz, vp]
@@ -178,6 +181,28 @@ def tiga_apply_csr(g: CsrRelation, x, w=None, reducer: int = SUM, out=None, argm
     msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)
     _ok(load_library().tiga_apply_csr(g.ref, _ptr(x), _dt(x), F, _ptr(w), ctypes.byref(msg), reducer, _ptr(out),
                                       _ptr(argmax), _ptr(ws), ws.numel(), _stream(stream)), "tiga_apply_csr")
+    _launches += 2
+    return out, argmax
+
+
+BUILTIN_WS_BYTES = 8 << 20
+
+
+def tiga_apply_csr_builtin_ws(g: CsrRelation, x, w=None, reducer: int = SUM, out=None, argmax=None, stream=None):
+    """tiga_apply_csr without a workspace argument: the library's fixed 8 MiB device array is the
+    scratch, for callers that may not allocate device memory.  Raises TigaError (status 6) when the
+    relation needs more than that.  Calls that overlap on the GPU race on the shared array.
+    `out` (and `argmax` for MAX) should be passed in by such callers; they are created here only
+    as a convenience when omitted.  Returns (out, argmax)."""
+    global _launches
+    F = x.shape[1]
+    if out is None:
+        out = torch.empty((g.n_dst, F), dtype=torch.float32, device=x.device)
+    if reducer == MAX and argmax is None:
+        argmax = torch.empty((g.n_dst, F), dtype=torch.int32, device=x.device)
+    msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)
+    _ok(load_library().tiga_apply_csr_builtin_ws(g.ref, _ptr(x), _dt(x), F, _ptr(w), ctypes.byref(msg), reducer,
+                                                 _ptr(out), _ptr(argmax), _stream(stream)), "tiga_apply_csr_builtin_ws")
     _launches += 2
     return out, argmax
 

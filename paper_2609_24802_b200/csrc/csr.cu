@@ -16,6 +16,7 @@
 //     fix-up kernel folds into the row, again in edge order.  No atomics in the forward, so
 //     results are reproducible.
 #include "common.cuh"
+#include <mutex>
 
 namespace tiga {
 
@@ -895,6 +896,44 @@ extern "C" tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dty
     return launch_status();
 }
 
+// ---- built-in scratch for callers that cannot allocate -------------------------------------
+// The array is part of this library's device image, so every GPU that loads the library
+// carries it until the process exits.  In host code its name is only a handle for the
+// runtime: the address a kernel can use comes from cudaGetSymbolAddress, looked up once per
+// device with that device current.
+static __device__ __align__(256) unsigned char g_builtin_ws[TIGA_BUILTIN_WS_BYTES];
+
+static tiga_status builtin_ws_address(void** out) {
+    constexpr int MAX_DEVICES = 64;
+    static void* cached[MAX_DEVICES] = {};
+    static std::mutex lock;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return TIGA_ERR_CUDA;
+    std::lock_guard<std::mutex> guard(lock);
+    if (!cached[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_builtin_ws) != cudaSuccess || !ptr) return TIGA_ERR_CUDA;
+        cached[dev] = ptr;
+    }
+    *out = cached[dev];
+    return TIGA_OK;
+}
+
+extern "C" tiga_status tiga_apply_csr_builtin_ws(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
+                                                 const float* w, const tiga_msg* msg, tiga_reducer reducer,
+                                                 float* out, int32_t* argmax, void* stream) {
+    // capacity first: a refusal touches neither the device nor the array
+    tiga_status st = check_csr(g);
+    if (st != TIGA_OK) return st;
+    if (F <= 0) return TIGA_ERR_INVALID_ARG;
+    if (reducer != TIGA_SUM && reducer != TIGA_MAX) return TIGA_ERR_INVALID_ARG;
+    if (tiga_csr_workspace_bytes(g, F, x_dtype, reducer, 0) > (size_t)TIGA_BUILTIN_WS_BYTES) return TIGA_ERR_TOO_LARGE;
+    void* ws = nullptr;
+    st = builtin_ws_address(&ws);
+    if (st != TIGA_OK) return st;
+    return tiga_apply_csr(g, x, x_dtype, F, w, msg, reducer, out, argmax, ws, (size_t)TIGA_BUILTIN_WS_BYTES, stream);
+}
+
 extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
                                                const float* w, const tiga_msg* msg, tiga_reducer reducer,
                                                const float* grad_out, const int32_t* argmax,
@@ -966,6 +1005,7 @@ extern "C" const char* tiga_status_string(tiga_status s) {
         case TIGA_ERR_WORKSPACE: return "workspace missing or too small";
         case TIGA_ERR_CUDA: return "CUDA runtime error";
         case TIGA_ERR_INVALID_GRAPH: return "malformed CSR relation";
+        case TIGA_ERR_TOO_LARGE: return "problem exceeds the library's built-in scratch capacity";
     }
     return "unknown status";
 }

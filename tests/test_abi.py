@@ -32,7 +32,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_status_strings(lib):
     assert lib.tiga_status_string(0) == "ok"
-    assert len({lib.tiga_status_string(s) for s in range(6)}) == 6
+    assert len({lib.tiga_status_string(s) for s in range(7)}) == 7
 
 
 def test_grid_matches_the_oracle_reading(lib):
