@@ -58,6 +58,8 @@ struct CsrParams {
     float* carry_val;        // [ntiles, F]
     int32_t* carry_arg;      // [ntiles, F] (max only)
     long long ntiles;
+    int* huge_count;         // narrow-row path: number of queued chunks of huge rows
+    int4* huge_list;         // (row, chunk, chunks of the row, first slot of the row)
     // backward
     const float* gy;
     float* gx;
@@ -343,204 +345,214 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_forward_kernel(const CsrParam
 
 // --------------------------------------------------------------------------------------------
 // Forward for narrow rows (one or two 16-byte vectors per feature row, e.g. F = 8 fp16).
-// A worker of G lanes would leave most of a warp idle here, so every THREAD owns IPT
-// consecutive items of the tile's merged "row ends + edges" sequence and walks them in order
-// with its reducer state in registers (all its gathers are issued up front).  Rows wholly
-// inside a thread's items are stored directly; the state of the row that is open at the end
-// of a thread's items is combined across threads by a segmented scan (warp shuffles, then the
-// eight warp totals), which hands every thread the partial state of the row that was already
-// open when its items began.  Merging stays in edge order, so results are reproducible.
+// A worker of G lanes would leave most of a warp idle here and a feature row is a single
+// 128-bit load, so the work is split by ROW CLASS instead:
+//   * every warp owns 32 consecutive rows; rows of at most ROW_SHORT edges are summed by
+//     their own lane, in edge order (empty rows cost one zero store);
+//   * longer rows (up to ROW_HUGE edges) are taken one at a time by the whole warp: lanes
+//     stride over the row's edges with coalesced index loads and 128-bit gathers, then a
+//     shuffle tree combines the 32 partial states (for max the tie rule "lowest edge position"
+//     makes the merge order irrelevant);
+//   * rows above ROW_HUGE edges are cut into ROW_HUGE-edge chunks that are queued in the
+//     workspace; a second kernel gives every chunk to a warp, a third folds the chunk states
+//     of a row in order.
+// All 32 results of a warp are stored together (one contiguous kilobyte for F = 8).
+// The summation tree is fixed, so results are reproducible.
 // --------------------------------------------------------------------------------------------
-constexpr int NARROW_IPT = CSR_TILE / CSR_THREADS;
+constexpr int ROW_SHORT = 16;
+constexpr int ROW_HUGE = 8192;
+
+template <int RED, int NV, int VW>
+__device__ __forceinline__ void tree_merge(State<RED, NV, VW>& s) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int i = 0; i < NV; ++i)
+#pragma unroll
+            for (int k = 0; k < VW; ++k) {
+                const float ov = __shfl_xor_sync(0xffffffffu, s.v[i][k], o);
+                if constexpr (RED == 0) {
+                    s.v[i][k] += ov;
+                } else {
+                    const int oa = __shfl_xor_sync(0xffffffffu, s.a[i][k], o);
+                    // larger message wins; equal messages: the lower edge position
+                    const bool take = oa >= 0 && (s.a[i][k] < 0 || ov > s.v[i][k] || (ov == s.v[i][k] && oa < s.a[i][k]));
+                    if (take) { s.v[i][k] = ov; s.a[i][k] = oa; }
+                }
+            }
+}
+
+// the whole warp reduces edges [es, es + n) of one row; every lane returns the total
+template <typename XT, int NV, int RED, int UNR = 4>
+__device__ __forceinline__ State<RED, NV, XTraits<XT>::VW> warp_row(const CsrParams& p, long long es, int n, int lane) {
+    constexpr int VW = XTraits<XT>::VW;
+    State<RED, NV, VW> s;
+    s.reset();
+    const uint4* __restrict__ xbase = static_cast<const uint4*>(p.x);
+    for (int k = lane; k < n; k += 32 * UNR) {
+        uint4 xv[UNR][NV];
+        float wv[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const bool in = k + 32 * u < n;
+            const long long e = es + (in ? k + 32 * u : k);
+            const long long c = ld_stream(p.col + e);
+            wv[u] = p.w ? ld_stream(p.w + e) : 1.f;
+#pragma unroll
+            for (int i = 0; i < NV; ++i) xv[u][i] = in ? __ldg(xbase + c * p.nvec + i) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            if (k + 32 * u < n) {
+                float xf[VW];
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    XTraits<XT>::unpack(xv[u][i], xf);
+#pragma unroll
+                    for (int q = 0; q < VW; ++q) s.message(i, q, wv[u], xf[q], (int)(es + k + 32 * u));
+                }
+            }
+        }
+    }
+    tree_merge<RED, NV, VW>(s);
+    return s;
+}
+
+template <typename XT, int NV, int RED>
+__device__ __forceinline__ void store_state(const CsrParams& p, float* out, int32_t* arg, const State<RED, NV, XTraits<XT>::VW>& s) {
+    constexpr int VW = XTraits<XT>::VW;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+#pragma unroll
+        for (int k = 0; k < VW; k += 4) {
+            st_stream(reinterpret_cast<float4*>(out + i * VW + k), make_float4(s.v[i][k], s.v[i][k + 1], s.v[i][k + 2], s.v[i][k + 3]));
+            if constexpr (RED != 0)
+                st_stream(reinterpret_cast<int4*>(arg + i * VW + k), make_int4(s.a[i][k], s.a[i][k + 1], s.a[i][k + 2], s.a[i][k + 3]));
+        }
+    }
+}
 
 template <typename XT, int NV, int RED, typename IT>
-__global__ void __launch_bounds__(CSR_THREADS) csr_forward_narrow_kernel(const CsrParams p) {
+__global__ void __launch_bounds__(CSR_THREADS) csr_rows_kernel(const CsrParams p) {
     constexpr int VW = XTraits<XT>::VW;
-    constexpr int IPT = NARROW_IPT;
-    constexpr int U = IPT / NV;                  // gathers in flight per thread
-    constexpr int NWARP = CSR_THREADS / 32;
     constexpr unsigned FULL = 0xffffffffu;
     using St = State<RED, NV, VW>;
-
-    __shared__ int s_ptr[CSR_TILE + 2];
-    __shared__ int s_col[CSR_TILE + CSR_TILE / 32 + 1];
-    __shared__ float s_w[CSR_TILE + CSR_TILE / 32 + 1];
-    __shared__ long long s_coord[2];
-    __shared__ int s_start[CSR_THREADS + 1];
-    __shared__ float s_tv[2][NWARP][NV * VW];     // [0] inclusive warp totals, [1] exclusive prefixes over warps
-    __shared__ int s_ta[2][NWARP][RED ? NV * VW : 1];
-    __shared__ int s_tf[2][NWARP];
-
-    const Tile t = stage_tile<IT, true>(p, s_ptr, s_col, s_w, s_coord);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const bool has_w = p.w != nullptr;
+    const IT* __restrict__ rowptr = static_cast<const IT*>(p.rowptr);
     const uint4* __restrict__ xbase = static_cast<const uint4*>(p.x);
-    const int total = t.nfin + t.ne;
+    const int lane = threadIdx.x & 31;
+    const long long row = ((long long)blockIdx.x * CSR_THREADS + threadIdx.x);      // warp-contiguous rows
+    const bool valid = row < p.n_dst;
+    const long long es = valid ? (long long)rowptr[row] : 0;
+    const long long ee = valid ? (long long)rowptr[row + 1] : 0;
+    const long long deg = ee - es;
 
-    // merge coordinates of this thread's first item: rows finished before diagonal d
-    const int d0 = tid * IPT < total ? tid * IPT : total;
-    const int d1 = (tid + 1) * IPT < total ? (tid + 1) * IPT : total;
-    {
-        int lo = 0, hi = t.nfin;
-        while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            if (s_ptr[mid + 1] + mid + 1 <= d0) lo = mid + 1; else hi = mid;
-        }
-        s_start[tid] = lo;
-        if (tid == 0) s_start[CSR_THREADS] = t.nfin;
-    }
-    __syncthreads();
-    const int r0 = s_start[tid], r1 = s_start[tid + 1];
-    const int ea = d0 - r0, eb = d1 - r1;         // this thread's edges [ea, eb), rows to finish [r0, r1)
-
-    auto store_row = [&](long long row, const St& s) {
-#pragma unroll
-        for (int i = 0; i < NV; ++i) {
-            float* o = p.out + row * p.F + (size_t)i * VW;
-#pragma unroll
-            for (int k = 0; k < VW; k += 4)
-                st_stream(reinterpret_cast<float4*>(o + k), make_float4(s.v[i][k], s.v[i][k + 1], s.v[i][k + 2], s.v[i][k + 3]));
-            if constexpr (RED != 0) {
-                int* ao = p.arg + row * p.F + (size_t)i * VW;
-#pragma unroll
-                for (int k = 0; k < VW; k += 4)
-                    st_stream(reinterpret_cast<int4*>(ao + k), make_int4(s.a[i][k], s.a[i][k + 1], s.a[i][k + 2], s.a[i][k + 3]));
-            }
-        }
-    };
-    // fold a partial state that comes EARLIER in edge order into s
-    auto merge_earlier = [&](St& s, int i, int k, float ov, int oa) {
-        if constexpr (RED == 0) {
-            s.v[i][k] = ov + s.v[i][k];
-        } else {
-            if (oa >= 0 && (s.a[i][k] < 0 || !(s.v[i][k] > ov))) { s.v[i][k] = ov; s.a[i][k] = oa; }
-        }
-    };
-
-    St st, head;
+    St st;
     st.reset();
-    head.reset();
-    int row = r0, hrow = -1;
-    bool head_open = false;
-    if (ea < eb || r0 < r1) {
-        int cur_end = row < t.nrows ? s_ptr[row + 1] : 0x7fffffff;
-        head_open = (s_ptr[row] < 0 ? 0 : s_ptr[row]) < ea;
-        auto finish_row = [&]() {
-            if (head_open) { head = st; hrow = row; head_open = false; }
-            else store_row(t.i0 + row, st);
-            st.reset();
-            ++row;
-            cur_end = row < t.nrows ? s_ptr[row + 1] : 0x7fffffff;
-        };
+    // short rows: one lane each, edge order
+    if (valid && deg <= ROW_SHORT) {
+        const int n = (int)deg;
+        for (int k = 0; k < n; k += 4) {
+            uint4 xv[4][NV];
+            float wv[4];
 #pragma unroll
-        for (int ub = 0; ub < IPT; ub += U) {
-            uint4 xv[U][NV];
-            float wv[U];
+            for (int u = 0; u < 4; ++u) {
+                const bool in = k + u < n;
+                const long long e = es + (in ? k + u : k);
+                const long long c = __ldg(p.col + e);
+                wv[u] = p.w ? __ldg(p.w + e) : 1.f;
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int e = ea + ub + u < eb ? ea + ub + u : (eb > ea ? eb - 1 : 0);
-                const long long c = (ea < eb) ? s_col[pad32(e)] : 0;
-                wv[u] = (has_w && ea < eb) ? s_w[pad32(e)] : 1.f;
-#pragma unroll
-                for (int i = 0; i < NV; ++i) xv[u][i] = (ea + ub + u < eb) ? __ldg(xbase + c * p.nvec + i) : make_uint4(0, 0, 0, 0);
+                for (int i = 0; i < NV; ++i) xv[u][i] = in ? __ldg(xbase + c * p.nvec + i) : make_uint4(0, 0, 0, 0);
             }
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int e = ea + ub + u;
-                if (e < eb) {
-                    while (e >= cur_end) finish_row();
+            for (int u = 0; u < 4; ++u) {
+                if (k + u < n) {
                     float xf[VW];
 #pragma unroll
                     for (int i = 0; i < NV; ++i) {
                         XTraits<XT>::unpack(xv[u][i], xf);
 #pragma unroll
-                        for (int k = 0; k < VW; ++k) st.message(i, k, wv[u], xf[k], (int)(t.e0 + e));
+                        for (int q = 0; q < VW; ++q) st.message(i, q, wv[u], xf[q], (int)(es + k + u));
                     }
                 }
             }
         }
-        while (row < r1) finish_row();
     }
-    // st is now the state of the row that is open after this thread's items (identity if none);
-    // it restarts the scan unless the thread lies wholly inside a row that began before it
-    int flag = head_open ? 0 : ((ea < eb || r0 < r1) ? 1 : 0);
-    St inc = st;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int of = __shfl_up_sync(FULL, flag, o);
-#pragma unroll
-        for (int i = 0; i < NV; ++i)
-#pragma unroll
-            for (int k = 0; k < VW; ++k) {
-                const float ov = __shfl_up_sync(FULL, inc.v[i][k], o);
-                int oa = 0;
-                if constexpr (RED != 0) oa = __shfl_up_sync(FULL, inc.a[i][k], o);
-                if (lane >= o && !flag) merge_earlier(inc, i, k, ov, oa);
-            }
-        if (lane >= o) flag |= of;
-    }
-    if (lane == 31) {
-#pragma unroll
-        for (int i = 0; i < NV; ++i)
-#pragma unroll
-            for (int k = 0; k < VW; ++k) {
-                s_tv[0][warp][i * VW + k] = inc.v[i][k];
-                if constexpr (RED != 0) s_ta[0][warp][i * VW + k] = inc.a[i][k];
-            }
-        s_tf[0][warp] = flag;
+    // longer rows go through a queue in shared memory that all warps of the CTA drain together,
+    // so one warp with several long rows does not hold the others back
+    __shared__ int q_row[CSR_THREADS];
+    __shared__ long long q_start[CSR_THREADS];
+    __shared__ int q_len[CSR_THREADS];
+    __shared__ int q_n, q_next;
+    if (threadIdx.x == 0) { q_n = 0; q_next = 0; }
+    __syncthreads();
+    const bool is_mid = valid && deg > ROW_SHORT && deg <= ROW_HUGE;
+    if (is_mid) {
+        const int slot = atomicAdd(&q_n, 1);
+        q_row[slot] = threadIdx.x; q_start[slot] = es; q_len[slot] = (int)deg;
     }
     __syncthreads();
-    if (tid < NV * VW) {
-        // exclusive scan over the eight warp totals, one feature per thread
-        float v = 0.f;
-        int a = -1;
-        for (int w2 = 0; w2 < NWARP; ++w2) {
-            s_tv[1][w2][tid] = v;
-            if constexpr (RED != 0) s_ta[1][w2][tid] = a;
-            const float tv = s_tv[0][w2][tid];
-            const int ta = RED ? s_ta[0][w2][RED ? tid : 0] : 0;
-            if (s_tf[0][w2]) { v = tv; a = ta; }
-            else if constexpr (RED == 0) v = v + tv;
-            else { if (ta >= 0 && (a < 0 || tv > v)) { v = tv; a = ta; } }
-        }
+    const int nmid = q_n;
+    const long long row0 = (long long)blockIdx.x * CSR_THREADS;
+    for (;;) {
+        int idx = 0;
+        if (lane == 0) idx = atomicAdd(&q_next, 1);
+        idx = __shfl_sync(FULL, idx, 0);
+        if (idx >= nmid) break;
+        const long long r = row0 + q_row[idx];
+        const long long rs = q_start[idx];
+        const int rn = q_len[idx];
+        const St tot = warp_row<XT, NV, RED>(p, rs, rn, lane);
+        if (lane == 0) store_state<XT, NV, RED>(p, p.out + r * p.F, RED ? p.arg + r * p.F : nullptr, tot);
     }
-    __syncthreads();
-    // exclusive prefix of this thread: the open row's state contributed by earlier threads
-    St pre;
-    const int ef = __shfl_up_sync(FULL, flag, 1);
-#pragma unroll
-    for (int i = 0; i < NV; ++i)
-#pragma unroll
-        for (int k = 0; k < VW; ++k) {
-            float ev = __shfl_up_sync(FULL, inc.v[i][k], 1);
-            int ea2 = -1;
-            if constexpr (RED != 0) ea2 = __shfl_up_sync(FULL, inc.a[i][k], 1);
-            if (lane == 0) { ev = 0.f; ea2 = -1; }
-            pre.v[i][k] = ev;
-            if constexpr (RED != 0) pre.a[i][k] = ea2;
-            if (lane == 0 || !ef) merge_earlier(pre, i, k, s_tv[1][warp][i * VW + k], RED ? s_ta[1][warp][RED ? i * VW + k : 0] : 0);
-        }
-    if (hrow >= 0) {
-#pragma unroll
-        for (int i = 0; i < NV; ++i)
-#pragma unroll
-            for (int k = 0; k < VW; ++k) merge_earlier(head, i, k, pre.v[i][k], RED ? pre.a[RED ? i : 0][RED ? k : 0] : 0);
-        store_row(t.i0 + hrow, head);
+    // huge rows: queue their chunks
+    if (valid && deg > ROW_HUGE) {
+        const int chunks = (int)((deg + ROW_HUGE - 1) / ROW_HUGE);
+        const int base = atomicAdd(p.huge_count, chunks);
+        for (int c = 0; c < chunks; ++c) p.huge_list[base + c] = make_int4((int)row, c, chunks, base);
     }
-    if (tid == CSR_THREADS - 1) {
-        // trailing unfinished row of the tile -> carry-out (inclusive value at the last thread)
-        const bool open = t.nrows > t.nfin && t.ne > (s_ptr[t.nfin] < 0 ? 0 : s_ptr[t.nfin]);
-        p.carry_row[blockIdx.x] = open ? (int32_t)(t.i0 + t.nfin) : -1;
-        if (open) {
-#pragma unroll
-            for (int i = 0; i < NV; ++i)
-#pragma unroll
-                for (int k = 0; k < VW; ++k) {
-                    if (!flag) merge_earlier(inc, i, k, s_tv[1][warp][i * VW + k], RED ? s_ta[1][warp][RED ? i * VW + k : 0] : 0);
-                    p.carry_val[(size_t)blockIdx.x * p.F + i * VW + k] = inc.v[i][k];
-                    if constexpr (RED != 0) p.carry_arg[(size_t)blockIdx.x * p.F + i * VW + k] = inc.a[i][k];
-                }
+    if (valid && deg <= ROW_SHORT)
+        store_state<XT, NV, RED>(p, p.out + row * p.F, RED ? p.arg + row * p.F : nullptr, st);
+}
+
+// one warp per queued chunk of a huge row
+template <typename XT, int NV, int RED, typename IT>
+__global__ void __launch_bounds__(CSR_THREADS) csr_huge_chunks_kernel(const CsrParams p) {
+    const IT* __restrict__ rowptr = static_cast<const IT*>(p.rowptr);
+    const int lane = threadIdx.x & 31;
+    const int nwarps = gridDim.x * (CSR_THREADS / 32);
+    const int total = *p.huge_count;
+    for (int idx = blockIdx.x * (CSR_THREADS / 32) + (threadIdx.x >> 5); idx < total; idx += nwarps) {
+        const int4 ent = p.huge_list[idx];
+        const long long es = (long long)rowptr[ent.x] + (long long)ent.y * ROW_HUGE;
+        const long long ee = (long long)rowptr[ent.x + 1];
+        const int n = (int)(ee - es < ROW_HUGE ? ee - es : ROW_HUGE);
+        const auto tot = warp_row<XT, NV, RED, (NV == 1 ? 8 : 4)>(p, es, n, lane);
+        if (lane == 0)
+            store_state<XT, NV, RED>(p, p.carry_val + (size_t)idx * p.F, RED ? p.carry_arg + (size_t)idx * p.F : nullptr, tot);
+    }
+}
+
+// fold the chunk states of every huge row in chunk (= edge) order; one thread per (row, feature)
+template <int RED>
+__global__ void csr_huge_fold_kernel(const CsrParams p) {
+    const int total = *p.huge_count;
+    const long long nthreads = (long long)gridDim.x * blockDim.x;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < (long long)total * p.F; t += nthreads) {
+        const int idx = (int)(t / p.F), f = (int)(t % p.F);
+        const int4 ent = p.huge_list[idx];
+        if (ent.y != 0) continue;
+        float v = p.carry_val[(size_t)idx * p.F + f];
+        int a = RED ? p.carry_arg[(size_t)idx * p.F + f] : 0;
+        for (int c = 1; c < ent.z; ++c) {
+            const float ov = p.carry_val[(size_t)(idx + c) * p.F + f];
+            if (RED == 0) v += ov;
+            else {
+                const int oa = p.carry_arg[(size_t)(idx + c) * p.F + f];
+                if (oa >= 0 && (a < 0 || ov > v)) { v = ov; a = oa; }
+            }
         }
+        p.out[(size_t)ent.x * p.F + f] = v;
+        if (RED) p.arg[(size_t)ent.x * p.F + f] = a;
     }
 }
 
@@ -759,8 +771,19 @@ static tiga_status launch_fwd_t(const CsrParams& p, cudaStream_t s) {
 
 template <typename XT, int RED, typename IT>
 static tiga_status launch_fwd_g(const CsrParams& p, int G, int VPL, cudaStream_t s) {
-    if (p.nvec == 1) { csr_forward_narrow_kernel<XT, 1, RED, IT><<<(unsigned)p.ntiles, CSR_THREADS, 0, s>>>(p); return launch_status(); }
-    if (p.nvec == 2) { csr_forward_narrow_kernel<XT, 2, RED, IT><<<(unsigned)p.ntiles, CSR_THREADS, 0, s>>>(p); return launch_status(); }
+    if (p.nvec <= 2) {
+        TIGA_CUDA_TRY(cudaMemsetAsync(p.huge_count, 0, sizeof(int), s));
+        const unsigned blocks = (unsigned)((p.n_dst + CSR_THREADS - 1) / CSR_THREADS);
+        if (p.nvec == 1) {
+            csr_rows_kernel<XT, 1, RED, IT><<<blocks, CSR_THREADS, 0, s>>>(p);
+            csr_huge_chunks_kernel<XT, 1, RED, IT><<<148 * 8, CSR_THREADS, 0, s>>>(p);
+        } else {
+            csr_rows_kernel<XT, 2, RED, IT><<<blocks, CSR_THREADS, 0, s>>>(p);
+            csr_huge_chunks_kernel<XT, 2, RED, IT><<<148 * 8, CSR_THREADS, 0, s>>>(p);
+        }
+        csr_huge_fold_kernel<RED><<<148 * 2, 256, 0, s>>>(p);
+        return launch_status();
+    }
     switch (G) {
         case 1: return launch_fwd_t<XT, 1, 1, RED, IT>(p, s);
         case 2: return launch_fwd_t<XT, 2, 1, RED, IT>(p, s);
@@ -823,6 +846,7 @@ extern "C" size_t tiga_csr_workspace_bytes(const tiga_csr* g, int32_t F, tiga_dt
     const size_t nt = (size_t)num_tiles(g) + 1;
     size_t b = align_up(nt * sizeof(int32_t), 256) + align_up(nt * F * sizeof(float), 256);
     if (reducer == TIGA_MAX) b += align_up(nt * F * sizeof(int32_t), 256);
+    b += 256 + align_up(nt * sizeof(int4), 256);      // queue of huge-row chunks (narrow-row path)
     return b + 256;
 }
 
@@ -880,6 +904,8 @@ extern "C" tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dty
     p.carry_row = cv.take<int32_t>((size_t)p.ntiles + 1);
     p.carry_val = cv.take<float>(((size_t)p.ntiles + 1) * F);
     p.carry_arg = reducer == TIGA_MAX ? cv.take<int32_t>(((size_t)p.ntiles + 1) * F) : nullptr;
+    p.huge_count = cv.take<int>(1);
+    p.huge_list = cv.take<int4>((size_t)p.ntiles + 1);      // >= 2 E / ROW_HUGE + 1 entries
 
     const bool i64 = g->rowptr_type == TIGA_I64;
     if (x_dtype == TIGA_F32) {
@@ -890,6 +916,7 @@ extern "C" tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dty
         else st = i64 ? launch_fwd_g<__half, 1, int64_t>(p, G, VPL, s) : launch_fwd_g<__half, 1, int32_t>(p, G, VPL, s);
     }
     if (st != TIGA_OK) return st;
+    if (nvec <= 2) return TIGA_OK;             // the row-class path has no tile carry-outs
     const long long work = p.ntiles * F;
     if (reducer == TIGA_SUM) csr_fixup_kernel<0><<<(unsigned)((work + 255) / 256), 256, 0, s>>>(p);
     else csr_fixup_kernel<1><<<(unsigned)((work + 255) / 256), 256, 0, s>>>(p);
