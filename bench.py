@@ -369,11 +369,16 @@ def cpu_baseline(w, seconds_hint=20):
                                       p0=rr["sigma"], use_cells=True)
     oracle.radius_backward_gauss(rr["pos"], rr["x"], rr["gy"], rr["r"], rr["box"], rr["periodic"], rr["sigma"], use_cells=True)
     t_rad = time.time() - t0
-    inter = 3 * c["E"] + 2 * int(cnt.sum())
-    return {"value": inter / (t_csr + t_rad), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+    lj = w["lj"]
+    t0 = time.time()
+    _, _, cnt3 = oracle.radius_forward(lj["pos"], None, lj["r"], lj["box"], lj["periodic"], oracle.MSG_LJ, 1.0, 1.0, use_cells=True)
+    t_lj = time.time() - t0
+    inter = 3 * c["E"] + 2 * int(cnt.sum()) + int(cnt3.sum())
+    return {"value": inter / (t_csr + t_rad + t_lj), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
             "sample": f"cfg1 CSR max fwd + sum fwd + sum bwd (3 x {c['E']} edges, {t_csr:.1f} s) + cfg2 radius Gaussian "
-                      f"fwd+bwd with the oracle's cell directory (2 x {int(cnt.sum())} pairs, {t_rad:.1f} s); "
-                      "max bwd, histogram and Lennard-Jones rows not sampled"}
+                      f"fwd+bwd with the oracle's cell directory (2 x {int(cnt.sum())} pairs, {t_rad:.1f} s) + cfg3 "
+                      f"Lennard-Jones with the cell directory ({int(cnt3.sum())} pairs, {t_lj:.1f} s); "
+                      "max bwd and histogram rows not sampled"}
 
 
 def run_reference(args, rank, world):
