@@ -188,7 +188,8 @@ tiga_status tiga_radius_bin(const float* pos, int64_t n, float r, const tiga_box
  * point i accumulates the messages of all j != i with |p_i - p_j| <= r (minimum image in
  * periodic dimensions; the predicate is decided exactly as in double precision) straight
  * into the sum reducer.  Neither an edge list nor per-edge messages are written.
- *   GAUSS / DIST : feat fp32 [n, F] (F multiple of 4, <= 128), out fp32 [n, F]
+ *   GAUSS / DIST : feat fp32 [n, F] (1 <= F <= 128; 128-bit accesses when F is a multiple
+ *                  of 4, scalar accesses otherwise), out fp32 [n, F]
  *   LJ           : feat ignored, F ignored, out fp32 [n, 4] = (Fx, Fy, Fz, e_i) with
  *                  F_i = sum_j 24 eps (2 (s/d)^12 - (s/d)^6) (p_i - p_j) / d^2 and
  *                  e_i = (1/2) sum_j 4 eps ((s/d)^12 - (s/d)^6)
@@ -203,7 +204,7 @@ tiga_status tiga_apply_radius(const float* pos, const float* feat, int64_t n, in
  *   grad_feat[j,:] = sum over i with j in N(i) of g_ij grad_out[i,:]
  *   grad_pos[k,:]  = -(1/sigma^2) sum over j in N(k) of g_kj (p_k - p_j)
  *                                  (grad_out[k].feat[j] + grad_out[j].feat[k])
- *   grad_feat : fp32 [n, F] or NULL;  grad_pos : fp32 [n, 3] or NULL.
+ *   grad_feat : fp32 [n, F] or NULL;  grad_pos : fp32 [n, 3] or NULL.  F must be a multiple of 4.
  *   reuse_plan != 0: ws still holds the bins of this very position snapshot (left there by
  *   tiga_apply_radius or tiga_radius_bin with the same n, r, box); otherwise it is rebuilt. */
 tiga_status tiga_apply_radius_backward(const float* pos, const float* feat, int64_t n, int32_t F,

@@ -271,7 +271,8 @@ __device__ __noinline__ bool exact_pair(const RadiusParams& p, int a, int b) {
 
 // MODE 0: Gaussian (DIST = false) or distance-weighted (DIST = true) forward; 1: Lennard-Jones;
 // 2: Gaussian backward.  MI: some periodic dimension has a single cell (explicit minimum image).
-template <int MODE, int LF, bool DIST, bool MI>
+// VEC: feature rows are 16-byte aligned (F % 4 == 0); otherwise the forward uses scalar accesses.
+template <int MODE, int LF, bool DIST, bool MI, bool VEC = true>
 __global__ void __launch_bounds__(TRAV_THREADS) radius_traverse_kernel(const __grid_constant__ RadiusParams p) {
     using SM = TravSmem<MODE>;
     constexpr int STAGE_CAP = SM::STAGE_CAP, QCAP = SM::QCAP, QSTRIDE = SM::QSTRIDE;
@@ -395,7 +396,10 @@ __global__ void __launch_bounds__(TRAV_THREADS) radius_traverse_kernel(const __g
                                     for (int u = 0; u < 4; ++u) {      // four gathered rows in flight
                                         e[u] = lq[t + u < n ? t + u : t];
                                         if (t + u >= n) e[u].y = 0.f;
-                                        x[u] = __ldg(reinterpret_cast<const float4*>(p.feat + (size_t)__float_as_int(e[u].x) * F) + fl);
+                                        const float* xr = p.feat + (size_t)__float_as_int(e[u].x) * F + fl * 4;
+                                        if (VEC) x[u] = __ldg(reinterpret_cast<const float4*>(xr));
+                                        else x[u] = make_float4(__ldg(xr), fl * 4 + 1 < F ? __ldg(xr + 1) : 0.f,
+                                                                fl * 4 + 2 < F ? __ldg(xr + 2) : 0.f, fl * 4 + 3 < F ? __ldg(xr + 3) : 0.f);
                                     }
 #pragma unroll
                                     for (int u = 0; u < 4; ++u) {
@@ -435,10 +439,16 @@ __global__ void __launch_bounds__(TRAV_THREADS) radius_traverse_kernel(const __g
                                 }
                             }
                             float* orow = (MODE == 0 ? p.out : p.gfeat);
-                            if (orow) {
+                            if (orow && VEC) {
                                 float4* o = reinterpret_cast<float4*>(orow + (size_t)oqq * F) + fl;
                                 if (!first) { const float4 old = *o; acc.x += old.x; acc.y += old.y; acc.z += old.z; acc.w += old.w; }
                                 *o = acc;
+                            } else if (orow) {
+                                float* o = orow + (size_t)oqq * F + fl * 4;
+                                const float a4[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+                                for (int c4 = 0; c4 < 4; ++c4)
+                                    if (fl * 4 + c4 < F) o[c4] = first ? a4[c4] : o[c4] + a4[c4];
                             }
                         }
                         if (MODE == 2) {
@@ -686,6 +696,13 @@ template <int MODE, int LF, bool DIST, bool MI>
 static tiga_status launch_traverse_t(const RadiusParams& p, cudaStream_t s) {
     const unsigned blocks = (unsigned)((p.ncells + TRAV_WARPS - 1) / TRAV_WARPS);
     constexpr int smem = TravSmem<MODE>::PER_WARP * TRAV_WARPS;
+    if (MODE == 0 && (p.F & 3)) {
+        // scalar feature accesses (only the forward supports widths that are not multiples of 4)
+        auto sk = radius_traverse_kernel<MODE == 0 ? 0 : MODE, LF, DIST, MI, MODE != 0>;
+        if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(sk, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        sk<<<blocks, TRAV_THREADS, smem, s>>>(p);
+        return launch_status();
+    }
     auto kern = radius_traverse_kernel<MODE, LF, DIST, MI>;
     if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     kern<<<blocks, TRAV_THREADS, smem, s>>>(p);
@@ -756,7 +773,7 @@ extern "C" tiga_status tiga_radius_bin(const float* pos, int64_t n, float r, con
 
 static tiga_status radius_common(RadiusParams* p, const float* pos, const float* feat, int64_t n, int32_t F,
                                  float r, const tiga_box* box, const tiga_msg* msg_p, void* ws, size_t ws_bytes,
-                                 int32_t** fill, RadiusLayout* lay) {
+                                 int32_t** fill, RadiusLayout* lay, int forward_only_widths) {
     if (!msg_p) return TIGA_ERR_INVALID_ARG;
     const tiga_msg msg = *msg_p;
     tiga_status st = fill_params(p, n, r, box);
@@ -766,7 +783,8 @@ static tiga_status radius_common(RadiusParams* p, const float* pos, const float*
         F = 4;
     } else if (msg.kind == TIGA_MSG_GAUSS || msg.kind == TIGA_MSG_DIST) {
         if (F <= 0) return TIGA_ERR_INVALID_ARG;
-        if (F % 4 || F > 128) return TIGA_ERR_UNSUPPORTED;
+        if (F > 128) return TIGA_ERR_UNSUPPORTED;
+        if ((F % 4) && forward_only_widths == 0) return TIGA_ERR_UNSUPPORTED;
         if (msg.kind == TIGA_MSG_GAUSS && !(msg.p0 > 0.f)) return TIGA_ERR_INVALID_ARG;
         if (n > 0 && (!feat || !aligned16(feat))) return TIGA_ERR_INVALID_ARG;
     } else {
@@ -785,7 +803,7 @@ extern "C" tiga_status tiga_apply_radius(const float* pos, const float* feat, in
     RadiusParams p{};
     int32_t* fill;
     RadiusLayout lay;
-    tiga_status st = radius_common(&p, pos, feat, n, F, r, box, msg, ws, ws_bytes, &fill, &lay);
+    tiga_status st = radius_common(&p, pos, feat, n, F, r, box, msg, ws, ws_bytes, &fill, &lay, 1);
     if (st != TIGA_OK) return st;
     if (n == 0) return TIGA_OK;
     if (!out || !aligned16(out)) return TIGA_ERR_INVALID_ARG;
@@ -807,7 +825,7 @@ extern "C" tiga_status tiga_apply_radius_backward(const float* pos, const float*
     RadiusParams p{};
     int32_t* fill;
     RadiusLayout lay;
-    tiga_status st = radius_common(&p, pos, feat, n, F, r, box, msg, ws, ws_bytes, &fill, &lay);
+    tiga_status st = radius_common(&p, pos, feat, n, F, r, box, msg, ws, ws_bytes, &fill, &lay, 0);
     if (st != TIGA_OK) return st;
     if (n == 0 || (!grad_feat && !grad_pos)) return TIGA_OK;
     if (!grad_out || !aligned16(grad_out)) return TIGA_ERR_INVALID_ARG;

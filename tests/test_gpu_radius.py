@@ -85,6 +85,20 @@ def test_gaussian_small(tiga, periodic, F):
     _check_gauss(tiga, pos, x, gy, r, np.ones(3, np.float32), [periodic] * 3, np.float32(float(r) / 2))
 
 
+@pytest.mark.parametrize("F", [1, 3, 6])
+def test_forward_widths_that_are_not_multiples_of_four(tiga, F):
+    n = 5000
+    pos = gen.uniform_points(n, 40 + F)
+    x = gen.normal_features(n, F, 40 + F, 31)
+    r = gen.radius_for_expected_neighbours(n, 32.0)
+    ones = np.ones(3, np.float32)
+    _check_gauss(tiga, pos, x, None, r, ones, [0, 0, 0], np.float32(float(r) / 2), backward=False)
+    _check_gauss(tiga, pos, x, None, r, ones, [1, 1, 1], np.float32(float(r) / 2), kind=tiga.MSG_DIST)
+    with pytest.raises(tiga.TigaError) as ei:      # the backward needs 128-bit rows
+        tiga.tiga_apply_radius_backward(dev(pos, torch), dev(x, torch), dev(x, torch), r, ones, [0, 0, 0], 0.1)
+    assert ei.value.status == 2
+
+
 def test_few_cells_mixed_periodicity_and_anisotropic_box(tiga):
     # the paper's tiny radius shape: 128 points, cutoff 0.35 (two cells per dimension)
     pos = gen.uniform_points(128, 7)
