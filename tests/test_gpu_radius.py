@@ -211,3 +211,24 @@ def test_cfg2_full_size_sampled_rows(tiga):
     assert rel_err(gx, b["gx"], b["Agx"]) <= GRAD_TOL
     assert rel_err(gp, b["gp"], b["Agp"]) <= GRAD_TOL
     assert np.max(np.abs(gp.astype(np.float64).sum(0))) < 1e-5 * b["Agp"].sum()     # translation invariance
+
+
+def test_cfg3_full_size(tiga):
+    """160^3 = 4,096,000 jittered-lattice particles, periodic, cutoff 2.5: 2048 sampled rows against
+    all-pairs brute force, every row against the oracle's cell-directory variant, and Newton's
+    third law over the whole system."""
+    c = gen.config("cfg3")
+    n = c["n"]
+    assert n == 4_096_000
+    out, count, _ = tiga.tiga_apply_radius(dev(c["pos"], torch), None, c["r"], c["box"], c["periodic"], tiga.MSG_LJ,
+                                           p0=1.0, p1=1.0, want_count=True)
+    out, count = host(out), host(count)
+    rows = np.sort(gen.rng(3, 78).choice(n, 2048, replace=False))
+    y, A, cnt = oracle.radius_forward(c["pos"], None, c["r"], c["box"], c["periodic"], oracle.MSG_LJ, 1.0, 1.0, rows=rows)
+    assert np.array_equal(count[rows], cnt)
+    assert rel_err(out[rows], y, A) <= SUM_TOL
+    y, A, cnt = oracle.radius_forward(c["pos"], None, c["r"], c["box"], c["periodic"], oracle.MSG_LJ, 1.0, 1.0, use_cells=True)
+    assert np.array_equal(count, cnt) and count.sum() % 2 == 0
+    assert rel_err(out, y, A) <= SUM_TOL
+    assert 50 < count.mean() < 58
+    assert np.max(np.abs(out[:, :3].astype(np.float64).sum(0))) < 1e-6 * A[:, :3].sum()
