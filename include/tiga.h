@@ -105,7 +105,8 @@ tiga_status tiga_validate_csr(const tiga_csr* g, int level, void* ws, size_t ws_
  *   out    : fp32 [n_dst, F].
  *   argmax : int32 [n_dst, F]; required for TIGA_MAX (needs n_edges < 2^31), ignored for TIGA_SUM.
  *   ws     : tiga_csr_workspace_bytes(g, F, x_dtype, reducer, 0) bytes; contents are scratch.
- * Rows longer than one tile are split and their partial states merged in edge order, so
+ * Long rows are split and their partial states merged in a fixed order (edge order for feature
+ * rows of 64 bytes and more; a fixed lane-strided tree for narrower rows), without atomics, so
  * results are reproducible from run to run. */
 tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
                            const float* w, const tiga_msg* msg, tiga_reducer reducer,

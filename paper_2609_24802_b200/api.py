@@ -168,6 +168,13 @@ def tiga_validate_csr(g: CsrRelation, level: int = 1, stream=None) -> None:
     _ok(load_library().tiga_validate_csr(g.ref, level, _ptr(ws), ws.numel(), _stream(stream)), "tiga_validate_csr")
 
 
+def _csr_forward_launches(x) -> int:
+    """Kernels one forward call launches: tile kernel + fix-up, or the three row-class kernels
+    when a feature row is at most 32 bytes."""
+    row_bytes = x.shape[1] * x.element_size()
+    return 3 if row_bytes <= 32 else 2
+
+
 def tiga_apply_csr(g: CsrRelation, x, w=None, reducer: int = SUM, out=None, argmax=None, ws=None, stream=None):
     """out[i,:] = reduce over the row's edges of w[e] * x[col[e],:].  Returns (out, argmax)."""
     global _launches
@@ -181,7 +188,7 @@ def tiga_apply_csr(g: CsrRelation, x, w=None, reducer: int = SUM, out=None, argm
     msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)
     _ok(load_library().tiga_apply_csr(g.ref, _ptr(x), _dt(x), F, _ptr(w), ctypes.byref(msg), reducer, _ptr(out),
                                       _ptr(argmax), _ptr(ws), ws.numel(), _stream(stream)), "tiga_apply_csr")
-    _launches += 2
+    _launches += _csr_forward_launches(x)
     return out, argmax
 
 
@@ -203,7 +210,7 @@ def tiga_apply_csr_builtin_ws(g: CsrRelation, x, w=None, reducer: int = SUM, out
     msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)
     _ok(load_library().tiga_apply_csr_builtin_ws(g.ref, _ptr(x), _dt(x), F, _ptr(w), ctypes.byref(msg), reducer,
                                                  _ptr(out), _ptr(argmax), _stream(stream)), "tiga_apply_csr_builtin_ws")
-    _launches += 2
+    _launches += _csr_forward_launches(x)
     return out, argmax
 
 

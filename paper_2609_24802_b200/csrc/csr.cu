@@ -760,9 +760,8 @@ static long long num_tiles(const tiga_csr* g) { return (g->n_dst + g->n_edges + 
 
 template <typename XT, int G, int VPL, int RED, typename IT>
 static tiga_status launch_fwd_t(const CsrParams& p, cudaStream_t s) {
-    constexpr int VW = XTraits<XT>::VW;
     constexpr int NW = CSR_THREADS / G;
-    const size_t dyn = (size_t)2 * NW * G * VPL * VW * sizeof(float) * (RED ? 2 : 1);
+    const size_t dyn = (size_t)2 * NW * G * VPL * XTraits<XT>::VW * sizeof(float) * (RED ? 2 : 1);
     auto kern = csr_forward_kernel<XT, G, VPL, RED, IT>;
     if (dyn > 16 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
     kern<<<(unsigned)p.ntiles, CSR_THREADS, dyn, s>>>(p);

@@ -74,3 +74,15 @@ def test_host_side_argument_errors(lib):
     assert cdll.tiga_csr_workspace_bytes(ctypes.byref(g), 64, 0, 0, 0) >= 2 * 64 * 4
     assert cdll.tiga_csr_degree_histogram(ctypes.byref(g), 256, 0, 256, None) == 1                          # nbins < 1
     assert cdll.tiga_validate_csr(ctypes.byref(g), 0, None, 0, None) == 0                                   # metadata only
+    # radius: message descriptor, widths, message parameters (all refused before any device access)
+    b.periodic[0] = b.periodic[1] = b.periodic[2] = 0
+    r = ctypes.c_float(0.1)
+    big = 1 << 30
+    assert cdll.tiga_apply_radius(256, 256, 100, 8, r, ctypes.byref(b), None, 256, None, 256, big, None) == 1          # no message
+    assert cdll.tiga_apply_radius(256, 256, 100, 132, r, ctypes.byref(b), ctypes.byref(_Msg(2, 0.1, 0.0)), 256, None, 256, big, None) == 2
+    assert cdll.tiga_apply_radius(256, 256, 100, 8, r, ctypes.byref(b), ctypes.byref(_Msg(2, 0.0, 0.0)), 256, None, 256, big, None) == 1    # sigma <= 0
+    assert cdll.tiga_apply_radius(256, None, 100, 4, r, ctypes.byref(b), ctypes.byref(_Msg(4, 1.0, 0.0)), 256, None, 256, big, None) == 1   # s <= 0
+    assert cdll.tiga_apply_radius(256, 256, 100, 8, r, ctypes.byref(b), ctypes.byref(_Msg(1, 0.0, 0.0)), 256, None, 256, big, None) == 2    # CSR message kind
+    assert cdll.tiga_apply_radius(256, 256, 100, 8, r, ctypes.byref(b), ctypes.byref(_Msg(2, 0.1, 0.0)), 256, None, 256, 64, None) == 3     # workspace
+    assert cdll.tiga_apply_radius_backward(256, 256, 100, 8, r, ctypes.byref(b), ctypes.byref(_Msg(4, 1.0, 1.0)), 256, 256, 256, 256, big, 0, None) == 2
+    assert cdll.tiga_apply_radius_backward(256, 256, 100, 6, r, ctypes.byref(b), ctypes.byref(_Msg(2, 0.1, 0.0)), 256, 256, 256, 256, big, 0, None) == 2
