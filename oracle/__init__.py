@@ -210,3 +210,49 @@ def radius_backward_gauss(pos, feat, gy, r, box, periodic, sigma, rows=None, use
                                           ctypes.c_int(int(use_cells)), _p(gx), _p(Agx), _p(gp), _p(Agp))
     assert rc == 0
     return dict(gx=gx, Agx=Agx, gp=gp, Agp=Agp)
+
+
+# ------------------------------------------------------------------------------ edge neural network
+def _mlp_args(W1, b1, W2, b2):
+    W1 = np.ascontiguousarray(W1, np.float64); b1 = np.ascontiguousarray(b1, np.float64)
+    W2 = np.ascontiguousarray(W2, np.float64); b2 = np.ascontiguousarray(b2, np.float64)
+    return W1, b1, W2, b2
+
+
+def radius_mlp_forward(pos, feat, r, box, periodic, W1, b1, W2, b2, use_cells=False):
+    """y_i = sum_{j in N(i)} [W2 relu(W1 [p_j - p_i; x_j] + b1) + b2]  (Appendix A).
+    Returns (y [n,Fout], A, count)."""
+    lib = _load()
+    pos, r, box, periodic = _geom(pos, r, box, periodic)
+    feat = np.ascontiguousarray(feat, np.float64)
+    W1, b1, W2, b2 = _mlp_args(W1, b1, W2, b2)
+    n, Fin = feat.shape
+    H, Fout = W1.shape[0], W2.shape[0]
+    assert W1.shape == (H, 3 + Fin) and W2.shape == (Fout, H) and H <= 64 and Fout <= 16 and 3 + Fin <= 64
+    y = np.empty((n, Fout)); A = np.empty((n, Fout)); cnt = np.empty(n, np.int32)
+    rc = lib.oracle_radius_mlp_forward(_p(pos), _p(feat), ctypes.c_int64(n), ctypes.c_int(Fin), ctypes.c_double(r),
+                                       _p(box), _p(periodic), _p(W1), _p(b1), _p(W2), _p(b2), ctypes.c_int(H),
+                                       ctypes.c_int(Fout), ctypes.c_int(int(use_cells)), _p(y), _p(A), _p(cnt))
+    assert rc == 0
+    return y, A, cnt
+
+
+def radius_mlp_backward(pos, feat, gy, r, box, periodic, W1, b1, W2, b2, use_cells=False):
+    """Returns dict with gx, gp, gW1, gb1, gW2, gb2 and their abs-sum companions A<name>."""
+    lib = _load()
+    pos, r, box, periodic = _geom(pos, r, box, periodic)
+    feat = np.ascontiguousarray(feat, np.float64); gy = np.ascontiguousarray(gy, np.float64)
+    W1, b1, W2, b2 = _mlp_args(W1, b1, W2, b2)
+    n, Fin = feat.shape
+    H, Fout = W1.shape[0], W2.shape[0]
+    shapes = dict(gx=(n, Fin), gp=(n, 3), gW1=W1.shape, gb1=b1.shape, gW2=W2.shape, gb2=b2.shape)
+    out = {}
+    args = []
+    for k, shp in shapes.items():
+        out[k] = np.empty(shp); out["A" + k] = np.empty(shp)
+        args += [_p(out[k]), _p(out["A" + k])]
+    rc = lib.oracle_radius_mlp_backward(_p(pos), _p(feat), _p(gy), ctypes.c_int64(n), ctypes.c_int(Fin),
+                                        ctypes.c_double(r), _p(box), _p(periodic), _p(W1), _p(b1), _p(W2), _p(b2),
+                                        ctypes.c_int(H), ctypes.c_int(Fout), ctypes.c_int(int(use_cells)), *args)
+    assert rc == 0
+    return out

@@ -501,3 +501,163 @@ int oracle_num_threads(void) {
 #endif
     return n;
 }
+
+/* ------------------------------------------------------------------ edge neural network
+ * Appendix A: over the radius relation N(i) = { j != i : |p_j - p_i| <= r },
+ *     y_i = sum over j in N(i) of [ W2 ReLU( W1 [p_j - p_i ; x_j] + b1 ) + b2 ]
+ * with the displacement taken source minus destination (minimum image where periodic) and the
+ * final bias inside the sum.  W1 is [H, 3 + Fin] row major, W2 is [Fout, H].
+ * Reverse mode with the membership frozen (Section 5), by the plain chain rule per ordered pair:
+ *     mbar = ybar_i,  W2bar += mbar a^T,  b2bar += mbar,  abar = W2^T mbar,
+ *     hbar = abar * [h > 0],  W1bar += hbar u^T,  b1bar += hbar,  ubar = W1^T hbar,
+ *     pbar_j += ubar[0:3],  pbar_i -= ubar[0:3],  xbar_j += ubar[3:].
+ * ReLU'(0) = 0.  Every output has a companion array with the sum of absolute contributions.
+ */
+typedef struct {
+    int Fin, H, Fout;
+    const double *W1, *b1, *W2, *b2;
+} mlp_t;
+
+/* forward of one ordered pair (i <- j); returns h (pre-activation) and u as well */
+static void mlp_pair(const rel_t* R, const double* feat, const mlp_t* M, int64_t i, int64_t j,
+                     const double D_ij[3], double* u, double* h, double* m) {
+    const int K = 3 + M->Fin;
+    for (int d = 0; d < 3; ++d) u[d] = -D_ij[d];              /* p_j - p_i */
+    for (int f = 0; f < M->Fin; ++f) u[3 + f] = feat[j * M->Fin + f];
+    for (int a = 0; a < M->H; ++a) {
+        double s = M->b1[a];
+        for (int k = 0; k < K; ++k) s += M->W1[a * K + k] * u[k];
+        h[a] = s;
+    }
+    for (int o = 0; o < M->Fout; ++o) {
+        double s = M->b2[o];
+        for (int a = 0; a < M->H; ++a) s += M->W2[o * M->H + a] * (h[a] > 0.0 ? h[a] : 0.0);
+        m[o] = s;
+    }
+    (void)R; (void)i;
+}
+
+int oracle_radius_mlp_forward(const double* pos, const double* feat, int64_t n, int Fin,
+                              double r, const double* len, const int32_t* periodic,
+                              const double* W1, const double* b1, const double* W2, const double* b2,
+                              int H, int Fout, int use_cells, double* y, double* A, int32_t* count) {
+    rel_t R;
+    rel_init(&R, pos, n, r, len, periodic);
+    grid_t G = { {0, 0, 0}, NULL, NULL };
+    if (use_cells && grid_build(&R, r, &G)) return 1;
+    mlp_t M = { Fin, H, Fout, W1, b1, W2, b2 };
+#pragma omp parallel
+    {
+        int64_t* buf = NULL;
+        int64_t cap = 0;
+        double u[64], h[64], m[16];
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t i = 0; i < n; ++i) {
+            for (int o = 0; o < Fout; ++o) { y[i * Fout + o] = 0.0; if (A) A[i * Fout + o] = 0.0; }
+            int32_t cnt = 0;
+            int64_t mc = use_cells ? candidates(&R, &G, i, &buf, &cap) : n;
+            for (int64_t t = 0; t < mc; ++t) {
+                int64_t j = use_cells ? buf[t] : t;
+                if (j == i) continue;
+                double D[3], d2;
+                if (!pair_d2(&R, i, j, D, &d2)) continue;
+                ++cnt;
+                mlp_pair(&R, feat, &M, i, j, D, u, h, m);
+                for (int o = 0; o < Fout; ++o) { y[i * Fout + o] += m[o]; if (A) A[i * Fout + o] += fabs(m[o]); }
+            }
+            if (count) count[i] = cnt;
+        }
+        free(buf);
+    }
+    free(G.start);
+    free(G.items);
+    return 0;
+}
+
+/* Outputs (each with its abs-sum companion): gx [n,Fin], gp [n,3], gW1 [H,3+Fin], gb1 [H],
+ * gW2 [Fout,H], gb2 [Fout].  Row k of gx / gp is gathered from the pairs in which k is the
+ * destination and those in which it is the source; parameter gradients are summed over the
+ * ordered pairs by their destination, per thread, and folded in thread order. */
+int oracle_radius_mlp_backward(const double* pos, const double* feat, const double* gy, int64_t n, int Fin,
+                               double r, const double* len, const int32_t* periodic,
+                               const double* W1, const double* b1, const double* W2, const double* b2,
+                               int H, int Fout, int use_cells,
+                               double* gx, double* Agx, double* gp, double* Agp,
+                               double* gW1, double* AgW1, double* gb1, double* Agb1,
+                               double* gW2, double* AgW2, double* gb2, double* Agb2) {
+    rel_t R;
+    rel_init(&R, pos, n, r, len, periodic);
+    grid_t G = { {0, 0, 0}, NULL, NULL };
+    if (use_cells && grid_build(&R, r, &G)) return 1;
+    mlp_t M = { Fin, H, Fout, W1, b1, W2, b2 };
+    const int K = 3 + Fin;
+    const int NP = H * K + H + Fout * H + Fout;
+    for (int e = 0; e < H * K; ++e) { gW1[e] = 0.0; AgW1[e] = 0.0; }
+    for (int e = 0; e < H; ++e) { gb1[e] = 0.0; Agb1[e] = 0.0; }
+    for (int e = 0; e < Fout * H; ++e) { gW2[e] = 0.0; AgW2[e] = 0.0; }
+    for (int e = 0; e < Fout; ++e) { gb2[e] = 0.0; Agb2[e] = 0.0; }
+#pragma omp parallel
+    {
+        int64_t* buf = NULL;
+        int64_t cap = 0;
+        double u[64], h[64], m[16], hb[64], ub[64];
+        double* acc = (double*)calloc((size_t)2 * NP, sizeof(double));     /* gradients, then abs sums */
+        double* aW1 = acc, *ab1 = aW1 + H * K, *aW2 = ab1 + H, *ab2 = aW2 + Fout * H;
+        double* sW1 = acc + NP, *sb1 = sW1 + H * K, *sW2 = sb1 + H, *sb2 = sW2 + Fout * H;
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t k = 0; k < n; ++k) {
+            for (int f = 0; f < Fin; ++f) { gx[k * Fin + f] = 0.0; Agx[k * Fin + f] = 0.0; }
+            for (int d = 0; d < 3; ++d) { gp[k * 3 + d] = 0.0; Agp[k * 3 + d] = 0.0; }
+            int64_t mc = use_cells ? candidates(&R, &G, k, &buf, &cap) : n;
+            for (int64_t t = 0; t < mc; ++t) {
+                int64_t o = use_cells ? buf[t] : t;
+                if (o == k) continue;
+                double D[3], d2;
+                for (int role = 0; role < 2; ++role) {
+                    /* role 0: k is the destination i, o the source j; role 1: o destination, k source */
+                    const int64_t i = role == 0 ? k : o, j = role == 0 ? o : k;
+                    if (!pair_d2(&R, i, j, D, &d2)) continue;
+                    mlp_pair(&R, feat, &M, i, j, D, u, h, m);
+                    for (int a = 0; a < H; ++a) {
+                        double s = 0.0;
+                        for (int q = 0; q < Fout; ++q) s += W2[q * H + a] * gy[i * Fout + q];
+                        hb[a] = h[a] > 0.0 ? s : 0.0;
+                    }
+                    for (int c = 0; c < K; ++c) {
+                        double s = 0.0;
+                        for (int a = 0; a < H; ++a) s += W1[a * K + c] * hb[a];
+                        ub[c] = s;
+                    }
+                    if (role == 0) {
+                        for (int d = 0; d < 3; ++d) { gp[k * 3 + d] -= ub[d]; Agp[k * 3 + d] += fabs(ub[d]); }
+                        for (int a = 0; a < H; ++a) {
+                            for (int c = 0; c < K; ++c) { aW1[a * K + c] += hb[a] * u[c]; sW1[a * K + c] += fabs(hb[a] * u[c]); }
+                            ab1[a] += hb[a]; sb1[a] += fabs(hb[a]);
+                            const double act = h[a] > 0.0 ? h[a] : 0.0;
+                            for (int q = 0; q < Fout; ++q) {
+                                aW2[q * H + a] += gy[i * Fout + q] * act;
+                                sW2[q * H + a] += fabs(gy[i * Fout + q] * act);
+                            }
+                        }
+                        for (int q = 0; q < Fout; ++q) { ab2[q] += gy[i * Fout + q]; sb2[q] += fabs(gy[i * Fout + q]); }
+                    } else {
+                        for (int d = 0; d < 3; ++d) { gp[k * 3 + d] += ub[d]; Agp[k * 3 + d] += fabs(ub[d]); }
+                        for (int f = 0; f < Fin; ++f) { gx[k * Fin + f] += ub[3 + f]; Agx[k * Fin + f] += fabs(ub[3 + f]); }
+                    }
+                }
+            }
+        }
+#pragma omp critical
+        {
+            for (int e = 0; e < H * K; ++e) { gW1[e] += aW1[e]; AgW1[e] += sW1[e]; }
+            for (int e = 0; e < H; ++e) { gb1[e] += ab1[e]; Agb1[e] += sb1[e]; }
+            for (int e = 0; e < Fout * H; ++e) { gW2[e] += aW2[e]; AgW2[e] += sW2[e]; }
+            for (int e = 0; e < Fout; ++e) { gb2[e] += ab2[e]; Agb2[e] += sb2[e]; }
+        }
+        free(acc);
+        free(buf);
+    }
+    free(G.start);
+    free(G.items);
+    return 0;
+}
