@@ -490,6 +490,34 @@ def run_paper_shapes(args):
         rows.append({"shape": f"dynamic radius (rebuilt every call), distance-weighted scalar sum, N={n}", "pairs": pairs, "F": 1,
                      "ms_median": med, "ms_min": lo, "ms_max": hi, "interactions_per_s": pairs / (med * 1e-3),
                      "paper": "1.84 ms at N=131,072 (PyG 80.24 ms, chunked Torch 1870 ms; RTX 5070 Ti)" if n == 131072 else "figure only"})
+    # differentiated edge network (Appendix A / supplementary study): 35,947 points on a synthetic closed
+    # surface, cutoff 0.015, 8 node features, 4 outputs; forward includes the relation rebuild
+    n = 35_947
+    pos, x, gy = to(gen.surface_points(n, args.seed)), to(gen.normal_features(n, 8, args.seed, 31)), to(gen.normal_features(n, 4, args.seed, 32))
+    ones, nonper = np.ones(3, np.float32), [0, 0, 0]
+    for hidden, paper in ((8, "fwd 0.86 ms, loss+bwd 0.72 ms (Torch 0.64 / 2.07)"), (16, "example width, no timing printed"),
+                          (32, "fwd 0.92 ms, loss+bwd 8.86 ms (Torch 0.94 / 2.42)")):
+        P = [to(a) for a in gen.mlp_params(8, hidden, 4, args.seed)]
+        out, cnt, ws = T.tiga_apply_radius_mlp(pos, x, 0.015, ones, nonper, *P, want_count=True)
+        pairs = int(cnt.sum().item())
+        fwd = median_ms(lambda: T.tiga_apply_radius_mlp(pos, x, 0.015, ones, nonper, *P, out=out, ws=ws))
+        bwd = median_ms(lambda: T.tiga_apply_radius_mlp_backward(pos, x, gy, 0.015, ones, nonper, *P, ws=ws, reuse_plan=True))
+        rows.append({"shape": f"edge network on a radius graph, 35,947 surface points, r=0.015, hidden {hidden}", "pairs": pairs,
+                     "ms_median": fwd[0], "ms_min": fwd[1], "ms_max": fwd[2], "backward_ms_median": bwd[0],
+                     "backward_ms_min": bwd[1], "backward_ms_max": bwd[2], "interactions_per_s": pairs / (fwd[0] * 1e-3),
+                     "paper": paper + " on the Stanford Bunny vertices, 356,260 edges (RTX 5070 Ti)"})
+    c = gen.config("cfg2", args.seed, F=8)
+    pos, x, gy = to(c["pos"]), to(c["x"]), to(gen.normal_features(c["n"], 4, args.seed, 33))
+    P = [to(a) for a in gen.mlp_params(8, 16, 4, args.seed)]
+    out, cnt, ws = T.tiga_apply_radius_mlp(pos, x, c["r"], c["box"], c["periodic"], *P, want_count=True)
+    pairs = int(cnt.sum().item())
+    fwd = median_ms(lambda: T.tiga_apply_radius_mlp(pos, x, c["r"], c["box"], c["periodic"], *P, out=out, ws=ws))
+    bwd = median_ms(lambda: T.tiga_apply_radius_mlp_backward(pos, x, gy, c["r"], c["box"], c["periodic"], *P, ws=ws, reuse_plan=True))
+    flop_f = 2.0 * (16 * 11 + 4 * 16) * pairs
+    rows.append({"shape": "edge network, 1,000,000 periodic points, 32 neighbours, 8 features, hidden 16", "pairs": pairs,
+                 "ms_median": fwd[0], "ms_min": fwd[1], "ms_max": fwd[2], "backward_ms_median": bwd[0],
+                 "backward_ms_min": bwd[1], "backward_ms_max": bwd[2], "interactions_per_s": pairs / (fwd[0] * 1e-3),
+                 "forward_tflops_fp32": flop_f / (fwd[0] * 1e-3) / 1e12, "paper": "not measured in the paper"})
     print(json.dumps({"case": "paper_shapes", "protocol": "warm, 4 warm-ups, 10 timed calls, median (min, max)", "rows": rows}))
 
 

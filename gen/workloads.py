@@ -18,7 +18,7 @@ __all__ = [
     "DEFAULT_SEED", "build_generators", "rng", "sha256_of", "rmat_csr", "rmat_edge",
     "edge_weights", "normal_features", "small_int_features", "small_int_weights",
     "uniform_points", "jittered_lattice", "hex_mesh_csr", "periodic_offset_csr",
-    "regular_random_csr", "radius_for_expected_neighbours", "config",
+    "regular_random_csr", "radius_for_expected_neighbours", "config", "surface_points", "mlp_params",
 ]
 
 DEFAULT_SEED = 20260921
@@ -258,3 +258,24 @@ def config(name: str, seed: int = DEFAULT_SEED, **over):
             d["w"] = None
         return d
     raise KeyError(name)
+
+
+def surface_points(n: int, seed: int = DEFAULT_SEED) -> np.ndarray:
+    """n points on a closed, bumpy surface inside the unit cube (a stand-in for a scanned mesh's
+    vertex list: positions only, roughly uniform over the surface)."""
+    g = rng(seed, 81)
+    v = g.standard_normal((n, 3))
+    v /= np.linalg.norm(v, axis=1, keepdims=True)
+    rad = 0.34 + 0.05 * np.sin(5.0 * v[:, 0]) * np.cos(3.0 * v[:, 1]) + 0.04 * v[:, 2] ** 2
+    return (0.5 + v * rad[:, None]).astype(np.float32)
+
+
+def mlp_params(f_in: int, hidden: int, f_out: int, seed: int = DEFAULT_SEED):
+    """Random edge-network parameters (W1 [hidden, 3+f_in], b1, W2 [f_out, hidden], b2), fp32."""
+    g = rng(seed, 82)
+    k = 3 + f_in
+    W1 = (g.uniform(-1, 1, (hidden, k)) / np.sqrt(k)).astype(np.float32)
+    b1 = (g.uniform(-1, 1, hidden) / np.sqrt(k)).astype(np.float32)
+    W2 = (g.uniform(-1, 1, (f_out, hidden)) / np.sqrt(hidden)).astype(np.float32)
+    b2 = (g.uniform(-1, 1, f_out) / np.sqrt(hidden)).astype(np.float32)
+    return W1, b1, W2, b2

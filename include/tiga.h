@@ -213,6 +213,44 @@ tiga_status tiga_apply_radius_backward(const float* pos, const float* feat, int6
                                        const float* grad_out, float* grad_feat, float* grad_pos,
                                        void* ws, size_t ws_bytes, int reuse_plan, void* stream);
 
+/* ----------------------------------------------------------------- radius, edge network */
+
+/* Shared edge-local network of the paper's Appendix A, evaluated per selected edge (i <- j):
+ *     m_ij = W2 ReLU( W1 [p_j - p_i ; x_j] + b1 ) + b2
+ * (displacement source minus destination, minimum image where periodic; the final bias is part
+ * of every message).  All four arrays are DEVICE pointers, row major. */
+typedef struct {
+    int32_t f_in;       /* node feature width, 1..13 */
+    int32_t hidden;     /* 8, 16 or 32 */
+    int32_t f_out;      /* 1..4 */
+    const float* W1;    /* [hidden, 3 + f_in]; columns 0..2 multiply the displacement */
+    const float* b1;    /* [hidden] */
+    const float* W2;    /* [f_out, hidden] */
+    const float* b2;    /* [f_out] */
+} tiga_edge_mlp;
+
+/* Fused generated-relation apply with the edge network as the message (Appendix A, Section 4.9):
+ *     out[i,:] = sum over j in N(i) of m_ij,   zero vector without neighbours.
+ *   feat : fp32 [n, f_in];  out : fp32 [n, f_out];  count : int32 [n] or NULL.
+ * Bins the points first (plan left in ws).  ws: tiga_radius_workspace_bytes(n, f_in, r, box, 0). */
+tiga_status tiga_apply_radius_mlp(const float* pos, const float* feat, int64_t n, float r, const tiga_box* box,
+                                  const tiga_edge_mlp* mlp, float* out, int32_t* count,
+                                  void* ws, size_t ws_bytes, void* stream);
+
+/* Reverse mode of tiga_apply_radius_mlp with the membership frozen (Section 5, Appendix A): the
+ * activations are recomputed per pair, nothing of size E is stored.
+ *   grad_out : fp32 [n, f_out]
+ *   grad_feat [n, f_in], grad_pos [n, 3], grad_W1 [hidden, 3 + f_in], grad_b1 [hidden],
+ *   grad_W2 [f_out, hidden], grad_b2 [f_out]: each fp32, overwritten, or NULL to skip.
+ * Feature and position gradients are owner-computed (no atomics, reproducible); the parameter
+ * gradients are summed with floating-point atomics and may differ in the last bits between runs.
+ * ReLU'(0) = 0.  reuse_plan as in tiga_apply_radius_backward. */
+tiga_status tiga_apply_radius_mlp_backward(const float* pos, const float* feat, int64_t n, float r, const tiga_box* box,
+                                           const tiga_edge_mlp* mlp, const float* grad_out,
+                                           float* grad_feat, float* grad_pos,
+                                           float* grad_W1, float* grad_b1, float* grad_W2, float* grad_b2,
+                                           void* ws, size_t ws_bytes, int reuse_plan, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -237,8 +237,10 @@ def radius_mlp_forward(pos, feat, r, box, periodic, W1, b1, W2, b2, use_cells=Fa
     return y, A, cnt
 
 
-def radius_mlp_backward(pos, feat, gy, r, box, periodic, W1, b1, W2, b2, use_cells=False):
-    """Returns dict with gx, gp, gW1, gb1, gW2, gb2 and their abs-sum companions A<name>."""
+def radius_mlp_backward(pos, feat, gy, r, box, periodic, W1, b1, W2, b2, use_cells=False, kink_eps=0.0):
+    """Returns dict with gx, gp, gW1, gb1, gW2, gb2, their abs-sum companions A<name>, and
+    ``kink`` (int32 [n]): 1 where some pair the point takes part in has a pre-activation with
+    |h| < kink_eps (the ReLU derivative is discontinuous there)."""
     lib = _load()
     pos, r, box, periodic = _geom(pos, r, box, periodic)
     feat = np.ascontiguousarray(feat, np.float64); gy = np.ascontiguousarray(gy, np.float64)
@@ -246,13 +248,14 @@ def radius_mlp_backward(pos, feat, gy, r, box, periodic, W1, b1, W2, b2, use_cel
     n, Fin = feat.shape
     H, Fout = W1.shape[0], W2.shape[0]
     shapes = dict(gx=(n, Fin), gp=(n, 3), gW1=W1.shape, gb1=b1.shape, gW2=W2.shape, gb2=b2.shape)
-    out = {}
+    out = {"kink": np.zeros(n, np.int32)}
     args = []
     for k, shp in shapes.items():
         out[k] = np.empty(shp); out["A" + k] = np.empty(shp)
         args += [_p(out[k]), _p(out["A" + k])]
     rc = lib.oracle_radius_mlp_backward(_p(pos), _p(feat), _p(gy), ctypes.c_int64(n), ctypes.c_int(Fin),
                                         ctypes.c_double(r), _p(box), _p(periodic), _p(W1), _p(b1), _p(W2), _p(b2),
-                                        ctypes.c_int(H), ctypes.c_int(Fout), ctypes.c_int(int(use_cells)), *args)
+                                        ctypes.c_int(H), ctypes.c_int(Fout), ctypes.c_int(int(use_cells)),
+                                        ctypes.c_double(float(kink_eps)), _p(out["kink"]), *args)
     assert rc == 0
     return out

@@ -512,6 +512,11 @@ int oracle_num_threads(void) {
  *     hbar = abar * [h > 0],  W1bar += hbar u^T,  b1bar += hbar,  ubar = W1^T hbar,
  *     pbar_j += ubar[0:3],  pbar_i -= ubar[0:3],  xbar_j += ubar[3:].
  * ReLU'(0) = 0.  Every output has a companion array with the sum of absolute contributions.
+ * ReLU makes the gradient discontinuous where a pre-activation crosses zero; a lower-precision
+ * evaluation can land on the other side there.  The backward therefore also reports, per
+ * point, whether any pair it takes part in has a pre-activation with |h| < kink_eps, so that a
+ * comparison can leave exactly those rows out (Section 5: ReLU-like kinks need appropriate
+ * test points).
  */
 typedef struct {
     int Fin, H, Fout;
@@ -581,7 +586,7 @@ int oracle_radius_mlp_forward(const double* pos, const double* feat, int64_t n, 
 int oracle_radius_mlp_backward(const double* pos, const double* feat, const double* gy, int64_t n, int Fin,
                                double r, const double* len, const int32_t* periodic,
                                const double* W1, const double* b1, const double* W2, const double* b2,
-                               int H, int Fout, int use_cells,
+                               int H, int Fout, int use_cells, double kink_eps, int32_t* kink,
                                double* gx, double* Agx, double* gp, double* Agp,
                                double* gW1, double* AgW1, double* gb1, double* Agb1,
                                double* gW2, double* AgW2, double* gb2, double* Agb2) {
@@ -608,6 +613,7 @@ int oracle_radius_mlp_backward(const double* pos, const double* feat, const doub
         for (int64_t k = 0; k < n; ++k) {
             for (int f = 0; f < Fin; ++f) { gx[k * Fin + f] = 0.0; Agx[k * Fin + f] = 0.0; }
             for (int d = 0; d < 3; ++d) { gp[k * 3 + d] = 0.0; Agp[k * 3 + d] = 0.0; }
+            if (kink) kink[k] = 0;
             int64_t mc = use_cells ? candidates(&R, &G, k, &buf, &cap) : n;
             for (int64_t t = 0; t < mc; ++t) {
                 int64_t o = use_cells ? buf[t] : t;
@@ -618,6 +624,7 @@ int oracle_radius_mlp_backward(const double* pos, const double* feat, const doub
                     const int64_t i = role == 0 ? k : o, j = role == 0 ? o : k;
                     if (!pair_d2(&R, i, j, D, &d2)) continue;
                     mlp_pair(&R, feat, &M, i, j, D, u, h, m);
+                    if (kink) for (int a = 0; a < H; ++a) if (fabs(h[a]) < kink_eps) kink[k] = 1;
                     for (int a = 0; a < H; ++a) {
                         double s = 0.0;
                         for (int q = 0; q < Fout; ++q) s += W2[q * H + a] * gy[i * Fout + q];

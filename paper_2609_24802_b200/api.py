@@ -17,7 +17,8 @@ __all__ = [
     "CsrRelation", "tiga_status_string", "tiga_csr_workspace_bytes", "tiga_validate_csr",
     "tiga_apply_csr", "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram",
     "tiga_radius_grid", "tiga_radius_workspace_bytes", "tiga_radius_bin",
-    "tiga_apply_radius", "tiga_apply_radius_backward", "launch_count",
+    "tiga_apply_radius", "tiga_apply_radius_backward", "tiga_apply_radius_mlp",
+    "tiga_apply_radius_mlp_backward", "launch_count",
 ]
 
 SUM, MAX = 0, 1
@@ -29,7 +30,7 @@ EXPORTS = [
     "tiga_status_string", "tiga_csr_workspace_bytes", "tiga_validate_csr", "tiga_apply_csr",
     "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram", "tiga_radius_grid",
     "tiga_radius_workspace_bytes", "tiga_radius_bin", "tiga_apply_radius",
-    "tiga_apply_radius_backward",
+    "tiga_apply_radius_backward", "tiga_apply_radius_mlp", "tiga_apply_radius_mlp_backward",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -53,6 +54,11 @@ class _Csr(ctypes.Structure):
 
 class _Box(ctypes.Structure):
     _fields_ = [("len", ctypes.c_float * 3), ("periodic", ctypes.c_int32 * 3)]
+
+
+class _EdgeMlp(ctypes.Structure):
+    _fields_ = [("f_in", ctypes.c_int32), ("hidden", ctypes.c_int32), ("f_out", ctypes.c_int32),
+                ("W1", ctypes.c_void_p), ("b1", ctypes.c_void_p), ("W2", ctypes.c_void_p), ("b2", ctypes.c_void_p)]
 
 
 _lib = None
@@ -97,6 +103,11 @@ def load_library() -> ctypes.CDLL:
     lib.tiga_apply_radius_backward.restype = ctypes.c_int
     lib.tiga_apply_radius_backward.argtypes = [vp, vp, i64, i32, f, ctypes.POINTER(_Box), ctypes.POINTER(_Msg), vp, vp, vp,
                                                vp, sz, ctypes.c_int, vp]
+    lib.tiga_apply_radius_mlp.restype = ctypes.c_int
+    lib.tiga_apply_radius_mlp.argtypes = [vp, vp, i64, f, ctypes.POINTER(_Box), ctypes.POINTER(_EdgeMlp), vp, vp, vp, sz, vp]
+    lib.tiga_apply_radius_mlp_backward.restype = ctypes.c_int
+    lib.tiga_apply_radius_mlp_backward.argtypes = [vp, vp, i64, f, ctypes.POINTER(_Box), ctypes.POINTER(_EdgeMlp), vp,
+                                                   vp, vp, vp, vp, vp, vp, vp, sz, ctypes.c_int, vp]
     _lib = lib
     return lib
 
@@ -325,3 +336,53 @@ def tiga_apply_radius_backward(pos, feat, grad_out, r: float, box, periodic, sig
         "tiga_apply_radius_backward")
     _launches += 1 if reuse_plan else 7
     return grad_feat, grad_pos
+
+
+def _edge_mlp(W1, b1, W2, b2):
+    for t in (W1, b1, W2, b2):
+        assert t.is_cuda and t.is_contiguous() and t.dtype == torch.float32
+    H, K = W1.shape
+    return _EdgeMlp(K - 3, H, W2.shape[0], W1.data_ptr(), b1.data_ptr(), W2.data_ptr(), b2.data_ptr())
+
+
+def tiga_apply_radius_mlp(pos, feat, r: float, box, periodic, W1, b1, W2, b2, out=None, count=None,
+                          want_count=False, ws=None, stream=None):
+    """out[i] = sum_{j in N(i)} [W2 relu(W1 [p_j - p_i; x_j] + b1) + b2].  Returns (out, count, ws)."""
+    global _launches
+    n = pos.shape[0]
+    m = _edge_mlp(W1, b1, W2, b2)
+    bx = _box(box, periodic)
+    if out is None:
+        out = torch.empty((n, m.f_out), dtype=torch.float32, device=pos.device)
+    if want_count and count is None:
+        count = torch.empty(n, dtype=torch.int32, device=pos.device)
+    if ws is None:
+        ws = _ws(tiga_radius_workspace_bytes(n, m.f_in, r, box, periodic), pos)
+    _ok(load_library().tiga_apply_radius_mlp(_ptr(pos), _ptr(feat), n, float(r), ctypes.byref(bx), ctypes.byref(m),
+                                             _ptr(out), _ptr(count), _ptr(ws), ws.numel(), _stream(stream)),
+        "tiga_apply_radius_mlp")
+    _launches += 7
+    return out, count, ws
+
+
+def tiga_apply_radius_mlp_backward(pos, feat, grad_out, r: float, box, periodic, W1, b1, W2, b2, ws=None,
+                                   reuse_plan=False, stream=None):
+    """Returns dict(grad_feat, grad_pos, grad_W1, grad_b1, grad_W2, grad_b2)."""
+    global _launches
+    n = pos.shape[0]
+    m = _edge_mlp(W1, b1, W2, b2)
+    bx = _box(box, periodic)
+    dev = pos.device
+    g = dict(grad_feat=torch.empty((n, m.f_in), device=dev), grad_pos=torch.empty((n, 3), device=dev),
+             grad_W1=torch.empty_like(W1), grad_b1=torch.empty_like(b1), grad_W2=torch.empty_like(W2),
+             grad_b2=torch.empty_like(b2))
+    if ws is None:
+        assert not reuse_plan
+        ws = _ws(tiga_radius_workspace_bytes(n, m.f_in, r, box, periodic, True), pos)
+    _ok(load_library().tiga_apply_radius_mlp_backward(_ptr(pos), _ptr(feat), n, float(r), ctypes.byref(bx), ctypes.byref(m),
+                                                      _ptr(grad_out), _ptr(g["grad_feat"]), _ptr(g["grad_pos"]),
+                                                      _ptr(g["grad_W1"]), _ptr(g["grad_b1"]), _ptr(g["grad_W2"]),
+                                                      _ptr(g["grad_b2"]), _ptr(ws), ws.numel(), int(bool(reuse_plan)),
+                                                      _stream(stream)), "tiga_apply_radius_mlp_backward")
+    _launches += 1 if reuse_plan else 7
+    return g

@@ -20,50 +20,13 @@
 // neighbour set equals the double-precision one.  Periodic images are formed by
 // subtracting the box length from whichever of the two coordinates lies next to the upper
 // face, which is exact in fp32, so wrapped pairs are as accurate as interior ones.
-#include "common.cuh"
-#include <math.h>
+#include "radius_shared.cuh"
 #include <type_traits>
 
 namespace tiga {
 
 constexpr int RAD_THREADS = 256;
 constexpr int SCAN_BLOCK = 2048;   // elements per CTA in the scan passes
-
-struct RadiusParams {
-    const float* pos;
-    const float* feat;
-    const float* gy;
-    float* out;
-    int32_t* count;
-    float* gfeat;
-    float* gpos;
-    int n;
-    int F;
-    float r;
-    float r2_lo, r2_hi;       // fp32 filter band around r^2
-    float r2_mid, r2_band;    // its centre and half width
-    double r2_exact;          // (double)r * (double)r
-    float len[3];
-    float inv_len[3];
-    int periodic[3];
-    int nc[3];
-    float invh[3];
-    float hcell[3];           // cell edge, len / nc
-    int ncells;
-    float p0, p1;             // message parameters
-    // plan (workspace)
-    int32_t* cell;
-    int32_t* cnt;
-    int32_t* cell_start;
-    int32_t* order_tmp;
-    int32_t* order;
-    float4* spos;             // positions in cell order, .w = original point id (bit pattern)
-    int32_t* blocksum;
-    // optional user copies of the plan
-    int32_t* u_cell;
-    int32_t* u_cell_start;
-    int32_t* u_order;
-};
 
 // ------------------------------------------------------------------------------ binning
 __global__ void bin_count_kernel(const RadiusParams p) {
@@ -197,37 +160,6 @@ __global__ void bin_sort_kernel(const RadiusParams p) {
 }
 
 // ------------------------------------------------------------------------------ traversal
-constexpr int TRAV_WARPS = 4;
-constexpr int TRAV_THREADS = TRAV_WARPS * 32;
-
-// The defining predicate in double precision (same operations as the plain definition).
-__device__ __noinline__ bool exact_within(const RadiusParams& p, const float4 a, const float4 b) {
-    const float pa[3] = {a.x, a.y, a.z}, pb[3] = {b.x, b.y, b.z};
-    double d2 = 0.0;
-#pragma unroll
-    for (int d = 0; d < 3; ++d) {
-        double t = __dsub_rn((double)pa[d], (double)pb[d]);
-        if (p.periodic[d]) {
-            const double L = (double)p.len[d];
-            t = __dsub_rn(t, __dmul_rn(L, rint(__ddiv_rn(t, L))));
-        }
-        const double sq = __dmul_rn(t, t);
-        d2 = (d == 0) ? sq : __dadd_rn(d2, sq);
-    }
-    return d2 <= p.r2_exact;
-}
-
-__device__ __forceinline__ float fast_exp2(float x) {
-    float r;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-    return r;
-}
-
-__device__ __forceinline__ float fast_rcp(float x) {
-    float r;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-    return r;
-}
 
 // One warp per query cell.
 //   staging : the candidates of the 27-cell stencil (contiguous ranges of the cell-sorted
@@ -246,9 +178,6 @@ __device__ __forceinline__ float fast_rcp(float x) {
 //             a query's list and evaluate the pair forces.
 // Lists hold QCAP entries per query and the stage STAGE_CAP candidates; when either fills up
 // the warp drains / processes and goes on, so any density works.
-constexpr int STAGE_PAD = 32;           // sentinels behind the staged candidates: no bounds checks
-constexpr int QB = 8;                   // queries per batch
-constexpr float FAR_AWAY = 1.0e18f;
 
 template <int MODE> struct TravSmem {
     // sized for the workloads' densities (about 216 / 351 candidates, 32 / 54 neighbours);
@@ -261,13 +190,6 @@ template <int MODE> struct TravSmem {
     static constexpr int MISC_BYTES = QB * 16 + QB * 4 * 2;          // query coordinates, counts, totals
     static constexpr int PER_WARP = STAGE_BYTES + LIST_BYTES + MISC_BYTES;
 };
-
-// exact predicate for the pair of original point ids (a, b)
-__device__ __noinline__ bool exact_pair(const RadiusParams& p, int a, int b) {
-    const float4 pa = make_float4(p.pos[3 * (size_t)a], p.pos[3 * (size_t)a + 1], p.pos[3 * (size_t)a + 2], 0.f);
-    const float4 pb = make_float4(p.pos[3 * (size_t)b], p.pos[3 * (size_t)b + 1], p.pos[3 * (size_t)b + 2], 0.f);
-    return exact_within(p, pa, pb);
-}
 
 // MODE 0: Gaussian (DIST = false) or distance-weighted (DIST = true) forward; 1: Lennard-Jones;
 // 2: Gaussian backward.  MI: some periodic dimension has a single cell (explicit minimum image).
@@ -626,12 +548,7 @@ static tiga_status make_grid(long long n, float r, const tiga_box* box, int nc[3
     return TIGA_OK;
 }
 
-struct RadiusLayout {
-    size_t bytes;
-    int nblocks;
-};
-
-static RadiusLayout carve_radius(RadiusParams* p, void* ws, int32_t** fill) {
+RadiusLayout carve_radius(RadiusParams* p, void* ws, int32_t** fill) {
     Carver cv(ws);
     const size_t n = (size_t)p->n, nc = (size_t)p->ncells;
     const int nblocks = (int)((nc + SCAN_BLOCK - 1) / SCAN_BLOCK);
@@ -646,7 +563,7 @@ static RadiusLayout carve_radius(RadiusParams* p, void* ws, int32_t** fill) {
     return RadiusLayout{cv.off, nblocks};
 }
 
-static tiga_status fill_params(RadiusParams* p, long long n, float r, const tiga_box* box) {
+tiga_status fill_params(RadiusParams* p, long long n, float r, const tiga_box* box) {
     int nc[3];
     float invh[3];
     tiga_status st = make_grid(n, r, box, nc, invh);
@@ -673,7 +590,7 @@ static tiga_status fill_params(RadiusParams* p, long long n, float r, const tiga
     return TIGA_OK;
 }
 
-static tiga_status run_binning(RadiusParams& p, int32_t* fill, int nblocks, cudaStream_t s) {
+tiga_status run_binning(RadiusParams& p, int32_t* fill, int nblocks, cudaStream_t s) {
     if (p.n == 0) return TIGA_OK;
     TIGA_CUDA_TRY(cudaMemsetAsync(p.cnt, 0, (2 * (size_t)p.ncells + 2) * sizeof(int32_t), s));
     const unsigned pb = (unsigned)((p.n + 255) / 256);

@@ -1,0 +1,101 @@
+// Pieces of the generated-radius path shared by radius.cu (binning, Gaussian / distance /
+// Lennard-Jones traversals) and radius_mlp.cu (edge-network message).
+#pragma once
+#include "common.cuh"
+#include <math.h>
+
+namespace tiga {
+
+constexpr int TRAV_WARPS = 4;
+constexpr int TRAV_THREADS = TRAV_WARPS * 32;
+constexpr int STAGE_PAD = 32;           // sentinels behind the staged candidates: no bounds checks
+constexpr int QB = 8;                   // queries per batch
+constexpr float FAR_AWAY = 1.0e18f;
+
+struct RadiusParams {
+    const float* pos;
+    const float* feat;
+    const float* gy;
+    float* out;
+    int32_t* count;
+    float* gfeat;
+    float* gpos;
+    int n;
+    int F;
+    float r;
+    float r2_lo, r2_hi;       // fp32 filter band around r^2
+    float r2_mid, r2_band;    // its centre and half width
+    double r2_exact;          // (double)r * (double)r
+    float len[3];
+    float inv_len[3];
+    int periodic[3];
+    int nc[3];
+    float invh[3];
+    float hcell[3];           // cell edge, len / nc
+    int ncells;
+    float p0, p1;             // message parameters
+    // edge network (radius_mlp.cu): device pointers to W1 [H, 3+Fin], b1 [H], W2 [Fout, H], b2 [Fout]
+    const float *W1, *b1, *W2, *b2;
+    float *gW1, *gb1, *gW2, *gb2;
+    int Fin, Fout;
+    // plan (workspace)
+    int32_t* cell;
+    int32_t* cnt;
+    int32_t* cell_start;
+    int32_t* order_tmp;
+    int32_t* order;
+    float4* spos;             // positions in cell order, .w = original point id (bit pattern)
+    int32_t* blocksum;
+    // optional user copies of the plan
+    int32_t* u_cell;
+    int32_t* u_cell_start;
+    int32_t* u_order;
+};
+
+struct RadiusLayout {
+    size_t bytes;
+    int nblocks;
+};
+
+// host side, defined in radius.cu
+tiga_status fill_params(RadiusParams* p, long long n, float r, const tiga_box* box);
+RadiusLayout carve_radius(RadiusParams* p, void* ws, int32_t** fill);
+tiga_status run_binning(RadiusParams& p, int32_t* fill, int nblocks, cudaStream_t s);
+
+// The defining predicate in double precision (same operations as the plain definition).
+static __device__ __noinline__ bool exact_within(const RadiusParams& p, const float4 a, const float4 b) {
+    const float pa[3] = {a.x, a.y, a.z}, pb[3] = {b.x, b.y, b.z};
+    double d2 = 0.0;
+#pragma unroll
+    for (int d = 0; d < 3; ++d) {
+        double t = __dsub_rn((double)pa[d], (double)pb[d]);
+        if (p.periodic[d]) {
+            const double L = (double)p.len[d];
+            t = __dsub_rn(t, __dmul_rn(L, rint(__ddiv_rn(t, L))));
+        }
+        const double sq = __dmul_rn(t, t);
+        d2 = (d == 0) ? sq : __dadd_rn(d2, sq);
+    }
+    return d2 <= p.r2_exact;
+}
+
+static __device__ __forceinline__ float fast_exp2(float x) {
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+static __device__ __forceinline__ float fast_rcp(float x) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+// exact predicate for the pair of original point ids (a, b)
+static __device__ __noinline__ bool exact_pair(const RadiusParams& p, int a, int b) {
+    const float4 pa = make_float4(p.pos[3 * (size_t)a], p.pos[3 * (size_t)a + 1], p.pos[3 * (size_t)a + 2], 0.f);
+    const float4 pb = make_float4(p.pos[3 * (size_t)b], p.pos[3 * (size_t)b + 1], p.pos[3 * (size_t)b + 2], 0.f);
+    return exact_within(p, pa, pb);
+}
+
+}  // namespace tiga

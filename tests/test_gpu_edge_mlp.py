@@ -1,0 +1,85 @@
+"""GPU parity of the edge-network message over the radius relation (paper Appendix A) against the
+fp64 oracle: outputs within 1e-5 and every gradient (features, positions, W1, b1, W2, b2) within
+1e-4 of the sum of absolute contributions; neighbour counts bit-exact."""
+import numpy as np
+import pytest
+
+import gen
+import oracle
+from parity import GRAD_TOL, SUM_TOL, dev, host, rel_err
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tiga():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2609_24802_b200 import api
+    return api
+
+
+def _check(tiga, pos, x, gy, r, box, per, params, use_cells=True, backward=True, kink_eps=1e-5, min_keep=0.95):
+    y, A, cnt = oracle.radius_mlp_forward(pos, x, r, box, per, *params, use_cells=use_cells)
+    pd, xd = dev(pos, torch), dev(x, torch)
+    P = [dev(a, torch) for a in params]
+    out, count, ws = tiga.tiga_apply_radius_mlp(pd, xd, r, box, per, *P, want_count=True)
+    assert np.array_equal(host(count), cnt), "neighbour counts must be bit exact"
+    assert rel_err(host(out), y, A) <= SUM_TOL
+    if backward:
+        # rows that touch a pre-activation within kink_eps of the ReLU kink are left out of the per-row
+        # comparison: fp32 and fp64 may take different sides there and the derivative jumps
+        ref = oracle.radius_mlp_backward(pos, x, gy, r, box, per, *params, use_cells=use_cells, kink_eps=kink_eps)
+        keep = ref["kink"] == 0
+        assert keep.mean() > min_keep
+        g = tiga.tiga_apply_radius_mlp_backward(pd, xd, dev(gy, torch), r, box, per, *P, ws=ws, reuse_plan=True)
+        for ours, name in (("grad_feat", "gx"), ("grad_pos", "gp")):
+            assert rel_err(host(g[ours])[keep], ref[name][keep], ref["A" + name][keep]) <= GRAD_TOL, name
+        for ours, name in (("grad_W1", "gW1"), ("grad_b1", "gb1"), ("grad_W2", "gW2"), ("grad_b2", "gb2")):
+            assert rel_err(host(g[ours]), ref[name], ref["A" + name]) <= GRAD_TOL, name
+        g2 = tiga.tiga_apply_radius_mlp_backward(pd, xd, dev(gy, torch), r, box, per, *P)      # rebuilds the bins
+        assert torch.equal(g["grad_feat"], g2["grad_feat"]) and torch.equal(g["grad_pos"], g2["grad_pos"])
+
+
+@pytest.mark.parametrize("periodic", [0, 1])
+@pytest.mark.parametrize("dims", [(8, 16, 4), (8, 8, 4), (8, 32, 4), (1, 8, 1), (5, 16, 3), (13, 32, 2)])
+def test_small_clouds(tiga, periodic, dims):
+    f_in, hidden, f_out = dims
+    n = 3000
+    pos = gen.uniform_points(n, 60 + hidden)
+    x = gen.normal_features(n, f_in, 61, 31)
+    gy = gen.normal_features(n, f_out, 61, 32)
+    r = gen.radius_for_expected_neighbours(n, 12.0)
+    _check(tiga, pos, x, gy, r, np.ones(3, np.float32), [periodic] * 3, gen.mlp_params(f_in, hidden, f_out, 7))
+
+
+def test_paper_example_shape(tiga):
+    # Appendix A: 128 points, 8 node features, hidden 16, 4 outputs, cutoff 0.35
+    pos = gen.uniform_points(128, 7)
+    x = gen.normal_features(128, 8, 7, 31)
+    gy = gen.normal_features(128, 4, 7, 32)
+    params = gen.mlp_params(8, 16, 4, 7)
+    ones = np.ones(3, np.float32)
+    _check(tiga, pos, x, gy, np.float32(0.35), ones, [0, 0, 0], params, use_cells=False)
+    _check(tiga, pos, x, gy, np.float32(0.35), ones, [1, 1, 1], params, use_cells=False)     # single cell, minimum image
+
+
+def test_dense_cluster_overflows_the_lists(tiga):
+    n = 2500
+    pos = gen.uniform_points(n, 15) * np.float32(0.1) + np.float32(0.3)
+    x = gen.normal_features(n, 8, 15, 31)
+    gy = gen.normal_features(n, 4, 15, 32)
+    # about 400 neighbours per point: many pre-activations per row, so a tighter kink margin
+    _check(tiga, pos, x, gy, np.float32(0.04), np.ones(3, np.float32), [0, 0, 0], gen.mlp_params(8, 16, 4, 9),
+           kink_eps=3e-6, min_keep=0.5)
+
+
+@pytest.mark.parametrize("hidden", [8, 32])
+def test_surface_stand_in(tiga, hidden):
+    """35,947 points on a closed surface with cutoff 0.015 (the size and radius of the paper's
+    differentiated edge-network study; the geometry itself is synthetic)."""
+    n = 35_947
+    pos = gen.surface_points(n, 3)
+    x = gen.normal_features(n, 8, 3, 31)
+    gy = gen.normal_features(n, 4, 3, 32)
+    _check(tiga, pos, x, gy, np.float32(0.015), np.ones(3, np.float32), [0, 0, 0], gen.mlp_params(8, hidden, 4, 3))
