@@ -195,7 +195,7 @@ template <int MODE> struct TravSmem {
 // 2: Gaussian backward.  MI: some periodic dimension has a single cell (explicit minimum image).
 // VEC: feature rows are 16-byte aligned (F % 4 == 0); otherwise the forward uses scalar accesses.
 template <int MODE, int LF, bool DIST, bool MI, bool VEC = true>
-__global__ void __launch_bounds__(TRAV_THREADS) radius_traverse_kernel(const __grid_constant__ RadiusParams p) {
+__global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_traverse_kernel(const __grid_constant__ RadiusParams p) {
     using SM = TravSmem<MODE>;
     constexpr int STAGE_CAP = SM::STAGE_CAP, QCAP = SM::QCAP, QSTRIDE = SM::QSTRIDE;
     constexpr unsigned FULL = 0xffffffffu;
