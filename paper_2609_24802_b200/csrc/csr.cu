@@ -22,6 +22,7 @@ namespace tiga {
 
 constexpr int CSR_THREADS = 256;
 constexpr int CSR_TILE = 2048;     // merge-path items per CTA
+constexpr int CSR_PAD = 8;         // readable entries behind a tile's staged edges
 
 template <typename XT> struct XTraits;
 template <> struct XTraits<float> {
@@ -131,8 +132,10 @@ __device__ Tile stage_tile(const CsrParams& p, int* s_ptr, int* s_col, float* s_
     for (int k = threadIdx.x; k < t.ne; k += CSR_THREADS) {
         const int kk = PADDED ? pad32(k) : k;
         s_col[kk] = ld_stream(p.col + t.e0 + k);
-        if (p.w) s_w[kk] = ld_stream(p.w + t.e0 + k);
+        s_w[kk] = p.w ? ld_stream(p.w + t.e0 + k) : 1.f;
     }
+    // a few valid entries behind the last edge: unrolled loops may load (never use) past their span
+    if (threadIdx.x < CSR_PAD) { s_col[(PADDED ? pad32(t.ne) : t.ne) + threadIdx.x] = 0; s_w[(PADDED ? pad32(t.ne) : t.ne) + threadIdx.x] = 0.f; }
     __syncthreads();
     return t;
 }
@@ -183,15 +186,15 @@ struct State {
 };
 
 template <typename XT, int G, int VPL, int RED, typename IT>
-__global__ void __launch_bounds__(CSR_THREADS) csr_forward_kernel(const CsrParams p) {
+__global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrParams p) {
     constexpr int VW = XTraits<XT>::VW;
     constexpr int NW = CSR_THREADS / G;          // workers per CTA
     constexpr int LV = G * VPL * VW;             // floats of one partial state
     constexpr int U = (VPL == 1) ? 4 : (VPL == 2 ? 2 : 1);   // gathers in flight per lane
 
     __shared__ int s_ptr[CSR_TILE + 2];
-    __shared__ int s_col[CSR_TILE];
-    __shared__ float s_w[CSR_TILE];
+    __shared__ int s_col[CSR_TILE + CSR_PAD];
+    __shared__ float s_w[CSR_TILE + CSR_PAD];
     __shared__ long long s_coord[2];
     __shared__ int s_tag[2 * NW];                // local row of head (even) / tail (odd) partial, -1 = none
     __shared__ unsigned char s_first[NW];        // tail partial starts its chain
@@ -202,8 +205,8 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_forward_kernel(const CsrParam
     const Tile t = stage_tile<IT>(p, s_ptr, s_col, s_w, s_coord);
     const int wk = threadIdx.x / G;
     const int ln = threadIdx.x % G;
-    const bool has_w = p.w != nullptr;
-    const uint4* __restrict__ xbase = static_cast<const uint4*>(p.x);
+    const uint4* __restrict__ xlane = static_cast<const uint4*>(p.x) + ln;
+    const unsigned nvec = (unsigned)p.nvec;
     const long long e0 = t.e0;
 
     bool act[VPL];
@@ -274,13 +277,13 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_forward_kernel(const CsrParam
             float wv[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const int ee = (e + u < b) ? e + u : b - 1;
-                const long long c = s_col[ee];
-                wv[u] = has_w ? s_w[ee] : 1.f;
-                const uint4* src = xbase + c * p.nvec;
+                // entries past the span are readable (next worker's edges or the pad) and never used
+                const unsigned c = (unsigned)s_col[e + u];
+                wv[u] = s_w[e + u];
+                const uint4* src = xlane + (unsigned long long)c * nvec;      // one 32 x 32 -> 64 multiply
 #pragma unroll
                 for (int i = 0; i < VPL; ++i)
-                    xv[u][i] = act[i] ? __ldg(src + i * G + ln) : make_uint4(0, 0, 0, 0);
+                    xv[u][i] = act[i] ? __ldg(src + i * G) : make_uint4(0, 0, 0, 0);
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
@@ -600,20 +603,20 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const Csr
     constexpr int NW = CSR_THREADS / G;
     constexpr int U = (VPL == 1) ? 4 : (VPL == 2 ? 2 : 1);
     __shared__ int s_ptr[CSR_TILE + 2];
-    __shared__ int s_col[CSR_TILE];
-    __shared__ float s_w[CSR_TILE];
+    __shared__ int s_col[CSR_TILE + CSR_PAD];
+    __shared__ float s_w[CSR_TILE + CSR_PAD];
     __shared__ float s_gw[CSR_TILE];
     __shared__ long long s_coord[2];
 
     const Tile t = stage_tile<IT>(p, s_ptr, s_col, s_w, s_coord);
     const int wk = threadIdx.x / G;
     const int ln = threadIdx.x % G;
-    const bool has_w = p.w != nullptr;
     // lanes of one worker stay converged; workers of one warp do not
     const unsigned wmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) & ~(G - 1)));
-    const float4* __restrict__ xbase = static_cast<const float4*>(p.x);
+    const float4* __restrict__ xlane = static_cast<const float4*>(p.x) + ln;
     const float4* __restrict__ gybase = reinterpret_cast<const float4*>(p.gy);
-    float4* gxbase = reinterpret_cast<float4*>(p.gx);
+    float4* gxlane = reinterpret_cast<float4*>(p.gx) + ln;
+    const unsigned nvec = (unsigned)p.nvec;
 
     bool act[VPL];
 #pragma unroll
@@ -638,13 +641,13 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const Csr
             float wv[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const int ee = (e + u < b) ? e + u : b - 1;
-                cv[u] = s_col[ee];
-                wv[u] = has_w ? s_w[ee] : 1.f;
+                // entries past the span are readable (next worker's edges or the pad) and never used
+                cv[u] = s_col[e + u];
+                wv[u] = s_w[e + u];
                 if (p.gw) {
 #pragma unroll
                     for (int i = 0; i < VPL; ++i)
-                        xv[u][i] = act[i] ? __ldg(xbase + (long long)cv[u] * p.nvec + i * G + ln) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        xv[u][i] = act[i] ? __ldg(xlane + (unsigned long long)(unsigned)cv[u] * nvec + i * G) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
 #pragma unroll
@@ -669,7 +672,7 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const Csr
 #pragma unroll
                         for (int i = 0; i < VPL; ++i)
                             if (act[i])
-                                atomicAdd(gxbase + (long long)cv[u] * p.nvec + i * G + ln,
+                                atomicAdd(gxlane + (unsigned long long)(unsigned)cv[u] * nvec + i * G,
                                           make_float4(wv[u] * g[i].x, wv[u] * g[i].y, wv[u] * g[i].z, wv[u] * g[i].w));
                     }
                 }
