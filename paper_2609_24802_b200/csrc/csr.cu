@@ -285,6 +285,20 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
                 for (int i = 0; i < VPL; ++i)
                     xv[u][i] = act[i] ? __ldg(src + i * G) : make_uint4(0, 0, 0, 0);
             }
+            if (e + U <= b && e + U <= cur_end) {
+                // common case: the whole batch lies inside the current row and the span
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    float xf[VW];
+#pragma unroll
+                    for (int i = 0; i < VPL; ++i) {
+                        XTraits<XT>::unpack(xv[u][i], xf);
+#pragma unroll
+                        for (int k = 0; k < VW; ++k) st.message(i, k, wv[u], xf[k], (int)(e0 + e + u));
+                    }
+                }
+                continue;
+            }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 if (e + u < b) {
