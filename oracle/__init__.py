@@ -212,6 +212,25 @@ def radius_backward_gauss(pos, feat, gy, r, box, periodic, sigma, rows=None, use
     return dict(gx=gx, Agx=Agx, gp=gp, Agp=Agp)
 
 
+# ------------------------------------------------------------------------------ generated kNN
+def knn(pos, feat, k, rows=None):
+    """Exact k nearest neighbours by the key (fp32 squared distance, index) and their neighbour
+    sum.  Returns (idx int32 [n_rows,k], d2 fp32 [n_rows,k], y fp64 [n_rows,F], A fp64)."""
+    lib = _load()
+    pos = np.ascontiguousarray(pos, dtype=np.float32)
+    feat = np.ascontiguousarray(feat, dtype=np.float64)
+    n = pos.shape[0]
+    F = feat.shape[1]
+    rows = None if rows is None else _i64(rows)
+    nr = n if rows is None else len(rows)
+    idx = np.empty((nr, k), np.int32); d2 = np.empty((nr, k), np.float32)
+    y = np.empty((nr, F), np.float64); A = np.empty((nr, F), np.float64)
+    rc = lib.oracle_knn(_p(pos), _p(feat), ctypes.c_int64(n), ctypes.c_int(F), ctypes.c_int(int(k)),
+                        _p(rows), ctypes.c_int64(nr), _p(idx), _p(d2), _p(y), _p(A))
+    assert rc == 0
+    return idx, d2, y, A
+
+
 # ------------------------------------------------------------------------------ edge neural network
 def _mlp_args(W1, b1, W2, b2):
     W1 = np.ascontiguousarray(W1, np.float64); b1 = np.ascontiguousarray(b1, np.float64)

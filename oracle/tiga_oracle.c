@@ -18,6 +18,8 @@
  *     Appendix A: the position derivative acts through the displacement of selected edges)
  *   - a cell directory (Section 4.9) used only to restrict candidates; the exact distance
  *     predicate is unchanged.
+ *   - the generated exact k-nearest-neighbour relation consumed by a neighbour sum
+ *     (Section 4.9; keys are (squared distance, source index)), by brute force over all sources.
  * Readings where the paper is silent (max reducer: empty row finalizes to 0 with arg -1,
  * ties go to the lowest edge position; periodic boxes use the minimum image; Gaussian and
  * Lennard-Jones messages; the cell-grid constants) are the build's own and are listed in
@@ -666,5 +668,66 @@ int oracle_radius_mlp_backward(const double* pos, const double* feat, const doub
     }
     free(G.start);
     free(G.items);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ generated exact kNN + neighbour sum
+ * Section 4.9 (generated kNN): every destination query examines all sources, keeps the k
+ * smallest ordering keys and consumes the selected source features without storing an
+ * adjacency.  A key is (squared distance, source index), so equal distances are ordered by
+ * index.  The evaluated workload (Section 7) is a neighbour sum with k = 16.
+ *
+ * Precision: the paper bounds this path to FP32 and computes reference distances by direct
+ * differences, not by the matrix-product identity.  The selection is an integer decision
+ * made by floating point, so it is taken here in that precision: the squared distance is
+ * the fp32 value  fl(fl(fl(dx*dx) + fl(dy*dy)) + fl(dz*dz))  with  dx = fl(x_i - x_j)  and
+ * no contraction (this file is compiled with -ffp-contract=off).  The neighbour sum itself
+ * is accumulated in double, in key order.
+ *
+ * Readings where the paper is silent: the query itself is not its own neighbour (j != i by
+ * index, as for the radius relation of Appendix A); with fewer than k other points the
+ * missing entries have index -1, distance +inf and contribute nothing.
+ *
+ * For each requested row (rows == NULL: all): idx [n_rows, k] and d2 [n_rows, k] in key
+ * order, y [n_rows, F] the neighbour sum, A the sum of absolute contributions.
+ */
+int oracle_knn(const float* pos, const double* feat, int64_t n, int F, int k,
+               const int64_t* rows, int64_t n_rows,
+               int32_t* idx, float* d2, double* y, double* A) {
+    if (k <= 0) return 1;
+    if (!rows) n_rows = n;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t t = 0; t < n_rows; ++t) {
+        const int64_t i = rows ? rows[t] : t;
+        int32_t* bi = idx + t * k;
+        float* bd = d2 + t * k;
+        int have = 0;
+        const float xi = pos[3 * i], yi = pos[3 * i + 1], zi = pos[3 * i + 2];
+        for (int64_t j = 0; j < n; ++j) {
+            if (j == i) continue;
+            const float dx = xi - pos[3 * j], dy = yi - pos[3 * j + 1], dz = zi - pos[3 * j + 2];
+            const float sx = dx * dx, sy = dy * dy, sz = dz * dz;
+            float s = sx + sy;
+            s = s + sz;
+            /* sources arrive in index order, so a candidate goes behind retained keys of equal distance */
+            if (have == k && !(s < bd[k - 1])) continue;
+            int at = have < k ? have : k - 1;
+            while (at > 0 && s < bd[at - 1]) { bd[at] = bd[at - 1]; bi[at] = bi[at - 1]; --at; }
+            bd[at] = s;
+            bi[at] = (int32_t)j;
+            if (have < k) ++have;
+        }
+        for (int u = have; u < k; ++u) { bi[u] = -1; bd[u] = INFINITY; }
+        for (int f = 0; f < F; ++f) {
+            double acc = 0.0, ab = 0.0;
+            for (int u = 0; u < have; ++u) {
+                const double c = feat[(int64_t)bi[u] * F + f];
+                acc += c;
+                ab += fabs(c);
+            }
+            y[t * F + f] = acc;
+            if (A) A[t * F + f] = ab;
+        }
+    }
     return 0;
 }
