@@ -19,6 +19,7 @@ __all__ = [
     "edge_weights", "normal_features", "small_int_features", "small_int_weights",
     "uniform_points", "jittered_lattice", "hex_mesh_csr", "periodic_offset_csr",
     "regular_random_csr", "radius_for_expected_neighbours", "config", "surface_points", "mlp_params",
+    "clustered_points",
 ]
 
 DEFAULT_SEED = 20260921
@@ -268,6 +269,20 @@ def surface_points(n: int, seed: int = DEFAULT_SEED) -> np.ndarray:
     v /= np.linalg.norm(v, axis=1, keepdims=True)
     rad = 0.34 + 0.05 * np.sin(5.0 * v[:, 0]) * np.cos(3.0 * v[:, 1]) + 0.04 * v[:, 2] ** 2
     return (0.5 + v * rad[:, None]).astype(np.float32)
+
+
+def clustered_points(n: int, seed: int = DEFAULT_SEED, blobs: int = 12, frac: float = 0.7) -> np.ndarray:
+    """Uneven density in the unit cube: ``frac`` of the points in tight Gaussian blobs (clipped to
+    the cube), the rest a thin uniform background.  Coordinates are k*2^-24."""
+    g = rng(seed, 83)
+    nb = int(n * frac)
+    centres = g.random((blobs, 3)) * 0.8 + 0.1
+    sig = g.uniform(0.004, 0.03, blobs)
+    which = g.integers(0, blobs, nb)
+    pts = centres[which] + g.standard_normal((nb, 3)) * sig[which, None]
+    pts = np.concatenate([pts, g.random((n - nb, 3))], 0)
+    pts = np.clip(pts, 0.0, 1.0 - 2.0**-24)
+    return (np.floor(pts * 2.0**24) * 2.0**-24).astype(np.float32)[g.permutation(n)]
 
 
 def mlp_params(f_in: int, hidden: int, f_out: int, seed: int = DEFAULT_SEED):

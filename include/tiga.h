@@ -251,6 +251,32 @@ tiga_status tiga_apply_radius_mlp_backward(const float* pos, const float* feat, 
                                            float* grad_W1, float* grad_b1, float* grad_W2, float* grad_b2,
                                            void* ws, size_t ws_bytes, int reuse_plan, void* stream);
 
+/* ----------------------------------------------------------------- generated exact kNN */
+
+#define TIGA_KNN_MAX_K 32
+
+/* Generated exact k-nearest-neighbour relation consumed by a neighbour sum without storing an
+ * adjacency (Section 4.9, generated kNN; Section 7: scalar neighbour sum with k = 16):
+ *     N_k(i) = the k sources j != i with the smallest keys (d2_ij, j),
+ *     out[i,:] = sum over j in N_k(i) of feat[j,:].
+ * The key's squared distance is the fp32 value fl(fl(fl(dx*dx) + fl(dy*dy)) + fl(dz*dz)) of the
+ * direct differences dx = fl(x_i - x_j), ... (the paper bounds this path to FP32 and uses direct
+ * differences); equal distances are ordered by source index.  The result is exact for that key
+ * on any input: a cell directory only orders the search (cells around the query first, farther
+ * shells while the k-th key could still improve), it never replaces the comparison of keys.
+ *   pos  : fp32 [n, 3] inside [0, len_d]; the box must not be periodic (TIGA_ERR_UNSUPPORTED)
+ *   feat : fp32 [n, F], F >= 1;  k : 1..TIGA_KNN_MAX_K (TIGA_ERR_UNSUPPORTED above)
+ *   out  : fp32 [n, F], fully overwritten
+ *   nbr  : int32 [n, k] or NULL, source indices in key order; nbr_d2 : fp32 [n, k] or NULL.
+ *          With fewer than k other points the missing entries are -1 and +inf and add nothing.
+ *   ws   : tiga_knn_workspace_bytes(n, k, box) bytes, 16-byte aligned; holds the bins afterwards.
+ * All array pointers are device pointers; the box is read on the host.  No backward exists for
+ * this relation (the paper generates none for it either). */
+size_t tiga_knn_workspace_bytes(int64_t n, int32_t k, const tiga_box* box);
+tiga_status tiga_apply_knn(const float* pos, const float* feat, int64_t n, int32_t F, int32_t k,
+                           const tiga_box* box, float* out, int32_t* nbr, float* nbr_d2,
+                           void* ws, size_t ws_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

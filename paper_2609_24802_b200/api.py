@@ -18,7 +18,7 @@ __all__ = [
     "tiga_apply_csr", "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram",
     "tiga_radius_grid", "tiga_radius_workspace_bytes", "tiga_radius_bin",
     "tiga_apply_radius", "tiga_apply_radius_backward", "tiga_apply_radius_mlp",
-    "tiga_apply_radius_mlp_backward", "launch_count",
+    "tiga_apply_radius_mlp_backward", "tiga_knn_workspace_bytes", "tiga_apply_knn", "launch_count",
 ]
 
 SUM, MAX = 0, 1
@@ -31,6 +31,7 @@ EXPORTS = [
     "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram", "tiga_radius_grid",
     "tiga_radius_workspace_bytes", "tiga_radius_bin", "tiga_apply_radius",
     "tiga_apply_radius_backward", "tiga_apply_radius_mlp", "tiga_apply_radius_mlp_backward",
+    "tiga_knn_workspace_bytes", "tiga_apply_knn",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -108,6 +109,10 @@ def load_library() -> ctypes.CDLL:
     lib.tiga_apply_radius_mlp_backward.restype = ctypes.c_int
     lib.tiga_apply_radius_mlp_backward.argtypes = [vp, vp, i64, f, ctypes.POINTER(_Box), ctypes.POINTER(_EdgeMlp), vp,
                                                    vp, vp, vp, vp, vp, vp, vp, sz, ctypes.c_int, vp]
+    lib.tiga_knn_workspace_bytes.restype = sz
+    lib.tiga_knn_workspace_bytes.argtypes = [i64, i32, ctypes.POINTER(_Box)]
+    lib.tiga_apply_knn.restype = ctypes.c_int
+    lib.tiga_apply_knn.argtypes = [vp, vp, i64, i32, i32, ctypes.POINTER(_Box), vp, vp, vp, vp, sz, vp]
     _lib = lib
     return lib
 
@@ -386,3 +391,30 @@ def tiga_apply_radius_mlp_backward(pos, feat, grad_out, r: float, box, periodic,
                                                       _stream(stream)), "tiga_apply_radius_mlp_backward")
     _launches += 1 if reuse_plan else 7
     return g
+
+
+def tiga_knn_workspace_bytes(n: int, k: int, box) -> int:
+    b = _box(box, (0, 0, 0))
+    return int(load_library().tiga_knn_workspace_bytes(n, k, ctypes.byref(b)))
+
+
+def tiga_apply_knn(pos, feat, k: int, box, periodic=(0, 0, 0), out=None, nbr=None, nbr_d2=None,
+                   want_nbr=True, ws=None, stream=None):
+    """out[i] = sum of feat[j] over the k nearest j != i by the key (fp32 squared distance, index).
+    Returns (out, nbr int32 [n,k] or None, nbr_d2 fp32 [n,k] or None, ws)."""
+    global _launches
+    n, F = feat.shape
+    b = _box(box, periodic)
+    dev = pos.device
+    if out is None:
+        out = torch.empty((n, F), dtype=torch.float32, device=dev)
+    if want_nbr and nbr is None:
+        nbr = torch.empty((n, k), dtype=torch.int32, device=dev)
+    if want_nbr and nbr_d2 is None:
+        nbr_d2 = torch.empty((n, k), dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = _ws(tiga_knn_workspace_bytes(n, k, box), pos)
+    _ok(load_library().tiga_apply_knn(_ptr(pos), _ptr(feat), n, F, int(k), ctypes.byref(b), _ptr(out), _ptr(nbr),
+                                      _ptr(nbr_d2), _ptr(ws), ws.numel(), _stream(stream)), "tiga_apply_knn")
+    _launches += 8
+    return out, nbr, nbr_d2, ws
