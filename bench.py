@@ -506,6 +506,17 @@ def run_paper_shapes(args):
                      "ms_median": fwd[0], "ms_min": fwd[1], "ms_max": fwd[2], "backward_ms_median": bwd[0],
                      "backward_ms_min": bwd[1], "backward_ms_max": bwd[2], "interactions_per_s": pairs / (fwd[0] * 1e-3),
                      "paper": paper + " on the Stanford Bunny vertices, 356,260 edges (RTX 5070 Ti)"})
+    # generated exact kNN, scalar neighbour sum, k = 16, relation rebuilt from the coordinates every call
+    knn_paper = {1024: "0.147 ms (Torch 0.244, PyG 1.775)", 16384: "6.32 ms (Torch 29.92, PyG 17.50)",
+                 131072: "172.37 ms (Torch 1908.43, PyG 393.21)"}
+    for n in (1024, 4096, 16384, 32768, 65536, 131072, 1_000_000, 4_000_000):
+        pos, x = to(gen.uniform_points(n, args.seed)), to(gen.normal_features(n, 1, args.seed, 31))
+        out, nbr, d2, ws = T.tiga_apply_knn(pos, x, 16, ones)
+        med, lo, hi = median_ms(lambda: T.tiga_apply_knn(pos, x, 16, ones, out=out, nbr=nbr, nbr_d2=d2, ws=ws))
+        rows.append({"shape": f"generated exact kNN, k=16, scalar neighbour sum, N={n}", "pairs": 16 * n, "F": 1,
+                     "ms_median": med, "ms_min": lo, "ms_max": hi, "interactions_per_s": 16 * n / (med * 1e-3),
+                     "paper": (knn_paper.get(n, "figure only") + " (RTX 5070 Ti, all-pairs scan)") if n <= 131072 else "beyond the paper's sizes"})
+        del pos, x, out, nbr, d2, ws
     c = gen.config("cfg2", args.seed, F=8)
     pos, x, gy = to(c["pos"]), to(c["x"]), to(gen.normal_features(c["n"], 4, args.seed, 33))
     P = [to(a) for a in gen.mlp_params(8, 16, 4, args.seed)]
@@ -555,6 +566,13 @@ def run_case(args):
             out, cnt, ws = T.tiga_apply_radius(pos, x, c["r"], c["box"], c["periodic"], T.MSG_GAUSS, p0=c["sigma"])
             T.tiga_apply_radius_backward(pos, x, gy, c["r"], c["box"], c["periodic"], c["sigma"], ws=ws, reuse_plan=True)
         units = c["n"]
+    elif args.case == "knn":
+        n = args.size or 1_000_000
+        pos, x = to(gen.uniform_points(n, args.seed)), to(gen.normal_features(n, 1, args.seed, 31))
+        out, nbr, d2, ws = T.tiga_apply_knn(pos, x, 16, np.ones(3, np.float32))
+        def run():
+            T.tiga_apply_knn(pos, x, 16, np.ones(3, np.float32), out=out, nbr=nbr, nbr_d2=d2, ws=ws)
+        units = n
     else:
         c = gen.config("cfg3", args.seed, m=args.size or 100)
         pos = to(c["pos"])
@@ -581,7 +599,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--seed", type=int, default=gen.DEFAULT_SEED)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", default=None, choices=["csr", "csr_large", "radius_gauss", "radius_lj", "paper_shapes"],
+    ap.add_argument("--case", default=None, choices=["csr", "csr_large", "radius_gauss", "radius_lj", "knn", "paper_shapes"],
                     help="run one traversal on a reduced replica (for profiler captures) instead of the benchmark")
     ap.add_argument("--size", type=int, default=0, help="--case size: R-MAT scale, number of points, or lattice side")
     args = ap.parse_args()

@@ -20,22 +20,28 @@
 //                     k-th key is no larger than the squared distance to the unexplored region, or
 //                     when the whole grid has been visited.
 //
-// Keys are (fp32 squared distance by direct differences in a fixed operation order, source index);
-// the k smallest are selected by rank counting, which also leaves them in key order.
+// Keys are (fp32 squared distance by direct differences in a fixed operation order, source index),
+// held as one 64-bit integer (distance bits above the index: squared distances are never negative,
+// so their bit patterns order like the values).  The k smallest of a list are selected by sorting
+// 32 keys at a time across the warp with a bitonic network of shuffles and merging the sorted
+// groups, which also leaves the selected keys in order, one per lane.
 #include "radius_shared.cuh"
 
 namespace tiga {
 
-constexpr int KNN_STAGE_CAP = 384;                 // staged candidates per chunk
+constexpr int KNN_STAGE_CAP = 256;                 // staged candidates per chunk
 constexpr int KNN_QCAP = 96;                       // list entries per query (cells kernel)
 constexpr int KNN_QSTRIDE = KNN_QCAP + 1;
 constexpr int KNN_RING_CAP = 128;                  // list entries of the rings kernel
 constexpr int KNN_STAGE_BYTES = (KNN_STAGE_CAP + STAGE_PAD) * 16;
 constexpr int KNN_LIST_BYTES = (QB * KNN_QSTRIDE * 8 + 15) / 16 * 16;
-constexpr int KNN_TMP_BYTES = TIGA_KNN_MAX_K * 8;
 constexpr int KNN_MISC_BYTES = QB * 16 + QB * 4 * 2;
-constexpr int KNN_PER_WARP = KNN_STAGE_BYTES + KNN_LIST_BYTES + KNN_TMP_BYTES + KNN_MISC_BYTES;
+constexpr int KNN_PER_WARP = KNN_STAGE_BYTES + KNN_LIST_BYTES + KNN_MISC_BYTES;
 constexpr int KNN_RING_BLOCKS = 148 * 4;
+constexpr double KNN_BALL_FACTOR = 2.0;            // expected points within the search radius, in units of k
+
+typedef unsigned long long knn_key;                // (bits of d2) << 32 | source index
+constexpr knn_key KNN_NO_KEY = ~0ull;
 
 struct KnnParams {
     RadiusParams rp;        // points, features, plan
@@ -57,67 +63,76 @@ static __device__ __forceinline__ float key_d2(const float qx, const float qy, c
     return __fadd_rn(__fadd_rn(__fmul_rn(dx, dx), __fmul_rn(dy, dy)), __fmul_rn(dz, dz));
 }
 
-static __device__ __forceinline__ bool key_less(const float2 a, const float2 b) {
-    return a.y < b.y || (a.y == b.y && __float_as_int(a.x) < __float_as_int(b.x));
-}
+static __device__ __forceinline__ int key_index(const knn_key v) { return (int)(unsigned)(v & 0xffffffffull); }
+static __device__ __forceinline__ float key_dist(const knn_key v) { return __uint_as_float((unsigned)(v >> 32)); }
 
-// Keeps the min(n, k) smallest keys of lq[0, n) and leaves them sorted in lq[0, min(n, k)).
-// Rank counting: keys are distinct (indices are), so the ranks are a permutation.  U entries per lane.
-template <int U>
-static __device__ __forceinline__ int select_k_u(float2* lq, float2* tmp, const int n, const int k, const int lane) {
-    float2 e[U];
-    int rank[U];
+// sorts 32 keys, one per lane, ascending by lane (bitonic network)
+static __device__ __forceinline__ knn_key sort32(knn_key v, const int lane) {
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-        const int t = lane + 32 * u;
-        e[u] = t < n ? lq[t] : make_float2(__int_as_float(0x7fffffff), __int_as_float(0x7f800000));
-        rank[u] = 0;
+    for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            const knn_key o = __shfl_xor_sync(0xffffffffu, v, stride);
+            const bool take_min = ((lane & stride) == 0) == ((lane & size) == 0);
+            v = ((v < o) == take_min) ? v : o;
+        }
     }
-    for (int t = 0; t < n; ++t) {
-        const float2 b = lq[t];
+    return v;
+}
+
+// a, b sorted ascending by lane: returns the 32 smallest of both, sorted
+static __device__ __forceinline__ knn_key merge_low32(const knn_key a, const knn_key b, const int lane) {
+    const knn_key br = __shfl_sync(0xffffffffu, b, 31 - lane);
+    knn_key c = a < br ? a : br;                              // the 32 smallest as a bitonic sequence
 #pragma unroll
-        for (int u = 0; u < U; ++u) rank[u] += key_less(b, e[u]) ? 1 : 0;
+    for (int stride = 16; stride > 0; stride >>= 1) {
+        const knn_key o = __shfl_xor_sync(0xffffffffu, c, stride);
+        c = ((c < o) == ((lane & stride) == 0)) ? c : o;
     }
-    __syncwarp();
-#pragma unroll
-    for (int u = 0; u < U; ++u)
-        if (lane + 32 * u < n && rank[u] < k) tmp[rank[u]] = e[u];
-    __syncwarp();
-    const int m = n < k ? n : k;
-    if (lane < m) lq[lane] = tmp[lane];
-    __syncwarp();
-    return m;
+    return c;
 }
 
-static __device__ __noinline__ int select_k(float2* lq, float2* tmp, const int n, const int k, const int lane) {
-    if (n <= 32) return select_k_u<1>(lq, tmp, n, k, lane);
-    if (n <= 64) return select_k_u<2>(lq, tmp, n, k, lane);
-    if (n <= 96) return select_k_u<3>(lq, tmp, n, k, lane);
-    return select_k_u<5>(lq, tmp, n, k, lane);
+// The 32 smallest keys of lq[0, n), sorted, lane t holding the t-th (KNN_NO_KEY beyond n).
+// List entries are (index, d2) pairs, which read as one little-endian 64-bit key.
+static __device__ __noinline__ knn_key select_sorted(const float2* lq, const int n, const int lane) {
+    const knn_key* l64 = reinterpret_cast<const knn_key*>(lq);
+    knn_key best = KNN_NO_KEY;
+    for (int base = 0; base < n; base += 32) {
+        knn_key v = base + lane < n ? l64[base + lane] : KNN_NO_KEY;
+        v = sort32(v, lane);
+        best = base == 0 ? v : merge_low32(best, v, lane);
+    }
+    return best;
 }
 
-// Writes the row of query i from its m <= k selected keys (sorted): indices, distances, neighbour sum.
-static __device__ __forceinline__ void emit_row(const KnnParams& P, const int i, const float2* top, const int m, const int lane) {
+// Writes the row of query i from its m <= k selected keys (lane t holds the t-th): indices,
+// distances, neighbour sum.
+static __device__ __forceinline__ void emit_row(const KnnParams& P, const int i, const knn_key top, const int m, const int lane) {
     const int k = P.k, F = P.rp.F;
+    const bool v = lane < m;
+    const int id = v ? key_index(top) : -1;
     if (lane < k) {
-        const bool v = lane < m;
-        if (P.nbr) P.nbr[(size_t)i * k + lane] = v ? __float_as_int(top[lane].x) : -1;
-        if (P.nbr_d2) P.nbr_d2[(size_t)i * k + lane] = v ? top[lane].y : __int_as_float(0x7f800000);
+        if (P.nbr) P.nbr[(size_t)i * k + lane] = id;
+        if (P.nbr_d2) P.nbr_d2[(size_t)i * k + lane] = v ? key_dist(top) : __int_as_float(0x7f800000);
     }
     const float* feat = P.rp.feat;
     if (F >= 8) {
-        for (int f = lane; f < F; f += 32) {
+        for (int f0 = 0; f0 < F; f0 += 32) {
+            const int f = f0 + lane;
             float acc = 0.f;
-            for (int t = 0; t < m; ++t) acc += __ldg(feat + (size_t)__float_as_int(top[t].x) * F + f);
-            P.out[(size_t)i * F + f] = acc;
+            for (int t = 0; t < m; ++t) {
+                const int idt = __shfl_sync(0xffffffffu, id, t);
+                if (f < F) acc += __ldg(feat + (size_t)idt * F + f);
+            }
+            if (f < F) P.out[(size_t)i * F + f] = acc;
         }
     } else {
-        const size_t row = lane < m ? (size_t)__float_as_int(top[lane].x) * F : 0;
+        const size_t row = v ? (size_t)id * F : 0;
         for (int f = 0; f < F; ++f) {
-            float v = lane < m ? __ldg(feat + row + f) : 0.f;
+            float x = v ? __ldg(feat + row + f) : 0.f;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if (lane == 0) P.out[(size_t)i * F + f] = v;
+            for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+            if (lane == 0) P.out[(size_t)i * F + f] = x;
         }
     }
 }
@@ -138,8 +153,7 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
     unsigned char* base = s_raw + (size_t)wib * KNN_PER_WARP;
     float4* stage = reinterpret_cast<float4*>(base);                                      // x, y, z, point id
     float2* list = reinterpret_cast<float2*>(base + KNN_STAGE_BYTES);                     // (point id, d2) per query
-    float2* tmp = reinterpret_cast<float2*>(base + KNN_STAGE_BYTES + KNN_LIST_BYTES);
-    float4* s_q = reinterpret_cast<float4*>(base + KNN_STAGE_BYTES + KNN_LIST_BYTES + KNN_TMP_BYTES);
+    float4* s_q = reinterpret_cast<float4*>(base + KNN_STAGE_BYTES + KNN_LIST_BYTES);
     int* s_n = reinterpret_cast<int*>(s_q + QB);
     float* s_tau = reinterpret_cast<float*>(s_n + QB);
     const unsigned lt_mask = (1u << lane) - 1u;
@@ -220,9 +234,8 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
         return v0;
     };
 
-    const bool single = total <= KNN_STAGE_CAP - 32;          // the whole stencil fits: stage it once
     int ns = 0;
-    if (single) stage_from(0, ns);
+    const bool single = stage_from(0, ns) >= total;           // the whole (pruned) stencil fits: staged once
 
     for (int qb0 = qs0; qb0 < qe0; qb0 += QB) {
         const int nq = (qe0 - qb0 < QB) ? qe0 - qb0 : QB;
@@ -267,8 +280,11 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
                     for (int q = 0; q < nq; ++q) {
                         const int n = s_n[q];
                         if (n > k) {
-                            const int m = select_k(list + q * KNN_QSTRIDE, tmp, n, k, lane);
-                            if (lane == 0) { s_n[q] = m; s_tau[q] = list[q * KNN_QSTRIDE + k - 1].y; }
+                            float2* lq = list + q * KNN_QSTRIDE;
+                            const knn_key top = select_sorted(lq, n, lane);
+                            __syncwarp();
+                            if (lane < k) reinterpret_cast<knn_key*>(lq)[lane] = top;
+                            if (lane == k - 1) { s_n[q] = k; s_tau[q] = key_dist(top); }
                         }
                     }
                     __syncwarp();
@@ -302,8 +318,7 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
             if (n < k) {
                 if (lane == 0) P.queue[atomicAdd(P.queue_n, 1)] = i;
             } else {
-                const int m = select_k(list + q * KNN_QSTRIDE, tmp, n, k, lane);
-                emit_row(P, i, list + q * KNN_QSTRIDE, m, lane);
+                emit_row(P, i, select_sorted(list + q * KNN_QSTRIDE, n, lane), k, lane);
             }
         }
     }
@@ -314,12 +329,10 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_rings_kernel(const __grid_co
     const RadiusParams& p = P.rp;
     constexpr unsigned FULL = 0xffffffffu;
     __shared__ float2 s_list[TRAV_WARPS][KNN_RING_CAP + 32];
-    __shared__ float2 s_tmp[TRAV_WARPS][TIGA_KNN_MAX_K];
 
     const int lane = threadIdx.x & 31;
     const int wib = threadIdx.x >> 5;
     float2* list = s_list[wib];
-    float2* tmp = s_tmp[wib];
     const unsigned lt_mask = (1u << lane) - 1u;
     const int k = P.k;
     const int nqueue = *P.queue_n;
@@ -335,6 +348,16 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_rings_kernel(const __grid_co
         int cnt = 0;
         float tau = 3.0e38f;
         __syncwarp();
+
+        // cuts the list back to its (at most k) smallest keys, sorted; k keys set the threshold
+        auto cut = [&]() {
+            const knn_key top = select_sorted(list, cnt, lane);
+            __syncwarp();
+            cnt = cnt < k ? cnt : k;
+            if (lane < cnt) reinterpret_cast<knn_key*>(list)[lane] = top;
+            if (cnt == k) tau = key_dist(__shfl_sync(FULL, top, k - 1));
+            __syncwarp();
+        };
 
         // one contiguous run of cell-ordered points [a, b) against the query
         auto run = [&](const int a, const int b) {
@@ -353,8 +376,7 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_rings_kernel(const __grid_co
                 cnt += __popc(m);
                 if (cnt > KNN_RING_CAP - 32) {
                     __syncwarp();
-                    cnt = select_k(list, tmp, cnt, k, lane);
-                    if (cnt == k) tau = list[k - 1].y;
+                    cut();
                 }
             }
         };
@@ -377,16 +399,14 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_rings_kernel(const __grid_co
             // farther than s cell edges away: k keys within that distance cannot be improved
             __syncwarp();
             if (cnt >= k) {
-                cnt = select_k(list, tmp, cnt, k, lane);          // sorted: the k-th key is the largest kept
-                tau = list[k - 1].y;
+                cut();                                            // sorted: the k-th key is the largest kept
                 const float g = (float)s * P.hmin;
                 if (tau <= g * g) break;
             }
             if (cx - s <= 0 && cy - s <= 0 && cz - s <= 0 && cx + s >= nx - 1 && cy + s >= ny - 1 && cz + s >= nz - 1) break;
         }
         __syncwarp();
-        cnt = select_k(list, tmp, cnt, k, lane);
-        emit_row(P, i, list, cnt, lane);
+        emit_row(P, i, select_sorted(list, cnt, lane), cnt < k ? cnt : k, lane);
         __syncwarp();
     }
 }
