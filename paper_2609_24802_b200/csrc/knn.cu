@@ -26,6 +26,7 @@
 // 32 keys at a time across the warp with a bitonic network of shuffles and merging the sorted
 // groups, which also leaves the selected keys in order, one per lane.
 #include "radius_shared.cuh"
+#include <type_traits>
 
 namespace tiga {
 
@@ -254,12 +255,13 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
         for (int q = 0; q < QB; ++q) { qcnt[q] = 0; tq[q] = s_tau[q]; }
 
         // all queries of the batch against the ns staged candidates
-        auto scan = [&](const int ns_) {
+        auto scan = [&](const int ns_, auto width) {
+            constexpr int NQ = decltype(width)::value;             // queries tested per trip (a short batch tests four)
             for (int cbase = 0; cbase < ns_; cbase += 32) {
                 const float4 pj = stage[cbase + lane];
                 int mx = 0;
 #pragma unroll
-                for (int q = 0; q < QB; ++q) {
+                for (int q = 0; q < NQ; ++q) {
                     const float4 qv = s_q[q];
                     const float d2 = key_d2(qv.x, qv.y, qv.z, pj.x, pj.y, pj.z);
                     const bool ok = d2 <= tq[q] && __float_as_int(pj.w) != __float_as_int(qv.w);
@@ -295,12 +297,13 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
         };
 
         if (single) {
-            scan(ns);
+            if (nq <= QB / 2) scan(ns, std::integral_constant<int, QB / 2>{});
+            else scan(ns, std::integral_constant<int, QB>{});
         } else {
             for (int v = 0; v < total;) {
                 int ns2;
                 v = stage_from(v, ns2);
-                scan(ns2);
+                scan(ns2, std::integral_constant<int, QB>{});
                 __syncwarp();
             }
         }
@@ -420,7 +423,7 @@ static float knn_search_radius(long long n, int k, const tiga_box* box) {
         lmax = (double)box->len[d] > lmax ? (double)box->len[d] : lmax;
     }
     if (n < 2) return (float)lmax;
-    const double h = cbrt(2.0 * (double)k * vol / ((double)n * 4.18879020478639));
+    const double h = cbrt(KNN_BALL_FACTOR * (double)k * vol / ((double)n * 4.18879020478639));
     return (float)(h < lmax ? h : lmax);
 }
 
