@@ -159,6 +159,22 @@ def bin_points(pos, r, box, periodic):
     return dict(ncell=ncell, invh=invh, cell=cell, cell_start=start, order=order)
 
 
+def csr_attention(rowptr, col, q, k, v, scale):
+    """Online-softmax reducer over the rows of a stored relation: returns (y, A, lse) in fp64."""
+    lib = _load()
+    rowptr = _i64(rowptr); col = _i32(col)
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    k = np.ascontiguousarray(k, dtype=np.float64)
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    n, D = q.shape
+    assert len(rowptr) == n + 1 and k.shape[1] == D and v.shape == k.shape
+    y = np.empty((n, D), np.float64); A = np.empty((n, D), np.float64); lse = np.empty(n, np.float64)
+    rc = lib.oracle_csr_attention(_p(rowptr), _p(col), ctypes.c_int64(n), _p(q), _p(k), _p(v), ctypes.c_int(D),
+                                  ctypes.c_double(float(scale)), _p(y), _p(A), _p(lse))
+    assert rc == 0
+    return y, A, lse
+
+
 # ------------------------------------------------------------------------------ radius
 def _geom(pos, r, box, periodic):
     pos = np.ascontiguousarray(pos, dtype=np.float64)      # exact for fp32 input

@@ -18,6 +18,8 @@
  *     Appendix A: the position derivative acts through the displacement of selected edges)
  *   - a cell directory (Section 4.9) used only to restrict candidates; the exact distance
  *     predicate is unchanged.
+ *   - the online-softmax reducer over the rows of a stored relation (Section 5; attention
+ *     appendix): the normalised exponential-weighted sum it evaluates, by the plain quotient.
  *   - the generated exact k-nearest-neighbour relation consumed by a neighbour sum
  *     (Section 4.9; keys are (squared distance, source index)), by brute force over all sources.
  * Readings where the paper is silent (max reducer: empty row finalizes to 0 with arg -1,
@@ -728,6 +730,54 @@ int oracle_knn(const float* pos, const double* feat, int64_t n, int F, int k,
             y[t * F + f] = acc;
             if (A) A[t * F + f] = ab;
         }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ online-softmax reducer over a stored relation
+ * Section 5 ("Online softmax") and the attention appendix: the edge function supplies a score
+ * and a value, s_e = scale * <q_d(e), k_s(e)> and v_s(e); the reducer's result for row i is
+ *     y_i = sum_e exp(s_e) v_s(e) / sum_e exp(s_e)        over the edges e of row i,
+ * the relation deciding which interactions are admissible (a triangular relation gives causal
+ * attention).  The streaming state (maximum, mass, accumulator) and its combine rule are a way
+ * of evaluating exactly this quotient, so the oracle is the quotient itself: per row the
+ * scores, their maximum, then the normalised sum, all in double, in edge order.
+ * Repeated edges are separate messages.  Reading for the empty row (the paper leaves it to the
+ * reducer's convention): zero vector, as for the sum reducer; lse = -inf.
+ *   q [n_dst, D], k [n_src, D], v [n_src, D];  y, A [n_dst, D];  lse [n_dst] = log sum_e exp(s_e).
+ * A receives sum_e softmax_e |v_s(e)|, the scale of the rounding error of y.
+ */
+int oracle_csr_attention(const int64_t* rowptr, const int32_t* col, int64_t n_dst,
+                         const double* q, const double* k, const double* v, int D, double scale,
+                         double* y, double* A, double* lse) {
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int64_t i = 0; i < n_dst; ++i) {
+        const int64_t b = rowptr[i], e = rowptr[i + 1];
+        double* yi = y + i * D;
+        double* Ai = A ? A + i * D : NULL;
+        for (int d = 0; d < D; ++d) { yi[d] = 0.0; if (Ai) Ai[d] = 0.0; }
+        if (b == e) { if (lse) lse[i] = -INFINITY; continue; }
+        double* s = (double*)malloc((size_t)(e - b) * sizeof(double));
+        double mx = -INFINITY;
+        for (int64_t t = b; t < e; ++t) {
+            const double* kj = k + (int64_t)col[t] * D;
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d) dot += q[i * D + d] * kj[d];
+            s[t - b] = scale * dot;
+            if (s[t - b] > mx) mx = s[t - b];
+        }
+        double mass = 0.0;
+        for (int64_t t = b; t < e; ++t) mass += exp(s[t - b] - mx);
+        for (int64_t t = b; t < e; ++t) {
+            const double pr = exp(s[t - b] - mx) / mass;
+            const double* vj = v + (int64_t)col[t] * D;
+            for (int d = 0; d < D; ++d) {
+                yi[d] += pr * vj[d];
+                if (Ai) Ai[d] += fabs(pr * vj[d]);
+            }
+        }
+        if (lse) lse[i] = mx + log(mass);
+        free(s);
     }
     return 0;
 }
