@@ -251,6 +251,27 @@ tiga_status tiga_apply_radius_mlp_backward(const float* pos, const float* feat, 
                                            float* grad_W1, float* grad_b1, float* grad_W2, float* grad_b2,
                                            void* ws, size_t ws_bytes, int reuse_plan, void* stream);
 
+/* ----------------------------------------------------------------- stored relation, online-softmax reducer */
+
+/* Online-softmax reducer over the rows of a stored relation (Section 5, "Online softmax and
+ * approximation"; the attention appendix): the edge function supplies a score and a value,
+ *     s_e = scale * <q[d(e),:], key[s(e),:]>,
+ *     out[i,:] = sum_e exp(s_e) value[s(e),:] / sum_e exp(s_e)      over the edges e of row i,
+ * evaluated with the streaming state (maximum, mass, accumulator) and the combine rule of that
+ * section; the relation decides which interactions exist (a triangular relation with the diagonal
+ * is causal attention).  Repeated edges are separate messages.  A row without edges yields the
+ * zero vector and lse = -inf (the reducer's empty-row convention, as for the sum reducer).
+ *   q : fp32 [n_dst, D];  key, value : fp32 [n_src, D];  D a multiple of 4, 4..128
+ *       (TIGA_ERR_UNSUPPORTED above 128);  out : fp32 [n_dst, D], fully overwritten
+ *   lse : fp32 [n_dst] or NULL, log of the row's total mass sum_e exp(s_e)
+ *   ws  : tiga_csr_attention_workspace_bytes(g, D) bytes, 16-byte aligned.
+ * All arrays are device pointers, g is read on the host.  Forward only (the paper has no
+ * streaming backward for this reducer).  No atomics: results are reproducible. */
+size_t tiga_csr_attention_workspace_bytes(const tiga_csr* g, int32_t D);
+tiga_status tiga_apply_csr_attention(const tiga_csr* g, const float* q, const float* key, const float* value,
+                                     int32_t D, float scale, float* out, float* lse,
+                                     void* ws, size_t ws_bytes, void* stream);
+
 /* ----------------------------------------------------------------- generated exact kNN */
 
 #define TIGA_KNN_MAX_K 32

@@ -18,7 +18,8 @@ __all__ = [
     "tiga_apply_csr", "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram",
     "tiga_radius_grid", "tiga_radius_workspace_bytes", "tiga_radius_bin",
     "tiga_apply_radius", "tiga_apply_radius_backward", "tiga_apply_radius_mlp",
-    "tiga_apply_radius_mlp_backward", "tiga_knn_workspace_bytes", "tiga_apply_knn", "launch_count",
+    "tiga_apply_radius_mlp_backward", "tiga_knn_workspace_bytes", "tiga_apply_knn",
+    "tiga_csr_attention_workspace_bytes", "tiga_apply_csr_attention", "launch_count",
 ]
 
 SUM, MAX = 0, 1
@@ -31,7 +32,7 @@ EXPORTS = [
     "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram", "tiga_radius_grid",
     "tiga_radius_workspace_bytes", "tiga_radius_bin", "tiga_apply_radius",
     "tiga_apply_radius_backward", "tiga_apply_radius_mlp", "tiga_apply_radius_mlp_backward",
-    "tiga_knn_workspace_bytes", "tiga_apply_knn",
+    "tiga_knn_workspace_bytes", "tiga_apply_knn", "tiga_csr_attention_workspace_bytes", "tiga_apply_csr_attention",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -109,6 +110,10 @@ def load_library() -> ctypes.CDLL:
     lib.tiga_apply_radius_mlp_backward.restype = ctypes.c_int
     lib.tiga_apply_radius_mlp_backward.argtypes = [vp, vp, i64, f, ctypes.POINTER(_Box), ctypes.POINTER(_EdgeMlp), vp,
                                                    vp, vp, vp, vp, vp, vp, vp, sz, ctypes.c_int, vp]
+    lib.tiga_csr_attention_workspace_bytes.restype = sz
+    lib.tiga_csr_attention_workspace_bytes.argtypes = [ctypes.POINTER(_Csr), i32]
+    lib.tiga_apply_csr_attention.restype = ctypes.c_int
+    lib.tiga_apply_csr_attention.argtypes = [ctypes.POINTER(_Csr), vp, vp, vp, i32, f, vp, vp, vp, sz, vp]
     lib.tiga_knn_workspace_bytes.restype = sz
     lib.tiga_knn_workspace_bytes.argtypes = [i64, i32, ctypes.POINTER(_Box)]
     lib.tiga_apply_knn.restype = ctypes.c_int
@@ -418,3 +423,25 @@ def tiga_apply_knn(pos, feat, k: int, box, periodic=(0, 0, 0), out=None, nbr=Non
                                       _ptr(nbr_d2), _ptr(ws), ws.numel(), _stream(stream)), "tiga_apply_knn")
     _launches += 8
     return out, nbr, nbr_d2, ws
+
+
+def tiga_csr_attention_workspace_bytes(g: CsrRelation, D: int) -> int:
+    return int(load_library().tiga_csr_attention_workspace_bytes(g.ref, int(D)))
+
+
+def tiga_apply_csr_attention(g: CsrRelation, q, key, value, scale: float, out=None, lse=None, want_lse=True,
+                             ws=None, stream=None):
+    """out[i] = sum_e softmax_e(scale * <q[i], key[col[e]]>) value[col[e]] over the edges of row i
+    (online-softmax reducer).  Returns (out, lse, ws)."""
+    global _launches
+    D = q.shape[1]
+    if out is None:
+        out = torch.empty((g.n_dst, D), dtype=torch.float32, device=q.device)
+    if want_lse and lse is None:
+        lse = torch.empty(g.n_dst, dtype=torch.float32, device=q.device)
+    if ws is None:
+        ws = _ws(tiga_csr_attention_workspace_bytes(g, D), q)
+    _ok(load_library().tiga_apply_csr_attention(g.ref, _ptr(q), _ptr(key), _ptr(value), D, float(scale), _ptr(out),
+                                                _ptr(lse), _ptr(ws), ws.numel(), _stream(stream)), "tiga_apply_csr_attention")
+    _launches += 2
+    return out, lse, ws
