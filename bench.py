@@ -506,6 +506,31 @@ def run_paper_shapes(args):
                      "ms_median": fwd[0], "ms_min": fwd[1], "ms_max": fwd[2], "backward_ms_median": bwd[0],
                      "backward_ms_min": bwd[1], "backward_ms_max": bwd[2], "interactions_per_s": pairs / (fwd[0] * 1e-3),
                      "paper": paper + " on the Stanford Bunny vertices, 356,260 edges (RTX 5070 Ti)"})
+    # online-softmax reducer: graph attention over the benchmark's stored relation and causal attention
+    # as a stored triangular relation (the appendix' example shape, longer)
+    c = gen.config("cfg1", args.seed)
+    g = T.CsrRelation(to(c["rowptr"]), to(c["col"]), c["n"])
+    q, k, v = (to(gen.normal_features(c["n"], 64, args.seed, 31 + i)) for i in range(3))
+    out, lse, ws = T.tiga_apply_csr_attention(g, q, k, v, 0.125)
+    med, lo, hi = median_ms(lambda: T.tiga_apply_csr_attention(g, q, k, v, 0.125, out=out, lse=lse, ws=ws))
+    rows.append({"shape": "online-softmax reducer (graph attention), R-MAT scale 20, 16,777,216 edges, width 64", "edges": c["E"],
+                 "F": 64, "ms_median": med, "ms_min": lo, "ms_max": hi, "edges_per_s": c["E"] / (med * 1e-3),
+                 "gather_GBps": c["E"] * 512 / (med * 1e-3) / 1e9, "paper": "not measured in the paper"})
+    del g, q, k, v, out, lse, ws
+    for n in (4096, 16384):
+        rp = torch.cat([torch.zeros(1, device=dev, dtype=torch.int64), torch.cumsum(torch.arange(1, n + 1, device=dev, dtype=torch.int64), 0)])
+        e = torch.arange(int(rp[-1].item()), device=dev, dtype=torch.int64)
+        col = (e - rp[torch.searchsorted(rp, e, right=True) - 1]).to(torch.int32)      # row i holds sources 0..i
+        del e
+        g = T.CsrRelation(rp, col, n)
+        q, k, v = (torch.randn((n, 64), device=dev) for _ in range(3))
+        out, lse, ws = T.tiga_apply_csr_attention(g, q, k, v, 0.125)
+        med, lo, hi = median_ms(lambda: T.tiga_apply_csr_attention(g, q, k, v, 0.125, out=out, lse=lse, ws=ws))
+        E = col.numel()
+        rows.append({"shape": f"online-softmax reducer, causal attention as a stored triangular relation, {n} tokens, width 64", "edges": E,
+                     "F": 64, "ms_median": med, "ms_min": lo, "ms_max": hi, "edges_per_s": E / (med * 1e-3),
+                     "paper": "appendix example (65 tokens) is a correctness check; the paper's dense streaming path is not timed"})
+        del g, q, k, v, out, lse, ws, rp, col
     # generated exact kNN, scalar neighbour sum, k = 16, relation rebuilt from the coordinates every call
     knn_paper = {1024: "0.147 ms (Torch 0.244, PyG 1.775)", 16384: "6.32 ms (Torch 29.92, PyG 17.50)",
                  131072: "172.37 ms (Torch 1908.43, PyG 393.21)"}
@@ -566,6 +591,14 @@ def run_case(args):
             out, cnt, ws = T.tiga_apply_radius(pos, x, c["r"], c["box"], c["periodic"], T.MSG_GAUSS, p0=c["sigma"])
             T.tiga_apply_radius_backward(pos, x, gy, c["r"], c["box"], c["periodic"], c["sigma"], ws=ws, reuse_plan=True)
         units = c["n"]
+    elif args.case == "attention":
+        c = gen.config("cfg1", args.seed, scale=args.size or 20)
+        g = T.CsrRelation(to(c["rowptr"]), to(c["col"]), c["n"])
+        q, k, v = (to(gen.normal_features(c["n"], 64, args.seed, 31 + i)) for i in range(3))
+        out, lse, ws = T.tiga_apply_csr_attention(g, q, k, v, 0.125)
+        def run():
+            T.tiga_apply_csr_attention(g, q, k, v, 0.125, out=out, lse=lse, ws=ws)
+        units = c["E"]
     elif args.case == "knn":
         n = args.size or 1_000_000
         pos, x = to(gen.uniform_points(n, args.seed)), to(gen.normal_features(n, 1, args.seed, 31))
@@ -599,7 +632,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--seed", type=int, default=gen.DEFAULT_SEED)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", default=None, choices=["csr", "csr_large", "radius_gauss", "radius_lj", "knn", "paper_shapes"],
+    ap.add_argument("--case", default=None, choices=["csr", "csr_large", "radius_gauss", "radius_lj", "knn", "attention", "paper_shapes"],
                     help="run one traversal on a reduced replica (for profiler captures) instead of the benchmark")
     ap.add_argument("--size", type=int, default=0, help="--case size: R-MAT scale, number of points, or lattice side")
     args = ap.parse_args()
