@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(HERE, "libtiga.so")
-SOURCES = ["csr.cu", "csr_attention.cu", "radius.cu", "radius_mlp.cu", "knn.cu"]
+SOURCES = ["csr.cu", "csr_attention.cu", "radius.cu", "radius_lj.cu", "radius_mlp.cu", "knn.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I" + INCLUDE, "-I" + CSRC]
 

@@ -764,7 +764,7 @@ extern "C" tiga_status tiga_apply_radius(const float* pos, const float* feat, in
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     st = run_binning(p, fill, lay.nblocks, s);
     if (st != TIGA_OK) return st;
-    if (msg->kind == TIGA_MSG_LJ) return launch_traverse<1, false>(p, s);
+    if (msg->kind == TIGA_MSG_LJ) return launch_lj_pairs(p, s);
     if (msg->kind == TIGA_MSG_DIST) return launch_traverse<0, true>(p, s);
     return launch_traverse<0, false>(p, s);
 }

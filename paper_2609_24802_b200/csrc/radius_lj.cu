@@ -1,0 +1,348 @@
+// Lennard-Jones message over the generated radius relation (fused cell-list traversal, paper
+// Section 4.9), evaluated once per unordered pair.
+//
+// The pair force is antisymmetric and the pair energy symmetric, so the row sums
+//     F_i = sum over j in N(i) of f_ij,   e_i = sum over j in N(i) of u_ij / 2
+// can be formed by visiting every unordered pair {i, j} once and adding f_ij to row i and -f_ij
+// to row j.  One warp owns a cell and tests its points against the points of the cell itself
+// (each pair once, by index order) and of the 13 neighbour cells whose offset is lexicographically
+// positive; the other 13 cells visit this one from their side.  That halves the candidate tests,
+// the staging and the force evaluations of a traversal that walks all 27 cells per row.
+//
+// The price is that a row is no longer summed by a single warp: contributions arrive through
+// 128-bit vector atomics (out must start at zero), so the summation order, and with it the last
+// bits of the result, can change from run to run.  Neighbour counts are integers and stay exact.
+//
+// Structure inside a warp (as in radius_traverse_kernel): the half stencil is staged in shared
+// memory in cell-local coordinates with periodic images applied (exact fp32 shifts), candidates
+// farther than the cutoff from the bounding box of the cell's points are dropped, phase A tests one
+// staged candidate per lane against eight queries and compacts accepted pairs into per-query
+// lists by ballots (pairs within the fp32 error band of the cutoff are decided in fp64), phase B
+// gives every query four lanes that evaluate its listed pairs.
+#include "radius_shared.cuh"
+#include <type_traits>
+
+namespace tiga {
+
+constexpr int LJ_STAGE_CAP = 256;
+constexpr int LJ_QCAP = 64;
+constexpr int LJ_QSTRIDE = LJ_QCAP + 1;
+constexpr int LJ_STAGE_BYTES = (LJ_STAGE_CAP + STAGE_PAD) * 16;
+constexpr int LJ_LIST_BYTES = (QB * LJ_QSTRIDE * 8 + 15) / 16 * 16;
+constexpr int LJ_MISC_BYTES = QB * 16 + QB * 4 + LJ_STAGE_CAP * 4;      // queries, list lengths, per-candidate counts
+constexpr int LJ_PER_WARP = LJ_STAGE_BYTES + LJ_LIST_BYTES + LJ_MISC_BYTES;
+
+template <bool MI, bool COUNT>
+__global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const __grid_constant__ RadiusParams p) {
+    constexpr unsigned FULL = 0xffffffffu;
+    extern __shared__ __align__(16) unsigned char s_raw[];
+
+    const int lane = threadIdx.x & 31;
+    const int wib = threadIdx.x >> 5;
+    const int cellid = blockIdx.x * TRAV_WARPS + wib;
+    if (cellid >= p.ncells) return;
+    unsigned char* base = s_raw + (size_t)wib * LJ_PER_WARP;
+    float4* stage = reinterpret_cast<float4*>(base);                                   // local x, y, z, point id
+    float2* list = reinterpret_cast<float2*>(base + LJ_STAGE_BYTES);                   // (stage slot, d2) per query
+    float4* s_q = reinterpret_cast<float4*>(base + LJ_STAGE_BYTES + LJ_LIST_BYTES);
+    int* s_n = reinterpret_cast<int*>(s_q + QB);
+    int* s_cnt = s_n + QB;                  // accepted pairs per staged candidate (only when counts are wanted)
+
+    const int c[3] = {cellid % p.nc[0], (cellid / p.nc[0]) % p.nc[1], cellid / (p.nc[0] * p.nc[1])};
+    const float org[3] = {(float)c[0] * p.hcell[0], (float)c[1] * p.hcell[1], (float)c[2] * p.hcell[2]};
+    const bool mi0 = MI && p.periodic[0] && p.nc[0] == 1, mi1 = MI && p.periodic[1] && p.nc[1] == 1, mi2 = MI && p.periodic[2] && p.nc[2] == 1;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    float4* out4 = reinterpret_cast<float4*>(p.out);
+
+    auto fold = [&](float& dx, float& dy, float& dz) {
+        if (MI) {          // periodic dimension folded into a single cell: explicit minimum image
+            if (mi0) dx -= p.len[0] * rintf(dx * p.inv_len[0]);
+            if (mi1) dy -= p.len[1] * rintf(dy * p.inv_len[1]);
+            if (mi2) dz -= p.len[2] * rintf(dz * p.inv_len[2]);
+        }
+    };
+
+    // ---- half stencil: lane 0 is the cell itself, lanes 1..13 the lexicographically positive offsets
+    int r_cs = 0, r_len = 0;
+    float r_off[3] = {0.f, 0.f, 0.f};
+    {
+        const int L = 13 + lane;
+        const int off[3] = {L % 3 - 1, (L / 3) % 3 - 1, L / 9 - 1};
+        bool ok = lane < 14;
+        int q[3] = {0, 0, 0};
+#pragma unroll
+        for (int d = 0; d < 3; ++d) {
+            r_off[d] = org[d];
+            if (p.nc[d] == 1) { ok = ok && off[d] == 0; continue; }
+            int v = c[d] + off[d];
+            if (v < 0) {
+                if (p.periodic[d]) { v += p.nc[d]; r_off[d] = org[d] + p.len[d]; }     // org is 0 here: exact
+                else ok = false;
+            } else if (v >= p.nc[d]) {
+                if (p.periodic[d]) { v -= p.nc[d]; r_off[d] = org[d] - p.len[d]; }     // exact (Sterbenz)
+                else ok = false;
+            }
+            q[d] = v;
+        }
+        if (ok) {
+            const int id = (q[2] * p.nc[1] + q[1]) * p.nc[0] + q[0];
+            r_cs = p.cell_start[id];
+            r_len = p.cell_start[id + 1] - r_cs;
+        }
+    }
+    // lane 0 resolved the cell itself: its run is the cell's own points (one load round trip fewer
+    // than asking for them first)
+    const int qs0 = __shfl_sync(FULL, r_cs, 0), nown = __shfl_sync(FULL, r_len, 0), qe0 = qs0 + nown;
+    if (nown == 0) return;
+    int r_incl = r_len;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(FULL, r_incl, o);
+        if (lane >= o) r_incl += t;
+    }
+    const int total = __shfl_sync(FULL, r_incl, 31);
+
+    // flattened stencil position v -> its run and address in the cell-ordered points
+    auto locate = [&](const int v, int& run) -> int {
+        int r = 0;
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) {                 // 14 runs: a four-step search
+            const int probe = __shfl_sync(FULL, r_incl, r + o - 1);
+            if (probe <= v) r += o;
+        }
+        run = r > 13 ? 13 : r;
+        return __shfl_sync(FULL, r_cs, run) + (v - (__shfl_sync(FULL, r_incl, run) - __shfl_sync(FULL, r_len, run)));
+    };
+    constexpr int SU = 4;                                 // staging groups in flight
+    // start fetching the first staging groups now: they arrive while the bounding box is formed
+#pragma unroll
+    for (int u = 0; u < SU; ++u) {
+        int run;
+        const int v = 32 * u + lane;
+        const int src = locate(v, run);
+        if (v < total) asm volatile("prefetch.global.L1 [%0];" ::"l"(p.spos + src));
+    }
+
+    // ---- bounding box of the cell's own points in local coordinates, one register per lane
+    float bb;
+    {
+        float blo[3] = {FAR_AWAY, FAR_AWAY, FAR_AWAY}, bhi[3] = {-FAR_AWAY, -FAR_AWAY, -FAR_AWAY};
+        for (int q = qs0 + lane; q < qe0; q += 32) {
+            const float4 pq = p.spos[q];
+            const float l[3] = {pq.x - org[0], pq.y - org[1], pq.z - org[2]};
+#pragma unroll
+            for (int d = 0; d < 3; ++d) { blo[d] = fminf(blo[d], l[d]); bhi[d] = fmaxf(bhi[d], l[d]); }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int d = 0; d < 3; ++d) {
+                blo[d] = fminf(blo[d], __shfl_xor_sync(FULL, blo[d], o));
+                bhi[d] = fmaxf(bhi[d], __shfl_xor_sync(FULL, bhi[d], o));
+            }
+        bb = lane == 0 ? blo[0] : lane == 1 ? blo[1] : lane == 2 ? blo[2] : lane == 3 ? bhi[0] : lane == 4 ? bhi[1] : bhi[2];
+        if (mi0 && (lane == 0 || lane == 3)) bb = lane == 0 ? -FAR_AWAY : FAR_AWAY;   // a dimension folded by the explicit
+        if (mi1 && (lane == 1 || lane == 4)) bb = lane == 1 ? -FAR_AWAY : FAR_AWAY;   // minimum image is not pruned
+        if (mi2 && (lane == 2 || lane == 5)) bb = lane == 2 ? -FAR_AWAY : FAR_AWAY;
+    }
+
+    const float s2 = p.p1 * p.p1, e24 = 24.f * p.p0, e2x = 2.f * p.p0;
+
+    // ---- all queries of the cell against the ns staged candidates; the first nself of them are the
+    //      cell's own points, in the same order as the queries
+    auto process_chunk = [&](const int ns, const int nself) {
+        if (lane < STAGE_PAD) stage[ns + lane] = make_float4(FAR_AWAY, FAR_AWAY, FAR_AWAY, __int_as_float(-1));
+        if (COUNT)
+            for (int k = lane; k < ns; k += 32) s_cnt[k] = 0;
+        for (int qb0 = qs0; qb0 < qe0; qb0 += QB) {
+            const int nq = (qe0 - qb0 < QB) ? qe0 - qb0 : QB;
+            __syncwarp();
+            if (lane < nq) {
+                const float4 pq = p.spos[qb0 + lane];
+                s_q[lane] = make_float4(pq.x - org[0], pq.y - org[1], pq.z - org[2], pq.w);
+            }
+            __syncwarp();
+            int qcnt[QB];
+#pragma unroll
+            for (int q = 0; q < QB; ++q) qcnt[q] = 0;
+
+            auto drain = [&]() {
+                __syncwarp();
+                if (lane == 0) {
+#pragma unroll
+                    for (int q = 0; q < QB; ++q) s_n[q] = qcnt[q];
+                }
+                __syncwarp();
+                const int q = lane >> 2, sub = lane & 3;
+                float fx = 0.f, fy = 0.f, fz = 0.f, en = 0.f;
+                int n = 0;
+                if (q < nq) {
+                    const float4 qv = s_q[q];
+                    n = s_n[q];
+                    const float2* lq = list + q * LJ_QSTRIDE;
+                    for (int t = sub; t < n; t += 8) {
+                        float2 e[2];
+                        float4 pj[2];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            e[u] = lq[t + 4 * u < n ? t + 4 * u : t];
+                            pj[u] = stage[__float_as_int(e[u].x)];
+                        }
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            if (t + 4 * u < n) {
+                                const float inv = fast_rcp(e[u].y);
+                                const float qq = s2 * inv;
+                                const float q3 = qq * qq * qq;
+                                const float fs = e24 * (2.f * q3 * q3 - q3) * inv;
+                                const float ee = e2x * (q3 * q3 - q3);
+                                float dx = qv.x - pj[u].x, dy = qv.y - pj[u].y, dz = qv.z - pj[u].z;
+                                fold(dx, dy, dz);
+                                const float gx = fs * dx, gy = fs * dy, gz = fs * dz;
+                                fx += gx; fy += gy; fz += gz; en += ee;
+                                const int idj = __float_as_int(pj[u].w);
+                                atomicAdd(out4 + idj, make_float4(-gx, -gy, -gz, ee));      // the pair's other row
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int o = 1; o <= 2; o <<= 1) {
+                    fx += __shfl_xor_sync(FULL, fx, o); fy += __shfl_xor_sync(FULL, fy, o);
+                    fz += __shfl_xor_sync(FULL, fz, o); en += __shfl_xor_sync(FULL, en, o);
+                }
+                if (q < nq && sub == 0 && n > 0) {
+                    const int idq = __float_as_int(s_q[q].w);
+                    atomicAdd(out4 + idq, make_float4(fx, fy, fz, en));
+                    if (COUNT) atomicAdd(p.count + idq, n);
+                }
+#pragma unroll
+                for (int q2 = 0; q2 < QB; ++q2) qcnt[q2] = 0;
+                __syncwarp();
+            };
+
+            // ---- phase A: one staged candidate per lane against the queries of the batch.
+            //      OWN: the group holds points of the cell itself, which pair only with later ones.
+            auto phase_a = [&](const int cbase, auto full_batch, auto own_group) -> bool {
+                constexpr bool FULLB = decltype(full_batch)::value;
+                constexpr bool OWN = decltype(own_group)::value;
+                const float4 pj = stage[cbase + lane];
+                const int idj = __float_as_int(pj.w);
+                const bool own = OWN && cbase + lane < nself;
+                float d2q[QB];
+                float nearest = FAR_AWAY;       // smallest |d2 - r^2| seen by this lane
+#pragma unroll
+                for (int q = 0; q < QB; ++q) {
+                    if (!FULLB && q >= nq) break;
+                    const float4 qv = s_q[q];
+                    float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
+                    fold(dx, dy, dz);
+                    float d2 = fmaf(dz, dz, fmaf(dy, dy, dx * dx));
+                    if (OWN && own && idj <= __float_as_int(qv.w)) d2 = FAR_AWAY;      // own cell: each pair once
+                    if (MI && idj < 0) d2 = FAR_AWAY;                                  // folded sentinels
+                    nearest = fminf(nearest, fabsf(d2 - p.r2_mid));
+                    d2q[q] = d2;
+                }
+                if (__any_sync(FULL, nearest <= p.r2_band)) {
+                    // some pair lies within the fp32 error band of the cutoff: decide it in fp64
+#pragma unroll
+                    for (int q = 0; q < QB; ++q) {
+                        if (!FULLB && q >= nq) break;
+                        if (fabsf(d2q[q] - p.r2_mid) <= p.r2_band)
+                            d2q[q] = exact_pair(p, __float_as_int(s_q[q].w), idj) ? fminf(d2q[q], p.r2_lo) : FAR_AWAY;
+                    }
+                }
+                int mx = 0, mine = 0;           // mine: queries that accepted this lane's candidate
+#pragma unroll
+                for (int q = 0; q < QB; ++q) {
+                    if (!FULLB && q >= nq) break;
+                    const bool ok = d2q[q] <= p.r2_lo;
+                    const unsigned m = __ballot_sync(FULL, ok);
+                    float2* dst = list + q * LJ_QSTRIDE + qcnt[q] + __popc(m & lt_mask);
+                    if (ok) *dst = make_float2(__int_as_float(cbase + lane), d2q[q]);
+                    if (COUNT) mine += ok ? 1 : 0;
+                    qcnt[q] += __popc(m);
+                    mx = qcnt[q] > mx ? qcnt[q] : mx;
+                }
+                if (COUNT && mine) s_cnt[cbase + lane] += mine;      // the slot belongs to this lane alone
+                return mx > LJ_QCAP - 32;
+            };
+
+            bool need = false;
+            for (int cbase = 0;; cbase += 32) {
+                const bool done = cbase >= ns;
+                if (done || need) drain();
+                if (done) break;
+                if (cbase < nself)
+                    need = (nq == QB) ? phase_a(cbase, std::true_type{}, std::true_type{}) : phase_a(cbase, std::false_type{}, std::true_type{});
+                else
+                    need = (nq == QB) ? phase_a(cbase, std::true_type{}, std::false_type{}) : phase_a(cbase, std::false_type{}, std::false_type{});
+            }
+        }
+        __syncwarp();
+        if (COUNT)                            // the candidates' side of the neighbour counts, one atomic per candidate
+            for (int k = lane; k < ns; k += 32) {
+                const int cnum = s_cnt[k];
+                if (cnum) atomicAdd(p.count + __float_as_int(stage[k].w), cnum);
+            }
+        __syncwarp();
+    };
+
+    // ---- flat staging of the kept candidates, a chunk at a time
+    for (int lo = 0; lo < total; lo += LJ_STAGE_CAP) {
+        const int nin = total - lo < LJ_STAGE_CAP ? total - lo : LJ_STAGE_CAP;
+        int nst = 0;
+        for (int k0 = 0; k0 < nin; k0 += 32 * SU) {
+            float4 c4[SU];
+            float ox[SU], oy[SU], oz[SU];
+#pragma unroll
+            for (int u = 0; u < SU; ++u) {                // all loads of the step first
+                const int k = k0 + 32 * u + lane;
+                int run;
+                const int src = locate(lo + k, run);
+                ox[u] = __shfl_sync(FULL, r_off[0], run); oy[u] = __shfl_sync(FULL, r_off[1], run); oz[u] = __shfl_sync(FULL, r_off[2], run);
+                c4[u] = k < nin ? __ldg(p.spos + src) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            const float lx = __shfl_sync(FULL, bb, 0), ly = __shfl_sync(FULL, bb, 1), lz = __shfl_sync(FULL, bb, 2);
+            const float hx = __shfl_sync(FULL, bb, 3), hy = __shfl_sync(FULL, bb, 4), hz = __shfl_sync(FULL, bb, 5);
+#pragma unroll
+            for (int u = 0; u < SU; ++u) {
+                if (k0 + 32 * u >= nin) break;
+                const float4 val = make_float4(c4[u].x - ox[u], c4[u].y - oy[u], c4[u].z - oz[u], c4[u].w);
+                const float ex = fmaxf(fmaxf(lx - val.x, val.x - hx), 0.f);
+                const float ey = fmaxf(fmaxf(ly - val.y, val.y - hy), 0.f);
+                const float ez = fmaxf(fmaxf(lz - val.z, val.z - hz), 0.f);
+                const bool keep = k0 + 32 * u + lane < nin && fmaf(ez, ez, fmaf(ey, ey, ex * ex)) <= p.r2_hi * 1.0001f;
+                const unsigned m = __ballot_sync(FULL, keep);
+                if (keep) stage[nst + __popc(m & lt_mask)] = val;
+                nst += __popc(m);
+            }
+        }
+        __syncwarp();
+        // the cell's own points come first in the flattened stencil and are never dropped
+        const int nself = lo < nown ? (nown - lo < LJ_STAGE_CAP ? nown - lo : LJ_STAGE_CAP) : 0;
+        process_chunk(nst, nself);
+    }
+}
+
+template <bool MI, bool COUNT>
+static tiga_status launch_lj_t(const RadiusParams& p, cudaStream_t s) {
+    const unsigned blocks = (unsigned)((p.ncells + TRAV_WARPS - 1) / TRAV_WARPS);
+    constexpr int smem = LJ_PER_WARP * TRAV_WARPS;
+    auto kern = radius_lj_pairs_kernel<MI, COUNT>;
+    if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    kern<<<blocks, TRAV_THREADS, smem, s>>>(p);
+    return launch_status();
+}
+
+tiga_status launch_lj_pairs(const RadiusParams& p, cudaStream_t s) {
+    // rows are accumulated by atomics from several warps: start from zero
+    TIGA_CUDA_TRY(cudaMemsetAsync(p.out, 0, (size_t)p.n * 4 * sizeof(float), s));
+    if (p.count) TIGA_CUDA_TRY(cudaMemsetAsync(p.count, 0, (size_t)p.n * sizeof(int32_t), s));
+    bool mi = false;
+    for (int d = 0; d < 3; ++d) mi = mi || (p.periodic[d] && p.nc[d] == 1);
+    if (p.count) return mi ? launch_lj_t<true, true>(p, s) : launch_lj_t<false, true>(p, s);
+    return mi ? launch_lj_t<true, false>(p, s) : launch_lj_t<false, false>(p, s);
+}
+
+}  // namespace tiga

@@ -61,6 +61,8 @@ struct RadiusLayout {
 tiga_status fill_params(RadiusParams* p, long long n, float r, const tiga_box* box);
 RadiusLayout carve_radius(RadiusParams* p, void* ws, int32_t** fill);
 tiga_status run_binning(RadiusParams& p, int32_t* fill, int nblocks, cudaStream_t s);
+// host side, defined in radius_lj.cu: zeroes out / count, then one launch (pairs visited once, rows summed by atomics)
+tiga_status launch_lj_pairs(const RadiusParams& p, cudaStream_t s);
 
 // The defining predicate in double precision (same operations as the plain definition).
 static __device__ __noinline__ bool exact_within(const RadiusParams& p, const float4 a, const float4 b) {
