@@ -526,32 +526,39 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_trav
     for (int lo = 0; lo < total || first_chunk; lo += STAGE_CAP) {
         const int ns = total - lo < STAGE_CAP ? total - lo : STAGE_CAP;
         int nst = 0;                                                         // candidates kept (warp uniform)
-        for (int k = lane; k < ns + (32 - (ns & 31)) % 32; k += 32) {        // whole warp trips: shuffles inside
-            const int v = lo + k;
-            int r = 0;
+        constexpr int SU = 4;                                                // staging groups in flight
+        for (int k0 = 0; k0 < ns; k0 += 32 * SU) {
+            float4 c4[SU];
+            float ox[SU], oy[SU], oz[SU];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const int probe = __shfl_sync(FULL, r_incl, r + o - 1);
-                if (probe <= v) r += o;
+            for (int u = 0; u < SU; ++u) {                                   // all loads of the step first
+                const int k = k0 + 32 * u + lane;
+                const int v = lo + k;
+                int r = 0;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const int probe = __shfl_sync(FULL, r_incl, r + o - 1);
+                    if (probe <= v) r += o;
+                }
+                r = r > 31 ? 31 : r;
+                const int src = __shfl_sync(FULL, r_cs, r) + (v - (__shfl_sync(FULL, r_incl, r) - __shfl_sync(FULL, r_len, r)));
+                ox[u] = __shfl_sync(FULL, r_off[0], r); oy[u] = __shfl_sync(FULL, r_off[1], r); oz[u] = __shfl_sync(FULL, r_off[2], r);
+                c4[u] = k < ns ? __ldg(p.spos + src) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            r = r > 31 ? 31 : r;
-            const int src = __shfl_sync(FULL, r_cs, r) + (v - (__shfl_sync(FULL, r_incl, r) - __shfl_sync(FULL, r_len, r)));
-            const float ox = __shfl_sync(FULL, r_off[0], r), oy = __shfl_sync(FULL, r_off[1], r), oz = __shfl_sync(FULL, r_off[2], r);
             const float lx = __shfl_sync(FULL, bb, 0), ly = __shfl_sync(FULL, bb, 1), lz = __shfl_sync(FULL, bb, 2);
             const float hx = __shfl_sync(FULL, bb, 3), hy = __shfl_sync(FULL, bb, 4), hz = __shfl_sync(FULL, bb, 5);
-            bool keep = false;
-            float4 val = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (k < ns) {
-                const float4 c4 = __ldg(p.spos + src);
-                val = make_float4(c4.x - ox, c4.y - oy, c4.z - oz, c4.w);
+#pragma unroll
+            for (int u = 0; u < SU; ++u) {
+                if (k0 + 32 * u >= ns) break;
+                const float4 val = make_float4(c4[u].x - ox[u], c4[u].y - oy[u], c4[u].z - oz[u], c4[u].w);
                 const float ex = fmaxf(fmaxf(lx - val.x, val.x - hx), 0.f);
                 const float ey = fmaxf(fmaxf(ly - val.y, val.y - hy), 0.f);
                 const float ez = fmaxf(fmaxf(lz - val.z, val.z - hz), 0.f);
-                keep = fmaf(ez, ez, fmaf(ey, ey, ex * ex)) <= p.r2_hi * 1.0001f;
+                const bool keep = k0 + 32 * u + lane < ns && fmaf(ez, ez, fmaf(ey, ey, ex * ex)) <= p.r2_hi * 1.0001f;
+                const unsigned m = __ballot_sync(FULL, keep);
+                if (keep) stage[nst + __popc(m & lt_mask)] = val;
+                nst += __popc(m);
             }
-            const unsigned m = __ballot_sync(FULL, keep);
-            if (keep) stage[nst + __popc(m & lt_mask)] = val;
-            nst += __popc(m);
         }
         __syncwarp();
         process_chunk(nst, first_chunk);
