@@ -8,11 +8,12 @@
 //   1. binning: cell id per point + per-cell counts, exclusive scan (reduce-then-scan, no
 //      inter-CTA waiting), scatter into cell order, per-cell rank sort by point id (which
 //      makes the scatter stable and therefore unique), sorted copy of the positions;
-//   2. traversal: one warp per query cell walks the 27 neighbouring cells (wrapped or
-//      clipped) as contiguous candidate ranges.  The lanes of a query split its candidates;
-//      accepted (source, weight) pairs go to lane-private lists in shared memory and are
-//      consumed with groups of lanes across the feature axis, so every gathered feature
-//      row is one coalesced 128-bit-per-lane request.
+//   2. traversal: one warp per query cell stages the 27 neighbouring cells (wrapped or
+//      clipped, contiguous ranges of the cell-ordered points) in shared memory, tests one
+//      staged candidate per lane against eight queries at a time, compacts accepted
+//      (source, weight) pairs into one list per query and consumes the lists with groups of
+//      lanes across the feature axis, so every gathered feature row is one coalesced
+//      128-bit-per-lane request.  (Lennard-Jones: radius_lj.cu; edge network: radius_mlp.cu.)
 //
 // Exact membership: the fp32 squared distance is only a filter.  A pair whose fp32 value
 // falls within a few ulps of r^2 is re-decided in fp64 with the defining formula
@@ -174,16 +175,16 @@ __global__ void bin_sort_kernel(const RadiusParams p) {
 //             (staged slot, d^2 or weight) where the displacement is needed again.
 //   phase B : MODE 0 (Gaussian / distance forward) and MODE 2 (Gaussian backward): LF lanes
 //             span one feature row with 128-bit accesses and 32 / LF queries advance together,
-//             four gathered rows in flight per lane; MODE 1 (Lennard-Jones): four lanes share
-//             a query's list and evaluate the pair forces.
+//             four gathered rows in flight per lane.  (The Lennard-Jones message has its own
+//             kernel in radius_lj.cu, which visits every unordered pair once.)
 // Lists hold QCAP entries per query and the stage STAGE_CAP candidates; when either fills up
 // the warp drains / processes and goes on, so any density works.
 
 template <int MODE> struct TravSmem {
-    // sized for the workloads' densities (about 216 / 351 candidates, 32 / 54 neighbours);
+    // sized for the workload's density (about 216 candidates before pruning, 32 neighbours);
     // denser inputs only mean more chunks and drains
-    static constexpr int STAGE_CAP = (MODE == 1) ? 384 : 256;      // candidates staged per chunk
-    static constexpr int QCAP = (MODE == 1) ? 96 : 80;             // list entries per query
+    static constexpr int STAGE_CAP = 256;                          // candidates staged per chunk
+    static constexpr int QCAP = 80;                                // list entries per query
     static constexpr int QSTRIDE = QCAP + 1;                       // odd stride: the lists of different queries fall in different banks
     static constexpr int STAGE_BYTES = (STAGE_CAP + STAGE_PAD) * 16;
     static constexpr int LIST_BYTES = (QB * QSTRIDE * 8 + 15) / 16 * 16;
@@ -191,7 +192,7 @@ template <int MODE> struct TravSmem {
     static constexpr int PER_WARP = STAGE_BYTES + LIST_BYTES + MISC_BYTES;
 };
 
-// MODE 0: Gaussian (DIST = false) or distance-weighted (DIST = true) forward; 1: Lennard-Jones;
+// MODE 0: Gaussian (DIST = false) or distance-weighted (DIST = true) forward;
 // 2: Gaussian backward.  MI: some periodic dimension has a single cell (explicit minimum image).
 // VEC: feature rows are 16-byte aligned (F % 4 == 0); otherwise the forward uses scalar accesses.
 template <int MODE, int LF, bool DIST, bool MI, bool VEC = true>
@@ -218,7 +219,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_trav
     const int c[3] = {cellid % p.nc[0], (cellid / p.nc[0]) % p.nc[1], cellid / (p.nc[0] * p.nc[1])};
     const float org[3] = {(float)c[0] * p.hcell[0], (float)c[1] * p.hcell[1], (float)c[2] * p.hcell[2]};
     const int F = p.F;
-    const float neg_c2 = (MODE != 1 && !DIST) ? -1.4426950408889634f / (2.f * p.p0 * p.p0) : 0.f;   // exp(-d2/(2 s^2)) = 2^(d2 * neg_c2)
+    const float neg_c2 = !DIST ? -1.4426950408889634f / (2.f * p.p0 * p.p0) : 0.f;   // exp(-d2/(2 s^2)) = 2^(d2 * neg_c2)
     const int fl = lane % LF, grp = lane / LF;
     const bool mi0 = MI && p.periodic[0] && p.nc[0] == 1, mi1 = MI && p.periodic[1] && p.nc[1] == 1, mi2 = MI && p.periodic[2] && p.nc[2] == 1;
     constexpr int QP = 32 / LF;
@@ -257,48 +258,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_trav
                     for (int q = 0; q < QB; ++q) { s_n[q] = qcnt[q]; s_tot[q] += qcnt[q]; }
                 }
                 __syncwarp();
-                if (MODE == 1) {
-                    // four lanes per query
-                    const int q = lane >> 2, sub = lane & 3;
-                    float fx = 0.f, fy = 0.f, fz = 0.f, en = 0.f;
-                    if (q < nq) {
-                        const float4 qv = s_q[q];
-                        const int n = s_n[q];
-                        const float s2 = p.p1 * p.p1, e24 = 24.f * p.p0, e2x = 2.f * p.p0;
-                        const float2* lq = list + q * QSTRIDE;
-                        for (int t = sub; t < n; t += 8) {
-                            float2 e[2];
-                            float4 pj[2];
-#pragma unroll
-                            for (int u = 0; u < 2; ++u) {
-                                e[u] = lq[t + 4 * u < n ? t + 4 * u : t];
-                                pj[u] = stage[__float_as_int(e[u].x)];
-                            }
-#pragma unroll
-                            for (int u = 0; u < 2; ++u) {
-                                const float inv = (t + 4 * u < n) ? fast_rcp(e[u].y) : 0.f;      // 0 switches the pair off
-                                const float qq = s2 * inv;
-                                const float q3 = qq * qq * qq;
-                                const float fs = e24 * (2.f * q3 * q3 - q3) * inv;
-                                float dx = qv.x - pj[u].x, dy = qv.y - pj[u].y, dz = qv.z - pj[u].z;
-                                fold(dx, dy, dz);
-                                fx = fmaf(fs, dx, fx); fy = fmaf(fs, dy, fy); fz = fmaf(fs, dz, fz);
-                                en = fmaf(e2x, q3 * q3 - q3, en);
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int o = 1; o <= 2; o <<= 1) {
-                        fx += __shfl_xor_sync(FULL, fx, o); fy += __shfl_xor_sync(FULL, fy, o);
-                        fz += __shfl_xor_sync(FULL, fz, o); en += __shfl_xor_sync(FULL, en, o);
-                    }
-                    if (q < nq && sub == 0) {
-                        float4* o = reinterpret_cast<float4*>(p.out) + __float_as_int(s_q[q].w);
-                        float4 a = make_float4(fx, fy, fz, en);
-                        if (!first) { const float4 old = *o; a.x += old.x; a.y += old.y; a.z += old.z; a.w += old.w; }
-                        *o = a;
-                    }
-                } else {
+                {
                     for (int pass = 0; pass * QP < nq; ++pass) {
                         const int qq = pass * QP + grp;
                         const bool valid = qq < nq && fvalid;
@@ -430,8 +390,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_trav
                     const bool ok = d2q[q] <= p.r2_lo;
                     const unsigned m = __ballot_sync(FULL, ok);
                     float val;
-                    if (MODE == 1) val = d2q[q];
-                    else val = DIST ? sqrtf(d2q[q]) : fast_exp2(d2q[q] * neg_c2);
+                    val = DIST ? sqrtf(d2q[q]) : fast_exp2(d2q[q] * neg_c2);
                     float2* dst = list + q * QSTRIDE + qcnt[q] + __popc(m & lt_mask);
                     if (ok) *dst = make_float2(MODE == 0 ? pj.w : __int_as_float(cbase + lane), val);
                     qcnt[q] += __popc(m);
@@ -671,7 +630,7 @@ static tiga_status launch_traverse_t(const RadiusParams& p, cudaStream_t s) {
 
 template <int MODE, bool DIST, bool MI>
 static tiga_status launch_traverse_lf(const RadiusParams& p, cudaStream_t s) {
-    switch (MODE == 1 ? 1 : feature_lanes(p.F)) {
+    switch (feature_lanes(p.F)) {
         case 1: return launch_traverse_t<MODE, 1, DIST, MI>(p, s);
         case 2: return launch_traverse_t<MODE, 2, DIST, MI>(p, s);
         case 4: return launch_traverse_t<MODE, 4, DIST, MI>(p, s);
