@@ -376,27 +376,69 @@ __global__ void __launch_bounds__(TRAV_THREADS) radius_mlp_kernel(const __grid_c
             if (lane >= o) r_incl += t;
         }
         const int total = __shfl_sync(FULL, r_incl, 31);
+        // bounding box of the cell's own points (local coordinates), one register per lane: a candidate
+        // farther than the cutoff from it is no neighbour of any of them and is not staged
+        float bb;
+        {
+            float blo[3] = {FAR_AWAY, FAR_AWAY, FAR_AWAY}, bhi[3] = {-FAR_AWAY, -FAR_AWAY, -FAR_AWAY};
+            for (int q = qs0 + lane; q < qe0; q += 32) {
+                const float4 pq = p.spos[q];
+                const float l[3] = {pq.x - org[0], pq.y - org[1], pq.z - org[2]};
+#pragma unroll
+                for (int d = 0; d < 3; ++d) { blo[d] = fminf(blo[d], l[d]); bhi[d] = fmaxf(bhi[d], l[d]); }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                for (int d = 0; d < 3; ++d) {
+                    blo[d] = fminf(blo[d], __shfl_xor_sync(FULL, blo[d], o));
+                    bhi[d] = fmaxf(bhi[d], __shfl_xor_sync(FULL, bhi[d], o));
+                }
+            bb = lane == 0 ? blo[0] : lane == 1 ? blo[1] : lane == 2 ? blo[2] : lane == 3 ? bhi[0] : lane == 4 ? bhi[1] : bhi[2];
+            if (mi0 && (lane == 0 || lane == 3)) bb = lane == 0 ? -FAR_AWAY : FAR_AWAY;   // a dimension folded by the explicit
+            if (mi1 && (lane == 1 || lane == 4)) bb = lane == 1 ? -FAR_AWAY : FAR_AWAY;   // minimum image is not pruned
+            if (mi2 && (lane == 2 || lane == 5)) bb = lane == 2 ? -FAR_AWAY : FAR_AWAY;
+        }
         bool first_chunk = true;
         for (int lo = 0; lo < total || first_chunk; lo += MLP_STAGE_CAP) {
             const int ns = total - lo < MLP_STAGE_CAP ? total - lo : MLP_STAGE_CAP;
-            for (int k = lane; k < ns + (32 - (ns & 31)) % 32; k += 32) {
-                const int v = lo + k;
-                int r = 0;
+            int nst = 0;                                                     // candidates kept (warp uniform)
+            constexpr int SU = 4;                                            // staging groups in flight
+            for (int k0 = 0; k0 < ns; k0 += 32 * SU) {
+                float4 c4[SU];
+                float ox[SU], oy[SU], oz[SU];
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    const int probe = __shfl_sync(FULL, r_incl, r + o - 1);
-                    if (probe <= v) r += o;
+                for (int u = 0; u < SU; ++u) {                               // all loads of the step first
+                    const int k = k0 + 32 * u + lane;
+                    const int v = lo + k;
+                    int r = 0;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const int probe = __shfl_sync(FULL, r_incl, r + o - 1);
+                        if (probe <= v) r += o;
+                    }
+                    r = r > 31 ? 31 : r;
+                    const int src = __shfl_sync(FULL, r_cs, r) + (v - (__shfl_sync(FULL, r_incl, r) - __shfl_sync(FULL, r_len, r)));
+                    ox[u] = __shfl_sync(FULL, r_off[0], r); oy[u] = __shfl_sync(FULL, r_off[1], r); oz[u] = __shfl_sync(FULL, r_off[2], r);
+                    c4[u] = k < ns ? __ldg(p.spos + src) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
-                r = r > 31 ? 31 : r;
-                const int src = __shfl_sync(FULL, r_cs, r) + (v - (__shfl_sync(FULL, r_incl, r) - __shfl_sync(FULL, r_len, r)));
-                const float ox = __shfl_sync(FULL, r_off[0], r), oy = __shfl_sync(FULL, r_off[1], r), oz = __shfl_sync(FULL, r_off[2], r);
-                if (k < ns) {
-                    const float4 c4 = __ldg(p.spos + src);
-                    stage[k] = make_float4(c4.x - ox, c4.y - oy, c4.z - oz, c4.w);
+                const float lx = __shfl_sync(FULL, bb, 0), ly = __shfl_sync(FULL, bb, 1), lz = __shfl_sync(FULL, bb, 2);
+                const float hx = __shfl_sync(FULL, bb, 3), hy = __shfl_sync(FULL, bb, 4), hz = __shfl_sync(FULL, bb, 5);
+#pragma unroll
+                for (int u = 0; u < SU; ++u) {
+                    if (k0 + 32 * u >= ns) break;
+                    const float4 val = make_float4(c4[u].x - ox[u], c4[u].y - oy[u], c4[u].z - oz[u], c4[u].w);
+                    const float ex = fmaxf(fmaxf(lx - val.x, val.x - hx), 0.f);
+                    const float ey = fmaxf(fmaxf(ly - val.y, val.y - hy), 0.f);
+                    const float ez = fmaxf(fmaxf(lz - val.z, val.z - hz), 0.f);
+                    const bool keep = k0 + 32 * u + lane < ns && fmaf(ez, ez, fmaf(ey, ey, ex * ex)) <= p.r2_hi * 1.0001f;
+                    const unsigned m = __ballot_sync(FULL, keep);
+                    if (keep) stage[nst + __popc(m & lt_mask)] = val;
+                    nst += __popc(m);
                 }
             }
             __syncwarp();
-            process_chunk(ns, first_chunk);
+            process_chunk(nst, first_chunk);
             first_chunk = false;
         }
     }
