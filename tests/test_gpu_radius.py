@@ -183,6 +183,52 @@ def test_lennard_jones_replica(tiga):
     assert np.max(np.abs(out[:, :3].astype(np.float64).sum(0))) < 1e-6 * A[:, :3].sum()
 
 
+def _separated_points(n, box, seed, dmin):
+    """Uniform points in the box with no pair closer than dmin (Lennard-Jones inputs never overlap)."""
+    pos = (gen.uniform_points(n, seed).astype(np.float64) * np.asarray(box, np.float64)).astype(np.float32)
+    d = pos[:, None, :].astype(np.float64) - pos[None, :, :]
+    d -= np.asarray(box, np.float64) * np.rint(d / np.asarray(box, np.float64))      # strictest reading: periodic in all
+    dist = np.sqrt((d * d).sum(2)) + np.eye(n) * 1e9
+    keep = np.ones(n, bool)
+    for i in range(n):
+        if keep[i]:
+            keep[(dist[i] < dmin) & (np.arange(n) > i)] = False
+    return pos[keep]
+
+
+@pytest.mark.parametrize("periodic", [(0, 0, 0), (1, 1, 1), (1, 0, 1), (0, 1, 0)])
+@pytest.mark.parametrize("cells", [(1, 1, 1), (2, 2, 2), (3, 3, 3), (4, 3, 2), (1, 5, 3), (6, 1, 1), (3, 4, 1)])
+def test_lennard_jones_small_grids(tiga, cells, periodic):
+    """Every unordered pair must be visited exactly once whatever the grid: one, two or three
+    cells per dimension, wrapped or clipped (a periodic dimension with fewer than three cells
+    collapses to one cell with the explicit minimum image)."""
+    r = np.float32(1.0)
+    box = np.array([c * 1.05 + 0.3 for c in cells], np.float32)       # floor(len / (r (1 + 2^-10))) = cells
+    if any(p and b <= 2.0 for p, b in zip(periodic, box)):
+        pytest.skip("a periodic dimension must be longer than twice the cutoff")
+    pos = _separated_points(600, box, 40 + sum(cells), 0.45)
+    grid, _ = tiga.tiga_radius_grid(len(pos), r, box, list(periodic))
+    expect = [1 if (p and c < 3) else c for c, p in zip(cells, periodic)]
+    cap = int(round((8 * len(pos)) ** (1 / 3) - 0.5))
+    assert list(grid) == [min(e, cap) for e in expect]
+    out, A = _check_lj(tiga, pos, r, box, list(periodic), eps=0.7, s=0.5)
+    assert np.max(np.abs(out[:, :3].astype(np.float64).sum(0))) < 1e-5 * max(A[:, :3].sum(), 1e-30)
+
+
+def test_lennard_jones_rows_are_summed_by_atomics(tiga):
+    """Two runs agree to rounding (the summation order of a row depends on scheduling) and the
+    neighbour counts, being integers, agree exactly."""
+    c = gen.config("cfg3", m=24)
+    pd = dev(c["pos"], torch)
+    a, ca, _ = tiga.tiga_apply_radius(pd, None, c["r"], c["box"], c["periodic"], tiga.MSG_LJ, p0=1.0, p1=1.0, want_count=True)
+    b, cb, _ = tiga.tiga_apply_radius(pd, None, c["r"], c["box"], c["periodic"], tiga.MSG_LJ, p0=1.0, p1=1.0, want_count=True)
+    assert torch.equal(ca, cb)
+    y, A, cnt = oracle.radius_forward(c["pos"], None, c["r"], c["box"], c["periodic"], oracle.MSG_LJ, 1.0, 1.0, use_cells=True)
+    assert np.max(np.abs(host(a).astype(np.float64) - host(b)) / A) <= 2 * SUM_TOL
+    nocount, none, _ = tiga.tiga_apply_radius(pd, None, c["r"], c["box"], c["periodic"], tiga.MSG_LJ, p0=1.0, p1=1.0)
+    assert none is None and rel_err(host(nocount), y, A) <= SUM_TOL
+
+
 # ------------------------------------------------------------------------------ full size
 def test_cfg2_full_size_sampled_rows(tiga):
     """1M points, periodic, F=32: 4096 sampled rows against all-pairs brute force, all rows
