@@ -656,8 +656,9 @@ def run_case(args):
     else:
         c = gen.config("cfg3", args.seed, m=args.size or 100)
         pos = to(c["pos"])
+        cnt = torch.empty(c["n"], dtype=torch.int32, device=dev) if args.with_count else None
         def run():
-            T.tiga_apply_radius(pos, None, c["r"], c["box"], c["periodic"], T.MSG_LJ, p0=1.0, p1=1.0)
+            T.tiga_apply_radius(pos, None, c["r"], c["box"], c["periodic"], T.MSG_LJ, p0=1.0, p1=1.0, count=cnt)
         units = c["n"]
     for _ in range(max(args.warmup, 1)):
         run()
@@ -681,6 +682,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--case", default=None, choices=["csr", "csr_large", "radius_gauss", "radius_lj", "knn", "attention", "paper_shapes"],
                     help="run one traversal on a reduced replica (for profiler captures) instead of the benchmark")
+    ap.add_argument("--with-count", action="store_true", help="--case radius_lj: also ask for the neighbour counts")
     ap.add_argument("--size", type=int, default=0, help="--case size: R-MAT scale, number of points, or lattice side")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

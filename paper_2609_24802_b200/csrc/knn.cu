@@ -38,6 +38,7 @@ constexpr int KNN_STAGE_BYTES = (KNN_STAGE_CAP + STAGE_PAD) * 16;
 constexpr int KNN_LIST_BYTES = (QB * KNN_QSTRIDE * 8 + 15) / 16 * 16;
 constexpr int KNN_MISC_BYTES = QB * 16 + QB * 4 * 2;
 constexpr int KNN_PER_WARP = KNN_STAGE_BYTES + KNN_LIST_BYTES + KNN_MISC_BYTES;
+static_assert(KNN_PER_WARP % 16 == 0 && KNN_LIST_BYTES % 16 == 0, "the stage and the queries are accessed as 16-byte vectors");
 constexpr int KNN_RING_BLOCKS = 148 * 4;
 constexpr double KNN_BALL_FACTOR = 2.0;            // expected points within the search radius, in units of k
 

@@ -190,6 +190,7 @@ template <int MODE> struct TravSmem {
     static constexpr int LIST_BYTES = (QB * QSTRIDE * 8 + 15) / 16 * 16;
     static constexpr int MISC_BYTES = QB * 16 + QB * 4 * 2;          // query coordinates, counts, totals
     static constexpr int PER_WARP = STAGE_BYTES + LIST_BYTES + MISC_BYTES;
+    static_assert(PER_WARP % 16 == 0 && LIST_BYTES % 16 == 0, "the stage and the queries are accessed as 16-byte vectors");
 };
 
 // MODE 0: Gaussian (DIST = false) or distance-weighted (DIST = true) forward;

@@ -28,12 +28,15 @@ constexpr int LJ_STAGE_CAP = 256;
 constexpr int LJ_QCAP = 64;
 constexpr int LJ_QSTRIDE = LJ_QCAP + 1;
 constexpr int LJ_STAGE_BYTES = (LJ_STAGE_CAP + STAGE_PAD) * 16;
-constexpr int LJ_LIST_BYTES = (QB * LJ_QSTRIDE * 8 + 15) / 16 * 16;
-constexpr int LJ_MISC_BYTES = QB * 16 + QB * 4 + LJ_STAGE_CAP * 4;      // queries, list lengths, per-candidate counts
-constexpr int LJ_PER_WARP = LJ_STAGE_BYTES + LJ_LIST_BYTES + LJ_MISC_BYTES;
+constexpr int LJQ = 4;                        // queries per batch in this kernel
+constexpr int LJ_LPQ = 32 / LJQ;              // lanes that share a query's list in phase B
+constexpr int LJ_LIST_BYTES = (LJQ * LJ_QSTRIDE * 8 + 15) / 16 * 16;
+constexpr int LJ_MISC_BYTES = LJQ * 16 + LJQ * 4;                         // queries, list lengths
+constexpr int LJ_PER_WARP = (LJ_STAGE_BYTES + LJ_LIST_BYTES + LJ_MISC_BYTES + 15) / 16 * 16;
+static_assert(LJ_STAGE_BYTES % 16 == 0 && LJ_LIST_BYTES % 16 == 0 && LJ_PER_WARP % 16 == 0, "the stage and the queries are accessed as 16-byte vectors");
 
 template <bool MI, bool COUNT>
-__global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const __grid_constant__ RadiusParams p) {
+__global__ void __launch_bounds__(TRAV_THREADS, 6) radius_lj_pairs_kernel(const __grid_constant__ RadiusParams p) {
     constexpr unsigned FULL = 0xffffffffu;
     extern __shared__ __align__(16) unsigned char s_raw[];
 
@@ -45,8 +48,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const 
     float4* stage = reinterpret_cast<float4*>(base);                                   // local x, y, z, point id
     float2* list = reinterpret_cast<float2*>(base + LJ_STAGE_BYTES);                   // (stage slot, d2) per query
     float4* s_q = reinterpret_cast<float4*>(base + LJ_STAGE_BYTES + LJ_LIST_BYTES);
-    int* s_n = reinterpret_cast<int*>(s_q + QB);
-    int* s_cnt = s_n + QB;                  // accepted pairs per staged candidate (only when counts are wanted)
+    int* s_n = reinterpret_cast<int*>(s_q + LJQ);
 
     const int c[3] = {cellid % p.nc[0], (cellid / p.nc[0]) % p.nc[1], cellid / (p.nc[0] * p.nc[1])};
     const float org[3] = {(float)c[0] * p.hcell[0], (float)c[1] * p.hcell[1], (float)c[2] * p.hcell[2]};
@@ -152,62 +154,64 @@ __global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const 
     //      cell's own points, in the same order as the queries
     auto process_chunk = [&](const int ns, const int nself) {
         if (lane < STAGE_PAD) stage[ns + lane] = make_float4(FAR_AWAY, FAR_AWAY, FAR_AWAY, __int_as_float(-1));
-        if (COUNT)
-            for (int k = lane; k < ns; k += 32) s_cnt[k] = 0;
-        for (int qb0 = qs0; qb0 < qe0; qb0 += QB) {
-            const int nq = (qe0 - qb0 < QB) ? qe0 - qb0 : QB;
+        for (int qb0 = qs0; qb0 < qe0; qb0 += LJQ) {
+            const int nq = (qe0 - qb0 < LJQ) ? qe0 - qb0 : LJQ;
             __syncwarp();
             if (lane < nq) {
                 const float4 pq = p.spos[qb0 + lane];
                 s_q[lane] = make_float4(pq.x - org[0], pq.y - org[1], pq.z - org[2], pq.w);
             }
             __syncwarp();
-            int qcnt[QB];
+            int qcnt[LJQ];
 #pragma unroll
-            for (int q = 0; q < QB; ++q) qcnt[q] = 0;
+            for (int q = 0; q < LJQ; ++q) qcnt[q] = 0;
 
             auto drain = [&]() {
                 __syncwarp();
                 if (lane == 0) {
 #pragma unroll
-                    for (int q = 0; q < QB; ++q) s_n[q] = qcnt[q];
+                    for (int q = 0; q < LJQ; ++q) s_n[q] = qcnt[q];
                 }
                 __syncwarp();
-                const int q = lane >> 2, sub = lane & 3;
+                const int q = lane / LJ_LPQ, sub = lane % LJ_LPQ;
                 float fx = 0.f, fy = 0.f, fz = 0.f, en = 0.f;
                 int n = 0;
                 if (q < nq) {
                     const float4 qv = s_q[q];
                     n = s_n[q];
                     const float2* lq = list + q * LJ_QSTRIDE;
-                    for (int t = sub; t < n; t += 8) {
+                    for (int t = sub; t < n; t += 2 * LJ_LPQ) {
                         float2 e[2];
                         float4 pj[2];
 #pragma unroll
                         for (int u = 0; u < 2; ++u) {
-                            e[u] = lq[t + 4 * u < n ? t + 4 * u : t];
+                            e[u] = lq[t + LJ_LPQ * u < n ? t + LJ_LPQ * u : t];
                             pj[u] = stage[__float_as_int(e[u].x)];
                         }
 #pragma unroll
                         for (int u = 0; u < 2; ++u) {
-                            if (t + 4 * u < n) {
-                                const float inv = fast_rcp(e[u].y);
-                                const float qq = s2 * inv;
-                                const float q3 = qq * qq * qq;
-                                const float fs = e24 * (2.f * q3 * q3 - q3) * inv;
-                                const float ee = e2x * (q3 * q3 - q3);
-                                float dx = qv.x - pj[u].x, dy = qv.y - pj[u].y, dz = qv.z - pj[u].z;
-                                fold(dx, dy, dz);
-                                const float gx = fs * dx, gy = fs * dy, gz = fs * dz;
-                                fx += gx; fy += gy; fz += gz; en += ee;
-                                const int idj = __float_as_int(pj[u].w);
+                            // the arithmetic runs for both slots of the step; an absent pair has inv = 0
+                            // (zero force and energy) and only its atomics are switched off
+                            const bool valid = t + LJ_LPQ * u < n;
+                            const float inv = valid ? fast_rcp(e[u].y) : 0.f;
+                            const float qq = s2 * inv;
+                            const float q3 = qq * qq * qq;
+                            const float fs = e24 * (2.f * q3 * q3 - q3) * inv;
+                            const float ee = e2x * (q3 * q3 - q3);
+                            float dx = qv.x - pj[u].x, dy = qv.y - pj[u].y, dz = qv.z - pj[u].z;
+                            fold(dx, dy, dz);
+                            const float gx = fs * dx, gy = fs * dy, gz = fs * dz;
+                            fx += gx; fy += gy; fz += gz; en += ee;
+                            const int idj = __float_as_int(pj[u].w);
+                            if (valid) {
                                 atomicAdd(out4 + idj, make_float4(-gx, -gy, -gz, ee));      // the pair's other row
+                                if (COUNT) atomicAdd(p.count + idj, 1);
                             }
                         }
                     }
                 }
 #pragma unroll
-                for (int o = 1; o <= 2; o <<= 1) {
+                for (int o = 1; o < LJ_LPQ; o <<= 1) {
                     fx += __shfl_xor_sync(FULL, fx, o); fy += __shfl_xor_sync(FULL, fy, o);
                     fz += __shfl_xor_sync(FULL, fz, o); en += __shfl_xor_sync(FULL, en, o);
                 }
@@ -217,7 +221,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const 
                     if (COUNT) atomicAdd(p.count + idq, n);
                 }
 #pragma unroll
-                for (int q2 = 0; q2 < QB; ++q2) qcnt[q2] = 0;
+                for (int q2 = 0; q2 < LJQ; ++q2) qcnt[q2] = 0;
                 __syncwarp();
             };
 
@@ -229,10 +233,10 @@ __global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const 
                 const float4 pj = stage[cbase + lane];
                 const int idj = __float_as_int(pj.w);
                 const bool own = OWN && cbase + lane < nself;
-                float d2q[QB];
+                float d2q[LJQ];
                 float nearest = FAR_AWAY;       // smallest |d2 - r^2| seen by this lane
 #pragma unroll
-                for (int q = 0; q < QB; ++q) {
+                for (int q = 0; q < LJQ; ++q) {
                     if (!FULLB && q >= nq) break;
                     const float4 qv = s_q[q];
                     float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
@@ -246,25 +250,23 @@ __global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const 
                 if (__any_sync(FULL, nearest <= p.r2_band)) {
                     // some pair lies within the fp32 error band of the cutoff: decide it in fp64
 #pragma unroll
-                    for (int q = 0; q < QB; ++q) {
+                    for (int q = 0; q < LJQ; ++q) {
                         if (!FULLB && q >= nq) break;
                         if (fabsf(d2q[q] - p.r2_mid) <= p.r2_band)
                             d2q[q] = exact_pair(p, __float_as_int(s_q[q].w), idj) ? fminf(d2q[q], p.r2_lo) : FAR_AWAY;
                     }
                 }
-                int mx = 0, mine = 0;           // mine: queries that accepted this lane's candidate
+                int mx = 0;
 #pragma unroll
-                for (int q = 0; q < QB; ++q) {
+                for (int q = 0; q < LJQ; ++q) {
                     if (!FULLB && q >= nq) break;
                     const bool ok = d2q[q] <= p.r2_lo;
                     const unsigned m = __ballot_sync(FULL, ok);
                     float2* dst = list + q * LJ_QSTRIDE + qcnt[q] + __popc(m & lt_mask);
                     if (ok) *dst = make_float2(__int_as_float(cbase + lane), d2q[q]);
-                    if (COUNT) mine += ok ? 1 : 0;
                     qcnt[q] += __popc(m);
                     mx = qcnt[q] > mx ? qcnt[q] : mx;
                 }
-                if (COUNT && mine) s_cnt[cbase + lane] += mine;      // the slot belongs to this lane alone
                 return mx > LJ_QCAP - 32;
             };
 
@@ -274,17 +276,12 @@ __global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const 
                 if (done || need) drain();
                 if (done) break;
                 if (cbase < nself)
-                    need = (nq == QB) ? phase_a(cbase, std::true_type{}, std::true_type{}) : phase_a(cbase, std::false_type{}, std::true_type{});
+                    need = (nq == LJQ) ? phase_a(cbase, std::true_type{}, std::true_type{}) : phase_a(cbase, std::false_type{}, std::true_type{});
                 else
-                    need = (nq == QB) ? phase_a(cbase, std::true_type{}, std::false_type{}) : phase_a(cbase, std::false_type{}, std::false_type{});
+                    need = (nq == LJQ) ? phase_a(cbase, std::true_type{}, std::false_type{}) : phase_a(cbase, std::false_type{}, std::false_type{});
             }
         }
         __syncwarp();
-        if (COUNT)                            // the candidates' side of the neighbour counts, one atomic per candidate
-            for (int k = lane; k < ns; k += 32) {
-                const int cnum = s_cnt[k];
-                if (cnum) atomicAdd(p.count + __float_as_int(stage[k].w), cnum);
-            }
         __syncwarp();
     };
 

@@ -37,6 +37,7 @@ template <int HID, bool BWD> struct MlpSmem {
     static constexpr int PAIR_STRIDE = 2 * HID + MLP_DIN + 4 + 1;                // hbar, u, a, ybar (+1: odd stride)
     static constexpr int PAIR_BYTES = BWD ? (32 * PAIR_STRIDE * 4 + 15) / 16 * 16 : 0;
     static constexpr int PER_WARP = STAGE_BYTES + LIST_BYTES + MISC_BYTES + PAIR_BYTES;
+    static_assert(PER_WARP % 16 == 0, "the stage and the queries are accessed as 16-byte vectors");
     static constexpr int TOTAL = CTA_BYTES + TRAV_WARPS * PER_WARP;
 };
 
