@@ -181,14 +181,17 @@ __global__ void bin_sort_kernel(const RadiusParams p) {
 // the warp drains / processes and goes on, so any density works.
 
 template <int MODE> struct TravSmem {
+    // queries per batch: the forward runs fastest with short batches and seven CTAs per SM, the
+    // backward (more registers per pair) with long batches
+    static constexpr int TQB = MODE == 0 ? 4 : QB;
     // sized for the workload's density (about 216 candidates before pruning, 32 neighbours);
     // denser inputs only mean more chunks and drains
     static constexpr int STAGE_CAP = 256;                          // candidates staged per chunk
     static constexpr int QCAP = 80;                                // list entries per query
     static constexpr int QSTRIDE = QCAP + 1;                       // odd stride: the lists of different queries fall in different banks
     static constexpr int STAGE_BYTES = (STAGE_CAP + STAGE_PAD) * 16;
-    static constexpr int LIST_BYTES = (QB * QSTRIDE * 8 + 15) / 16 * 16;
-    static constexpr int MISC_BYTES = QB * 16 + QB * 4 * 2;          // query coordinates, counts, totals
+    static constexpr int LIST_BYTES = (TQB * QSTRIDE * 8 + 15) / 16 * 16;
+    static constexpr int MISC_BYTES = TQB * 16 + TQB * 4 * 2;          // query coordinates, counts, totals
     static constexpr int PER_WARP = STAGE_BYTES + LIST_BYTES + MISC_BYTES;
     static_assert(PER_WARP % 16 == 0 && LIST_BYTES % 16 == 0, "the stage and the queries are accessed as 16-byte vectors");
 };
@@ -197,9 +200,9 @@ template <int MODE> struct TravSmem {
 // 2: Gaussian backward.  MI: some periodic dimension has a single cell (explicit minimum image).
 // VEC: feature rows are 16-byte aligned (F % 4 == 0); otherwise the forward uses scalar accesses.
 template <int MODE, int LF, bool DIST, bool MI, bool VEC = true>
-__global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_traverse_kernel(const __grid_constant__ RadiusParams p) {
+__global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_traverse_kernel(const __grid_constant__ RadiusParams p) {
     using SM = TravSmem<MODE>;
-    constexpr int STAGE_CAP = SM::STAGE_CAP, QCAP = SM::QCAP, QSTRIDE = SM::QSTRIDE;
+    constexpr int STAGE_CAP = SM::STAGE_CAP, QCAP = SM::QCAP, QSTRIDE = SM::QSTRIDE, TQB = SM::TQB;
     constexpr unsigned FULL = 0xffffffffu;
     extern __shared__ __align__(16) unsigned char s_raw[];
 
@@ -214,8 +217,8 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_trav
     float4* stage = reinterpret_cast<float4*>(base);
     float2* list = reinterpret_cast<float2*>(base + SM::STAGE_BYTES);
     float4* s_q = reinterpret_cast<float4*>(base + SM::STAGE_BYTES + SM::LIST_BYTES);   // local x, y, z, point id
-    int* s_n = reinterpret_cast<int*>(s_q + QB);                                        // list lengths of the drain in progress
-    int* s_tot = s_n + QB;                                                              // neighbours found so far in this chunk
+    int* s_n = reinterpret_cast<int*>(s_q + TQB);                                        // list lengths of the drain in progress
+    int* s_tot = s_n + TQB;                                                              // neighbours found so far in this chunk
 
     const int c[3] = {cellid % p.nc[0], (cellid / p.nc[0]) % p.nc[1], cellid / (p.nc[0] * p.nc[1])};
     const float org[3] = {(float)c[0] * p.hcell[0], (float)c[1] * p.hcell[1], (float)c[2] * p.hcell[2]};
@@ -238,8 +241,8 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_trav
     // ---- all queries of the cell against the ns candidates currently staged
     auto process_chunk = [&](const int ns, const bool first_chunk) {
         if (lane < STAGE_PAD) stage[ns + lane] = make_float4(FAR_AWAY, FAR_AWAY, FAR_AWAY, __int_as_float(-1));
-        for (int qb0 = qs0; qb0 < qe0; qb0 += QB) {
-            const int nq = (qe0 - qb0 < QB) ? qe0 - qb0 : QB;
+        for (int qb0 = qs0; qb0 < qe0; qb0 += TQB) {
+            const int nq = (qe0 - qb0 < TQB) ? qe0 - qb0 : TQB;
             __syncwarp();
             if (lane < nq) {
                 const float4 pq = p.spos[qb0 + lane];
@@ -247,16 +250,16 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_trav
                 s_tot[lane] = 0;
             }
             __syncwarp();
-            int qcnt[QB];                         // list lengths (warp uniform, kept in registers)
+            int qcnt[TQB];                         // list lengths (warp uniform, kept in registers)
 #pragma unroll
-            for (int q = 0; q < QB; ++q) qcnt[q] = 0;
+            for (int q = 0; q < TQB; ++q) qcnt[q] = 0;
             bool first = first_chunk;
 
             auto drain = [&]() {
                 __syncwarp();
                 if (lane == 0) {
 #pragma unroll
-                    for (int q = 0; q < QB; ++q) { s_n[q] = qcnt[q]; s_tot[q] += qcnt[q]; }
+                    for (int q = 0; q < TQB; ++q) { s_n[q] = qcnt[q]; s_tot[q] += qcnt[q]; }
                 }
                 __syncwarp();
                 {
@@ -351,20 +354,20 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_trav
                     }
                 }
 #pragma unroll
-                for (int q = 0; q < QB; ++q) qcnt[q] = 0;
+                for (int q = 0; q < TQB; ++q) qcnt[q] = 0;
                 first = false;
                 __syncwarp();
             };
 
             // ---- phase A: one staged candidate per lane against the queries of the batch
             auto phase_a = [&](const int cbase, auto full_batch) -> bool {
-                constexpr bool FULLB = decltype(full_batch)::value;     // all QB queries present: no trip tests
+                constexpr bool FULLB = decltype(full_batch)::value;     // all TQB queries present: no trip tests
                 const float4 pj = stage[cbase + lane];
                 const int idj = __float_as_int(pj.w);
-                float d2q[QB];
+                float d2q[TQB];
                 float nearest = FAR_AWAY;       // smallest |d2 - r^2| seen by this lane
 #pragma unroll
-                for (int q = 0; q < QB; ++q) {
+                for (int q = 0; q < TQB; ++q) {
                     if (!FULLB && q >= nq) break;
                     const float4 qv = s_q[q];
                     float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
@@ -378,7 +381,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_trav
                     // some pair lies within the fp32 error band of the cutoff: decide it in fp64 and
                     // move it clear of the band (the change of d2 is below the fp32 error itself)
 #pragma unroll
-                    for (int q = 0; q < QB; ++q) {
+                    for (int q = 0; q < TQB; ++q) {
                         if (!FULLB && q >= nq) break;
                         if (fabsf(d2q[q] - p.r2_mid) <= p.r2_band)
                             d2q[q] = exact_pair(p, __float_as_int(s_q[q].w), idj) ? fminf(d2q[q], p.r2_lo) : FAR_AWAY;
@@ -386,7 +389,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_trav
                 }
                 int mx = 0;
 #pragma unroll
-                for (int q = 0; q < QB; ++q) {
+                for (int q = 0; q < TQB; ++q) {
                     if (!FULLB && q >= nq) break;
                     const bool ok = d2q[q] <= p.r2_lo;
                     const unsigned m = __ballot_sync(FULL, ok);
@@ -406,7 +409,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 5 : 0)) radius_trav
                 const bool done = cbase >= ns;
                 if (done || need) drain();
                 if (done) break;
-                need = (nq == QB) ? phase_a(cbase, std::true_type{}) : phase_a(cbase, std::false_type{});
+                need = (nq == TQB) ? phase_a(cbase, std::true_type{}) : phase_a(cbase, std::false_type{});
             }
             if (p.count && lane < nq) {
                 const int oq = __float_as_int(s_q[lane].w);
