@@ -30,13 +30,14 @@
 
 namespace tiga {
 
+constexpr int KQB = 4;                             // queries per batch (cells kernel)
 constexpr int KNN_STAGE_CAP = 256;                 // staged candidates per chunk
 constexpr int KNN_QCAP = 96;                       // list entries per query (cells kernel)
 constexpr int KNN_QSTRIDE = KNN_QCAP + 1;
 constexpr int KNN_RING_CAP = 128;                  // list entries of the rings kernel
 constexpr int KNN_STAGE_BYTES = (KNN_STAGE_CAP + STAGE_PAD) * 16;
-constexpr int KNN_LIST_BYTES = (QB * KNN_QSTRIDE * 8 + 15) / 16 * 16;
-constexpr int KNN_MISC_BYTES = QB * 16 + QB * 4 * 2;
+constexpr int KNN_LIST_BYTES = (KQB * KNN_QSTRIDE * 8 + 15) / 16 * 16;
+constexpr int KNN_MISC_BYTES = KQB * 16 + KQB * 4 * 2;
 constexpr int KNN_PER_WARP = KNN_STAGE_BYTES + KNN_LIST_BYTES + KNN_MISC_BYTES;
 static_assert(KNN_PER_WARP % 16 == 0 && KNN_LIST_BYTES % 16 == 0, "the stage and the queries are accessed as 16-byte vectors");
 constexpr int KNN_RING_BLOCKS = 148 * 4;
@@ -156,8 +157,8 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
     float4* stage = reinterpret_cast<float4*>(base);                                      // x, y, z, point id
     float2* list = reinterpret_cast<float2*>(base + KNN_STAGE_BYTES);                     // (point id, d2) per query
     float4* s_q = reinterpret_cast<float4*>(base + KNN_STAGE_BYTES + KNN_LIST_BYTES);
-    int* s_n = reinterpret_cast<int*>(s_q + QB);
-    float* s_tau = reinterpret_cast<float*>(s_n + QB);
+    int* s_n = reinterpret_cast<int*>(s_q + KQB);
+    float* s_tau = reinterpret_cast<float*>(s_n + KQB);
     const unsigned lt_mask = (1u << lane) - 1u;
     const int k = P.k;
 
@@ -239,10 +240,10 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
     int ns = 0;
     const bool single = stage_from(0, ns) >= total;           // the whole (pruned) stencil fits: staged once
 
-    for (int qb0 = qs0; qb0 < qe0; qb0 += QB) {
-        const int nq = (qe0 - qb0 < QB) ? qe0 - qb0 : QB;
+    for (int qb0 = qs0; qb0 < qe0; qb0 += KQB) {
+        const int nq = (qe0 - qb0 < KQB) ? qe0 - qb0 : KQB;
         __syncwarp();
-        if (lane < QB) {
+        if (lane < KQB) {
             // absent queries sit far away with a negative threshold: they accept nothing
             const float4 pq = lane < nq ? p.spos[qb0 + lane] : make_float4(FAR_AWAY, FAR_AWAY, FAR_AWAY, __int_as_float(-2));
             s_q[lane] = pq;
@@ -250,10 +251,10 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
             s_tau[lane] = lane < nq ? P.h2 : -1.f;
         }
         __syncwarp();
-        int qcnt[QB];
-        float tq[QB];
+        int qcnt[KQB];
+        float tq[KQB];
 #pragma unroll
-        for (int q = 0; q < QB; ++q) { qcnt[q] = 0; tq[q] = s_tau[q]; }
+        for (int q = 0; q < KQB; ++q) { qcnt[q] = 0; tq[q] = s_tau[q]; }
 
         // all queries of the batch against the ns staged candidates
         auto scan = [&](const int ns_, auto width) {
@@ -277,7 +278,7 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
                     __syncwarp();
                     if (lane == 0) {
 #pragma unroll
-                        for (int q = 0; q < QB; ++q) s_n[q] = qcnt[q];
+                        for (int q = 0; q < KQB; ++q) s_n[q] = qcnt[q];
                     }
                     __syncwarp();
                     for (int q = 0; q < nq; ++q) {
@@ -292,19 +293,19 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
                     }
                     __syncwarp();
 #pragma unroll
-                    for (int q = 0; q < QB; ++q) { qcnt[q] = s_n[q]; tq[q] = s_tau[q]; }
+                    for (int q = 0; q < KQB; ++q) { qcnt[q] = s_n[q]; tq[q] = s_tau[q]; }
                 }
             }
         };
 
         if (single) {
-            if (nq <= QB / 2) scan(ns, std::integral_constant<int, QB / 2>{});
-            else scan(ns, std::integral_constant<int, QB>{});
+            if (nq <= KQB / 2) scan(ns, std::integral_constant<int, KQB / 2>{});
+            else scan(ns, std::integral_constant<int, KQB>{});
         } else {
             for (int v = 0; v < total;) {
                 int ns2;
                 v = stage_from(v, ns2);
-                scan(ns2, std::integral_constant<int, QB>{});
+                scan(ns2, std::integral_constant<int, KQB>{});
                 __syncwarp();
             }
         }
@@ -313,7 +314,7 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
         __syncwarp();
         if (lane == 0) {
 #pragma unroll
-            for (int q = 0; q < QB; ++q) s_n[q] = qcnt[q];
+            for (int q = 0; q < KQB; ++q) s_n[q] = qcnt[q];
         }
         __syncwarp();
         for (int q = 0; q < nq; ++q) {
