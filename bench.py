@@ -374,6 +374,49 @@ def run_ours(args, rank, world, local_rank):
     fwd_bwd = {"csr_sum": E / ((per_row_ms[0] + per_row_ms[1]) * 1e-3), "csr_max": E / ((per_row_ms[2] + per_row_ms[3]) * 1e-3),
                "radius_gauss": counts["rad_pairs"] / ((per_row_ms[5] + per_row_ms[6]) * 1e-3)}
 
+    # ---- the stored-relation forward in detail: three bandwidth fractions, the L2 gather ceiling,
+    #      warm and flushed L2 (outside the timed step; rank 0 only)
+    def timed(fn, reps=10, before=None):
+        ts = []
+        for _ in range(reps):
+            if before is not None:
+                before()
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record(stream); fn(); b.record(stream); torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return statistics.median(ts)
+
+    gen_t = torch.Generator(device=dev); gen_t.manual_seed(args.seed)
+    table = torch.randn((60 * 2**20 // (4 * F), F), device=dev, generator=gen_t)              # 60 MiB of 256-byte rows: fits L2
+    ridx = torch.randint(0, table.shape[0], (E,), device=dev, generator=gen_t, dtype=torch.int32)
+    sink = torch.zeros(1, device=dev)
+    for _ in range(3):
+        T.tiga_probe_row_gather(table, ridx, sink)
+    t_l2 = timed(lambda: T.tiga_probe_row_gather(table, ridx, sink))
+    t_col = timed(lambda: T.tiga_probe_row_gather(d["x"], d["col"], sink))                 # the workload's own index stream and table
+    l2_peak = E * 4.0 * F / (t_l2 * 1e-3)
+    flush_buf = torch.empty(512 * 2**20, dtype=torch.uint8, device=dev)
+    fwd_call = lambda: T.tiga_apply_csr(g, d["x"], d["w"], T.SUM, out=out_sum, ws=ws_csr)
+    t_warm = timed(fwd_call)
+    t_cold = timed(fwd_call, before=lambda: flush_buf.zero_())
+    touched = int(torch.unique(d["col"]).numel())
+    t_fwd = per_row_ms[0]
+    b_min = 4.0 * (N + 1) + 8.0 * E + 4.0 * F * touched + 4.0 * F * N
+    b_dram = TRAFFIC_PER_UNIT["csr_sum_fwd"][1] * E
+    csr_detail = {
+        "row": "csr_sum_fwd", "ms_in_step": round(t_fwd, 4), "ms_back_to_back_warm_l2": round(t_warm, 4),
+        "ms_l2_flushed_512MiB_write_between_calls": round(t_cold, 4),
+        "f_alg": row_report["csr_sum_fwd"]["frac"], "f_dram": b_dram / (t_fwd * 1e-3) / (hbm_gbs * 1e9),
+        "f_min": b_min / (t_fwd * 1e-3) / (hbm_gbs * 1e9),
+        "bytes_alg": models["csr_sum_fwd"]["work"], "bytes_dram_ncu_scaled": b_dram, "bytes_min": b_min, "touched_source_rows": touched,
+        "l2_gather_peak_GBps": l2_peak / 1e9,
+        "l2_gather_peak_note": "tiga_probe_row_gather: 16.8M uniform random 256-byte row gathers from a 60 MiB table",
+        "gather_of_own_index_stream_ms": round(t_col, 4),
+        "T_l2roof_over_T": (E * 4.0 * F / l2_peak) / (t_fwd * 1e-3),
+        "T_own_gather_over_T": t_col / t_fwd,
+    }
+    del table, ridx, flush_buf
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -391,7 +434,7 @@ def run_ours(args, rank, world, local_rank):
                      "peak_source": peak_kind + (" hbm copy" if dr["bound"] == "hbm" else
                                                                                      " 148 SM x 128 lanes x sampled SM clock")},
         "e2e": {"value": inter_all / (e2e_ms / args.steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": launches, "clocks": clocks,
+        "gpu_launches": launches, "clocks": clocks, "csr_detail": csr_detail,
     }
     if not args.no_cpu_baseline and world >= 1:
         line["cpu_baseline"] = cpu_baseline(w, seconds_hint=20)

@@ -251,6 +251,16 @@ tiga_status tiga_apply_radius_mlp_backward(const float* pos, const float* feat, 
                                            float* grad_W1, float* grad_b1, float* grad_W2, float* grad_b2,
                                            void* ws, size_t ws_bytes, int reuse_plan, void* stream);
 
+/* Measurement probe, no counterpart in the paper: gathers n_idx rows of row_bytes bytes
+ * (a multiple of 16, at most 512) from `table` by index with 128-bit loads, one row per group of
+ * row_bytes / 16 lanes, four rows in flight per lane, and folds them into `sink` (fp32 [1]) so
+ * that nothing is optimised away.  The benchmark times it on a table that fits L2 to obtain the
+ * L2 -> SM gather bandwidth that bounds the stored-relation forward when the gathered rows are
+ * cache resident.  table, idx (int32 [n_idx], every entry in [0, n_rows)) and sink are device
+ * pointers. */
+tiga_status tiga_probe_row_gather(const void* table, int64_t n_rows, int32_t row_bytes,
+                                  const int32_t* idx, int64_t n_idx, float* sink, void* stream);
+
 /* ----------------------------------------------------------------- stored relation, online-softmax reducer */
 
 /* Online-softmax reducer over the rows of a stored relation (Section 5, "Online softmax and

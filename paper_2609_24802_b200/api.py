@@ -19,7 +19,7 @@ __all__ = [
     "tiga_radius_grid", "tiga_radius_workspace_bytes", "tiga_radius_bin",
     "tiga_apply_radius", "tiga_apply_radius_backward", "tiga_apply_radius_mlp",
     "tiga_apply_radius_mlp_backward", "tiga_knn_workspace_bytes", "tiga_apply_knn",
-    "tiga_csr_attention_workspace_bytes", "tiga_apply_csr_attention", "launch_count",
+    "tiga_csr_attention_workspace_bytes", "tiga_apply_csr_attention", "tiga_probe_row_gather", "launch_count",
 ]
 
 SUM, MAX = 0, 1
@@ -33,6 +33,7 @@ EXPORTS = [
     "tiga_radius_workspace_bytes", "tiga_radius_bin", "tiga_apply_radius",
     "tiga_apply_radius_backward", "tiga_apply_radius_mlp", "tiga_apply_radius_mlp_backward",
     "tiga_knn_workspace_bytes", "tiga_apply_knn", "tiga_csr_attention_workspace_bytes", "tiga_apply_csr_attention",
+    "tiga_probe_row_gather",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -110,6 +111,8 @@ def load_library() -> ctypes.CDLL:
     lib.tiga_apply_radius_mlp_backward.restype = ctypes.c_int
     lib.tiga_apply_radius_mlp_backward.argtypes = [vp, vp, i64, f, ctypes.POINTER(_Box), ctypes.POINTER(_EdgeMlp), vp,
                                                    vp, vp, vp, vp, vp, vp, vp, sz, ctypes.c_int, vp]
+    lib.tiga_probe_row_gather.restype = ctypes.c_int
+    lib.tiga_probe_row_gather.argtypes = [vp, i64, i32, vp, i64, vp, vp]
     lib.tiga_csr_attention_workspace_bytes.restype = sz
     lib.tiga_csr_attention_workspace_bytes.argtypes = [ctypes.POINTER(_Csr), i32]
     lib.tiga_apply_csr_attention.restype = ctypes.c_int
@@ -445,3 +448,14 @@ def tiga_apply_csr_attention(g: CsrRelation, q, key, value, scale: float, out=No
                                                 _ptr(lse), _ptr(ws), ws.numel(), _stream(stream)), "tiga_apply_csr_attention")
     _launches += 2
     return out, lse, ws
+
+
+def tiga_probe_row_gather(table, idx, sink, stream=None) -> None:
+    """Measurement probe: gathers table[idx[k], :] for every k (rows of 16..512 bytes) and folds
+    them into sink[0]; timed by the benchmark to obtain the L2 -> SM gather ceiling."""
+    global _launches
+    n_rows = table.shape[0]
+    row_bytes = table.shape[1] * table.element_size()
+    _ok(load_library().tiga_probe_row_gather(_ptr(table), n_rows, row_bytes, _ptr(idx), idx.numel(), _ptr(sink),
+                                             _stream(stream)), "tiga_probe_row_gather")
+    _launches += 1

@@ -607,6 +607,28 @@ __global__ void degree_hist_kernel(const IT* __restrict__ rowptr, long long n, i
         if (s_hist[k]) atomicAdd(hist + k, (unsigned long long)s_hist[k]);
 }
 
+// Measurement probe: index-driven row gathers with the access shape of the forward (one row per
+// group of LN lanes, 128-bit loads, four rows in flight), folded into one number.
+template <int LN>
+__global__ void __launch_bounds__(256) row_gather_probe_kernel(const uint4* __restrict__ table, const int32_t* __restrict__ idx,
+                                                               long long n_idx, float* sink) {
+    const int ln = threadIdx.x % LN;
+    const long long groups = (long long)gridDim.x * (blockDim.x / LN);
+    const long long g0 = (long long)blockIdx.x * (blockDim.x / LN) + threadIdx.x / LN;
+    float acc = 0.f;
+    for (long long k = g0 * 4; k < n_idx; k += groups * 4) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long long kk = k + u < n_idx ? k + u : k;
+            v[u] = __ldg(table + (unsigned long long)(unsigned)__ldg(idx + kk) * LN + ln);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) acc += __uint_as_float(v[u].x) + __uint_as_float(v[u].y) + __uint_as_float(v[u].z) + __uint_as_float(v[u].w);
+    }
+    if (acc == 123.456f) atomicAdd(sink, acc);      // keeps the loads alive; practically never taken
+}
+
 template <typename IT>
 __global__ void validate_kernel(const IT* __restrict__ rowptr, const int32_t* __restrict__ col,
                                 long long n_dst, long long n_src, long long n_edges, int* flags) {
@@ -921,4 +943,25 @@ extern "C" const char* tiga_status_string(tiga_status s) {
         case TIGA_ERR_TOO_LARGE: return "problem exceeds the library's built-in scratch capacity";
     }
     return "unknown status";
+}
+
+extern "C" tiga_status tiga_probe_row_gather(const void* table, int64_t n_rows, int32_t row_bytes,
+                                             const int32_t* idx, int64_t n_idx, float* sink, void* stream) {
+    if (!table || !idx || !sink || n_rows <= 0 || n_idx < 0 || !aligned16(table)) return TIGA_ERR_INVALID_ARG;
+    if (row_bytes < 16 || row_bytes > 512 || (row_bytes & 15)) return TIGA_ERR_INVALID_ARG;
+    const int ln = row_bytes / 16;
+    if (ln & (ln - 1)) return TIGA_ERR_UNSUPPORTED;      // 16, 32, 64, 128, 256 or 512 bytes per row
+    if (n_idx == 0) return TIGA_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const unsigned blocks = 148 * 8;
+    const uint4* t = static_cast<const uint4*>(table);
+    switch (ln) {
+        case 1: row_gather_probe_kernel<1><<<blocks, 256, 0, s>>>(t, idx, n_idx, sink); break;
+        case 2: row_gather_probe_kernel<2><<<blocks, 256, 0, s>>>(t, idx, n_idx, sink); break;
+        case 4: row_gather_probe_kernel<4><<<blocks, 256, 0, s>>>(t, idx, n_idx, sink); break;
+        case 8: row_gather_probe_kernel<8><<<blocks, 256, 0, s>>>(t, idx, n_idx, sink); break;
+        case 16: row_gather_probe_kernel<16><<<blocks, 256, 0, s>>>(t, idx, n_idx, sink); break;
+        default: row_gather_probe_kernel<32><<<blocks, 256, 0, s>>>(t, idx, n_idx, sink); break;
+    }
+    return launch_status();
 }
