@@ -231,3 +231,18 @@ def test_cfg4_full_size(tiga):
     assert np.array_equal(host(hist), ref) and int(host(mx)[0]) == rmx
     y, A, _ = oracle.csr_forward(c["rowptr"], c["col"], c["x"], None, oracle.SUM)
     assert rel_err(out, y, A) <= SUM_TOL
+
+
+def test_row_gather_probe_runs_and_checks_its_arguments(tiga):
+    table = torch.randn((4096, 64), device="cuda")
+    idx = torch.randint(0, 4096, (100_000,), device="cuda", dtype=torch.int32)
+    sink = torch.zeros(1, device="cuda")
+    tiga.tiga_probe_row_gather(table, idx, sink)
+    torch.cuda.synchronize()
+    assert torch.isfinite(sink).all()
+    with pytest.raises(tiga.TigaError) as e:
+        tiga.tiga_probe_row_gather(torch.randn((16, 3), device="cuda"), idx[:4] % 16, sink)      # 12-byte rows
+    assert e.value.status == 1
+    with pytest.raises(tiga.TigaError) as e:
+        tiga.tiga_probe_row_gather(torch.randn((16, 12), device="cuda"), idx[:4] % 16, sink)     # 48-byte rows: not a power of two
+    assert e.value.status == 2
