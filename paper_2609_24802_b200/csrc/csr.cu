@@ -572,7 +572,8 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const Csr
 // Backward, max reducer: the cotangent of (i, f) goes through the selected edge only.
 // One thread per (i, f).  The features of a row often select the same edge (always, for a row with
 // one edge), so a warp first sums the edge-gradient contributions of lanes that share an edge
-// (the two most frequent leading edges of a warp, the rest go out one by one; more rounds measured slower): one atomic per edge instead of
+// (two rounds, each for the edge of the lowest lane not served yet; what is left goes out one by
+// one: more rounds measured slower): one atomic per edge instead of
 // up to 32 on the same address.
 __global__ void csr_backward_max_kernel(const CsrParams p) {
     constexpr unsigned FULL = 0xffffffffu;
