@@ -55,7 +55,9 @@ struct State {
     }
 };
 
-template <typename XT, int G, int VPL, int RED, typename IT>
+// EXACT: the feature row fills the worker exactly (nvec == G * VPL): row stride and lane activity
+// are compile-time constants, which removes address arithmetic and predicates from the edge loop.
+template <typename XT, int G, int VPL, int RED, typename IT, bool EXACT>
 __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrParams p) {
     constexpr int VW = XTraits<XT>::VW;
     constexpr int NW = CSR_THREADS / G;          // workers per CTA
@@ -76,23 +78,24 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
     const int wk = threadIdx.x / G;
     const int ln = threadIdx.x % G;
     const uint4* __restrict__ xlane = static_cast<const uint4*>(p.x) + ln;
-    const unsigned nvec = (unsigned)p.nvec;
+    const unsigned nvec = EXACT ? (unsigned)(G * VPL) : (unsigned)p.nvec;
+    const int F = EXACT ? G * VPL * VW : p.F;
     const long long e0 = t.e0;
 
     bool act[VPL];
 #pragma unroll
-    for (int i = 0; i < VPL; ++i) act[i] = (i * G + ln) < p.nvec;
+    for (int i = 0; i < VPL; ++i) act[i] = EXACT ? true : (i * G + ln) < p.nvec;
 
     auto store_row = [&](long long row, const State<RED, VPL, VW>& s) {
 #pragma unroll
         for (int i = 0; i < VPL; ++i) {
             if (!act[i]) continue;
-            float* o = p.out + row * p.F + (size_t)(i * G + ln) * VW;
+            float* o = p.out + row * F + (size_t)(i * G + ln) * VW;
 #pragma unroll
             for (int k = 0; k < VW; k += 4)
                 st_stream(reinterpret_cast<float4*>(o + k), make_float4(s.v[i][k], s.v[i][k + 1], s.v[i][k + 2], s.v[i][k + 3]));
             if constexpr (RED != 0) {
-                int* ao = p.arg + row * p.F + (size_t)(i * G + ln) * VW;
+                int* ao = p.arg + row * F + (size_t)(i * G + ln) * VW;
 #pragma unroll
                 for (int k = 0; k < VW; k += 4)
                     st_stream(reinterpret_cast<int4*>(ao + k), make_int4(s.a[i][k], s.a[i][k + 1], s.a[i][k + 2], s.a[i][k + 3]));
@@ -219,7 +222,7 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
 #pragma unroll
             for (int i = 0; i < VPL; ++i) {
                 if (!act[i]) continue;
-                const size_t o = (size_t)blockIdx.x * p.F + (size_t)(i * G + ln) * VW;
+                const size_t o = (size_t)blockIdx.x * F + (size_t)(i * G + ln) * VW;
 #pragma unroll
                 for (int k = 0; k < VW; ++k) {
                     p.carry_val[o + k] = st.v[i][k];
@@ -696,7 +699,7 @@ template <typename XT, int G, int VPL, int RED, typename IT>
 static tiga_status launch_fwd_t(const CsrParams& p, cudaStream_t s) {
     constexpr int NW = CSR_THREADS / G;
     const size_t dyn = (size_t)2 * NW * G * VPL * XTraits<XT>::VW * sizeof(float) * (RED ? 2 : 1);
-    auto kern = csr_forward_kernel<XT, G, VPL, RED, IT>;
+    auto kern = p.nvec == G * VPL ? csr_forward_kernel<XT, G, VPL, RED, IT, true> : csr_forward_kernel<XT, G, VPL, RED, IT, false>;
     if (dyn > 16 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
     kern<<<(unsigned)p.ntiles, CSR_THREADS, dyn, s>>>(p);
     return launch_status();
