@@ -65,8 +65,8 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
     constexpr int U = (VPL == 1) ? 4 : (VPL == 2 ? 2 : 1);   // gathers in flight per lane
 
     __shared__ int s_ptr[CSR_TILE + 2];
-    __shared__ int s_col[CSR_TILE + CSR_PAD];
-    __shared__ float s_w[CSR_TILE + CSR_PAD];
+    __shared__ __align__(16) int s_col[CSR_TILE + CSR_PAD];
+    __shared__ __align__(16) float s_w[CSR_TILE + CSR_PAD];
     __shared__ long long s_coord[2];
     __shared__ int s_tag[2 * NW];                // local row of head (even) / tail (odd) partial, -1 = none
     __shared__ unsigned char s_first[NW];        // tail partial starts its chain
@@ -133,7 +133,8 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
     if (ln == 0) { s_tag[2 * wk] = -1; s_tag[2 * wk + 1] = -1; s_first[wk] = 0; }
     if (threadIdx.x == 0) p.carry_row[blockIdx.x] = -1;
 
-    const int chunk = (t.ne + NW - 1) / NW;
+    // spans start on multiples of U, so a step's U indices and weights are one vector load each
+    const int chunk = ((t.ne + NW - 1) / NW + U - 1) / U * U;
     const int a = wk * chunk;
     const int b = (a + chunk < t.ne) ? a + chunk : t.ne;
 
@@ -148,11 +149,23 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
         for (int e = a; e < b; e += U) {
             uint4 xv[U][VPL];
             float wv[U];
+            int cv[U];
+            // entries past the span are readable (next worker's edges or the pad) and never used
+            if constexpr (U == 4) {
+                const int4 c4 = *reinterpret_cast<const int4*>(s_col + e);
+                const float4 w4 = *reinterpret_cast<const float4*>(s_w + e);
+                cv[0] = c4.x; cv[1] = c4.y; cv[2] = c4.z; cv[3] = c4.w;
+                wv[0] = w4.x; wv[1] = w4.y; wv[2] = w4.z; wv[3] = w4.w;
+            } else if constexpr (U == 2) {
+                const int2 c2 = *reinterpret_cast<const int2*>(s_col + e);
+                const float2 w2 = *reinterpret_cast<const float2*>(s_w + e);
+                cv[0] = c2.x; cv[1] = c2.y; wv[0] = w2.x; wv[1] = w2.y;
+            } else {
+                cv[0] = s_col[e]; wv[0] = s_w[e];
+            }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                // entries past the span are readable (next worker's edges or the pad) and never used
-                const unsigned c = (unsigned)s_col[e + u];
-                wv[u] = s_w[e + u];
+                const unsigned c = (unsigned)cv[u];
                 const uint4* src = xlane + (unsigned long long)c * nvec;      // one 32 x 32 -> 64 multiply
 #pragma unroll
                 for (int i = 0; i < VPL; ++i)
