@@ -46,15 +46,16 @@ struct AttState {
     }
 };
 
-template <int G, typename IT>
+// EXACT: the row fills the worker exactly (D == 4 G): constant row stride, no lane predicates.
+template <int G, typename IT, bool EXACT>
 __global__ void __launch_bounds__(CSR_THREADS) csr_attention_kernel(const CsrParams p) {
     constexpr int NW = CSR_THREADS / G;          // workers per CTA
     constexpr int LV = G * 4;                    // floats of one partial accumulator
     constexpr int U = 4;                         // edges per step
 
     __shared__ int s_ptr[CSR_TILE + 2];
-    __shared__ int s_col[CSR_TILE + CSR_PAD];
-    __shared__ float s_w[CSR_TILE + CSR_PAD];
+    __shared__ __align__(16) int s_col[CSR_TILE + CSR_PAD];
+    __shared__ __align__(16) float s_w[CSR_TILE + CSR_PAD];
     __shared__ long long s_coord[2];
     __shared__ int s_tag[2 * NW];                // local row of head (even) / tail (odd) partial, -1 = none
     __shared__ unsigned char s_first[NW];        // tail partial starts its chain
@@ -66,8 +67,9 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_attention_kernel(const CsrPar
     const int wk = threadIdx.x / G;
     const int ln = threadIdx.x % G;
     const unsigned wmask = G == 32 ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
-    const unsigned nvec = (unsigned)p.nvec;
-    const bool act = ln < p.nvec;
+    const unsigned nvec = EXACT ? (unsigned)G : (unsigned)p.nvec;
+    const int F = EXACT ? 4 * G : p.F;
+    const bool act = EXACT ? true : ln < p.nvec;
     const float4* __restrict__ qlane = reinterpret_cast<const float4*>(p.q) + ln;
     const float4* __restrict__ klane = reinterpret_cast<const float4*>(p.key) + ln;
     const float4* __restrict__ vlane = reinterpret_cast<const float4*>(p.x) + ln;
@@ -82,7 +84,7 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_attention_kernel(const CsrPar
     };
     auto store_row = [&](long long row, const AttState& s) {
         const float inv = s.l > 0.f ? 1.f / s.l : 0.f;
-        if (act) st_stream(reinterpret_cast<float4*>(p.out + row * p.F) + ln, make_float4(s.o[0] * inv, s.o[1] * inv, s.o[2] * inv, s.o[3] * inv));
+        if (act) st_stream(reinterpret_cast<float4*>(p.out + row * F) + ln, make_float4(s.o[0] * inv, s.o[1] * inv, s.o[2] * inv, s.o[3] * inv));
         if (ln == 0) {
             const float lse = s.l > 0.f ? (s.m + log2f(s.l)) * ATT_LN2 : ATT_NEG_INF;
             p.gw[row] = lse;                     // workspace copy, read by the fix-up
@@ -111,7 +113,8 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_attention_kernel(const CsrPar
     if (ln == 0) { s_tag[2 * wk] = -1; s_tag[2 * wk + 1] = -1; s_first[wk] = 0; }
     if (threadIdx.x == 0) p.carry_row[blockIdx.x] = -1;
 
-    const int chunk = (t.ne + NW - 1) / NW;
+    // spans start on multiples of U, so a step's U indices are one vector load
+    const int chunk = ((t.ne + NW - 1) / NW + U - 1) / U * U;
     const int a = wk * chunk;
     const int b = (a + chunk < t.ne) ? a + chunk : t.ne;
 
@@ -126,10 +129,12 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_attention_kernel(const CsrPar
         float4 qv = load_q(r);
         for (int e = a; e < b; e += U) {
             float4 kv[U], vv[U];
+            // entries past the span are readable (next worker's edges or the pad) and never used
+            const int4 c4 = *reinterpret_cast<const int4*>(s_col + e);
+            const int cv[U] = {c4.x, c4.y, c4.z, c4.w};
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                // entries past the span are readable (next worker's edges or the pad) and never used
-                const unsigned long long off = (unsigned long long)(unsigned)s_col[e + u] * nvec;
+                const unsigned long long off = (unsigned long long)(unsigned)cv[u] * nvec;
                 kv[u] = act ? __ldg(klane + off) : zero4;
                 vv[u] = act ? __ldg(vlane + off) : zero4;
             }
@@ -209,7 +214,7 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_attention_kernel(const CsrPar
                 p.carry_row[blockIdx.x] = (int32_t)(t.i0 + r);
                 p.carry_ml[blockIdx.x] = make_float2(st.m, st.l);
             }
-            if (act) *(reinterpret_cast<float4*>(p.carry_val + (size_t)blockIdx.x * p.F) + ln) = make_float4(st.o[0], st.o[1], st.o[2], st.o[3]);
+            if (act) *(reinterpret_cast<float4*>(p.carry_val + (size_t)blockIdx.x * F) + ln) = make_float4(st.o[0], st.o[1], st.o[2], st.o[3]);
         }
     }
 }
@@ -245,7 +250,8 @@ __global__ void csr_attention_fixup_kernel(const CsrParams p) {
 template <int G, typename IT>
 static tiga_status launch_attention_t(const CsrParams& p, cudaStream_t s) {
     constexpr int smem = 2 * (CSR_THREADS / G) * G * 4 * (int)sizeof(float);
-    csr_attention_kernel<G, IT><<<(unsigned)p.ntiles, CSR_THREADS, smem, s>>>(p);
+    if (p.nvec == G) csr_attention_kernel<G, IT, true><<<(unsigned)p.ntiles, CSR_THREADS, smem, s>>>(p);
+    else csr_attention_kernel<G, IT, false><<<(unsigned)p.ntiles, CSR_THREADS, smem, s>>>(p);
     const long long work = p.ntiles * p.F;
     csr_attention_fixup_kernel<<<(unsigned)((work + 255) / 256), 256, 0, s>>>(p);
     return launch_status();
