@@ -198,8 +198,9 @@ template <int MODE> struct TravSmem {
 
 // MODE 0: Gaussian (DIST = false) or distance-weighted (DIST = true) forward;
 // 2: Gaussian backward.  MI: some periodic dimension has a single cell (explicit minimum image).
-// VEC: feature rows are 16-byte aligned (F % 4 == 0); otherwise the forward uses scalar accesses.
-template <int MODE, int LF, bool DIST, bool MI, bool VEC = true>
+// VEC: 0 = scalar feature accesses (F % 4 != 0, forward only); 1 = 128-bit accesses, F % 4 == 0;
+// 2 = additionally F == 4 LF exactly, so the row stride is a compile-time constant.
+template <int MODE, int LF, bool DIST, bool MI, int VEC = 1>
 __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_traverse_kernel(const __grid_constant__ RadiusParams p) {
     using SM = TravSmem<MODE>;
     constexpr int STAGE_CAP = SM::STAGE_CAP, QCAP = SM::QCAP, QSTRIDE = SM::QSTRIDE, TQB = SM::TQB;
@@ -222,12 +223,12 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
 
     const int c[3] = {cellid % p.nc[0], (cellid / p.nc[0]) % p.nc[1], cellid / (p.nc[0] * p.nc[1])};
     const float org[3] = {(float)c[0] * p.hcell[0], (float)c[1] * p.hcell[1], (float)c[2] * p.hcell[2]};
-    const int F = p.F;
+    const int F = VEC == 2 ? 4 * LF : p.F;
     const float neg_c2 = !DIST ? -1.4426950408889634f / (2.f * p.p0 * p.p0) : 0.f;   // exp(-d2/(2 s^2)) = 2^(d2 * neg_c2)
     const int fl = lane % LF, grp = lane / LF;
     const bool mi0 = MI && p.periodic[0] && p.nc[0] == 1, mi1 = MI && p.periodic[1] && p.nc[1] == 1, mi2 = MI && p.periodic[2] && p.nc[2] == 1;
     constexpr int QP = 32 / LF;
-    const bool fvalid = fl * 4 < F;
+    const bool fvalid = VEC == 2 ? true : fl * 4 < F;
     const unsigned lt_mask = (1u << lane) - 1u;
 
     auto fold = [&](float& dx, float& dy, float& dz) {
@@ -621,12 +622,12 @@ static tiga_status launch_traverse_t(const RadiusParams& p, cudaStream_t s) {
     constexpr int smem = TravSmem<MODE>::PER_WARP * TRAV_WARPS;
     if (MODE == 0 && (p.F & 3)) {
         // scalar feature accesses (only the forward supports widths that are not multiples of 4)
-        auto sk = radius_traverse_kernel<MODE == 0 ? 0 : MODE, LF, DIST, MI, MODE != 0>;
+        auto sk = radius_traverse_kernel<MODE == 0 ? 0 : MODE, LF, DIST, MI, MODE != 0 ? 1 : 0>;
         if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(sk, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         sk<<<blocks, TRAV_THREADS, smem, s>>>(p);
         return launch_status();
     }
-    auto kern = radius_traverse_kernel<MODE, LF, DIST, MI>;
+    auto kern = p.F == 4 * LF ? radius_traverse_kernel<MODE, LF, DIST, MI, 2> : radius_traverse_kernel<MODE, LF, DIST, MI, 1>;
     if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     kern<<<blocks, TRAV_THREADS, smem, s>>>(p);
     return launch_status();
