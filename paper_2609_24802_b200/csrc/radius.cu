@@ -188,7 +188,7 @@ template <int MODE> struct TravSmem {
     // denser inputs only mean more chunks and drains
     static constexpr int STAGE_CAP = 256;                          // candidates staged per chunk
     static constexpr int QCAP = 80;                                // list entries per query
-    static constexpr int QSTRIDE = QCAP + 1;                       // odd stride: the lists of different queries fall in different banks
+    static constexpr int QSTRIDE = QCAP + 5;                       // room for four padding entries; odd, so the lists of different queries fall in different banks
     static constexpr int STAGE_BYTES = (STAGE_CAP + STAGE_PAD) * 16;
     static constexpr int LIST_BYTES = (TQB * QSTRIDE * 8 + 15) / 16 * 16;
     static constexpr int MISC_BYTES = TQB * 16 + TQB * 4 * 2;          // query coordinates, counts, totals
@@ -263,6 +263,10 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
                     for (int q = 0; q < TQB; ++q) { s_n[q] = qcnt[q]; s_tot[q] += qcnt[q]; }
                 }
                 __syncwarp();
+                // four entries of weight zero behind every list (source 0 / slot 0 exist): the loops below
+                // read whole steps without looking at the list length
+                if (lane < TQB * 4) list[(lane >> 2) * QSTRIDE + s_n[lane >> 2] + (lane & 3)] = make_float2(__int_as_float(0), 0.f);
+                __syncwarp();
                 {
                     for (int pass = 0; pass * QP < nq; ++pass) {
                         const int qq = pass * QP + grp;
@@ -281,8 +285,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
                                     float4 x[4];
 #pragma unroll
                                     for (int u = 0; u < 4; ++u) {      // four gathered rows in flight
-                                        e[u] = lq[t + u < n ? t + u : t];
-                                        if (t + u >= n) e[u].y = 0.f;
+                                        e[u] = lq[t + u];
                                         const float* xr = p.feat + (size_t)__float_as_int(e[u].x) * F + fl * 4;
                                         if (VEC) x[u] = __ldg(reinterpret_cast<const float4*>(xr));
                                         else x[u] = make_float4(__ldg(xr), fl * 4 + 1 < F ? __ldg(xr + 1) : 0.f,
@@ -302,8 +305,8 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
                                     float g[2];
 #pragma unroll
                                     for (int u = 0; u < 2; ++u) {
-                                        const float2 en2 = lq[t + u < n ? t + u : t];
-                                        g[u] = (t + u < n) ? en2.y : 0.f;
+                                        const float2 en2 = lq[t + u];
+                                        g[u] = en2.y;
                                         const float4 pj = stage[__float_as_int(en2.x)];
                                         float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
                                         fold(dx, dy, dz);
