@@ -95,15 +95,33 @@ static __device__ __forceinline__ knn_key merge_low32(const knn_key a, const knn
     return c;
 }
 
+// two independent groups of 32 keys sorted side by side (the shuffles of one hide behind the other's)
+static __device__ __forceinline__ void sort32x2(knn_key& a, knn_key& b, const int lane) {
+#pragma unroll
+    for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            const knn_key oa = __shfl_xor_sync(0xffffffffu, a, stride);
+            const knn_key ob = __shfl_xor_sync(0xffffffffu, b, stride);
+            const bool take_min = ((lane & stride) == 0) == ((lane & size) == 0);
+            a = ((a < oa) == take_min) ? a : oa;
+            b = ((b < ob) == take_min) ? b : ob;
+        }
+    }
+}
+
 // The 32 smallest keys of lq[0, n), sorted, lane t holding the t-th (KNN_NO_KEY beyond n).
 // List entries are (index, d2) pairs, which read as one little-endian 64-bit key.
 static __device__ __noinline__ knn_key select_sorted(const float2* lq, const int n, const int lane) {
     const knn_key* l64 = reinterpret_cast<const knn_key*>(lq);
-    knn_key best = KNN_NO_KEY;
-    for (int base = 0; base < n; base += 32) {
-        knn_key v = base + lane < n ? l64[base + lane] : KNN_NO_KEY;
-        v = sort32(v, lane);
-        best = base == 0 ? v : merge_low32(best, v, lane);
+    if (n <= 32) return sort32(lane < n ? l64[lane] : KNN_NO_KEY, lane);
+    knn_key best = l64[lane];
+    knn_key v = 32 + lane < n ? l64[32 + lane] : KNN_NO_KEY;
+    sort32x2(best, v, lane);
+    best = merge_low32(best, v, lane);
+    for (int base = 64; base < n; base += 32) {
+        v = sort32(base + lane < n ? l64[base + lane] : KNN_NO_KEY, lane);
+        best = merge_low32(best, v, lane);
     }
     return best;
 }
