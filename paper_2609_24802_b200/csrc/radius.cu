@@ -169,8 +169,8 @@ __global__ void bin_sort_kernel(const RadiusParams p) {
 //             are exact or act on numbers of the size of a cell, so the fp32 displacement is
 //             accurate to a few ulps of the cell size on both sides of a periodic face.
 //   phase A : every lane keeps one staged candidate in registers and tests it against the
-//             queries of the cell, eight queries per batch (their coordinates are broadcast
-//             from shared memory).  Accepted pairs are compacted with a warp ballot into one
+//             queries of the cell, four (forward) or eight (backward) queries per batch (their
+//             coordinates are broadcast from shared memory).  Accepted pairs are compacted with a warp ballot into one
 //             contiguous list per query: (source, weight) for the forward messages,
 //             (staged slot, d^2 or weight) where the displacement is needed again.
 //   phase B : MODE 0 (Gaussian / distance forward) and MODE 2 (Gaussian backward): LF lanes
