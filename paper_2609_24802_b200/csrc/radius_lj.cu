@@ -31,9 +31,17 @@ constexpr int LJ_STAGE_BYTES = (LJ_STAGE_CAP + STAGE_PAD) * 16;
 constexpr int LJQ = 4;                        // queries per batch in this kernel
 constexpr int LJ_LPQ = 32 / LJQ;              // lanes that share a query's list in phase B
 constexpr int LJ_LIST_BYTES = (LJQ * LJ_QSTRIDE * 8 + 15) / 16 * 16;
-constexpr int LJ_MISC_BYTES = LJQ * 16 + LJQ * 4;                         // queries, list lengths
+constexpr int LJ_MISC_BYTES = LJQ * 16 + 3 * LJQ * 4 + LJQ * 4;             // queries, their coordinates by component, list lengths
 constexpr int LJ_PER_WARP = (LJ_STAGE_BYTES + LJ_LIST_BYTES + LJ_MISC_BYTES + 15) / 16 * 16;
 static_assert(LJ_STAGE_BYTES % 16 == 0 && LJ_LIST_BYTES % 16 == 0 && LJ_PER_WARP % 16 == 0, "the stage and the queries are accessed as 16-byte vectors");
+
+// two fp32 values per register pair: sm_100 executes add / mul / fma on both with one instruction
+typedef unsigned long long f32x2;
+static __device__ __forceinline__ f32x2 pack2(float a, float b) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
+static __device__ __forceinline__ void unpack2(f32x2 v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+static __device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 r; asm("sub.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+static __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 r; asm("mul.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+static __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
 
 template <bool MI, bool COUNT>
 __global__ void __launch_bounds__(TRAV_THREADS, 6) radius_lj_pairs_kernel(const __grid_constant__ RadiusParams p) {
@@ -48,7 +56,8 @@ __global__ void __launch_bounds__(TRAV_THREADS, 6) radius_lj_pairs_kernel(const 
     float4* stage = reinterpret_cast<float4*>(base);                                   // local x, y, z, point id
     float2* list = reinterpret_cast<float2*>(base + LJ_STAGE_BYTES);                   // (stage slot, d2) per query
     float4* s_q = reinterpret_cast<float4*>(base + LJ_STAGE_BYTES + LJ_LIST_BYTES);
-    int* s_n = reinterpret_cast<int*>(s_q + LJQ);
+    float* s_qc = reinterpret_cast<float*>(s_q + LJQ);        // x[LJQ], y[LJQ], z[LJQ]: read two queries at a time
+    int* s_n = reinterpret_cast<int*>(s_qc + 3 * LJQ);
 
     const int c[3] = {cellid % p.nc[0], (cellid / p.nc[0]) % p.nc[1], cellid / (p.nc[0] * p.nc[1])};
     const float org[3] = {(float)c[0] * p.hcell[0], (float)c[1] * p.hcell[1], (float)c[2] * p.hcell[2]};
@@ -157,9 +166,15 @@ __global__ void __launch_bounds__(TRAV_THREADS, 6) radius_lj_pairs_kernel(const 
         for (int qb0 = qs0; qb0 < qe0; qb0 += LJQ) {
             const int nq = (qe0 - qb0 < LJQ) ? qe0 - qb0 : LJQ;
             __syncwarp();
-            if (lane < nq) {
-                const float4 pq = p.spos[qb0 + lane];
-                s_q[lane] = make_float4(pq.x - org[0], pq.y - org[1], pq.z - org[2], pq.w);
+            if (lane < LJQ) {
+                // absent queries of a short batch sit far away: whatever is computed for them is never used
+                float4 lq4 = make_float4(FAR_AWAY, FAR_AWAY, FAR_AWAY, __int_as_float(-2));
+                if (lane < nq) {
+                    const float4 pq = p.spos[qb0 + lane];
+                    lq4 = make_float4(pq.x - org[0], pq.y - org[1], pq.z - org[2], pq.w);
+                }
+                s_q[lane] = lq4;
+                s_qc[lane] = lq4.x; s_qc[LJQ + lane] = lq4.y; s_qc[2 * LJQ + lane] = lq4.z;
             }
             __syncwarp();
             int qcnt[LJQ];
@@ -235,17 +250,36 @@ __global__ void __launch_bounds__(TRAV_THREADS, 6) radius_lj_pairs_kernel(const 
                 const bool own = OWN && cbase + lane < nself;
                 float d2q[LJQ];
                 float nearest = FAR_AWAY;       // smallest |d2 - r^2| seen by this lane
+                if constexpr (!MI) {
+                    // squared distances of two queries per instruction (same operations and roundings as
+                    // the scalar form: a product, then two fused multiply-adds)
+                    const f32x2 px = pack2(pj.x, pj.x), py = pack2(pj.y, pj.y), pz = pack2(pj.z, pj.z);
+                    const f32x2* qx2 = reinterpret_cast<const f32x2*>(s_qc);
 #pragma unroll
-                for (int q = 0; q < LJQ; ++q) {
-                    if (!FULLB && q >= nq) break;
-                    const float4 qv = s_q[q];
-                    float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
-                    fold(dx, dy, dz);
-                    float d2 = fmaf(dz, dz, fmaf(dy, dy, dx * dx));
-                    if (OWN && own && idj <= __float_as_int(qv.w)) d2 = FAR_AWAY;      // own cell: each pair once
-                    if (MI && idj < 0) d2 = FAR_AWAY;                                  // folded sentinels
-                    nearest = fminf(nearest, fabsf(d2 - p.r2_mid));
-                    d2q[q] = d2;
+                    for (int h = 0; h < LJQ / 2; ++h) {
+                        if (!FULLB && 2 * h >= nq) break;
+                        const f32x2 dx = sub2(qx2[h], px), dy = sub2(qx2[LJQ / 2 + h], py), dz = sub2(qx2[LJQ + h], pz);
+                        unpack2(fma2(dz, dz, fma2(dy, dy, mul2(dx, dx))), d2q[2 * h], d2q[2 * h + 1]);
+                    }
+#pragma unroll
+                    for (int q = 0; q < LJQ; ++q) {
+                        if (!FULLB && q >= nq) break;
+                        if (OWN && own && idj <= __float_as_int(s_q[q].w)) d2q[q] = FAR_AWAY;      // own cell: each pair once
+                        nearest = fminf(nearest, fabsf(d2q[q] - p.r2_mid));
+                    }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < LJQ; ++q) {
+                        if (!FULLB && q >= nq) break;
+                        const float4 qv = s_q[q];
+                        float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
+                        fold(dx, dy, dz);
+                        float d2 = fmaf(dz, dz, fmaf(dy, dy, dx * dx));
+                        if (OWN && own && idj <= __float_as_int(qv.w)) d2 = FAR_AWAY;      // own cell: each pair once
+                        if (idj < 0) d2 = FAR_AWAY;                                        // folded sentinels
+                        nearest = fminf(nearest, fabsf(d2 - p.r2_mid));
+                        d2q[q] = d2;
+                    }
                 }
                 if (__any_sync(FULL, nearest <= p.r2_band)) {
                     // some pair lies within the fp32 error band of the cutoff: decide it in fp64
