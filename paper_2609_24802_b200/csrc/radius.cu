@@ -191,7 +191,7 @@ template <int MODE> struct TravSmem {
     static constexpr int QSTRIDE = QCAP + 5;                       // room for four padding entries; odd, so the lists of different queries fall in different banks
     static constexpr int STAGE_BYTES = (STAGE_CAP + STAGE_PAD) * 16;
     static constexpr int LIST_BYTES = (TQB * QSTRIDE * 8 + 15) / 16 * 16;
-    static constexpr int MISC_BYTES = TQB * 16 + TQB * 4 * 2;          // query coordinates, counts, totals
+    static constexpr int MISC_BYTES = TQB * 16 + 3 * TQB * 4 + TQB * 4 * 2;   // queries, their coordinates by component, counts, totals
     static constexpr int PER_WARP = STAGE_BYTES + LIST_BYTES + MISC_BYTES;
     static_assert(PER_WARP % 16 == 0 && LIST_BYTES % 16 == 0, "the stage and the queries are accessed as 16-byte vectors");
 };
@@ -218,7 +218,8 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
     float4* stage = reinterpret_cast<float4*>(base);
     float2* list = reinterpret_cast<float2*>(base + SM::STAGE_BYTES);
     float4* s_q = reinterpret_cast<float4*>(base + SM::STAGE_BYTES + SM::LIST_BYTES);   // local x, y, z, point id
-    int* s_n = reinterpret_cast<int*>(s_q + TQB);                                        // list lengths of the drain in progress
+    float* s_qc = reinterpret_cast<float*>(s_q + TQB);                                  // x[TQB], y[TQB], z[TQB]: read two queries at a time
+    int* s_n = reinterpret_cast<int*>(s_qc + 3 * TQB);                                  // list lengths of the drain in progress
     int* s_tot = s_n + TQB;                                                              // neighbours found so far in this chunk
 
     const int c[3] = {cellid % p.nc[0], (cellid / p.nc[0]) % p.nc[1], cellid / (p.nc[0] * p.nc[1])};
@@ -245,9 +246,15 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
         for (int qb0 = qs0; qb0 < qe0; qb0 += TQB) {
             const int nq = (qe0 - qb0 < TQB) ? qe0 - qb0 : TQB;
             __syncwarp();
-            if (lane < nq) {
-                const float4 pq = p.spos[qb0 + lane];
-                s_q[lane] = make_float4(pq.x - org[0], pq.y - org[1], pq.z - org[2], pq.w);
+            if (lane < TQB) {
+                // absent queries of a short batch sit far away: whatever is computed for them is never used
+                float4 lq4 = make_float4(FAR_AWAY, FAR_AWAY, FAR_AWAY, __int_as_float(-2));
+                if (lane < nq) {
+                    const float4 pq = p.spos[qb0 + lane];
+                    lq4 = make_float4(pq.x - org[0], pq.y - org[1], pq.z - org[2], pq.w);
+                }
+                s_q[lane] = lq4;
+                s_qc[lane] = lq4.x; s_qc[TQB + lane] = lq4.y; s_qc[2 * TQB + lane] = lq4.z;
                 s_tot[lane] = 0;
             }
             __syncwarp();
@@ -370,16 +377,35 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
                 const int idj = __float_as_int(pj.w);
                 float d2q[TQB];
                 float nearest = FAR_AWAY;       // smallest |d2 - r^2| seen by this lane
+                if constexpr (!MI && MODE == 0) {
+                    // squared distances of two queries per packed instruction (same operations and roundings
+                    // as the scalar form: a product, then two fused multiply-adds)
+                    const f32x2 px = pack2(pj.x, pj.x), py = pack2(pj.y, pj.y), pz = pack2(pj.z, pj.z);
+                    const f32x2* qx2 = reinterpret_cast<const f32x2*>(s_qc);
 #pragma unroll
-                for (int q = 0; q < TQB; ++q) {
-                    if (!FULLB && q >= nq) break;
-                    const float4 qv = s_q[q];
-                    float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
-                    fold(dx, dy, dz);
-                    float d2 = fmaf(dz, dz, fmaf(dy, dy, dx * dx));
-                    if (idj == __float_as_int(qv.w) || (MI && idj < 0)) d2 = FAR_AWAY;     // self (by index); folded sentinels
-                    nearest = fminf(nearest, fabsf(d2 - p.r2_mid));
-                    d2q[q] = d2;
+                    for (int h = 0; h < TQB / 2; ++h) {
+                        if (!FULLB && 2 * h >= nq) break;
+                        const f32x2 dx = sub2(qx2[h], px), dy = sub2(qx2[TQB / 2 + h], py), dz = sub2(qx2[TQB + h], pz);
+                        unpack2(fma2(dz, dz, fma2(dy, dy, mul2(dx, dx))), d2q[2 * h], d2q[2 * h + 1]);
+                    }
+#pragma unroll
+                    for (int q = 0; q < TQB; ++q) {
+                        if (!FULLB && q >= nq) break;
+                        if (idj == __float_as_int(s_q[q].w)) d2q[q] = FAR_AWAY;            // self (by index)
+                        nearest = fminf(nearest, fabsf(d2q[q] - p.r2_mid));
+                    }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < TQB; ++q) {
+                        if (!FULLB && q >= nq) break;
+                        const float4 qv = s_q[q];
+                        float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
+                        fold(dx, dy, dz);
+                        float d2 = fmaf(dz, dz, fmaf(dy, dy, dx * dx));
+                        if (idj == __float_as_int(qv.w) || (MI && idj < 0)) d2 = FAR_AWAY; // self (by index); folded sentinels
+                        nearest = fminf(nearest, fabsf(d2 - p.r2_mid));
+                        d2q[q] = d2;
+                    }
                 }
                 if (__any_sync(FULL, nearest <= p.r2_band)) {
                     // some pair lies within the fp32 error band of the cutoff: decide it in fp64 and

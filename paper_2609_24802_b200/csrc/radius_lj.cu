@@ -35,14 +35,6 @@ constexpr int LJ_MISC_BYTES = LJQ * 16 + 3 * LJQ * 4 + LJQ * 4;             // q
 constexpr int LJ_PER_WARP = (LJ_STAGE_BYTES + LJ_LIST_BYTES + LJ_MISC_BYTES + 15) / 16 * 16;
 static_assert(LJ_STAGE_BYTES % 16 == 0 && LJ_LIST_BYTES % 16 == 0 && LJ_PER_WARP % 16 == 0, "the stage and the queries are accessed as 16-byte vectors");
 
-// two fp32 values per register pair: sm_100 executes add / mul / fma on both with one instruction
-typedef unsigned long long f32x2;
-static __device__ __forceinline__ f32x2 pack2(float a, float b) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
-static __device__ __forceinline__ void unpack2(f32x2 v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
-static __device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 r; asm("sub.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
-static __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 r; asm("mul.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
-static __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
-
 template <bool MI, bool COUNT>
 __global__ void __launch_bounds__(TRAV_THREADS, 6) radius_lj_pairs_kernel(const __grid_constant__ RadiusParams p) {
     constexpr unsigned FULL = 0xffffffffu;

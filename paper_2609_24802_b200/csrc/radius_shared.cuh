@@ -93,6 +93,14 @@ static __device__ __forceinline__ float fast_rcp(float x) {
     return r;
 }
 
+// two fp32 values per register pair: sm_100 executes add / mul / fma on both with one instruction
+typedef unsigned long long f32x2;
+static __device__ __forceinline__ f32x2 pack2(float a, float b) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
+static __device__ __forceinline__ void unpack2(f32x2 v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+static __device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 r; asm("sub.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+static __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 r; asm("mul.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+static __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
+
 // exact predicate for the pair of original point ids (a, b)
 static __device__ __noinline__ bool exact_pair(const RadiusParams& p, int a, int b) {
     const float4 pa = make_float4(p.pos[3 * (size_t)a], p.pos[3 * (size_t)a + 1], p.pos[3 * (size_t)a + 2], 0.f);
