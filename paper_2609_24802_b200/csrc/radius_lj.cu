@@ -36,7 +36,7 @@ constexpr int LJ_PER_WARP = (LJ_STAGE_BYTES + LJ_LIST_BYTES + LJ_MISC_BYTES + 15
 static_assert(LJ_STAGE_BYTES % 16 == 0 && LJ_LIST_BYTES % 16 == 0 && LJ_PER_WARP % 16 == 0, "the stage and the queries are accessed as 16-byte vectors");
 
 template <bool MI, bool COUNT>
-__global__ void __launch_bounds__(TRAV_THREADS, 6) radius_lj_pairs_kernel(const __grid_constant__ RadiusParams p) {
+__global__ void __launch_bounds__(TRAV_THREADS, COUNT ? 8 : 7) radius_lj_pairs_kernel(const __grid_constant__ RadiusParams p) {
     constexpr unsigned FULL = 0xffffffffu;
     extern __shared__ __align__(16) unsigned char s_raw[];
 
