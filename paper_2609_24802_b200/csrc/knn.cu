@@ -31,7 +31,7 @@
 namespace tiga {
 
 constexpr int KQB = 4;                             // queries per batch (cells kernel)
-constexpr int KNN_STAGE_CAP = 256;                 // staged candidates per chunk
+constexpr int KNN_STAGE_CAP = 192;                 // staged candidates per chunk
 constexpr int KNN_QCAP = 96;                       // list entries per query (cells kernel)
 constexpr int KNN_QSTRIDE = KNN_QCAP + 1;
 constexpr int KNN_RING_CAP = 128;                  // list entries of the rings kernel
