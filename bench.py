@@ -165,11 +165,11 @@ def combine_ranks(dist, device, total_ms, e2e_ms, interactions):
 # `roofline.traffic` to a full launch: bytes per particle / point / edge of one launch.
 TRAFFIC_PER_UNIT = {
     "radius_lj_fwd": ("particle", 48.4),          # profiles/radius_lj_pairs_1M.md: 32.4 B measured + the 16-byte row that leaves L2 at full size
-    "radius_gauss_fwd": ("point", 191.3),         # profiles/radius_traverse_gaussian_300k.md
-    "radius_gauss_bwd": ("point", 360.0),
+    "radius_gauss_fwd": ("point", 186.7),         # profiles/radius_traverse_gaussian_300k.md
+    "radius_gauss_bwd": ("point", 364.6),
     "csr_sum_fwd": ("edge", 21.1),                # profiles/csr_kernels_rmat_scale18.md
-    "csr_sum_bwd": ("edge", 45.4),
-    "csr_max_bwd": ("edge", 52.0),
+    "csr_sum_bwd": ("edge", 45.3),
+    "csr_max_bwd": ("edge", 52.1),
 }
 
 
