@@ -382,42 +382,64 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_rings_kernel(const __grid_co
             __syncwarp();
         };
 
-        // one contiguous run of cell-ordered points [a, b) against the query
-        auto run = [&](const int a, const int b) {
-            for (int v0 = a; v0 < b; v0 += 32) {
-                const int v = v0 + lane;
-                bool ok = false;
-                float4 c4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                float d2 = 0.f;
-                if (v < b) {
-                    c4 = __ldg(p.spos + v);
-                    d2 = key_d2(qx, qy, qz, c4.x, c4.y, c4.z);
-                    ok = d2 <= tau && __float_as_int(c4.w) != i;
-                }
-                const unsigned m = __ballot_sync(FULL, ok);
-                if (ok) list[cnt + __popc(m & lt_mask)] = make_float2(c4.w, d2);
-                cnt += __popc(m);
-                if (cnt > KNN_RING_CAP - 32) {
-                    __syncwarp();
-                    cut();
-                }
-            }
-        };
-
         for (int s = 0; s <= smax; ++s) {
             const int z0 = max(cz - s, 0), z1 = min(cz + s, nz - 1);
             const int y0 = max(cy - s, 0), y1 = min(cy + s, ny - 1);
             const int x0 = max(cx - s, 0), x1 = min(cx + s, nx - 1);
-            for (int z = z0; z <= z1; ++z)
-                for (int y = y0; y <= y1; ++y) {
+            const int wy = y1 - y0 + 1, nrow = (z1 - z0 + 1) * wy;
+            // the (y, z) rows of the shell, sixteen at a time: every lane resolves one contiguous run of
+            // cell-ordered points (a face row is one run over the whole x range, an inner row has its two
+            // end cells), then the runs are walked as one flat sequence so that all loads are independent
+            for (int rbase = 0; rbase < nrow; rbase += 16) {
+                const int rr = rbase + (lane >> 1), side = lane & 1;
+                int ra = 0, rlen = 0;
+                if (rr < nrow) {
+                    const int z = z0 + rr / wy, y = y0 + rr % wy;
                     const int row = (z * ny + y) * nx;
-                    if (z - cz == s || cz - z == s || y - cy == s || cy - y == s) {
-                        run(p.cell_start[row + x0], p.cell_start[row + x1 + 1]);      // a face row of the shell: whole x range
-                    } else {
-                        if (cx - s >= 0) run(p.cell_start[row + cx - s], p.cell_start[row + cx - s + 1]);
-                        if (s > 0 && cx + s < nx) run(p.cell_start[row + cx + s], p.cell_start[row + cx + s + 1]);
+                    const bool face = z - cz == s || cz - z == s || y - cy == s || cy - y == s;
+                    int xa = -1, xb = -1;                                  // cells [xa, xb]
+                    if (face) { if (side == 0) { xa = x0; xb = x1; } }
+                    else if (side == 0) { if (cx - s >= 0) xa = xb = cx - s; }
+                    else if (s > 0 && cx + s < nx) xa = xb = cx + s;
+                    if (xa >= 0) {
+                        ra = p.cell_start[row + xa];
+                        rlen = p.cell_start[row + xb + 1] - ra;
                     }
                 }
+                int rincl = rlen;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int t2 = __shfl_up_sync(FULL, rincl, o);
+                    if (lane >= o) rincl += t2;
+                }
+                const int total = __shfl_sync(FULL, rincl, 31);
+                for (int v0 = 0; v0 < total; v0 += 32) {
+                    const int v = v0 + lane;
+                    int r = 0;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const int probe = __shfl_sync(FULL, rincl, r + o - 1);
+                        if (probe <= v) r += o;
+                    }
+                    r = r > 31 ? 31 : r;
+                    const int src = __shfl_sync(FULL, ra, r) + (v - (__shfl_sync(FULL, rincl, r) - __shfl_sync(FULL, rlen, r)));
+                    bool ok = false;
+                    float4 c4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float d2 = 0.f;
+                    if (v < total) {
+                        c4 = __ldg(p.spos + src);
+                        d2 = key_d2(qx, qy, qz, c4.x, c4.y, c4.z);
+                        ok = d2 <= tau && __float_as_int(c4.w) != i;
+                    }
+                    const unsigned m = __ballot_sync(FULL, ok);
+                    if (ok) list[cnt + __popc(m & lt_mask)] = make_float2(c4.w, d2);
+                    cnt += __popc(m);
+                    if (cnt > KNN_RING_CAP - 32) {
+                        __syncwarp();
+                        cut();
+                    }
+                }
+            }
             // every point whose cell differs by more than s from the query's in some dimension is
             // farther than s cell edges away: k keys within that distance cannot be improved
             __syncwarp();
