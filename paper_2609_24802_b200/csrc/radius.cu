@@ -307,11 +307,12 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
                             } else {
                                 const float4 xk = __ldg(reinterpret_cast<const float4*>(p.feat + (size_t)oqq * F) + fl);
                                 const float4 gk = __ldg(reinterpret_cast<const float4*>(p.gy + (size_t)oqq * F) + fl);
-                                for (int t = 0; t < n; t += 2) {
-                                    float4 e[2], xj[2], gj[2];
-                                    float g[2];
+                                constexpr int BU = 4;      // pairs in flight per lane
+                                for (int t = 0; t < n; t += BU) {
+                                    float4 e[BU], xj[BU], gj[BU];
+                                    float g[BU];
 #pragma unroll
-                                    for (int u = 0; u < 2; ++u) {
+                                    for (int u = 0; u < BU; ++u) {
                                         const float2 en2 = lq[t + u];
                                         g[u] = en2.y;
                                         const float4 pj = stage[__float_as_int(en2.x)];
@@ -323,7 +324,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
                                         gj[u] = __ldg(reinterpret_cast<const float4*>(p.gy + row) + fl);
                                     }
 #pragma unroll
-                                    for (int u = 0; u < 2; ++u) {
+                                    for (int u = 0; u < BU; ++u) {
                                         acc.x = fmaf(g[u], gj[u].x, acc.x); acc.y = fmaf(g[u], gj[u].y, acc.y);
                                         acc.z = fmaf(g[u], gj[u].z, acc.z); acc.w = fmaf(g[u], gj[u].w, acc.w);
                                         float part = gk.x * xj[u].x;
