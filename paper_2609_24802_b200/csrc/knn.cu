@@ -11,7 +11,7 @@
 //                     27-cell stencil, so a query that finds k keys <= h^2 there is finished: no
 //                     point outside the stencil can have a smaller key.  The stencil is staged in
 //                     shared memory (candidates farther than h from the bounding box of the
-//                     cell's points are dropped), one candidate per lane is tested against eight
+//                     cell's points are dropped), one candidate per lane is tested against four
 //                     queries, accepted keys are compacted into per-query lists by ballots, and a
 //                     list that fills up is cut back to its k smallest keys, which also tightens
 //                     that query's acceptance threshold.

@@ -10,7 +10,7 @@
 //      makes the scatter stable and therefore unique), sorted copy of the positions;
 //   2. traversal: one warp per query cell stages the 27 neighbouring cells (wrapped or
 //      clipped, contiguous ranges of the cell-ordered points) in shared memory, tests one
-//      staged candidate per lane against eight queries at a time, compacts accepted
+//      staged candidate per lane against a batch of four or eight queries, compacts accepted
 //      (source, weight) pairs into one list per query and consumes the lists with groups of
 //      lanes across the feature axis, so every gathered feature row is one coalesced
 //      128-bit-per-lane request.  (Lennard-Jones: radius_lj.cu; edge network: radius_mlp.cu.)

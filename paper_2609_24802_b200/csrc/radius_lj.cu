@@ -16,9 +16,9 @@
 // Structure inside a warp (as in radius_traverse_kernel): the half stencil is staged in shared
 // memory in cell-local coordinates with periodic images applied (exact fp32 shifts), candidates
 // farther than the cutoff from the bounding box of the cell's points are dropped, phase A tests one
-// staged candidate per lane against eight queries and compacts accepted pairs into per-query
+// staged candidate per lane against four queries and compacts accepted pairs into per-query
 // lists by ballots (pairs within the fp32 error band of the cutoff are decided in fp64), phase B
-// gives every query four lanes that evaluate its listed pairs.
+// gives every query eight lanes that evaluate its listed pairs.
 #include "radius_shared.cuh"
 #include <type_traits>
 

@@ -9,7 +9,7 @@ namespace tiga {
 constexpr int TRAV_WARPS = 4;
 constexpr int TRAV_THREADS = TRAV_WARPS * 32;
 constexpr int STAGE_PAD = 32;           // sentinels behind the staged candidates: no bounds checks
-constexpr int QB = 8;                   // queries per batch
+constexpr int QB = 8;                   // queries per batch (kernels that run faster with four define their own width)
 constexpr float FAR_AWAY = 1.0e18f;
 
 struct RadiusParams {
