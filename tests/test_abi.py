@@ -86,3 +86,30 @@ def test_host_side_argument_errors(lib):
     assert cdll.tiga_apply_radius(256, 256, 100, 8, r, ctypes.byref(b), ctypes.byref(_Msg(2, 0.1, 0.0)), 256, None, 256, 64, None) == 3     # workspace
     assert cdll.tiga_apply_radius_backward(256, 256, 100, 8, r, ctypes.byref(b), ctypes.byref(_Msg(4, 1.0, 1.0)), 256, 256, 256, 256, big, 0, None) == 2
     assert cdll.tiga_apply_radius_backward(256, 256, 100, 6, r, ctypes.byref(b), ctypes.byref(_Msg(2, 0.1, 0.0)), 256, 256, 256, 256, big, 0, None) == 2
+
+
+def test_knn_and_attention_host_checks(lib):
+    """Workspace sizing and argument checks of the widened entry points run on the host only."""
+    cdll = lib.load_library()
+    from paper_2609_24802_b200.api import _Box, _Csr
+    box = _Box()
+    for d in range(3):
+        box.len[d] = 1.0
+        box.periodic[d] = 0
+    small = cdll.tiga_knn_workspace_bytes(1000, 16, ctypes.byref(box))
+    large = cdll.tiga_knn_workspace_bytes(1_000_000, 16, ctypes.byref(box))
+    assert 0 < small < large
+    assert cdll.tiga_knn_workspace_bytes(1000, 33, ctypes.byref(box)) == 0          # k above the envelope
+    assert cdll.tiga_knn_workspace_bytes(1000, 0, ctypes.byref(box)) == 0
+    box.periodic[1] = 1
+    assert cdll.tiga_knn_workspace_bytes(1000, 16, ctypes.byref(box)) == 0          # periodic boxes are not supported
+    # statuses without touching a device: bad k, periodic box, bad width
+    assert cdll.tiga_apply_knn(None, None, 10, 1, 0, ctypes.byref(box), None, None, None, None, 0, None) == 1
+    assert cdll.tiga_apply_knn(None, None, 10, 1, 4, ctypes.byref(box), None, None, None, None, 0, None) == 2
+    g = _Csr(0, 0, 0, 1_000_000, 1_000_000, 16_000_000)
+    assert cdll.tiga_csr_attention_workspace_bytes(ctypes.byref(g), 64) > cdll.tiga_csr_attention_workspace_bytes(ctypes.byref(g), 8) > 0
+    assert cdll.tiga_csr_attention_workspace_bytes(ctypes.byref(g), 6) == 0
+    assert cdll.tiga_csr_attention_workspace_bytes(ctypes.byref(g), 256) == 0
+    assert cdll.tiga_apply_csr_attention(ctypes.byref(g), None, None, None, 6, ctypes.c_float(1.0), None, None, None, 0, None) == 1
+    assert cdll.tiga_apply_csr_attention(ctypes.byref(g), None, None, None, 132, ctypes.c_float(1.0), None, None, None, 0, None) == 2
+    assert cdll.tiga_probe_row_gather(None, 10, 256, None, 10, None, None) == 1
