@@ -717,7 +717,22 @@ def run_case(args):
     ev1.record()
     torch.cuda.synchronize()
     ms = ev0.elapsed_time(ev1) / args.steps
-    print(json.dumps({"case": args.case, "units": units, "ms_per_step": ms, "units_per_s": units / (ms * 1e-3)}))
+    rec = {"case": args.case, "units": units, "ms_per_step": ms, "units_per_s": units / (ms * 1e-3)}
+    if args.case == "csr_large":
+        # the HBM-stream test: the three bandwidth fractions against the measured copy bandwidth
+        peaks = measured_peaks()
+        hbm = peaks[0] * 1e9
+        E, N = c["E"], c["n"]
+        b_alg = E * (4 + 16) + N * (8 + 32)                       # col + one 16-byte source row per edge; rowptr + fp32 output row per row
+        touched = int(torch.unique(g.col).numel()) if E <= (1 << 28) else None
+        b_min = 8.0 * (N + 1) + 4.0 * E + 16.0 * (touched if touched is not None else 2.7e7) + 32.0 * N
+        b_dram = 35.5e9 * E / float(1 << 30)                      # profiles/csr_large_cfg4_dram_traffic.md, per edge
+        rec.update({"f_alg": b_alg / (ms * 1e-3) / hbm, "f_dram": b_dram / (ms * 1e-3) / hbm, "f_min": b_min / (ms * 1e-3) / hbm,
+                    "bytes_alg": b_alg, "bytes_dram_ncu": b_dram, "bytes_min": b_min,
+                    "bytes_dram_note": "ncu capture at full size scaled by edges: meaningful at scale 26 only (smaller feature tables fit L2)",
+                    "touched_source_rows": touched if touched is not None else "2.7e7 (analytic, R-MAT scale 26)",
+                    "peak_GBps": peaks[0], "peak_source": peaks[2] if len(peaks) > 2 else "measured"})
+    print(json.dumps(rec))
 
 
 def main():
