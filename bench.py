@@ -727,7 +727,18 @@ def run_case(args):
         touched = int(torch.unique(g.col).numel()) if E <= (1 << 28) else None
         b_min = 8.0 * (N + 1) + 4.0 * E + 16.0 * (touched if touched is not None else 2.7e7) + 32.0 * N
         b_dram = 35.5e9 * E / float(1 << 30)                      # profiles/csr_large_cfg4_dram_traffic.md, per edge
-        rec.update({"f_alg": b_alg / (ms * 1e-3) / hbm, "f_dram": b_dram / (ms * 1e-3) / hbm, "f_min": b_min / (ms * 1e-3) / hbm,
+        sink = torch.zeros(1, device=dev)
+        for _ in range(2):
+            T.tiga_probe_row_gather(x, g.col, sink)
+        pa = torch.cuda.Event(enable_timing=True); pb = torch.cuda.Event(enable_timing=True)
+        pa.record()
+        for _ in range(3):
+            T.tiga_probe_row_gather(x, g.col, sink)
+        pb.record(); torch.cuda.synchronize()
+        t_gather = pa.elapsed_time(pb) / 3
+        rec.update({"gather_of_own_index_stream_ms": t_gather, "T_own_gather_over_T": t_gather / ms,
+                    "gather_note": "tiga_probe_row_gather on the same col stream and feature table: the gathers alone, no row sums, no output",
+                    "f_alg": b_alg / (ms * 1e-3) / hbm, "f_dram": b_dram / (ms * 1e-3) / hbm, "f_min": b_min / (ms * 1e-3) / hbm,
                     "bytes_alg": b_alg, "bytes_dram_ncu": b_dram, "bytes_min": b_min,
                     "bytes_dram_note": "ncu capture at full size scaled by edges: meaningful at scale 26 only (smaller feature tables fit L2)",
                     "touched_source_rows": touched if touched is not None else "2.7e7 (analytic, R-MAT scale 26)",
