@@ -143,21 +143,20 @@ __global__ void bin_scatter_kernel(const RadiusParams p, int32_t* fill) {
     p.order_tmp[slot] = i;
 }
 
-// One warp per cell: rank of every member among the members' point ids -> stable order,
-// and the sorted copy of the positions.
+// One thread per scattered slot: the rank of its point among the point ids of its cell gives
+// the stable order (cell, then index) and the place of the sorted copy of the position.
+// Neighbouring threads belong to the same cell and read the same few slots.
 __global__ void bin_sort_kernel(const RadiusParams p) {
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (warp >= p.ncells) return;
-    const int s = p.cell_start[warp], e = p.cell_start[warp + 1];
-    for (int t = s + lane; t < e; t += 32) {
-        const int id = p.order_tmp[t];
-        int rank = 0;
-        for (int u = s; u < e; ++u) rank += (p.order_tmp[u] < id) ? 1 : 0;
-        p.order[s + rank] = id;
-        if (p.u_order) p.u_order[s + rank] = id;
-        p.spos[s + rank] = make_float4(p.pos[3 * (size_t)id], p.pos[3 * (size_t)id + 1], p.pos[3 * (size_t)id + 2], __int_as_float(id));
-    }
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= p.n) return;
+    const int id = p.order_tmp[t];
+    const int c = p.cell[id];
+    const int s = p.cell_start[c], e = p.cell_start[c + 1];
+    int rank = 0;
+    for (int u = s; u < e; ++u) rank += (p.order_tmp[u] < id) ? 1 : 0;
+    p.order[s + rank] = id;
+    if (p.u_order) p.u_order[s + rank] = id;
+    p.spos[s + rank] = make_float4(p.pos[3 * (size_t)id], p.pos[3 * (size_t)id + 1], p.pos[3 * (size_t)id + 2], __int_as_float(id));
 }
 
 // ------------------------------------------------------------------------------ traversal
@@ -636,7 +635,7 @@ tiga_status run_binning(RadiusParams& p, int32_t* fill, int nblocks, cudaStream_
     scan_blocksums_kernel<<<1, 1024, 0, s>>>(p, nblocks);
     scan_apply_kernel<<<nblocks, RAD_THREADS, 0, s>>>(p);
     bin_scatter_kernel<<<pb, 256, 0, s>>>(p, fill);
-    bin_sort_kernel<<<(unsigned)(((size_t)p.ncells * 32 + 255) / 256), 256, 0, s>>>(p);
+    bin_sort_kernel<<<pb, 256, 0, s>>>(p);
     return launch_status();
 }
 
