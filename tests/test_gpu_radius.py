@@ -153,11 +153,11 @@ def test_gaussian_mid_replica(tiga):
 
 
 # ------------------------------------------------------------------------------ Lennard-Jones
-def _check_lj(tiga, pos, r, box, per, eps=1.0, s=1.0, use_cells=False):
+def _check_lj(tiga, pos, r, box, per, eps=1.0, s=1.0, use_cells=False, tol=SUM_TOL):
     y, A, cnt = oracle.radius_forward(pos, None, r, box, per, oracle.MSG_LJ, eps, s, use_cells=use_cells)
     out, count, _ = tiga.tiga_apply_radius(dev(pos, torch), None, r, box, per, tiga.MSG_LJ, p0=eps, p1=s, want_count=True)
     assert np.array_equal(host(count), cnt)
-    assert rel_err(host(out), y, A) <= SUM_TOL
+    assert rel_err(host(out), y, A) <= tol
     return host(out), A
 
 
@@ -220,6 +220,24 @@ def test_lennard_jones_small_grids(tiga, cells, periodic):
     assert list(grid) == [min(e, cap) for e in expect]
     out, A = _check_lj(tiga, pos, r, box, list(periodic), eps=0.7, s=0.5)
     assert np.max(np.abs(out[:, :3].astype(np.float64).sum(0))) < 1e-5 * max(A[:, :3].sum(), 1e-30)
+
+
+def test_lennard_jones_dense_cells_span_several_stage_chunks(tiga):
+    """Hundreds of points per cell: the cell's own points alone overflow the stage, so the half
+    stencil is processed in several chunks and the own-cell rule (each pair once, by index) is
+    applied across chunk borders."""
+    box = np.array([6.0, 6.0, 6.0], np.float32)
+    pos = _separated_points(2600, box, 77, 0.25)
+    assert len(pos) > 1800
+    # The pair force goes like d^-14, so a relative error e of d^2 is an error 7 e of the force, and the
+    # closest pairs dominate the sums.  A coordinate relative to the cell corner carries an fp32
+    # rounding of 2^-24 times the cell edge (3 here, against 0.25 between the closest points):
+    # e = 2 * 2^-24 * 3 / 0.25, which is added to the usual tolerance.  Counts stay exact.
+    tol = SUM_TOL + 7.0 * 2.0 * 2.0 ** -24 * 3.0 / 0.25
+    for periodic in ([0, 0, 0], [1, 1, 1]):
+        grid, _ = tiga.tiga_radius_grid(len(pos), np.float32(2.0), box, periodic)
+        assert max(grid) <= 2
+        _check_lj(tiga, pos, np.float32(2.0), box, periodic, eps=0.3, s=0.3, tol=tol)
 
 
 def test_lennard_jones_rows_are_summed_by_atomics(tiga):
