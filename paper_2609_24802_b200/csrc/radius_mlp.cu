@@ -9,7 +9,9 @@
 // one staged candidate per lane tested against eight queries, ballot compaction into one list
 // per query.  What differs is phase B: every lane takes one accepted pair and evaluates the
 // whole network for it with the weights broadcast from shared memory (input padded to 4 KQ,
-// hidden width HID in registers); pair messages are combined with a shuffle tree.
+// hidden width HID in registers).  The pairs of all queries of a batch form one flat sequence,
+// 32 per step, so short neighbour lists do not leave lanes idle; per-query sums are segmented
+// shuffle reductions (fixed order: reproducible).
 //
 // Backward, owner computes: for query k and neighbour m a lane evaluates the pair twice,
 //   (k <- m) gives the parameter gradients and -ubar[0:3] for pbar_k,
@@ -33,7 +35,8 @@ template <int HID, bool BWD> struct MlpSmem {
     static constexpr int CTA_BYTES = (W_FLOATS * (BWD ? 2 : 1) * 4 + 15) / 16 * 16;   // weights (+ gradient accumulators)
     static constexpr int STAGE_BYTES = (MLP_STAGE_CAP + STAGE_PAD) * 16;
     static constexpr int LIST_BYTES = (QB * MLP_QSTRIDE * 4 + 15) / 16 * 16;
-    static constexpr int MISC_BYTES = QB * 16 + QB * 4 * 2;
+    static constexpr int ACC_W = 16;                                             // per-query accumulator: outputs, or pbar (3) + xbar (13)
+    static constexpr int MISC_BYTES = QB * 16 + QB * 4 * 2 + QB * ACC_W * 4;
     static constexpr int PAIR_STRIDE = 2 * HID + MLP_DIN + 4 + 1;                // hbar, u, a, ybar (+1: odd stride)
     static constexpr int PAIR_BYTES = BWD ? (32 * PAIR_STRIDE * 4 + 15) / 16 * 16 : 0;
     static constexpr int PER_WARP = STAGE_BYTES + LIST_BYTES + MISC_BYTES + PAIR_BYTES;
@@ -123,6 +126,7 @@ __global__ void __launch_bounds__(TRAV_THREADS) radius_mlp_kernel(const __grid_c
     float4* s_q = reinterpret_cast<float4*>(base + SM::STAGE_BYTES + SM::LIST_BYTES);
     int* s_n = reinterpret_cast<int*>(s_q + QB);
     int* s_tot = s_n + QB;
+    float* s_acc = reinterpret_cast<float*>(s_tot + QB);          // [QB][ACC_W] sums of the drain in progress
     float* pairbuf = reinterpret_cast<float*>(base + SM::STAGE_BYTES + SM::LIST_BYTES + SM::MISC_BYTES);
 
     const bool mi0 = MI && p.periodic[0] && p.nc[0] == 1, mi1 = MI && p.periodic[1] && p.nc[1] == 1, mi2 = MI && p.periodic[2] && p.nc[2] == 1;
@@ -164,23 +168,46 @@ __global__ void __launch_bounds__(TRAV_THREADS) radius_mlp_kernel(const __grid_c
                 bool first = first_chunk;
 
                 auto drain = [&]() {
+                    constexpr int ACC_W = SM::ACC_W;
                     __syncwarp();
                     if (lane == 0) {
 #pragma unroll
                         for (int q = 0; q < QB; ++q) { s_n[q] = qcnt[q]; s_tot[q] += qcnt[q]; }
                     }
+                    for (int e = lane; e < QB * ACC_W; e += 32) s_acc[e] = 0.f;
                     __syncwarp();
-                    for (int q = 0; q < nq; ++q) {
-                        const int n = s_n[q];
+                    // The accepted pairs of all queries of the batch form one flat sequence, 32 pairs per step
+                    // whatever the list lengths (a query with a dozen neighbours would otherwise leave most of
+                    // a step idle).  Lanes of one query are neighbours in that sequence, so per-query sums are
+                    // segmented reductions; the first lane of a segment adds the sum to the query's accumulator.
+                    int pre[QB + 1];
+                    pre[0] = 0;
+#pragma unroll
+                    for (int q = 0; q < QB; ++q) pre[q + 1] = pre[q] + (q < nq ? s_n[q] : 0);
+                    const int npairs = pre[QB];
+                    for (int t0 = 0; t0 < npairs; t0 += 32) {
+                        const int f = t0 + lane;
+                        const bool valid = f < npairs;
+                        int q = 0;
+#pragma unroll
+                        for (int j = 1; j < QB; ++j) q += (f >= pre[j]) ? 1 : 0;
+                        q = q < nq ? q : nq - 1;
+                        int tq = 0;
+#pragma unroll
+                        for (int j = 0; j < QB; ++j) tq = (j == q) ? f - pre[j] : tq;
+                        const int key = valid ? q : -1 - lane;               // idle lanes form segments of their own
                         const float4 qv = s_q[q];
                         const int oq = __float_as_int(qv.w);
-                        const int* lq = list + q * MLP_QSTRIDE;
+                        float4 pj = make_float4(0.f, 0.f, 0.f, __int_as_float(0));
+                        if (valid) pj = stage[list[q * MLP_QSTRIDE + tq]];
+                        float dx = pj.x - qv.x, dy = pj.y - qv.y, dz = pj.z - qv.z;      // source minus destination
+                        fold(dx, dy, dz);
+                        constexpr int NV = BWD ? KU : 4;
+                        float red[NV];
+#pragma unroll
+                        for (int i = 0; i < NV; ++i) red[i] = 0.f;
                         if constexpr (!BWD) {
-                            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                            for (int t = lane; t < n; t += 32) {
-                                const float4 pj = stage[lq[t]];
-                                float dx = pj.x - qv.x, dy = pj.y - qv.y, dz = pj.z - qv.z;      // source minus destination
-                                fold(dx, dy, dz);
+                            if (valid) {
                                 float u[KU], h[HID], m[4];
                                 u[0] = dx; u[1] = dy; u[2] = dz;
                                 const float* xr = p.feat + (size_t)__float_as_int(pj.w) * Fin;
@@ -188,95 +215,95 @@ __global__ void __launch_bounds__(TRAV_THREADS) radius_mlp_kernel(const __grid_c
                                 for (int k = 3; k < KU; ++k) u[k] = (k - 3 < Fin) ? __ldg(xr + k - 3) : 0.f;
                                 mlp_forward<HID, KQ>(sW1, sb1, sW2, sb2, u, h, m);
 #pragma unroll
-                                for (int o = 0; o < 4; ++o) acc[o] += m[o];
-                            }
-#pragma unroll
-                            for (int o = 0; o < 4; ++o)
-#pragma unroll
-                                for (int s = 16; s > 0; s >>= 1) acc[o] += __shfl_xor_sync(FULL, acc[o], s);
-                            if (lane < Fout) {
-                                float* dst = p.out + (size_t)oq * Fout + lane;
-                                const float v = lane == 0 ? acc[0] : (lane == 1 ? acc[1] : (lane == 2 ? acc[2] : acc[3]));
-                                *dst = first ? v : *dst + v;
+                                for (int o = 0; o < 4; ++o) red[o] = m[o];
                             }
                         } else {
-                            float gyk[4], xk[KU], gxk[KU], gpk[3] = {0.f, 0.f, 0.f};
+                            float* mine = pairbuf + lane * PS;
+                            if (valid) {
+                                const int om = __float_as_int(pj.w);
+                                float gyk[4], gym[4];
 #pragma unroll
-                            for (int o = 0; o < 4; ++o) gyk[o] = o < Fout ? __ldg(p.gy + (size_t)oq * Fout + o) : 0.f;
-#pragma unroll
-                            for (int k = 0; k < KU; ++k) { xk[k] = (k >= 3 && k - 3 < Fin) ? __ldg(p.feat + (size_t)oq * Fin + k - 3) : 0.f; gxk[k] = 0.f; }
-                            for (int t0 = 0; t0 < n; t0 += 32) {
-                                const int t = t0 + lane;
-                                float* mine = pairbuf + lane * PS;
-                                if (t < n) {
-                                    const float4 pj = stage[lq[t]];
-                                    const int om = __float_as_int(pj.w);
-                                    float dx = pj.x - qv.x, dy = pj.y - qv.y, dz = pj.z - qv.z;
-                                    fold(dx, dy, dz);
-                                    float u[KU], h[HID], m[4], hb[HID], ub[KU];
-                                    // pair (k <- m): parameter gradients and the destination part of pbar_k
-                                    u[0] = dx; u[1] = dy; u[2] = dz;
-                                    const float* xr = p.feat + (size_t)om * Fin;
-#pragma unroll
-                                    for (int k = 3; k < KU; ++k) u[k] = (k - 3 < Fin) ? __ldg(xr + k - 3) : 0.f;
-                                    mlp_forward<HID, KQ>(sW1, sb1, sW2, sb2, u, h, m);
-                                    mlp_backward<HID, KQ>(sW1, sW2, h, gyk, hb, ub);
-                                    gpk[0] -= ub[0]; gpk[1] -= ub[1]; gpk[2] -= ub[2];
-#pragma unroll
-                                    for (int a = 0; a < HID; ++a) { mine[a] = hb[a]; mine[HID + MLP_DIN + a] = fmaxf(h[a], 0.f); }
-#pragma unroll
-                                    for (int k = 0; k < MLP_DIN; ++k) mine[HID + k] = k < KU ? u[k < KU ? k : 0] : 0.f;
-#pragma unroll
-                                    for (int o = 0; o < 4; ++o) mine[2 * HID + MLP_DIN + o] = gyk[o];
-                                    // pair (m <- k): xbar_k and the source part of pbar_k
-                                    float gym[4];
-#pragma unroll
-                                    for (int o = 0; o < 4; ++o) gym[o] = o < Fout ? __ldg(p.gy + (size_t)om * Fout + o) : 0.f;
-                                    u[0] = -dx; u[1] = -dy; u[2] = -dz;
-#pragma unroll
-                                    for (int k = 3; k < KU; ++k) u[k] = xk[k];
-                                    mlp_forward<HID, KQ>(sW1, sb1, sW2, sb2, u, h, m);
-                                    mlp_backward<HID, KQ>(sW1, sW2, h, gym, hb, ub);
-                                    gpk[0] += ub[0]; gpk[1] += ub[1]; gpk[2] += ub[2];
-#pragma unroll
-                                    for (int k = 3; k < KU; ++k) gxk[k] += ub[k];
+                                for (int o = 0; o < 4; ++o) {
+                                    gyk[o] = o < Fout ? __ldg(p.gy + (size_t)oq * Fout + o) : 0.f;
+                                    gym[o] = o < Fout ? __ldg(p.gy + (size_t)om * Fout + o) : 0.f;
                                 }
-                                __syncwarp();
-                                const int np = n - t0 < 32 ? n - t0 : 32;
-                                for (int pp = 0; pp < np; ++pp) {
-                                    const float* pb = pairbuf + pp * PS;
-                                    const float uk = pb[HID + k1];
+                                float u[KU], h[HID], m[4], hb[HID], ub[KU];
+                                // pair (k <- m): parameter gradients and the destination part of pbar_k
+                                u[0] = dx; u[1] = dy; u[2] = dz;
+                                const float* xr = p.feat + (size_t)om * Fin;
 #pragma unroll
-                                    for (int i = 0; i < HID / 2; ++i) gW1acc[i] = fmaf(pb[a0 + 2 * i], uk, gW1acc[i]);
-                                    if (lane < HID) {
-                                        const float act = pb[HID + MLP_DIN + lane];
+                                for (int k = 3; k < KU; ++k) u[k] = (k - 3 < Fin) ? __ldg(xr + k - 3) : 0.f;
+                                mlp_forward<HID, KQ>(sW1, sb1, sW2, sb2, u, h, m);
+                                mlp_backward<HID, KQ>(sW1, sW2, h, gyk, hb, ub);
+                                red[0] = -ub[0]; red[1] = -ub[1]; red[2] = -ub[2];
 #pragma unroll
-                                        for (int o = 0; o < 4; ++o) gW2acc[o] = fmaf(pb[2 * HID + MLP_DIN + o], act, gW2acc[o]);
-                                        gb1acc += pb[lane];
-                                    }
-                                    if (lane < 4) gb2acc += pb[2 * HID + MLP_DIN + lane];
-                                }
-                                __syncwarp();
+                                for (int a = 0; a < HID; ++a) { mine[a] = hb[a]; mine[HID + MLP_DIN + a] = fmaxf(h[a], 0.f); }
+#pragma unroll
+                                for (int k = 0; k < MLP_DIN; ++k) mine[HID + k] = k < KU ? u[k < KU ? k : 0] : 0.f;
+#pragma unroll
+                                for (int o = 0; o < 4; ++o) mine[2 * HID + MLP_DIN + o] = gyk[o];
+                                // pair (m <- k): xbar_k and the source part of pbar_k
+                                const float* xq = p.feat + (size_t)oq * Fin;
+                                u[0] = -dx; u[1] = -dy; u[2] = -dz;
+#pragma unroll
+                                for (int k = 3; k < KU; ++k) u[k] = (k - 3 < Fin) ? __ldg(xq + k - 3) : 0.f;
+                                mlp_forward<HID, KQ>(sW1, sb1, sW2, sb2, u, h, m);
+                                mlp_backward<HID, KQ>(sW1, sW2, h, gym, hb, ub);
+                                red[0] += ub[0]; red[1] += ub[1]; red[2] += ub[2];
+#pragma unroll
+                                for (int k = 3; k < KU; ++k) red[k] = ub[k];
                             }
+                            __syncwarp();
+                            const int np = npairs - t0 < 32 ? npairs - t0 : 32;
+                            for (int pp = 0; pp < np; ++pp) {
+                                const float* pb = pairbuf + pp * PS;
+                                const float uk = pb[HID + k1];
 #pragma unroll
-                            for (int s = 16; s > 0; s >>= 1) {
+                                for (int i = 0; i < HID / 2; ++i) gW1acc[i] = fmaf(pb[a0 + 2 * i], uk, gW1acc[i]);
+                                if (lane < HID) {
+                                    const float act = pb[HID + MLP_DIN + lane];
 #pragma unroll
-                                for (int d = 0; d < 3; ++d) gpk[d] += __shfl_xor_sync(FULL, gpk[d], s);
-#pragma unroll
-                                for (int k = 3; k < KU; ++k) gxk[k] += __shfl_xor_sync(FULL, gxk[k], s);
+                                    for (int o = 0; o < 4; ++o) gW2acc[o] = fmaf(pb[2 * HID + MLP_DIN + o], act, gW2acc[o]);
+                                    gb1acc += pb[lane];
+                                }
+                                if (lane < 4) gb2acc += pb[2 * HID + MLP_DIN + lane];
                             }
-                            if (lane == 0) {
-                                if (p.gpos) {
-                                    float* o = p.gpos + 3 * (size_t)oq;
+                        }
+                        // segmented sums over the lanes of one query
 #pragma unroll
-                                    for (int d = 0; d < 3; ++d) o[d] = first ? gpk[d] : o[d] + gpk[d];
-                                }
-                                if (p.gfeat) {
-                                    float* o = p.gfeat + (size_t)oq * Fin;
+                        for (int d = 1; d < 32; d <<= 1) {
+                            const int kd = __shfl_down_sync(FULL, key, d);
+                            const bool same = lane + d < 32 && kd == key;
 #pragma unroll
-                                    for (int k = 3; k < KU; ++k)
-                                        if (k - 3 < Fin) o[k - 3] = first ? gxk[k] : o[k - 3] + gxk[k];
-                                }
+                            for (int i = 0; i < NV; ++i) {
+                                const float vd = __shfl_down_sync(FULL, red[i], d);
+                                if (same) red[i] += vd;
+                            }
+                        }
+                        const int kprev = __shfl_up_sync(FULL, key, 1);
+                        if (valid && (lane == 0 || kprev != key)) {
+#pragma unroll
+                            for (int i = 0; i < NV; ++i) s_acc[q * ACC_W + i] += red[i];     // one first lane per query and step
+                        }
+                        __syncwarp();
+                    }
+                    // the batch's rows
+                    if constexpr (!BWD) {
+                        const int q = lane >> 2, o = lane & 3;
+                        if (q < nq && o < Fout) {
+                            float* dst = p.out + (size_t)__float_as_int(s_q[q].w) * Fout + o;
+                            const float v = s_acc[q * ACC_W + o];
+                            *dst = first ? v : *dst + v;
+                        }
+                    } else {
+                        for (int e = lane; e < nq * ACC_W; e += 32) {
+                            const int q = e / ACC_W, cidx = e % ACC_W;
+                            const int oq = __float_as_int(s_q[q].w);
+                            const float v = s_acc[e];
+                            if (cidx < 3) {
+                                if (p.gpos) { float* o = p.gpos + 3 * (size_t)oq + cidx; *o = first ? v : *o + v; }
+                            } else if (cidx - 3 < Fin && cidx < KU) {
+                                if (p.gfeat) { float* o = p.gfeat + (size_t)oq * Fin + cidx - 3; *o = first ? v : *o + v; }
                             }
                         }
                     }
