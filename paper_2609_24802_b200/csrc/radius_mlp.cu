@@ -68,26 +68,25 @@ __device__ __forceinline__ void mlp_forward(const float* sW1, const float* sb1, 
     }
 }
 
-// hbar = (W2^T ybar) * [h > 0],  ubar = W1^T hbar
-template <int HID, int KQ>
+// hbar = (W2^T ybar) * [h > 0],  ubar = W1^T hbar.  hbar is consumed entry by entry (and parked in
+// shared memory where the parameter gradients need it), so it never occupies HID registers.
+template <int HID, int KQ, bool STORE>
 __device__ __forceinline__ void mlp_backward(const float* sW1, const float* sW2, const float (&h)[HID], const float (&gy)[4],
-                                             float (&hb)[HID], float (&ub)[4 * KQ]) {
-#pragma unroll
-    for (int a = 0; a < HID; ++a) {
-        float s = sW2[a] * gy[0];
-        s = fmaf(sW2[HID + a], gy[1], s); s = fmaf(sW2[2 * HID + a], gy[2], s); s = fmaf(sW2[3 * HID + a], gy[3], s);
-        hb[a] = h[a] > 0.f ? s : 0.f;
-    }
+                                             float* hb_out, float (&ub)[4 * KQ]) {
 #pragma unroll
     for (int c = 0; c < 4 * KQ; ++c) ub[c] = 0.f;
 #pragma unroll
     for (int a = 0; a < HID; ++a) {
+        float s = sW2[a] * gy[0];
+        s = fmaf(sW2[HID + a], gy[1], s); s = fmaf(sW2[2 * HID + a], gy[2], s); s = fmaf(sW2[3 * HID + a], gy[3], s);
+        const float hb = h[a] > 0.f ? s : 0.f;
+        if (STORE) hb_out[a] = hb;
         const float4* w = reinterpret_cast<const float4*>(sW1 + a * MLP_DIN);
 #pragma unroll
         for (int q = 0; q < KQ; ++q) {
             const float4 w4 = w[q];
-            ub[4 * q] = fmaf(w4.x, hb[a], ub[4 * q]); ub[4 * q + 1] = fmaf(w4.y, hb[a], ub[4 * q + 1]);
-            ub[4 * q + 2] = fmaf(w4.z, hb[a], ub[4 * q + 2]); ub[4 * q + 3] = fmaf(w4.w, hb[a], ub[4 * q + 3]);
+            ub[4 * q] = fmaf(w4.x, hb, ub[4 * q]); ub[4 * q + 1] = fmaf(w4.y, hb, ub[4 * q + 1]);
+            ub[4 * q + 2] = fmaf(w4.z, hb, ub[4 * q + 2]); ub[4 * q + 3] = fmaf(w4.w, hb, ub[4 * q + 3]);
         }
     }
 }
@@ -227,17 +226,17 @@ __global__ void __launch_bounds__(TRAV_THREADS) radius_mlp_kernel(const __grid_c
                                     gyk[o] = o < Fout ? __ldg(p.gy + (size_t)oq * Fout + o) : 0.f;
                                     gym[o] = o < Fout ? __ldg(p.gy + (size_t)om * Fout + o) : 0.f;
                                 }
-                                float u[KU], h[HID], m[4], hb[HID], ub[KU];
+                                float u[KU], h[HID], m[4], ub[KU];
                                 // pair (k <- m): parameter gradients and the destination part of pbar_k
                                 u[0] = dx; u[1] = dy; u[2] = dz;
                                 const float* xr = p.feat + (size_t)om * Fin;
 #pragma unroll
                                 for (int k = 3; k < KU; ++k) u[k] = (k - 3 < Fin) ? __ldg(xr + k - 3) : 0.f;
                                 mlp_forward<HID, KQ>(sW1, sb1, sW2, sb2, u, h, m);
-                                mlp_backward<HID, KQ>(sW1, sW2, h, gyk, hb, ub);
+                                mlp_backward<HID, KQ, true>(sW1, sW2, h, gyk, mine, ub);       // hbar goes straight to the pair buffer
                                 red[0] = -ub[0]; red[1] = -ub[1]; red[2] = -ub[2];
 #pragma unroll
-                                for (int a = 0; a < HID; ++a) { mine[a] = hb[a]; mine[HID + MLP_DIN + a] = fmaxf(h[a], 0.f); }
+                                for (int a = 0; a < HID; ++a) mine[HID + MLP_DIN + a] = fmaxf(h[a], 0.f);
 #pragma unroll
                                 for (int k = 0; k < MLP_DIN; ++k) mine[HID + k] = k < KU ? u[k < KU ? k : 0] : 0.f;
 #pragma unroll
@@ -248,7 +247,7 @@ __global__ void __launch_bounds__(TRAV_THREADS) radius_mlp_kernel(const __grid_c
 #pragma unroll
                                 for (int k = 3; k < KU; ++k) u[k] = (k - 3 < Fin) ? __ldg(xq + k - 3) : 0.f;
                                 mlp_forward<HID, KQ>(sW1, sb1, sW2, sb2, u, h, m);
-                                mlp_backward<HID, KQ>(sW1, sW2, h, gym, hb, ub);
+                                mlp_backward<HID, KQ, false>(sW1, sW2, h, gym, nullptr, ub);
                                 red[0] += ub[0]; red[1] += ub[1]; red[2] += ub[2];
 #pragma unroll
                                 for (int k = 3; k < KU; ++k) red[k] = ub[k];
