@@ -91,8 +91,11 @@ __device__ __forceinline__ void mlp_backward(const float* sW1, const float* sW2,
     }
 }
 
+// resident CTAs per SM the kernel is compiled for (register budget) and launched with (persistent grid)
+template <int HID, bool BWD> constexpr int mlp_ctas_per_sm() { return BWD ? (HID <= 16 ? 3 : 2) : (HID <= 16 ? 4 : 3); }
+
 template <int HID, int KQ, bool BWD, bool MI>
-__global__ void __launch_bounds__(TRAV_THREADS) radius_mlp_kernel(const __grid_constant__ RadiusParams p) {
+__global__ void __launch_bounds__(TRAV_THREADS, mlp_ctas_per_sm<HID, BWD>()) radius_mlp_kernel(const __grid_constant__ RadiusParams p) {
     using SM = MlpSmem<HID, BWD>;
     constexpr unsigned FULL = 0xffffffffu;
     constexpr int KU = 4 * KQ;
@@ -501,7 +504,7 @@ static tiga_status launch_mlp_t(const RadiusParams& p, cudaStream_t s) {
     auto kern = radius_mlp_kernel<HID, KQ, BWD, MI>;
     if (SM::TOTAL > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::TOTAL));
     long long blocks = (p.ncells + TRAV_WARPS - 1) / TRAV_WARPS;
-    const long long cap = 148LL * (BWD ? 2 : 6);       // persistent: parameter gradients are folded once per CTA
+    const long long cap = 148LL * mlp_ctas_per_sm<HID, BWD>();       // persistent: parameter gradients are folded once per CTA
     if (blocks > cap) blocks = cap;
     kern<<<(unsigned)blocks, TRAV_THREADS, SM::TOTAL, s>>>(p);
     return launch_status();
