@@ -251,6 +251,15 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
                 if (lane < nq) {
                     const float4 pq = p.spos[qb0 + lane];
                     lq4 = make_float4(pq.x - org[0], pq.y - org[1], pq.z - org[2], pq.w);
+                    if (MODE == 2) {
+                        // the backward reads the query's own feature and cotangent rows at the start of
+                        // its pass: ask for them now, they arrive during phase A
+                        const size_t rowq = (size_t)__float_as_int(pq.w) * F;
+                        for (int off = 0; off < F; off += 32) {
+                            asm volatile("prefetch.global.L1 [%0];" ::"l"(p.feat + rowq + off));
+                            asm volatile("prefetch.global.L1 [%0];" ::"l"(p.gy + rowq + off));
+                        }
+                    }
                 }
                 s_q[lane] = lq4;
                 s_qc[lane] = lq4.x; s_qc[TQB + lane] = lq4.y; s_qc[2 * TQB + lane] = lq4.z;
