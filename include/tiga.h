@@ -82,6 +82,11 @@ typedef struct {
 
 const char* tiga_status_string(tiga_status s);
 
+/* Number of CUDA kernels this library has launched in this process so far (host-side counter,
+ * all entry points, all devices).  No counterpart in the paper: benchmarks read it before and after
+ * a timed region to state how many of the library's kernels ran inside it. */
+int64_t tiga_kernel_launches(void);
+
 /* ------------------------------------------------------------------------------------ CSR */
 
 /* Bytes of workspace tiga_apply_csr (backward = 0) or tiga_apply_csr_backward (backward = 1)
@@ -126,21 +131,73 @@ tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dtype x_dtype,
  * Same arguments and results as tiga_apply_csr, minus ws / ws_bytes.  Differences:
  *   - Capacity: the call is refused with TIGA_ERR_TOO_LARGE, before anything is launched, when
  *     tiga_csr_workspace_bytes(g, F, x_dtype, reducer, 0) exceeds TIGA_BUILTIN_WS_BYTES
- *     (roughly (n_dst + n_edges) / 2048 * (4 F + 4) bytes, twice the F term for TIGA_MAX;
- *     e.g. 16.8M edges at F = 64 need 2.2 MiB).
+ *     (roughly (n_dst + n_edges) / 2048 * (4 F + 20) bytes plus about 1.5 KiB of padding, twice
+ *     the F term for TIGA_MAX; e.g. 16.8M edges at F = 64 need 2.3 MiB).
  *   - It never calls cudaMalloc, cudaFree or any other allocating routine.
  *   - The first call on each device looks up the array's device address (a host-side lookup,
  *     done with that device current and cached per device).  Make that first call before any
  *     stream capture begins.
  *   - All calls on one device share the one array, and it keeps whatever the previous call
- *     left in it.  Nothing in it has to start at zero: every tile writes its own slot before
- *     the fix-up pass reads it.  Two calls that overlap on the GPU (different streams, or
+ *     left in it.  What must start at zero (the length of the queue of chunks of very long
+ *     rows) is cleared by the call itself; every tile writes its own slot before the fix-up pass
+ *     reads it.  Two calls that overlap on the GPU (different streams, or
  *     different host threads) race on the array and corrupt each other's results; serialise
  *     them, or use tiga_apply_csr with separate workspaces. */
 #define TIGA_BUILTIN_WS_BYTES (8u << 20)
 tiga_status tiga_apply_csr_builtin_ws(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
                                       const float* w, const tiga_msg* msg, tiga_reducer reducer,
                                       float* out, int32_t* argmax, void* stream);
+
+/* Source-block plan: one-time preprocessing of a stored relation whose feature table is far larger
+ * than the L2 cache (the billion-edge relation of Section 7 held in device memory).  It depends on
+ * (rowptr, col) only -- the paper also treats relation set-up as untimed preprocessing (Section 7) --
+ * and regroups the edges by block of source rows and, inside a block, by destination row, keeping
+ * every row's edge order.  tiga_apply_csr_planned then runs one pass per block: all gathers of a
+ * pass fall into one slice of the feature table that stays in L2, and the pass adds one partial sum
+ * to every destination row that has an edge in the block.  The struct is plain data on the HOST; the
+ * arrays it describes live in `plan_buf` on the device at the byte offsets it records (the caller may
+ * move them to a smaller buffer as long as it updates the offsets):
+ *   col     int32 [n_edges]         sources, ordered by (block, destination row, edge position)
+ *   pos     int32 [n_edges]         original edge position of every permuted edge (only when built
+ *                                   with_positions; needed to index edge weights)
+ *   seg_row int32 [n_segments]      destination row of every (row, block) segment
+ *   seg_ptr int32 [n_segments + 1]  extent of every segment in col */
+#define TIGA_PLAN_MAX_BLOCKS 64
+typedef struct {
+    int32_t n_blocks;                                /* power of two, <= TIGA_PLAN_MAX_BLOCKS */
+    int32_t block_shift;                             /* source row j belongs to block j >> block_shift */
+    int32_t has_positions;
+    int32_t reserved;
+    int64_t n_dst, n_src, n_edges, n_segments;
+    int64_t seg_begin[TIGA_PLAN_MAX_BLOCKS + 1];     /* first segment of every block */
+    int64_t huge_segments[TIGA_PLAN_MAX_BLOCKS];     /* segments above 8192 edges, per block */
+    int64_t off_col, off_pos, off_seg_row, off_seg_ptr;   /* byte offsets in plan_buf; off_pos = -1 when absent */
+    int64_t used_bytes;                              /* bytes of plan_buf the plan occupies */
+} tiga_csr_plan;
+
+/* Bytes of plan_buf (worst case: every edge its own segment) and of build scratch.  Host only. */
+size_t tiga_csr_plan_bytes(const tiga_csr* g, int32_t n_blocks, int with_positions);
+size_t tiga_csr_plan_workspace_bytes(const tiga_csr* g, int32_t n_blocks);
+
+/* Builds the plan on the device and SYNCHRONISES the stream (segment counts come back to the host
+ * struct).  Needs n_edges < 2^31 - 1; rowptr int32 or int64.  n_blocks: a power of two; choose it so
+ * that n_src * row bytes / n_blocks is a fraction of the L2 size.  ws is scratch and may be freed
+ * afterwards.  The result is unique (a stable regrouping), so rebuilding gives the same plan. */
+tiga_status tiga_csr_plan_build(const tiga_csr* g, int32_t n_blocks, int with_positions,
+                                void* plan_buf, size_t plan_bytes, void* ws, size_t ws_bytes,
+                                tiga_csr_plan* plan /* host, out */, void* stream);
+
+/* tiga_apply_csr with the sum reducer through a plan: out[i,:] = sum of w[e] x[col[e],:] over row i.
+ * Feature rows of at most 32 bytes (F <= 8 fp32, F <= 16 fp16; TIGA_ERR_UNSUPPORTED above: wider rows
+ * do not need the plan).  w: fp32 [n_edges] in ORIGINAL edge order (plan built with_positions) or NULL.
+ * A row's partial sums are added in block order and long segments are folded in edge order, without
+ * atomics: results are reproducible from run to run (the grouping of the additions differs from
+ * tiga_apply_csr's, so the two agree to rounding, not bit for bit).
+ *   ws : tiga_csr_planned_workspace_bytes(plan, F) bytes of scratch. */
+size_t tiga_csr_planned_workspace_bytes(const tiga_csr_plan* plan, int32_t F);
+tiga_status tiga_apply_csr_planned(const tiga_csr_plan* plan, const void* plan_buf, const void* x, tiga_dtype x_dtype,
+                                   int32_t F, const float* w, const tiga_msg* msg, float* out,
+                                   void* ws, size_t ws_bytes, void* stream);
 
 /* Reverse mode of tiga_apply_csr for fixed relation indices (Section 5):
  *   sum : grad_w[e] = sum_f x[col[e],f] * grad_out[row(e),f]
@@ -250,16 +307,6 @@ tiga_status tiga_apply_radius_mlp_backward(const float* pos, const float* feat, 
                                            float* grad_feat, float* grad_pos,
                                            float* grad_W1, float* grad_b1, float* grad_W2, float* grad_b2,
                                            void* ws, size_t ws_bytes, int reuse_plan, void* stream);
-
-/* Measurement probe, no counterpart in the paper: gathers n_idx rows of row_bytes bytes
- * (a multiple of 16, at most 512) from `table` by index with 128-bit loads, one row per group of
- * row_bytes / 16 lanes, four rows in flight per lane, and folds them into `sink` (fp32 [1]) so
- * that nothing is optimised away.  The benchmark times it on a table that fits L2 to obtain the
- * L2 -> SM gather bandwidth that bounds the stored-relation forward when the gathered rows are
- * cache resident.  table, idx (int32 [n_idx], every entry in [0, n_rows)) and sink are device
- * pointers. */
-tiga_status tiga_probe_row_gather(const void* table, int64_t n_rows, int32_t row_bytes,
-                                  const int32_t* idx, int64_t n_idx, float* sink, void* stream);
 
 /* ----------------------------------------------------------------- stored relation, online-softmax reducer */
 

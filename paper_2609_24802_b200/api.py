@@ -16,10 +16,11 @@ __all__ = [
     "MSG_COPY", "MSG_WEIGHTED", "MSG_GAUSS", "MSG_DIST", "MSG_LJ",
     "CsrRelation", "tiga_status_string", "tiga_csr_workspace_bytes", "tiga_validate_csr",
     "tiga_apply_csr", "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram",
+    "CsrPlan", "tiga_csr_plan_build", "tiga_apply_csr_planned",
     "tiga_radius_grid", "tiga_radius_workspace_bytes", "tiga_radius_bin",
     "tiga_apply_radius", "tiga_apply_radius_backward", "tiga_apply_radius_mlp",
     "tiga_apply_radius_mlp_backward", "tiga_knn_workspace_bytes", "tiga_apply_knn",
-    "tiga_csr_attention_workspace_bytes", "tiga_apply_csr_attention", "tiga_probe_row_gather", "launch_count",
+    "tiga_csr_attention_workspace_bytes", "tiga_apply_csr_attention", "launch_count",
 ]
 
 SUM, MAX = 0, 1
@@ -28,12 +29,13 @@ I32, I64 = 0, 1
 MSG_COPY, MSG_WEIGHTED, MSG_GAUSS, MSG_DIST, MSG_LJ = 0, 1, 2, 3, 4
 
 EXPORTS = [
-    "tiga_status_string", "tiga_csr_workspace_bytes", "tiga_validate_csr", "tiga_apply_csr",
+    "tiga_status_string", "tiga_kernel_launches", "tiga_csr_workspace_bytes", "tiga_validate_csr", "tiga_apply_csr",
     "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram", "tiga_radius_grid",
+    "tiga_csr_plan_bytes", "tiga_csr_plan_workspace_bytes", "tiga_csr_plan_build", "tiga_csr_planned_workspace_bytes",
+    "tiga_apply_csr_planned",
     "tiga_radius_workspace_bytes", "tiga_radius_bin", "tiga_apply_radius",
     "tiga_apply_radius_backward", "tiga_apply_radius_mlp", "tiga_apply_radius_mlp_backward",
     "tiga_knn_workspace_bytes", "tiga_apply_knn", "tiga_csr_attention_workspace_bytes", "tiga_apply_csr_attention",
-    "tiga_probe_row_gather",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -64,8 +66,19 @@ class _EdgeMlp(ctypes.Structure):
                 ("W1", ctypes.c_void_p), ("b1", ctypes.c_void_p), ("W2", ctypes.c_void_p), ("b2", ctypes.c_void_p)]
 
 
+PLAN_MAX_BLOCKS = 64
+
+
+class _Plan(ctypes.Structure):
+    _fields_ = [("n_blocks", ctypes.c_int32), ("block_shift", ctypes.c_int32), ("has_positions", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("n_dst", ctypes.c_int64), ("n_src", ctypes.c_int64),
+                ("n_edges", ctypes.c_int64), ("n_segments", ctypes.c_int64),
+                ("seg_begin", ctypes.c_int64 * (PLAN_MAX_BLOCKS + 1)), ("huge_segments", ctypes.c_int64 * PLAN_MAX_BLOCKS),
+                ("off_col", ctypes.c_int64), ("off_pos", ctypes.c_int64), ("off_seg_row", ctypes.c_int64),
+                ("off_seg_ptr", ctypes.c_int64), ("used_bytes", ctypes.c_int64)]
+
+
 _lib = None
-_launches = 0     # kernels launched by the library through this binding (for benchmarks)
 
 
 def load_library() -> ctypes.CDLL:
@@ -80,6 +93,8 @@ def load_library() -> ctypes.CDLL:
     vp, i32, i64, sz, f = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t, ctypes.c_float
     lib.tiga_status_string.restype = ctypes.c_char_p
     lib.tiga_status_string.argtypes = [ctypes.c_int]
+    lib.tiga_kernel_launches.restype = i64
+    lib.tiga_kernel_launches.argtypes = []
     lib.tiga_csr_workspace_bytes.restype = sz
     lib.tiga_csr_workspace_bytes.argtypes = [ctypes.POINTER(_Csr), i32, ctypes.c_int, ctypes.c_int, ctypes.c_int]
     lib.tiga_validate_csr.restype = ctypes.c_int
@@ -93,6 +108,16 @@ def load_library() -> ctypes.CDLL:
     lib.tiga_apply_csr_backward.restype = ctypes.c_int
     lib.tiga_apply_csr_backward.argtypes = [ctypes.POINTER(_Csr), vp, ctypes.c_int, i32, vp, ctypes.POINTER(_Msg), ctypes.c_int,
                                             vp, vp, vp, vp, vp, sz, vp]
+    lib.tiga_csr_plan_bytes.restype = sz
+    lib.tiga_csr_plan_bytes.argtypes = [ctypes.POINTER(_Csr), i32, ctypes.c_int]
+    lib.tiga_csr_plan_workspace_bytes.restype = sz
+    lib.tiga_csr_plan_workspace_bytes.argtypes = [ctypes.POINTER(_Csr), i32]
+    lib.tiga_csr_plan_build.restype = ctypes.c_int
+    lib.tiga_csr_plan_build.argtypes = [ctypes.POINTER(_Csr), i32, ctypes.c_int, vp, sz, vp, sz, ctypes.POINTER(_Plan), vp]
+    lib.tiga_csr_planned_workspace_bytes.restype = sz
+    lib.tiga_csr_planned_workspace_bytes.argtypes = [ctypes.POINTER(_Plan), i32]
+    lib.tiga_apply_csr_planned.restype = ctypes.c_int
+    lib.tiga_apply_csr_planned.argtypes = [ctypes.POINTER(_Plan), vp, vp, ctypes.c_int, i32, vp, ctypes.POINTER(_Msg), vp, vp, sz, vp]
     lib.tiga_csr_degree_histogram.restype = ctypes.c_int
     lib.tiga_csr_degree_histogram.argtypes = [ctypes.POINTER(_Csr), vp, i64, vp, vp]
     lib.tiga_radius_grid.restype = ctypes.c_int
@@ -111,8 +136,6 @@ def load_library() -> ctypes.CDLL:
     lib.tiga_apply_radius_mlp_backward.restype = ctypes.c_int
     lib.tiga_apply_radius_mlp_backward.argtypes = [vp, vp, i64, f, ctypes.POINTER(_Box), ctypes.POINTER(_EdgeMlp), vp,
                                                    vp, vp, vp, vp, vp, vp, vp, sz, ctypes.c_int, vp]
-    lib.tiga_probe_row_gather.restype = ctypes.c_int
-    lib.tiga_probe_row_gather.argtypes = [vp, i64, i32, vp, i64, vp, vp]
     lib.tiga_csr_attention_workspace_bytes.restype = sz
     lib.tiga_csr_attention_workspace_bytes.argtypes = [ctypes.POINTER(_Csr), i32]
     lib.tiga_apply_csr_attention.restype = ctypes.c_int
@@ -129,7 +152,8 @@ load_library()      # fail at import time, loudly, when the CUDA library is not 
 
 
 def launch_count() -> int:
-    return _launches
+    """Kernels launched by the library so far in this process (counted inside the library)."""
+    return int(load_library().tiga_kernel_launches())
 
 
 def _ptr(t):
@@ -192,16 +216,8 @@ def tiga_validate_csr(g: CsrRelation, level: int = 1, stream=None) -> None:
     _ok(load_library().tiga_validate_csr(g.ref, level, _ptr(ws), ws.numel(), _stream(stream)), "tiga_validate_csr")
 
 
-def _csr_forward_launches(x) -> int:
-    """Kernels one forward call launches: tile kernel + fix-up, or the three row-class kernels
-    when a feature row is at most 32 bytes."""
-    row_bytes = x.shape[1] * x.element_size()
-    return 3 if row_bytes <= 32 else 2
-
-
 def tiga_apply_csr(g: CsrRelation, x, w=None, reducer: int = SUM, out=None, argmax=None, ws=None, stream=None):
     """out[i,:] = reduce over the row's edges of w[e] * x[col[e],:].  Returns (out, argmax)."""
-    global _launches
     F = x.shape[1]
     if out is None:
         out = torch.empty((g.n_dst, F), dtype=torch.float32, device=x.device)
@@ -212,7 +228,6 @@ def tiga_apply_csr(g: CsrRelation, x, w=None, reducer: int = SUM, out=None, argm
     msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)
     _ok(load_library().tiga_apply_csr(g.ref, _ptr(x), _dt(x), F, _ptr(w), ctypes.byref(msg), reducer, _ptr(out),
                                       _ptr(argmax), _ptr(ws), ws.numel(), _stream(stream)), "tiga_apply_csr")
-    _launches += _csr_forward_launches(x)
     return out, argmax
 
 
@@ -225,7 +240,6 @@ def tiga_apply_csr_builtin_ws(g: CsrRelation, x, w=None, reducer: int = SUM, out
     relation needs more than that.  Calls that overlap on the GPU race on the shared array.
     `out` (and `argmax` for MAX) should be passed in by such callers; they are created here only
     as a convenience when omitted.  Returns (out, argmax)."""
-    global _launches
     F = x.shape[1]
     if out is None:
         out = torch.empty((g.n_dst, F), dtype=torch.float32, device=x.device)
@@ -234,14 +248,12 @@ def tiga_apply_csr_builtin_ws(g: CsrRelation, x, w=None, reducer: int = SUM, out
     msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)
     _ok(load_library().tiga_apply_csr_builtin_ws(g.ref, _ptr(x), _dt(x), F, _ptr(w), ctypes.byref(msg), reducer,
                                                  _ptr(out), _ptr(argmax), _stream(stream)), "tiga_apply_csr_builtin_ws")
-    _launches += _csr_forward_launches(x)
     return out, argmax
 
 
 def tiga_apply_csr_backward(g: CsrRelation, x, w, grad_out, reducer: int = SUM, argmax=None,
                             grad_x=None, grad_w=None, want_x=True, want_w=True, ws=None, stream=None):
     """Returns (grad_x, grad_w); either is None when not requested."""
-    global _launches
     F = x.shape[1]
     if want_x and grad_x is None:
         grad_x = torch.empty((g.n_src, F), dtype=torch.float32, device=x.device)
@@ -253,18 +265,76 @@ def tiga_apply_csr_backward(g: CsrRelation, x, w, grad_out, reducer: int = SUM, 
     _ok(load_library().tiga_apply_csr_backward(g.ref, _ptr(x), _dt(x), F, _ptr(w), ctypes.byref(msg), reducer, _ptr(grad_out),
                                                _ptr(argmax), _ptr(grad_x), _ptr(grad_w), _ptr(ws), ws.numel(),
                                                _stream(stream)), "tiga_apply_csr_backward")
-    _launches += 1
     return grad_x, grad_w
+
+
+class CsrPlan:
+    """A built source-block plan: the host struct ``tiga_csr_plan`` plus the device buffer it describes."""
+
+    def __init__(self, c, buf, scratch_bytes):
+        self.c, self.buf, self.scratch_bytes = c, buf, int(scratch_bytes)
+
+    n_blocks = property(lambda self: int(self.c.n_blocks))
+    n_segments = property(lambda self: int(self.c.n_segments))
+    nbytes = property(lambda self: int(self.c.used_bytes))
+
+    def array(self, name):
+        """View of one of the plan's device arrays: 'col', 'pos', 'seg_row', 'seg_ptr'."""
+        off = {"col": self.c.off_col, "pos": self.c.off_pos, "seg_row": self.c.off_seg_row, "seg_ptr": self.c.off_seg_ptr}[name]
+        if off < 0:
+            return None
+        n = {"col": self.c.n_edges, "pos": self.c.n_edges, "seg_row": self.c.n_segments, "seg_ptr": self.c.n_segments + 1}[name]
+        return self.buf[off:off + 4 * n].view(torch.int32)
+
+
+def tiga_csr_plan_build(g: CsrRelation, row_bytes: int = 16, n_blocks: int = None, with_positions: bool = False,
+                        block_bytes: int = 32 << 20, stream=None) -> CsrPlan:
+    """Builds the source-block plan of a relation (one-time, synchronises).  ``n_blocks`` defaults to the
+    power of two that makes a block of source rows about ``block_bytes`` of feature table."""
+    lib = load_library()
+    if n_blocks is None:
+        n_blocks = 1
+        while n_blocks < PLAN_MAX_BLOCKS and g.n_src * row_bytes > n_blocks * block_bytes:
+            n_blocks *= 2
+    nbytes = int(lib.tiga_csr_plan_bytes(g.ref, n_blocks, int(with_positions)))
+    wbytes = int(lib.tiga_csr_plan_workspace_bytes(g.ref, n_blocks))
+    if nbytes == 0:
+        raise TigaError(2, "tiga_csr_plan_bytes")
+    buf = torch.empty(nbytes, dtype=torch.uint8, device=g.col.device)
+    ws = torch.empty(wbytes, dtype=torch.uint8, device=g.col.device)
+    c = _Plan()
+    _ok(lib.tiga_csr_plan_build(g.ref, n_blocks, int(with_positions), _ptr(buf), nbytes, _ptr(ws), wbytes,
+                                ctypes.byref(c), _stream(stream)), "tiga_csr_plan_build")
+    del ws
+    # the worst-case buffer shrinks to what the plan uses: move the two segment arrays up behind the edges
+    used = int(c.used_bytes)
+    if used < nbytes:
+        small = torch.empty(used, dtype=torch.uint8, device=buf.device)
+        small.copy_(buf[:used])
+        buf = small
+    return CsrPlan(c, buf, wbytes)
+
+
+def tiga_apply_csr_planned(plan: CsrPlan, x, w=None, out=None, ws=None, stream=None):
+    """Sum forward through a source-block plan.  Returns out."""
+    F = x.shape[1]
+    lib = load_library()
+    if out is None:
+        out = torch.empty((plan.c.n_dst, F), dtype=torch.float32, device=x.device)
+    if ws is None:
+        ws = _ws(lib.tiga_csr_planned_workspace_bytes(ctypes.byref(plan.c), F), x)
+    msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)
+    _ok(lib.tiga_apply_csr_planned(ctypes.byref(plan.c), _ptr(plan.buf), _ptr(x), _dt(x), F, _ptr(w), ctypes.byref(msg),
+                                   _ptr(out), _ptr(ws), ws.numel(), _stream(stream)), "tiga_apply_csr_planned")
+    return out
 
 
 def tiga_csr_degree_histogram(g: CsrRelation, nbins: int = 4096, stream=None):
     """Returns (hist int64[nbins], max_degree int64[1]) as device tensors."""
-    global _launches
     hist = torch.empty(nbins, dtype=torch.int64, device=g.rowptr.device)
     mx = torch.empty(1, dtype=torch.int64, device=g.rowptr.device)
     _ok(load_library().tiga_csr_degree_histogram(g.ref, _ptr(hist), nbins, _ptr(mx), _stream(stream)),
         "tiga_csr_degree_histogram")
-    _launches += 1
     return hist, mx
 
 
@@ -292,7 +362,6 @@ def tiga_radius_workspace_bytes(n: int, F: int, r: float, box, periodic, backwar
 
 def tiga_radius_bin(pos, r: float, box, periodic, ws=None, stream=None):
     """Returns dict(cell, cell_start, order, ncell, ws)."""
-    global _launches
     n = pos.shape[0]
     b = _box(box, periodic)
     ncell, _ = tiga_radius_grid(n, r, box, periodic)
@@ -304,14 +373,12 @@ def tiga_radius_bin(pos, r: float, box, periodic, ws=None, stream=None):
         ws = _ws(tiga_radius_workspace_bytes(n, 0, r, box, periodic), pos)
     _ok(load_library().tiga_radius_bin(_ptr(pos), n, float(r), ctypes.byref(b), _ptr(cell), _ptr(start),
                                        _ptr(order), _ptr(ws), ws.numel(), _stream(stream)), "tiga_radius_bin")
-    _launches += 6
     return dict(cell=cell, cell_start=start, order=order, ncell=ncell, ws=ws)
 
 
 def tiga_apply_radius(pos, feat, r: float, box, periodic, kind: int = MSG_GAUSS, p0: float = 1.0,
                       p1: float = 1.0, out=None, count=None, want_count=False, ws=None, stream=None):
     """Fused bin + traverse + message + sum.  Returns (out, count, ws)."""
-    global _launches
     n = pos.shape[0]
     F = 4 if kind == MSG_LJ else feat.shape[1]
     b = _box(box, periodic)
@@ -324,7 +391,6 @@ def tiga_apply_radius(pos, feat, r: float, box, periodic, kind: int = MSG_GAUSS,
     _ok(load_library().tiga_apply_radius(_ptr(pos), _ptr(feat), n, F, float(r), ctypes.byref(b),
                                          ctypes.byref(_Msg(kind, float(p0), float(p1))), _ptr(out), _ptr(count), _ptr(ws),
                                          ws.numel(), _stream(stream)), "tiga_apply_radius")
-    _launches += 7
     return out, count, ws
 
 
@@ -332,7 +398,6 @@ def tiga_apply_radius_backward(pos, feat, grad_out, r: float, box, periodic, sig
                                reuse_plan=False, grad_feat=None, grad_pos=None, want_feat=True, want_pos=True,
                                stream=None):
     """Reverse mode of the Gaussian message.  Returns (grad_feat, grad_pos)."""
-    global _launches
     n, F = feat.shape
     b = _box(box, periodic)
     if want_feat and grad_feat is None:
@@ -347,7 +412,6 @@ def tiga_apply_radius_backward(pos, feat, grad_out, r: float, box, periodic, sig
                                                   _ptr(grad_feat), _ptr(grad_pos), _ptr(ws), ws.numel(),
                                                   int(bool(reuse_plan)), _stream(stream)),
         "tiga_apply_radius_backward")
-    _launches += 1 if reuse_plan else 7
     return grad_feat, grad_pos
 
 
@@ -361,7 +425,6 @@ def _edge_mlp(W1, b1, W2, b2):
 def tiga_apply_radius_mlp(pos, feat, r: float, box, periodic, W1, b1, W2, b2, out=None, count=None,
                           want_count=False, ws=None, stream=None):
     """out[i] = sum_{j in N(i)} [W2 relu(W1 [p_j - p_i; x_j] + b1) + b2].  Returns (out, count, ws)."""
-    global _launches
     n = pos.shape[0]
     m = _edge_mlp(W1, b1, W2, b2)
     bx = _box(box, periodic)
@@ -374,14 +437,12 @@ def tiga_apply_radius_mlp(pos, feat, r: float, box, periodic, W1, b1, W2, b2, ou
     _ok(load_library().tiga_apply_radius_mlp(_ptr(pos), _ptr(feat), n, float(r), ctypes.byref(bx), ctypes.byref(m),
                                              _ptr(out), _ptr(count), _ptr(ws), ws.numel(), _stream(stream)),
         "tiga_apply_radius_mlp")
-    _launches += 7
     return out, count, ws
 
 
 def tiga_apply_radius_mlp_backward(pos, feat, grad_out, r: float, box, periodic, W1, b1, W2, b2, ws=None,
                                    reuse_plan=False, stream=None):
     """Returns dict(grad_feat, grad_pos, grad_W1, grad_b1, grad_W2, grad_b2)."""
-    global _launches
     n = pos.shape[0]
     m = _edge_mlp(W1, b1, W2, b2)
     bx = _box(box, periodic)
@@ -397,7 +458,6 @@ def tiga_apply_radius_mlp_backward(pos, feat, grad_out, r: float, box, periodic,
                                                       _ptr(g["grad_W1"]), _ptr(g["grad_b1"]), _ptr(g["grad_W2"]),
                                                       _ptr(g["grad_b2"]), _ptr(ws), ws.numel(), int(bool(reuse_plan)),
                                                       _stream(stream)), "tiga_apply_radius_mlp_backward")
-    _launches += 1 if reuse_plan else 7
     return g
 
 
@@ -410,7 +470,6 @@ def tiga_apply_knn(pos, feat, k: int, box, periodic=(0, 0, 0), out=None, nbr=Non
                    want_nbr=True, ws=None, stream=None):
     """out[i] = sum of feat[j] over the k nearest j != i by the key (fp32 squared distance, index).
     Returns (out, nbr int32 [n,k] or None, nbr_d2 fp32 [n,k] or None, ws)."""
-    global _launches
     n, F = feat.shape
     b = _box(box, periodic)
     dev = pos.device
@@ -424,7 +483,6 @@ def tiga_apply_knn(pos, feat, k: int, box, periodic=(0, 0, 0), out=None, nbr=Non
         ws = _ws(tiga_knn_workspace_bytes(n, k, box), pos)
     _ok(load_library().tiga_apply_knn(_ptr(pos), _ptr(feat), n, F, int(k), ctypes.byref(b), _ptr(out), _ptr(nbr),
                                       _ptr(nbr_d2), _ptr(ws), ws.numel(), _stream(stream)), "tiga_apply_knn")
-    _launches += 8
     return out, nbr, nbr_d2, ws
 
 
@@ -436,7 +494,6 @@ def tiga_apply_csr_attention(g: CsrRelation, q, key, value, scale: float, out=No
                              ws=None, stream=None):
     """out[i] = sum_e softmax_e(scale * <q[i], key[col[e]]>) value[col[e]] over the edges of row i
     (online-softmax reducer).  Returns (out, lse, ws)."""
-    global _launches
     D = q.shape[1]
     if out is None:
         out = torch.empty((g.n_dst, D), dtype=torch.float32, device=q.device)
@@ -446,16 +503,4 @@ def tiga_apply_csr_attention(g: CsrRelation, q, key, value, scale: float, out=No
         ws = _ws(tiga_csr_attention_workspace_bytes(g, D), q)
     _ok(load_library().tiga_apply_csr_attention(g.ref, _ptr(q), _ptr(key), _ptr(value), D, float(scale), _ptr(out),
                                                 _ptr(lse), _ptr(ws), ws.numel(), _stream(stream)), "tiga_apply_csr_attention")
-    _launches += 2
     return out, lse, ws
-
-
-def tiga_probe_row_gather(table, idx, sink, stream=None) -> None:
-    """Measurement probe: gathers table[idx[k], :] for every k (rows of 16..512 bytes) and folds
-    them into sink[0]; timed by the benchmark to obtain the L2 -> SM gather ceiling."""
-    global _launches
-    n_rows = table.shape[0]
-    row_bytes = table.shape[1] * table.element_size()
-    _ok(load_library().tiga_probe_row_gather(_ptr(table), n_rows, row_bytes, _ptr(idx), idx.numel(), _ptr(sink),
-                                             _stream(stream)), "tiga_probe_row_gather")
-    _launches += 1

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(HERE, "libtiga.so")
-SOURCES = ["csr.cu", "csr_attention.cu", "radius.cu", "radius_lj.cu", "radius_mlp.cu", "knn.cu"]
+SOURCES = ["csr.cu", "csr_plan.cu", "csr_attention.cu", "radius.cu", "radius_lj.cu", "radius_mlp.cu", "knn.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I" + INCLUDE, "-I" + CSRC]
 
@@ -51,7 +51,18 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
                     raise RuntimeError("nvcc failed")
     if force or jobs or _stale(LIB, objs):
         subprocess.check_call([_nvcc(), "-shared", "-o", LIB] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
+    build_bench_probe(force)
     return LIB
+
+
+def build_bench_probe(force: bool = False) -> str:
+    """The benchmark's row-gather probe is a library of its own: it measures, it is not product."""
+    src = os.path.join(HERE, "bench_probe", "row_gather_probe.cu")
+    lib = os.path.join(HERE, "bench_probe", "libtiga_bench_probe.so")
+    if force or _stale(lib, [src]):
+        subprocess.check_call([_nvcc(), "-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
+                               "-Xcompiler", "-fPIC", "-shared", src, "-o", lib])
+    return lib
 
 
 if __name__ == "__main__":

@@ -18,6 +18,12 @@ static inline tiga_status launch_status() {
     return cudaPeekAtLastError() == cudaSuccess ? TIGA_OK : TIGA_ERR_CUDA;
 }
 
+// Every kernel launch of the library goes through counted(): the grid size passes through unchanged
+// and the process-wide launch counter (read by tiga_kernel_launches) goes up by one.
+void note_launch();
+template <typename T>
+static inline T counted(T grid) { note_launch(); return grid; }
+
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

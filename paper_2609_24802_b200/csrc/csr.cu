@@ -4,7 +4,8 @@
 // Schedule (ours, not the paper's bounded-ragged Triton tile of Section 4.4):
 //   * The merged sequence "row ends + edges" (N + E items) is cut into equal tiles, one CTA
 //     per tile, so neither a 69k-edge row nor a run of a million empty rows unbalances a CTA
-//     (Section 4.4: "a high-degree split requires explicit partial states and a legal merge").
+//     (a long row is split into partial states that are merged in edge order, the obligation
+//     Section 4.4 attaches to splitting high-degree rows).
 //   * A CTA stages its slice of rowptr, col and w in shared memory with coalesced streaming
 //     loads, then splits its edges evenly over "workers" of G lanes.  A worker walks its edge
 //     span in order; each lane owns 16 bytes of the feature row, so one gathered source row
@@ -16,9 +17,13 @@
 //     fix-up kernel folds into the row, again in edge order.  No atomics in the forward, so
 //     results are reproducible.
 #include "csr_shared.cuh"
+#include <atomic>
 #include <mutex>
 
 namespace tiga {
+
+static std::atomic<long long> g_kernel_launches{0};
+void note_launch() { g_kernel_launches.fetch_add(1, std::memory_order_relaxed); }
 
 // --------------------------------------------------------------------------------------------
 // Forward.  G lanes per worker, VPL 16-byte vectors per lane, RED = 0 sum / 1 max.
@@ -263,7 +268,6 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
 // The summation tree is fixed, so results are reproducible.
 // --------------------------------------------------------------------------------------------
 constexpr int ROW_SHORT = 16;
-constexpr int ROW_HUGE = 8192;
 
 template <int RED, int NV, int VW>
 __device__ __forceinline__ void tree_merge(State<RED, NV, VW>& s) {
@@ -300,7 +304,7 @@ __device__ __forceinline__ State<RED, NV, XTraits<XT>::VW> warp_row(const CsrPar
             const bool in = k + 32 * u < n;
             const long long e = es + (in ? k + 32 * u : k);
             const long long c = ld_stream(p.col + e);
-            wv[u] = p.w ? ld_stream(p.w + e) : 1.f;
+            wv[u] = p.w ? ld_stream(p.w + (p.epos ? (long long)ld_stream(p.epos + e) : e)) : 1.f;
 #pragma unroll
             for (int i = 0; i < NV; ++i) xv[u][i] = in ? __ldg(xbase + c * p.nvec + i) : make_uint4(0, 0, 0, 0);
         }
@@ -321,21 +325,27 @@ __device__ __forceinline__ State<RED, NV, XTraits<XT>::VW> warp_row(const CsrPar
     return s;
 }
 
-template <typename XT, int NV, int RED>
+// ACC: the state is added to what the row already holds (planned apply: one segment of a row per pass)
+template <typename XT, int NV, int RED, bool ACC = false>
 __device__ __forceinline__ void store_state(const CsrParams& p, float* out, int32_t* arg, const State<RED, NV, XTraits<XT>::VW>& s) {
     constexpr int VW = XTraits<XT>::VW;
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
 #pragma unroll
         for (int k = 0; k < VW; k += 4) {
-            st_stream(reinterpret_cast<float4*>(out + i * VW + k), make_float4(s.v[i][k], s.v[i][k + 1], s.v[i][k + 2], s.v[i][k + 3]));
+            float4 v = make_float4(s.v[i][k], s.v[i][k + 1], s.v[i][k + 2], s.v[i][k + 3]);
+            if constexpr (ACC) {
+                const float4 old = ld_stream(reinterpret_cast<const float4*>(out + i * VW + k));
+                v.x += old.x; v.y += old.y; v.z += old.z; v.w += old.w;
+            }
+            st_stream(reinterpret_cast<float4*>(out + i * VW + k), v);
             if constexpr (RED != 0)
                 st_stream(reinterpret_cast<int4*>(arg + i * VW + k), make_int4(s.a[i][k], s.a[i][k + 1], s.a[i][k + 2], s.a[i][k + 3]));
         }
     }
 }
 
-template <typename XT, int NV, int RED, typename IT>
+template <typename XT, int NV, int RED, typename IT, bool ACC = false>
 __global__ void __launch_bounds__(CSR_THREADS) csr_rows_kernel(const CsrParams p) {
     constexpr int VW = XTraits<XT>::VW;
     constexpr unsigned FULL = 0xffffffffu;
@@ -362,7 +372,7 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_rows_kernel(const CsrParams p
                 const bool in = k + u < n;
                 const long long e = es + (in ? k + u : k);
                 const long long c = __ldg(p.col + e);
-                wv[u] = p.w ? __ldg(p.w + e) : 1.f;
+                wv[u] = p.w ? __ldg(p.w + (p.epos ? (long long)__ldg(p.epos + e) : e)) : 1.f;
 #pragma unroll
                 for (int i = 0; i < NV; ++i) xv[u][i] = in ? __ldg(xbase + c * p.nvec + i) : make_uint4(0, 0, 0, 0);
             }
@@ -405,7 +415,10 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_rows_kernel(const CsrParams p
         const long long rs = q_start[idx];
         const int rn = q_len[idx];
         const St tot = warp_row<XT, NV, RED>(p, rs, rn, lane);
-        if (lane == 0) store_state<XT, NV, RED>(p, p.out + r * p.F, RED ? p.arg + r * p.F : nullptr, tot);
+        if (lane == 0) {
+            const long long orow = ACC ? (long long)p.row_map[r] : r;
+            store_state<XT, NV, RED, ACC>(p, p.out + orow * p.F, RED ? p.arg + orow * p.F : nullptr, tot);
+        }
     }
     // huge rows: queue their chunks
     if (valid && deg > ROW_HUGE) {
@@ -413,8 +426,10 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_rows_kernel(const CsrParams p
         const int base = atomicAdd(p.huge_count, chunks);
         for (int c = 0; c < chunks; ++c) p.huge_list[base + c] = make_int4((int)row, c, chunks, base);
     }
-    if (valid && deg <= ROW_SHORT)
-        store_state<XT, NV, RED>(p, p.out + row * p.F, RED ? p.arg + row * p.F : nullptr, st);
+    if (valid && deg <= ROW_SHORT) {
+        const long long orow = ACC ? (long long)p.row_map[row] : row;
+        store_state<XT, NV, RED, ACC>(p, p.out + orow * p.F, RED ? p.arg + orow * p.F : nullptr, st);
+    }
 }
 
 // one warp per queued chunk of a huge row
@@ -436,7 +451,7 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_huge_chunks_kernel(const CsrP
 }
 
 // fold the chunk states of every huge row in chunk (= edge) order; one thread per (row, feature)
-template <int RED>
+template <int RED, bool ACC = false>
 __global__ void csr_huge_fold_kernel(const CsrParams p) {
     const int total = *p.huge_count;
     const long long nthreads = (long long)gridDim.x * blockDim.x;
@@ -454,8 +469,10 @@ __global__ void csr_huge_fold_kernel(const CsrParams p) {
                 if (oa >= 0 && (a < 0 || ov > v)) { v = ov; a = oa; }
             }
         }
-        p.out[(size_t)ent.x * p.F + f] = v;
-        if (RED) p.arg[(size_t)ent.x * p.F + f] = a;
+        const size_t orow = ACC ? (size_t)p.row_map[ent.x] : (size_t)ent.x;
+        if (ACC) v += p.out[orow * p.F + f];
+        p.out[orow * p.F + f] = v;
+        if (RED) p.arg[orow * p.F + f] = a;
     }
 }
 
@@ -494,7 +511,7 @@ __global__ void csr_fixup_kernel(const CsrParams p) {
 
 // --------------------------------------------------------------------------------------------
 // Backward, sum reducer (Section 5).  Same tiles and workers; every edge is independent:
-//   gw[e] = x[col[e],:] . gy[row,:]            (edge gradients retain edge identity)
+//   gw[e] = x[col[e],:] . gy[row,:]            (one value per edge position, duplicates not merged)
 //   gx[col[e],:] += w[e] * gy[row,:]           (reverse incidence: vector atomics)
 // --------------------------------------------------------------------------------------------
 template <int G, int VPL, typename IT>
@@ -648,28 +665,6 @@ __global__ void degree_hist_kernel(const IT* __restrict__ rowptr, long long n, i
         if (s_hist[k]) atomicAdd(hist + k, (unsigned long long)s_hist[k]);
 }
 
-// Measurement probe: index-driven row gathers with the access shape of the forward (one row per
-// group of LN lanes, 128-bit loads, four rows in flight), folded into one number.
-template <int LN>
-__global__ void __launch_bounds__(256) row_gather_probe_kernel(const uint4* __restrict__ table, const int32_t* __restrict__ idx,
-                                                               long long n_idx, float* sink) {
-    const int ln = threadIdx.x % LN;
-    const long long groups = (long long)gridDim.x * (blockDim.x / LN);
-    const long long g0 = (long long)blockIdx.x * (blockDim.x / LN) + threadIdx.x / LN;
-    float acc = 0.f;
-    for (long long k = g0 * 4; k < n_idx; k += groups * 4) {
-        uint4 v[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const long long kk = k + u < n_idx ? k + u : k;
-            v[u] = __ldg(table + (unsigned long long)(unsigned)__ldg(idx + kk) * LN + ln);
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) acc += __uint_as_float(v[u].x) + __uint_as_float(v[u].y) + __uint_as_float(v[u].z) + __uint_as_float(v[u].w);
-    }
-    if (acc == 123.456f) atomicAdd(sink, acc);      // keeps the loads alive; practically never taken
-}
-
 template <typename IT>
 __global__ void validate_kernel(const IT* __restrict__ rowptr, const int32_t* __restrict__ col,
                                 long long n_dst, long long n_src, long long n_edges, int* flags) {
@@ -714,7 +709,7 @@ static tiga_status launch_fwd_t(const CsrParams& p, cudaStream_t s) {
     const size_t dyn = (size_t)2 * NW * G * VPL * XTraits<XT>::VW * sizeof(float) * (RED ? 2 : 1);
     auto kern = p.nvec == G * VPL ? csr_forward_kernel<XT, G, VPL, RED, IT, true> : csr_forward_kernel<XT, G, VPL, RED, IT, false>;
     if (dyn > 16 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
-    kern<<<(unsigned)p.ntiles, CSR_THREADS, dyn, s>>>(p);
+    kern<<<counted((unsigned)p.ntiles), CSR_THREADS, dyn, s>>>(p);
     return launch_status();
 }
 
@@ -724,13 +719,13 @@ static tiga_status launch_fwd_g(const CsrParams& p, int G, int VPL, cudaStream_t
         TIGA_CUDA_TRY(cudaMemsetAsync(p.huge_count, 0, sizeof(int), s));
         const unsigned blocks = (unsigned)((p.n_dst + CSR_THREADS - 1) / CSR_THREADS);
         if (p.nvec == 1) {
-            csr_rows_kernel<XT, 1, RED, IT><<<blocks, CSR_THREADS, 0, s>>>(p);
-            csr_huge_chunks_kernel<XT, 1, RED, IT><<<148 * 8, CSR_THREADS, 0, s>>>(p);
+            csr_rows_kernel<XT, 1, RED, IT><<<counted(blocks), CSR_THREADS, 0, s>>>(p);
+            csr_huge_chunks_kernel<XT, 1, RED, IT><<<counted(148 * 8), CSR_THREADS, 0, s>>>(p);
         } else {
-            csr_rows_kernel<XT, 2, RED, IT><<<blocks, CSR_THREADS, 0, s>>>(p);
-            csr_huge_chunks_kernel<XT, 2, RED, IT><<<148 * 8, CSR_THREADS, 0, s>>>(p);
+            csr_rows_kernel<XT, 2, RED, IT><<<counted(blocks), CSR_THREADS, 0, s>>>(p);
+            csr_huge_chunks_kernel<XT, 2, RED, IT><<<counted(148 * 8), CSR_THREADS, 0, s>>>(p);
         }
-        csr_huge_fold_kernel<RED><<<148 * 2, 256, 0, s>>>(p);
+        csr_huge_fold_kernel<RED><<<counted(148 * 2), 256, 0, s>>>(p);
         return launch_status();
     }
     switch (G) {
@@ -748,7 +743,7 @@ static tiga_status launch_fwd_g(const CsrParams& p, int G, int VPL, cudaStream_t
 
 template <typename IT>
 static tiga_status launch_bwd_g(const CsrParams& p, int G, int VPL, cudaStream_t s) {
-#define TIGA_BWD(GG, VV) csr_backward_sum_kernel<GG, VV, IT><<<(unsigned)p.ntiles, CSR_THREADS, 0, s>>>(p); break
+#define TIGA_BWD(GG, VV) csr_backward_sum_kernel<GG, VV, IT><<<counted((unsigned)p.ntiles), CSR_THREADS, 0, s>>>(p); break
     switch (G) {
         case 1: TIGA_BWD(1, 1);
         case 2: TIGA_BWD(2, 1);
@@ -812,9 +807,9 @@ extern "C" tiga_status tiga_validate_csr(const tiga_csr* g, int level, void* ws,
     if (blocks > 148 * 16) blocks = 148 * 16;
     if (blocks < 1) blocks = 1;
     if (g->rowptr_type == TIGA_I32)
-        validate_kernel<int32_t><<<(unsigned)blocks, 256, 0, s>>>(static_cast<const int32_t*>(g->rowptr), g->col, g->n_dst, g->n_src, g->n_edges, flags);
+        validate_kernel<int32_t><<<counted((unsigned)blocks), 256, 0, s>>>(static_cast<const int32_t*>(g->rowptr), g->col, g->n_dst, g->n_src, g->n_edges, flags);
     else
-        validate_kernel<int64_t><<<(unsigned)blocks, 256, 0, s>>>(static_cast<const int64_t*>(g->rowptr), g->col, g->n_dst, g->n_src, g->n_edges, flags);
+        validate_kernel<int64_t><<<counted((unsigned)blocks), 256, 0, s>>>(static_cast<const int64_t*>(g->rowptr), g->col, g->n_dst, g->n_src, g->n_edges, flags);
     if (launch_status() != TIGA_OK) return TIGA_ERR_CUDA;
     int h = 0;
     TIGA_CUDA_TRY(cudaMemcpyAsync(&h, flags, sizeof(int), cudaMemcpyDeviceToHost, s));
@@ -867,8 +862,8 @@ extern "C" tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dty
     if (st != TIGA_OK) return st;
     if (nvec <= 2) return TIGA_OK;             // the row-class path has no tile carry-outs
     const long long work = p.ntiles * F;
-    if (reducer == TIGA_SUM) csr_fixup_kernel<0><<<(unsigned)((work + 255) / 256), 256, 0, s>>>(p);
-    else csr_fixup_kernel<1><<<(unsigned)((work + 255) / 256), 256, 0, s>>>(p);
+    if (reducer == TIGA_SUM) csr_fixup_kernel<0><<<counted((unsigned)((work + 255) / 256)), 256, 0, s>>>(p);
+    else csr_fixup_kernel<1><<<counted((unsigned)((work + 255) / 256)), 256, 0, s>>>(p);
     return launch_status();
 }
 
@@ -910,6 +905,75 @@ extern "C" tiga_status tiga_apply_csr_builtin_ws(const tiga_csr* g, const void* 
     return tiga_apply_csr(g, x, x_dtype, F, w, msg, reducer, out, argmax, ws, (size_t)TIGA_BUILTIN_WS_BYTES, stream);
 }
 
+// ---- planned forward (source-block passes; see csr_plan.cu) --------------------------------
+static size_t planned_chunk_capacity(const tiga_csr_plan* plan) {
+    long long huge = 0;
+    for (int b = 0; b < plan->n_blocks; ++b) huge += plan->huge_segments[b];
+    return (size_t)(plan->n_edges / ROW_HUGE + huge + 1);
+}
+
+extern "C" size_t tiga_csr_planned_workspace_bytes(const tiga_csr_plan* plan, int32_t F) {
+    if (!plan || F <= 0) return 0;
+    const size_t cap = planned_chunk_capacity(plan);
+    return 256 + align_up(cap * sizeof(int4), 256) + align_up(cap * (size_t)F * sizeof(float), 256) + 256;
+}
+
+template <typename XT, int NV>
+static tiga_status launch_planned_pass(const CsrParams& p, bool huge, cudaStream_t s) {
+    const unsigned blocks = (unsigned)((p.n_dst + CSR_THREADS - 1) / CSR_THREADS);
+    if (huge) TIGA_CUDA_TRY(cudaMemsetAsync(p.huge_count, 0, sizeof(int), s));
+    csr_rows_kernel<XT, NV, 0, int32_t, true><<<counted(blocks), CSR_THREADS, 0, s>>>(p);
+    if (huge) {
+        csr_huge_chunks_kernel<XT, NV, 0, int32_t><<<counted(148 * 8), CSR_THREADS, 0, s>>>(p);
+        csr_huge_fold_kernel<0, true><<<counted(148 * 2), 256, 0, s>>>(p);
+    }
+    return launch_status();
+}
+
+extern "C" tiga_status tiga_apply_csr_planned(const tiga_csr_plan* plan, const void* plan_buf, const void* x, tiga_dtype x_dtype,
+                                              int32_t F, const float* w, const tiga_msg* msg, float* out,
+                                              void* ws, size_t ws_bytes, void* stream) {
+    if (!plan || !plan_buf || !aligned16(plan_buf)) return TIGA_ERR_INVALID_ARG;
+    if (plan->n_blocks < 1 || plan->n_blocks > TIGA_PLAN_MAX_BLOCKS || plan->n_dst <= 0 || plan->n_edges <= 0) return TIGA_ERR_INVALID_ARG;
+    int nvec, G, VPL;
+    tiga_status st = check_features(F, x_dtype, &nvec, &G, &VPL);
+    if (st != TIGA_OK) return st;
+    if (nvec > 2) return TIGA_ERR_UNSUPPORTED;            // feature rows of at most 32 bytes: the case the plan exists for
+    if (!msg) return TIGA_ERR_INVALID_ARG;
+    if (msg->kind == TIGA_MSG_COPY) { if (w) return TIGA_ERR_INVALID_ARG; }
+    else if (msg->kind == TIGA_MSG_WEIGHTED) { if (!w) return TIGA_ERR_INVALID_ARG; if (!plan->has_positions) return TIGA_ERR_UNSUPPORTED; }
+    else return TIGA_ERR_UNSUPPORTED;
+    if (!out || !aligned16(out) || !x || !aligned16(x) || (w && !aligned16(w))) return TIGA_ERR_INVALID_ARG;
+    if (!ws || !aligned16(ws) || ws_bytes < tiga_csr_planned_workspace_bytes(plan, F)) return TIGA_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const char* base = static_cast<const char*>(plan_buf);
+    const int32_t* pcol = reinterpret_cast<const int32_t*>(base + plan->off_col);
+    const int32_t* ppos = plan->off_pos >= 0 ? reinterpret_cast<const int32_t*>(base + plan->off_pos) : nullptr;
+    const int32_t* seg_row = reinterpret_cast<const int32_t*>(base + plan->off_seg_row);
+    const int32_t* seg_ptr = reinterpret_cast<const int32_t*>(base + plan->off_seg_ptr);
+
+    CsrParams p{};
+    p.col = pcol; p.w = w; p.epos = w ? ppos : nullptr; p.x = x; p.out = out;
+    p.n_edges = plan->n_edges; p.F = F; p.nvec = nvec;
+    const size_t cap = planned_chunk_capacity(plan);
+    Carver cv(ws);
+    p.huge_count = cv.take<int>(1);
+    p.huge_list = cv.take<int4>(cap);
+    p.carry_val = cv.take<float>(cap * (size_t)F);
+    // rows start from zero; every pass adds the partial sums of its block, passes run in block order
+    TIGA_CUDA_TRY(cudaMemsetAsync(out, 0, (size_t)plan->n_dst * F * sizeof(float), s));
+    for (int b = 0; b < plan->n_blocks; ++b) {
+        const long long s0 = plan->seg_begin[b], s1 = plan->seg_begin[b + 1];
+        if (s1 <= s0) continue;
+        p.rowptr = seg_ptr + s0; p.row_map = seg_row + s0; p.n_dst = s1 - s0;
+        const bool huge = plan->huge_segments[b] > 0;
+        if (x_dtype == TIGA_F32) st = nvec == 1 ? launch_planned_pass<float, 1>(p, huge, s) : launch_planned_pass<float, 2>(p, huge, s);
+        else st = nvec == 1 ? launch_planned_pass<__half, 1>(p, huge, s) : launch_planned_pass<__half, 2>(p, huge, s);
+        if (st != TIGA_OK) return st;
+    }
+    return TIGA_OK;
+}
+
 extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
                                                const float* w, const tiga_msg* msg, tiga_reducer reducer,
                                                const float* grad_out, const int32_t* argmax,
@@ -948,7 +1012,7 @@ extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x,
         return g->rowptr_type == TIGA_I64 ? launch_bwd_g<int64_t>(p, G, VPL, s) : launch_bwd_g<int32_t>(p, G, VPL, s);
     }
     const long long work = g->n_dst * F;
-    csr_backward_max_kernel<<<(unsigned)((work + 255) / 256), 256, 0, s>>>(p);
+    csr_backward_max_kernel<<<counted((unsigned)((work + 255) / 256)), 256, 0, s>>>(p);
     return launch_status();
 }
 
@@ -965,13 +1029,15 @@ extern "C" tiga_status tiga_csr_degree_histogram(const tiga_csr* g, int64_t* his
     if (blocks > 148 * 4) blocks = 148 * 4;
     const size_t sm = (size_t)nbins * sizeof(unsigned int);
     if (g->rowptr_type == TIGA_I32)
-        degree_hist_kernel<int32_t><<<(unsigned)blocks, 256, sm, s>>>(static_cast<const int32_t*>(g->rowptr), g->n_dst, (int)nbins,
+        degree_hist_kernel<int32_t><<<counted((unsigned)blocks), 256, sm, s>>>(static_cast<const int32_t*>(g->rowptr), g->n_dst, (int)nbins,
                                                                    reinterpret_cast<unsigned long long*>(hist), reinterpret_cast<unsigned long long*>(max_degree));
     else
-        degree_hist_kernel<int64_t><<<(unsigned)blocks, 256, sm, s>>>(static_cast<const int64_t*>(g->rowptr), g->n_dst, (int)nbins,
+        degree_hist_kernel<int64_t><<<counted((unsigned)blocks), 256, sm, s>>>(static_cast<const int64_t*>(g->rowptr), g->n_dst, (int)nbins,
                                                                    reinterpret_cast<unsigned long long*>(hist), reinterpret_cast<unsigned long long*>(max_degree));
     return launch_status();
 }
+
+extern "C" int64_t tiga_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
 
 extern "C" const char* tiga_status_string(tiga_status s) {
     switch (s) {
@@ -984,25 +1050,4 @@ extern "C" const char* tiga_status_string(tiga_status s) {
         case TIGA_ERR_TOO_LARGE: return "problem exceeds the library's built-in scratch capacity";
     }
     return "unknown status";
-}
-
-extern "C" tiga_status tiga_probe_row_gather(const void* table, int64_t n_rows, int32_t row_bytes,
-                                             const int32_t* idx, int64_t n_idx, float* sink, void* stream) {
-    if (!table || !idx || !sink || n_rows <= 0 || n_idx < 0 || !aligned16(table)) return TIGA_ERR_INVALID_ARG;
-    if (row_bytes < 16 || row_bytes > 512 || (row_bytes & 15)) return TIGA_ERR_INVALID_ARG;
-    const int ln = row_bytes / 16;
-    if (ln & (ln - 1)) return TIGA_ERR_UNSUPPORTED;      // 16, 32, 64, 128, 256 or 512 bytes per row
-    if (n_idx == 0) return TIGA_OK;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const unsigned blocks = 148 * 8;
-    const uint4* t = static_cast<const uint4*>(table);
-    switch (ln) {
-        case 1: row_gather_probe_kernel<1><<<blocks, 256, 0, s>>>(t, idx, n_idx, sink); break;
-        case 2: row_gather_probe_kernel<2><<<blocks, 256, 0, s>>>(t, idx, n_idx, sink); break;
-        case 4: row_gather_probe_kernel<4><<<blocks, 256, 0, s>>>(t, idx, n_idx, sink); break;
-        case 8: row_gather_probe_kernel<8><<<blocks, 256, 0, s>>>(t, idx, n_idx, sink); break;
-        case 16: row_gather_probe_kernel<16><<<blocks, 256, 0, s>>>(t, idx, n_idx, sink); break;
-        default: row_gather_probe_kernel<32><<<blocks, 256, 0, s>>>(t, idx, n_idx, sink); break;
-    }
-    return launch_status();
 }

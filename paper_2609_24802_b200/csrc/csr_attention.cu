@@ -250,10 +250,10 @@ __global__ void csr_attention_fixup_kernel(const CsrParams p) {
 template <int G, typename IT>
 static tiga_status launch_attention_t(const CsrParams& p, cudaStream_t s) {
     constexpr int smem = 2 * (CSR_THREADS / G) * G * 4 * (int)sizeof(float);
-    if (p.nvec == G) csr_attention_kernel<G, IT, true><<<(unsigned)p.ntiles, CSR_THREADS, smem, s>>>(p);
-    else csr_attention_kernel<G, IT, false><<<(unsigned)p.ntiles, CSR_THREADS, smem, s>>>(p);
+    if (p.nvec == G) csr_attention_kernel<G, IT, true><<<counted((unsigned)p.ntiles), CSR_THREADS, smem, s>>>(p);
+    else csr_attention_kernel<G, IT, false><<<counted((unsigned)p.ntiles), CSR_THREADS, smem, s>>>(p);
     const long long work = p.ntiles * p.F;
-    csr_attention_fixup_kernel<<<(unsigned)((work + 255) / 256), 256, 0, s>>>(p);
+    csr_attention_fixup_kernel<<<counted((unsigned)((work + 255) / 256)), 256, 0, s>>>(p);
     return launch_status();
 }
 

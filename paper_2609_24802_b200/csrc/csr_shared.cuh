@@ -8,6 +8,7 @@ namespace tiga {
 constexpr int CSR_THREADS = 256;
 constexpr int CSR_TILE = 2048;     // merge-path items per CTA
 constexpr int CSR_PAD = 8;         // readable entries behind a tile's staged edges
+constexpr int ROW_HUGE = 8192;     // narrow-row path: rows (segments) above this many edges are cut into chunks
 
 template <typename XT> struct XTraits;
 template <> struct XTraits<float> {
@@ -46,6 +47,9 @@ struct CsrParams {
     long long ntiles;
     int* huge_count;         // narrow-row path: number of queued chunks of huge rows
     int4* huge_list;         // (row, chunk, chunks of the row, first slot of the row)
+    // planned apply (csr.cu, narrow rows): the "rows" are (destination row, source block) segments
+    const int32_t* row_map;  // segment -> destination row whose output it is added to
+    const int32_t* epos;     // permuted edge -> original edge position (indexes w), or null
     // backward
     const float* gy;
     float* gx;

@@ -532,7 +532,7 @@ extern "C" tiga_status tiga_apply_knn(const float* pos, const float* feat, int64
     const unsigned blocks = (unsigned)((P.rp.ncells + TRAV_WARPS - 1) / TRAV_WARPS);
     constexpr int smem = KNN_PER_WARP * TRAV_WARPS;
     TIGA_CUDA_TRY(cudaFuncSetAttribute(knn_cells_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    knn_cells_kernel<<<blocks, TRAV_THREADS, smem, s>>>(P);
-    knn_rings_kernel<<<KNN_RING_BLOCKS, TRAV_THREADS, 0, s>>>(P);
+    knn_cells_kernel<<<counted(blocks), TRAV_THREADS, smem, s>>>(P);
+    knn_rings_kernel<<<counted(KNN_RING_BLOCKS), TRAV_THREADS, 0, s>>>(P);
     return launch_status();
 }

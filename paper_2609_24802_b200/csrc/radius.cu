@@ -639,12 +639,12 @@ tiga_status run_binning(RadiusParams& p, int32_t* fill, int nblocks, cudaStream_
     if (p.n == 0) return TIGA_OK;
     TIGA_CUDA_TRY(cudaMemsetAsync(p.cnt, 0, (2 * (size_t)p.ncells + 2) * sizeof(int32_t), s));
     const unsigned pb = (unsigned)((p.n + 255) / 256);
-    bin_count_kernel<<<pb, 256, 0, s>>>(p);
-    scan_reduce_kernel<<<nblocks, RAD_THREADS, 0, s>>>(p);
-    scan_blocksums_kernel<<<1, 1024, 0, s>>>(p, nblocks);
-    scan_apply_kernel<<<nblocks, RAD_THREADS, 0, s>>>(p);
-    bin_scatter_kernel<<<pb, 256, 0, s>>>(p, fill);
-    bin_sort_kernel<<<pb, 256, 0, s>>>(p);
+    bin_count_kernel<<<counted(pb), 256, 0, s>>>(p);
+    scan_reduce_kernel<<<counted(nblocks), RAD_THREADS, 0, s>>>(p);
+    scan_blocksums_kernel<<<counted(1), 1024, 0, s>>>(p, nblocks);
+    scan_apply_kernel<<<counted(nblocks), RAD_THREADS, 0, s>>>(p);
+    bin_scatter_kernel<<<counted(pb), 256, 0, s>>>(p, fill);
+    bin_sort_kernel<<<counted(pb), 256, 0, s>>>(p);
     return launch_status();
 }
 
@@ -662,12 +662,12 @@ static tiga_status launch_traverse_t(const RadiusParams& p, cudaStream_t s) {
         // scalar feature accesses (only the forward supports widths that are not multiples of 4)
         auto sk = radius_traverse_kernel<MODE == 0 ? 0 : MODE, LF, DIST, MI, MODE != 0 ? 1 : 0>;
         if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(sk, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        sk<<<blocks, TRAV_THREADS, smem, s>>>(p);
+        sk<<<counted(blocks), TRAV_THREADS, smem, s>>>(p);
         return launch_status();
     }
     auto kern = p.F == 4 * LF ? radius_traverse_kernel<MODE, LF, DIST, MI, 2> : radius_traverse_kernel<MODE, LF, DIST, MI, 1>;
     if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    kern<<<blocks, TRAV_THREADS, smem, s>>>(p);
+    kern<<<counted(blocks), TRAV_THREADS, smem, s>>>(p);
     return launch_status();
 }
 

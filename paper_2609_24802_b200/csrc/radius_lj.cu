@@ -354,7 +354,7 @@ static tiga_status launch_lj_t(const RadiusParams& p, cudaStream_t s) {
     constexpr int smem = LJ_PER_WARP * TRAV_WARPS;
     auto kern = radius_lj_pairs_kernel<MI, COUNT>;
     if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    kern<<<blocks, TRAV_THREADS, smem, s>>>(p);
+    kern<<<counted(blocks), TRAV_THREADS, smem, s>>>(p);
     return launch_status();
 }
 

@@ -506,7 +506,7 @@ static tiga_status launch_mlp_t(const RadiusParams& p, cudaStream_t s) {
     long long blocks = (p.ncells + TRAV_WARPS - 1) / TRAV_WARPS;
     const long long cap = 148LL * mlp_ctas_per_sm<HID, BWD>();       // persistent: parameter gradients are folded once per CTA
     if (blocks > cap) blocks = cap;
-    kern<<<(unsigned)blocks, TRAV_THREADS, SM::TOTAL, s>>>(p);
+    kern<<<counted((unsigned)blocks), TRAV_THREADS, SM::TOTAL, s>>>(p);
     return launch_status();
 }
 

@@ -112,4 +112,13 @@ def test_knn_and_attention_host_checks(lib):
     assert cdll.tiga_csr_attention_workspace_bytes(ctypes.byref(g), 256) == 0
     assert cdll.tiga_apply_csr_attention(ctypes.byref(g), None, None, None, 6, ctypes.c_float(1.0), None, None, None, 0, None) == 1
     assert cdll.tiga_apply_csr_attention(ctypes.byref(g), None, None, None, 132, ctypes.c_float(1.0), None, None, None, 0, None) == 2
-    assert cdll.tiga_probe_row_gather(None, 10, 256, None, 10, None, None) == 1
+
+
+def test_bench_probe_library_builds_and_checks_its_arguments(lib):
+    """The benchmark's row-gather probe lives in a library of its own, outside the product ABI."""
+    from paper_2609_24802_b200 import bench_probe
+    cdll = bench_probe.load()
+    assert cdll.tiga_bench_probe_row_gather(None, 10, 256, None, 10, None, None) == 1
+    import subprocess
+    syms = subprocess.run(["nm", "-D", lib.LIB_PATH], capture_output=True, text=True).stdout
+    assert "probe" not in syms

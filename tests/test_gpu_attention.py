@@ -6,7 +6,7 @@ import pytest
 
 import gen
 import oracle
-from parity import SUM_TOL, dev, host, rel_err
+from parity import SUM_TOL, Guard, dev, host, rel_err
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -21,10 +21,16 @@ def tiga():
 
 def _check(tiga, rowptr, col, n_src, q, k, v, scale, rowptr_dtype=np.int32, tol=SUM_TOL):
     g = tiga.CsrRelation(dev(rowptr.astype(rowptr_dtype), torch), dev(col, torch), n_src)
-    out, lse, _ = tiga.tiga_apply_csr_attention(g, dev(q, torch), dev(k, torch), dev(v, torch), scale)
-    torch.cuda.synchronize()
+    guard = Guard(torch)
+    out, lse, _ = tiga.tiga_apply_csr_attention(g, dev(q, torch), dev(k, torch), dev(v, torch), scale,
+                                                out=guard.empty(q.shape), lse=guard.empty((q.shape[0],)),
+                                                ws=guard.workspace(tiga.tiga_csr_attention_workspace_bytes(g, q.shape[1])))
+    guard.check()
     y, A, ref_lse = oracle.csr_attention(rowptr, col, q, k, v, np.float32(scale))
-    assert rel_err(host(out), y, A) <= tol
+    err = rel_err(host(out), y, A)
+    if tol > SUM_TOL:
+        print(f"online softmax: largest normalised error {err:.3e} (widened tolerance {tol:.3e}, plain {SUM_TOL:.0e})")
+    assert err <= tol
     got = host(lse).astype(np.float64)
     empty = np.isneginf(ref_lse)
     assert np.array_equal(np.isneginf(got), empty)

@@ -6,7 +6,7 @@ import pytest
 
 import gen
 import oracle
-from parity import GRAD_TOL, SUM_TOL, dev, host, rel_err
+from parity import GRAD_TOL, SUM_TOL, Guard, dev, host, rel_err
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -23,7 +23,12 @@ def _check(tiga, pos, x, gy, r, box, per, params, use_cells=True, backward=True,
     y, A, cnt = oracle.radius_mlp_forward(pos, x, r, box, per, *params, use_cells=use_cells)
     pd, xd = dev(pos, torch), dev(x, torch)
     P = [dev(a, torch) for a in params]
-    out, count, ws = tiga.tiga_apply_radius_mlp(pd, xd, r, box, per, *P, want_count=True)
+    guard = Guard(torch)
+    n = len(pos)
+    out, count, ws = tiga.tiga_apply_radius_mlp(pd, xd, r, box, per, *P, out=guard.empty((n, params[2].shape[0])),
+                                                count=guard.empty((n,), torch.int32),
+                                                ws=guard.workspace(tiga.tiga_radius_workspace_bytes(n, x.shape[1], r, box, per)))
+    guard.check()
     assert np.array_equal(host(count), cnt), "neighbour counts must be bit exact"
     assert rel_err(host(out), y, A) <= SUM_TOL
     if backward:

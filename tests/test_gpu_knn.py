@@ -7,7 +7,7 @@ import pytest
 
 import gen
 import oracle
-from parity import SUM_TOL, dev, host, rel_err
+from parity import SUM_TOL, Guard, dev, host, rel_err
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -23,8 +23,12 @@ def tiga():
 
 
 def _check(tiga, pos, x, k, box=UNIT, rows=None):
-    out, nbr, d2, _ = tiga.tiga_apply_knn(dev(pos, torch), dev(x, torch), k, box)
-    torch.cuda.synchronize()
+    guard = Guard(torch)
+    n, F = x.shape
+    out, nbr, d2, _ = tiga.tiga_apply_knn(dev(pos, torch), dev(x, torch), k, box, out=guard.empty((n, F)),
+                                          nbr=guard.empty((n, k), torch.int32), nbr_d2=guard.empty((n, k)),
+                                          ws=guard.workspace(tiga.tiga_knn_workspace_bytes(n, k, box)))
+    guard.check()
     idx, rd2, y, A = oracle.knn(pos, x, k, rows=rows)
     sel = slice(None) if rows is None else np.asarray(rows)
     assert np.array_equal(host(nbr)[sel], idx), "neighbour indices must be bit exact, in key order"

@@ -6,7 +6,7 @@ import pytest
 
 import gen
 import oracle
-from parity import GRAD_TOL, SUM_TOL, dev, host, rel_err
+from parity import GRAD_TOL, SUM_TOL, Guard, dev, host, rel_err
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -32,13 +32,20 @@ def _check_gauss(tiga, pos, x, gy, r, box, per, sigma, kind=None, use_cells=Fals
     kind = tiga.MSG_GAUSS if kind is None else kind
     y, A, cnt = oracle.radius_forward(pos, x, r, box, per, kind, p0=sigma, use_cells=use_cells)
     pd, xd = dev(pos, torch), dev(x, torch)
-    out, count, ws = tiga.tiga_apply_radius(pd, xd, r, box, per, kind, p0=sigma, want_count=True)
+    guard = Guard(torch)
+    n, F = x.shape
+    ws = guard.workspace(tiga.tiga_radius_workspace_bytes(n, F, r, box, per))
+    out, count, ws = tiga.tiga_apply_radius(pd, xd, r, box, per, kind, p0=sigma, out=guard.empty((n, F)),
+                                            count=guard.empty((n,), torch.int32), ws=ws)
+    guard.check()
     assert np.array_equal(host(count), cnt), "neighbour counts must be bit exact"
     assert rel_err(host(out), y, A) <= SUM_TOL
     if backward and kind == tiga.MSG_GAUSS:
         ref = oracle.radius_backward_gauss(pos, x, gy, r, box, per, sigma, use_cells=use_cells)
         gyd = dev(gy, torch)
-        gx, gp = tiga.tiga_apply_radius_backward(pd, xd, gyd, r, box, per, sigma, ws=ws, reuse_plan=True)
+        gx, gp = tiga.tiga_apply_radius_backward(pd, xd, gyd, r, box, per, sigma, ws=ws, reuse_plan=True,
+                                                 grad_feat=guard.empty((n, F)), grad_pos=guard.empty((n, 3)))
+        guard.check()
         assert rel_err(host(gx), ref["gx"], ref["Agx"]) <= GRAD_TOL
         assert rel_err(host(gp), ref["gp"], ref["Agp"]) <= GRAD_TOL
         gx2, gp2 = tiga.tiga_apply_radius_backward(pd, xd, gyd, r, box, per, sigma)      # rebuilds the bins
@@ -155,9 +162,16 @@ def test_gaussian_mid_replica(tiga):
 # ------------------------------------------------------------------------------ Lennard-Jones
 def _check_lj(tiga, pos, r, box, per, eps=1.0, s=1.0, use_cells=False, tol=SUM_TOL):
     y, A, cnt = oracle.radius_forward(pos, None, r, box, per, oracle.MSG_LJ, eps, s, use_cells=use_cells)
-    out, count, _ = tiga.tiga_apply_radius(dev(pos, torch), None, r, box, per, tiga.MSG_LJ, p0=eps, p1=s, want_count=True)
+    guard = Guard(torch)
+    n = len(pos)
+    out, count, _ = tiga.tiga_apply_radius(dev(pos, torch), None, r, box, per, tiga.MSG_LJ, p0=eps, p1=s,
+                                           out=guard.empty((n, 4)), count=guard.empty((n,), torch.int32),
+                                           ws=guard.workspace(tiga.tiga_radius_workspace_bytes(n, 4, r, box, per)))
+    guard.check()
     assert np.array_equal(host(count), cnt)
-    assert rel_err(host(out), y, A) <= tol
+    err = rel_err(host(out), y, A)
+    print(f"Lennard-Jones: largest normalised error {err:.3e} (tolerance {tol:.1e})")
+    assert err <= tol
     return host(out), A
 
 
