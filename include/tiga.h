@@ -148,55 +148,51 @@ tiga_status tiga_apply_csr_builtin_ws(const tiga_csr* g, const void* x, tiga_dty
                                       const float* w, const tiga_msg* msg, tiga_reducer reducer,
                                       float* out, int32_t* argmax, void* stream);
 
-/* Source-block plan: one-time preprocessing of a stored relation whose feature table is far larger
+/* Hot-source plan: one-time preprocessing of a stored relation whose feature table is far larger
  * than the L2 cache (the billion-edge relation of Section 7 held in device memory).  It depends on
- * (rowptr, col) only -- the paper also treats relation set-up as untimed preprocessing (Section 7) --
- * and regroups the edges by block of source rows and, inside a block, by destination row, keeping
- * every row's edge order.  tiga_apply_csr_planned then runs one pass per block: all gathers of a
- * pass fall into one slice of the feature table that stays in L2, and the pass adds one partial sum
- * to every destination row that has an edge in the block.  The struct is plain data on the HOST; the
- * arrays it describes live in `plan_buf` on the device at the byte offsets it records (the caller may
- * move them to a smaller buffer as long as it updates the offsets):
- *   col     int32 [n_edges]         sources, ordered by (block, destination row, edge position)
- *   pos     int32 [n_edges]         original edge position of every permuted edge (only when built
- *                                   with_positions; needed to index edge weights)
- *   seg_row int32 [n_segments]      destination row of every (row, block) segment
- *   seg_ptr int32 [n_segments + 1]  extent of every segment in col */
-#define TIGA_PLAN_MAX_BLOCKS 64
+ * (rowptr, col) only -- the paper also treats relation set-up as untimed preprocessing (Section 7).
+ * In a skewed relation a small set of sources receives most of the edges; the plan selects the
+ * sources named by the most edges (at most max_hot_rows, all those with an in-degree of
+ * min_hot_degree or more), numbers them densely and rewrites the index stream so that a hot source is
+ * addressed by its rank and any other source j by n_hot + j.  tiga_apply_csr_planned copies the hot
+ * rows of the feature table into one compact, L2-resident table and runs the unchanged row-major
+ * traversal over the rewritten indices.  Edges are visited in the same order as without the plan:
+ * sums, maxima and argmax positions are bit-identical to tiga_apply_csr's.
+ * The struct is plain data on the HOST; the arrays it describes live in `plan_buf` on the device at the
+ * byte offsets it records:
+ *   col    int32 [n_edges]   rewritten source indices, in edge order
+ *   hot_id int32 [n_hot]     source row of every hot rank, ascending */
 typedef struct {
-    int32_t n_blocks;                                /* power of two, <= TIGA_PLAN_MAX_BLOCKS */
-    int32_t block_shift;                             /* source row j belongs to block j >> block_shift */
-    int32_t has_positions;
-    int32_t reserved;
-    int64_t n_dst, n_src, n_edges, n_segments;
-    int64_t seg_begin[TIGA_PLAN_MAX_BLOCKS + 1];     /* first segment of every block */
-    int64_t huge_segments[TIGA_PLAN_MAX_BLOCKS];     /* segments above 8192 edges, per block */
-    int64_t off_col, off_pos, off_seg_row, off_seg_ptr;   /* byte offsets in plan_buf; off_pos = -1 when absent */
-    int64_t used_bytes;                              /* bytes of plan_buf the plan occupies */
+    int64_t n_dst, n_src, n_edges;
+    int64_t n_hot;               /* hot sources */
+    int64_t min_hot_degree;      /* every hot source is named by at least this many edges (0: none is hot) */
+    int64_t hot_edges;           /* edges whose source is hot */
+    int64_t off_col, off_hot_id; /* byte offsets in plan_buf */
+    int64_t used_bytes;          /* bytes of plan_buf the plan occupies */
 } tiga_csr_plan;
 
-/* Bytes of plan_buf (worst case: every edge its own segment) and of build scratch.  Host only. */
-size_t tiga_csr_plan_bytes(const tiga_csr* g, int32_t n_blocks, int with_positions);
-size_t tiga_csr_plan_workspace_bytes(const tiga_csr* g, int32_t n_blocks);
+/* Bytes of plan_buf and of build scratch.  Host only. */
+size_t tiga_csr_plan_bytes(const tiga_csr* g, int64_t max_hot_rows);
+size_t tiga_csr_plan_workspace_bytes(const tiga_csr* g);
 
-/* Builds the plan on the device and SYNCHRONISES the stream (segment counts come back to the host
- * struct).  Needs n_edges < 2^31 - 1; rowptr int32 or int64.  n_blocks: a power of two; choose it so
- * that n_src * row bytes / n_blocks is a fraction of the L2 size.  ws is scratch and may be freed
- * afterwards.  The result is unique (a stable regrouping), so rebuilding gives the same plan. */
-tiga_status tiga_csr_plan_build(const tiga_csr* g, int32_t n_blocks, int with_positions,
-                                void* plan_buf, size_t plan_bytes, void* ws, size_t ws_bytes,
-                                tiga_csr_plan* plan /* host, out */, void* stream);
+/* Builds the plan on the device and SYNCHRONISES the stream twice (the in-degree histogram and the
+ * counts come back to the host).  Needs n_src + max_hot_rows < 2^31.  max_hot_rows: choose it so that
+ * max_hot_rows * row bytes is about half the L2 size.  ws is scratch and may be freed afterwards.  In-
+ * degrees of 4095 and more are not told apart: if more than max_hot_rows sources reach that, none is
+ * hot.  The result is unique, so rebuilding gives the same plan. */
+tiga_status tiga_csr_plan_build(const tiga_csr* g, int64_t max_hot_rows, void* plan_buf, size_t plan_bytes,
+                                void* ws, size_t ws_bytes, tiga_csr_plan* plan /* host, out */, void* stream);
 
-/* tiga_apply_csr with the sum reducer through a plan: out[i,:] = sum of w[e] x[col[e],:] over row i.
- * Feature rows of at most 32 bytes (F <= 8 fp32, F <= 16 fp16; TIGA_ERR_UNSUPPORTED above: wider rows
- * do not need the plan).  w: fp32 [n_edges] in ORIGINAL edge order (plan built with_positions) or NULL.
- * A row's partial sums are added in block order and long segments are folded in edge order, without
- * atomics: results are reproducible from run to run (the grouping of the additions differs from
- * tiga_apply_csr's, so the two agree to rounding, not bit for bit).
- *   ws : tiga_csr_planned_workspace_bytes(plan, F) bytes of scratch. */
-size_t tiga_csr_planned_workspace_bytes(const tiga_csr_plan* plan, int32_t F);
-tiga_status tiga_apply_csr_planned(const tiga_csr_plan* plan, const void* plan_buf, const void* x, tiga_dtype x_dtype,
-                                   int32_t F, const float* w, const tiga_msg* msg, float* out,
+/* tiga_apply_csr through a plan built for this very relation (same arguments and results, bit for
+ * bit).  Feature rows of at most 32 bytes (F <= 8 fp32, F <= 16 fp16; TIGA_ERR_UNSUPPORTED above:
+ * wider rows are served by the tile kernels, which the plan does not change).
+ *   ws : tiga_csr_planned_workspace_bytes(...) bytes: the compact table of hot rows plus the
+ *        forward's own scratch. */
+size_t tiga_csr_planned_workspace_bytes(const tiga_csr* g, const tiga_csr_plan* plan, int32_t F, tiga_dtype x_dtype,
+                                        tiga_reducer reducer);
+tiga_status tiga_apply_csr_planned(const tiga_csr* g, const tiga_csr_plan* plan, const void* plan_buf,
+                                   const void* x, tiga_dtype x_dtype, int32_t F, const float* w, const tiga_msg* msg,
+                                   tiga_reducer reducer, float* out, int32_t* argmax,
                                    void* ws, size_t ws_bytes, void* stream);
 
 /* Reverse mode of tiga_apply_csr for fixed relation indices (Section 5):

@@ -16,7 +16,7 @@ __all__ = [
     "MSG_COPY", "MSG_WEIGHTED", "MSG_GAUSS", "MSG_DIST", "MSG_LJ",
     "CsrRelation", "tiga_status_string", "tiga_csr_workspace_bytes", "tiga_validate_csr",
     "tiga_apply_csr", "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram",
-    "CsrPlan", "tiga_csr_plan_build", "tiga_apply_csr_planned",
+    "CsrPlan", "tiga_csr_plan_build", "tiga_csr_planned_workspace_bytes", "tiga_apply_csr_planned",
     "tiga_radius_grid", "tiga_radius_workspace_bytes", "tiga_radius_bin",
     "tiga_apply_radius", "tiga_apply_radius_backward", "tiga_apply_radius_mlp",
     "tiga_apply_radius_mlp_backward", "tiga_knn_workspace_bytes", "tiga_apply_knn",
@@ -66,16 +66,10 @@ class _EdgeMlp(ctypes.Structure):
                 ("W1", ctypes.c_void_p), ("b1", ctypes.c_void_p), ("W2", ctypes.c_void_p), ("b2", ctypes.c_void_p)]
 
 
-PLAN_MAX_BLOCKS = 64
-
-
 class _Plan(ctypes.Structure):
-    _fields_ = [("n_blocks", ctypes.c_int32), ("block_shift", ctypes.c_int32), ("has_positions", ctypes.c_int32),
-                ("reserved", ctypes.c_int32), ("n_dst", ctypes.c_int64), ("n_src", ctypes.c_int64),
-                ("n_edges", ctypes.c_int64), ("n_segments", ctypes.c_int64),
-                ("seg_begin", ctypes.c_int64 * (PLAN_MAX_BLOCKS + 1)), ("huge_segments", ctypes.c_int64 * PLAN_MAX_BLOCKS),
-                ("off_col", ctypes.c_int64), ("off_pos", ctypes.c_int64), ("off_seg_row", ctypes.c_int64),
-                ("off_seg_ptr", ctypes.c_int64), ("used_bytes", ctypes.c_int64)]
+    _fields_ = [("n_dst", ctypes.c_int64), ("n_src", ctypes.c_int64), ("n_edges", ctypes.c_int64), ("n_hot", ctypes.c_int64),
+                ("min_hot_degree", ctypes.c_int64), ("hot_edges", ctypes.c_int64), ("off_col", ctypes.c_int64),
+                ("off_hot_id", ctypes.c_int64), ("used_bytes", ctypes.c_int64)]
 
 
 _lib = None
@@ -109,15 +103,16 @@ def load_library() -> ctypes.CDLL:
     lib.tiga_apply_csr_backward.argtypes = [ctypes.POINTER(_Csr), vp, ctypes.c_int, i32, vp, ctypes.POINTER(_Msg), ctypes.c_int,
                                             vp, vp, vp, vp, vp, sz, vp]
     lib.tiga_csr_plan_bytes.restype = sz
-    lib.tiga_csr_plan_bytes.argtypes = [ctypes.POINTER(_Csr), i32, ctypes.c_int]
+    lib.tiga_csr_plan_bytes.argtypes = [ctypes.POINTER(_Csr), i64]
     lib.tiga_csr_plan_workspace_bytes.restype = sz
-    lib.tiga_csr_plan_workspace_bytes.argtypes = [ctypes.POINTER(_Csr), i32]
+    lib.tiga_csr_plan_workspace_bytes.argtypes = [ctypes.POINTER(_Csr)]
     lib.tiga_csr_plan_build.restype = ctypes.c_int
-    lib.tiga_csr_plan_build.argtypes = [ctypes.POINTER(_Csr), i32, ctypes.c_int, vp, sz, vp, sz, ctypes.POINTER(_Plan), vp]
+    lib.tiga_csr_plan_build.argtypes = [ctypes.POINTER(_Csr), i64, vp, sz, vp, sz, ctypes.POINTER(_Plan), vp]
     lib.tiga_csr_planned_workspace_bytes.restype = sz
-    lib.tiga_csr_planned_workspace_bytes.argtypes = [ctypes.POINTER(_Plan), i32]
+    lib.tiga_csr_planned_workspace_bytes.argtypes = [ctypes.POINTER(_Csr), ctypes.POINTER(_Plan), i32, ctypes.c_int, ctypes.c_int]
     lib.tiga_apply_csr_planned.restype = ctypes.c_int
-    lib.tiga_apply_csr_planned.argtypes = [ctypes.POINTER(_Plan), vp, vp, ctypes.c_int, i32, vp, ctypes.POINTER(_Msg), vp, vp, sz, vp]
+    lib.tiga_apply_csr_planned.argtypes = [ctypes.POINTER(_Csr), ctypes.POINTER(_Plan), vp, vp, ctypes.c_int, i32, vp,
+                                           ctypes.POINTER(_Msg), ctypes.c_int, vp, vp, vp, sz, vp]
     lib.tiga_csr_degree_histogram.restype = ctypes.c_int
     lib.tiga_csr_degree_histogram.argtypes = [ctypes.POINTER(_Csr), vp, i64, vp, vp]
     lib.tiga_radius_grid.restype = ctypes.c_int
@@ -269,64 +264,62 @@ def tiga_apply_csr_backward(g: CsrRelation, x, w, grad_out, reducer: int = SUM, 
 
 
 class CsrPlan:
-    """A built source-block plan: the host struct ``tiga_csr_plan`` plus the device buffer it describes."""
+    """A built hot-source plan: the host struct ``tiga_csr_plan``, the device buffer it describes and
+    the relation it was built for."""
 
-    def __init__(self, c, buf, scratch_bytes):
-        self.c, self.buf, self.scratch_bytes = c, buf, int(scratch_bytes)
+    def __init__(self, g, c, buf, scratch_bytes):
+        self.g, self.c, self.buf, self.scratch_bytes = g, c, buf, int(scratch_bytes)
 
-    n_blocks = property(lambda self: int(self.c.n_blocks))
-    n_segments = property(lambda self: int(self.c.n_segments))
+    n_hot = property(lambda self: int(self.c.n_hot))
+    hot_edges = property(lambda self: int(self.c.hot_edges))
+    min_hot_degree = property(lambda self: int(self.c.min_hot_degree))
     nbytes = property(lambda self: int(self.c.used_bytes))
 
     def array(self, name):
-        """View of one of the plan's device arrays: 'col', 'pos', 'seg_row', 'seg_ptr'."""
-        off = {"col": self.c.off_col, "pos": self.c.off_pos, "seg_row": self.c.off_seg_row, "seg_ptr": self.c.off_seg_ptr}[name]
-        if off < 0:
-            return None
-        n = {"col": self.c.n_edges, "pos": self.c.n_edges, "seg_row": self.c.n_segments, "seg_ptr": self.c.n_segments + 1}[name]
+        """View of one of the plan's device arrays: 'col' or 'hot_id'."""
+        off, n = {"col": (self.c.off_col, self.c.n_edges), "hot_id": (self.c.off_hot_id, self.c.n_hot)}[name]
         return self.buf[off:off + 4 * n].view(torch.int32)
 
 
-def tiga_csr_plan_build(g: CsrRelation, row_bytes: int = 16, n_blocks: int = None, with_positions: bool = False,
-                        block_bytes: int = 32 << 20, stream=None) -> CsrPlan:
-    """Builds the source-block plan of a relation (one-time, synchronises).  ``n_blocks`` defaults to the
-    power of two that makes a block of source rows about ``block_bytes`` of feature table."""
+def tiga_csr_plan_build(g: CsrRelation, max_hot_rows: int = None, row_bytes: int = 16, hot_bytes: int = 48 << 20,
+                        stream=None) -> CsrPlan:
+    """Builds the hot-source plan of a relation (one-time, synchronises).  ``max_hot_rows`` defaults to
+    as many rows as fit ``hot_bytes`` of compact feature table."""
     lib = load_library()
-    if n_blocks is None:
-        n_blocks = 1
-        while n_blocks < PLAN_MAX_BLOCKS and g.n_src * row_bytes > n_blocks * block_bytes:
-            n_blocks *= 2
-    nbytes = int(lib.tiga_csr_plan_bytes(g.ref, n_blocks, int(with_positions)))
-    wbytes = int(lib.tiga_csr_plan_workspace_bytes(g.ref, n_blocks))
+    if max_hot_rows is None:
+        max_hot_rows = max(1, hot_bytes // row_bytes)
+    max_hot_rows = int(min(max_hot_rows, g.n_src))
+    nbytes = int(lib.tiga_csr_plan_bytes(g.ref, max_hot_rows))
+    wbytes = int(lib.tiga_csr_plan_workspace_bytes(g.ref))
     if nbytes == 0:
         raise TigaError(2, "tiga_csr_plan_bytes")
     buf = torch.empty(nbytes, dtype=torch.uint8, device=g.col.device)
     ws = torch.empty(wbytes, dtype=torch.uint8, device=g.col.device)
     c = _Plan()
-    _ok(lib.tiga_csr_plan_build(g.ref, n_blocks, int(with_positions), _ptr(buf), nbytes, _ptr(ws), wbytes,
-                                ctypes.byref(c), _stream(stream)), "tiga_csr_plan_build")
-    del ws
-    # the worst-case buffer shrinks to what the plan uses: move the two segment arrays up behind the edges
-    used = int(c.used_bytes)
-    if used < nbytes:
-        small = torch.empty(used, dtype=torch.uint8, device=buf.device)
-        small.copy_(buf[:used])
-        buf = small
-    return CsrPlan(c, buf, wbytes)
+    _ok(lib.tiga_csr_plan_build(g.ref, max_hot_rows, _ptr(buf), nbytes, _ptr(ws), wbytes, ctypes.byref(c), _stream(stream)),
+        "tiga_csr_plan_build")
+    return CsrPlan(g, c, buf, wbytes)
 
 
-def tiga_apply_csr_planned(plan: CsrPlan, x, w=None, out=None, ws=None, stream=None):
-    """Sum forward through a source-block plan.  Returns out."""
+def tiga_csr_planned_workspace_bytes(plan: CsrPlan, F: int, x_dtype: int = F32, reducer: int = SUM) -> int:
+    return int(load_library().tiga_csr_planned_workspace_bytes(plan.g.ref, ctypes.byref(plan.c), F, x_dtype, reducer))
+
+
+def tiga_apply_csr_planned(plan: CsrPlan, x, w=None, reducer: int = SUM, out=None, argmax=None, ws=None, stream=None):
+    """tiga_apply_csr through a hot-source plan.  Returns (out, argmax)."""
     F = x.shape[1]
-    lib = load_library()
+    g = plan.g
     if out is None:
-        out = torch.empty((plan.c.n_dst, F), dtype=torch.float32, device=x.device)
+        out = torch.empty((g.n_dst, F), dtype=torch.float32, device=x.device)
+    if reducer == MAX and argmax is None:
+        argmax = torch.empty((g.n_dst, F), dtype=torch.int32, device=x.device)
     if ws is None:
-        ws = _ws(lib.tiga_csr_planned_workspace_bytes(ctypes.byref(plan.c), F), x)
+        ws = _ws(tiga_csr_planned_workspace_bytes(plan, F, _dt(x), reducer), x)
     msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)
-    _ok(lib.tiga_apply_csr_planned(ctypes.byref(plan.c), _ptr(plan.buf), _ptr(x), _dt(x), F, _ptr(w), ctypes.byref(msg),
-                                   _ptr(out), _ptr(ws), ws.numel(), _stream(stream)), "tiga_apply_csr_planned")
-    return out
+    _ok(load_library().tiga_apply_csr_planned(g.ref, ctypes.byref(plan.c), _ptr(plan.buf), _ptr(x), _dt(x), F, _ptr(w),
+                                              ctypes.byref(msg), reducer, _ptr(out), _ptr(argmax), _ptr(ws), ws.numel(),
+                                              _stream(stream)), "tiga_apply_csr_planned")
+    return out, argmax
 
 
 def tiga_csr_degree_histogram(g: CsrRelation, nbins: int = 4096, stream=None):

@@ -254,104 +254,196 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
 // --------------------------------------------------------------------------------------------
 // Forward for narrow rows (one or two 16-byte vectors per feature row, e.g. F = 8 fp16).
 // A worker of G lanes would leave most of a warp idle here and a feature row is a single
-// 128-bit load, so the work is split by ROW CLASS instead:
-//   * every warp owns 32 consecutive rows; rows of at most ROW_SHORT edges are summed by
-//     their own lane, in edge order (empty rows cost one zero store);
-//   * longer rows (up to ROW_HUGE edges) are taken one at a time by the whole warp: lanes
-//     stride over the row's edges with coalesced index loads and 128-bit gathers, then a
-//     shuffle tree combines the 32 partial states (for max the tie rule "lowest edge position"
-//     makes the merge order irrelevant);
+// 128-bit load, so the work is split by ROW CLASS instead.  Every thread looks at one row
+// (a warp at 32 consecutive rows):
+//   * rows of at most ROW_OWN edges are summed by their own lane, in edge order (empty rows cost
+//     one zero store; all 32 results of a warp leave as one contiguous kilobyte for F = 8);
+//   * rows of up to ROW_GROUP edges are queued in shared memory and taken by GROUPS of eight lanes,
+//     four rows per warp at a time: lanes stride over the row's edges, then the eight partial states
+//     are combined by a halving exchange that leaves every lane with its share of the row's result,
+//     so the row is stored by the group as one coalesced request;
+//   * rows of up to ROW_HUGE edges are queued for whole warps (coalesced index loads, 128-bit
+//     gathers, the same exchange over 32 lanes);
 //   * rows above ROW_HUGE edges are cut into ROW_HUGE-edge chunks that are queued in the
 //     workspace; a second kernel gives every chunk to a warp, a third folds the chunk states
 //     of a row in order.
-// All 32 results of a warp are stored together (one contiguous kilobyte for F = 8).
-// The summation tree is fixed, so results are reproducible.
+// The summation tree of every class is fixed, so results are reproducible (for max the tie rule
+// "lowest edge position" makes the merge order irrelevant).
 // --------------------------------------------------------------------------------------------
-constexpr int ROW_SHORT = 16;
+constexpr int ROW_OWN = 4;
+constexpr int ROW_GROUP = 64;
+constexpr int ROW_HUGE = 8192;
+constexpr int GROUP_LANES = 8;
 
-template <int RED, int NV, int VW>
-__device__ __forceinline__ void tree_merge(State<RED, NV, VW>& s) {
+// Where a source row lives.  HOT (planned apply): col values below n_hot address the compact copy of the
+// hot source rows, the others (minus n_hot) the feature table; both bases are set up once per thread.
+template <bool HOT>
+struct Sources {
+    const uint4* cold;
+    const uint4* hot;
+    unsigned n_hot, nvec;
+    __device__ __forceinline__ explicit Sources(const CsrParams& p) {
+        nvec = (unsigned)p.nvec;
+        n_hot = HOT ? (unsigned)p.n_hot : 0u;
+        cold = static_cast<const uint4*>(p.x) - (size_t)n_hot * nvec;
+        hot = HOT ? static_cast<const uint4*>(p.x_hot) : cold;
+    }
+    __device__ __forceinline__ const uint4* row(unsigned c) const {
+        const uint4* base = (HOT && c < n_hot) ? hot : cold;
+        return base + (unsigned long long)c * nvec;          // one 32 x 32 -> 64 multiply
+    }
+};
+
+// Combines the states of the L lanes of an aligned group by a halving exchange: at every step a lane
+// sends the half of its values that its partner keeps and folds the partner's half into its own, so
+// the number of values per lane halves while the number of lanes summed doubles; once one value is
+// left the remaining steps are plain butterflies.  Afterwards lane gl of the group holds, in its first
+// kept<C, L>() entries, the group totals of the values starting at spread_index<NVAL, L>(gl).
+template <int RED, int C, int J, int L>
+struct Spread {
+    static __device__ __forceinline__ void run(float* v, int* a, int gl) {
+        if constexpr ((1 << J) < L) {
+            constexpr int o = 1 << J;
+            constexpr unsigned FULL = 0xffffffffu;
+            if constexpr (C > 1) {
+                constexpr int H = C / 2;
+                const bool up = (gl & o) != 0;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-        for (int i = 0; i < NV; ++i)
-#pragma unroll
-            for (int k = 0; k < VW; ++k) {
-                const float ov = __shfl_xor_sync(0xffffffffu, s.v[i][k], o);
-                if constexpr (RED == 0) {
-                    s.v[i][k] += ov;
-                } else {
-                    const int oa = __shfl_xor_sync(0xffffffffu, s.a[i][k], o);
-                    // larger message wins; equal messages: the lower edge position
-                    const bool take = oa >= 0 && (s.a[i][k] < 0 || ov > s.v[i][k] || (ov == s.v[i][k] && oa < s.a[i][k]));
-                    if (take) { s.v[i][k] = ov; s.a[i][k] = oa; }
+                for (int k = 0; k < H; ++k) {
+                    const float send = up ? v[k] : v[k + H];
+                    const float keep = up ? v[k + H] : v[k];
+                    const float got = __shfl_xor_sync(FULL, send, o);
+                    if constexpr (RED == 0) {
+                        v[k] = keep + got;
+                    } else {
+                        const int sa = up ? a[k] : a[k + H];
+                        const int ka = up ? a[k + H] : a[k];
+                        const int ga = __shfl_xor_sync(FULL, sa, o);
+                        // larger message wins; equal messages: the lower edge position
+                        const bool take = ga >= 0 && (ka < 0 || got > keep || (got == keep && ga < ka));
+                        v[k] = take ? got : keep;
+                        a[k] = take ? ga : ka;
+                    }
                 }
+                Spread<RED, H, J + 1, L>::run(v, a, gl);
+            } else {
+                const float got = __shfl_xor_sync(FULL, v[0], o);
+                if constexpr (RED == 0) {
+                    v[0] += got;
+                } else {
+                    const int ga = __shfl_xor_sync(FULL, a[0], o);
+                    const bool take = ga >= 0 && (a[0] < 0 || got > v[0] || (got == v[0] && ga < a[0]));
+                    if (take) { v[0] = got; a[0] = ga; }
+                }
+                Spread<RED, 1, J + 1, L>::run(v, a, gl);
             }
+        }
+    }
+};
+
+template <int NVAL, int L>
+__device__ __forceinline__ int spread_index(int gl) {
+    int base = 0;
+#pragma unroll
+    for (int j = 0; (1 << j) < L && (NVAL >> j) > 1; ++j) base += ((gl >> j) & 1) * (NVAL >> (j + 1));
+    return base;
 }
 
-// the whole warp reduces edges [es, es + n) of one row; every lane returns the total
-template <typename XT, int NV, int RED, int UNR = 4>
-__device__ __forceinline__ State<RED, NV, XTraits<XT>::VW> warp_row(const CsrParams& p, long long es, int n, int lane) {
+// lanes of the group stride over edges [es, es + n) of one row; every lane returns its partial state.
+// W: the relation has edge weights (otherwise every message is the source row itself).  The indices of
+// the next step are requested before the gathers of the current one are consumed, so an index load and
+// a gather are in flight at the same time instead of one after the other.
+template <typename XT, int NV, int RED, int L, int UNR, bool HOT, bool W>
+__device__ __forceinline__ State<RED, NV, XTraits<XT>::VW> strided_row(const CsrParams& p, const Sources<HOT>& src, long long es, int n, int gl) {
     constexpr int VW = XTraits<XT>::VW;
     State<RED, NV, VW> s;
     s.reset();
-    const uint4* __restrict__ xbase = static_cast<const uint4*>(p.x);
-    for (int k = lane; k < n; k += 32 * UNR) {
+    const int32_t* __restrict__ colp = p.col + es;
+    const float* __restrict__ wp = W ? p.w + es : nullptr;
+    unsigned cn[UNR];
+    float wn[UNR];
+    auto fetch = [&](int k) {
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const int idx = k + L * u;
+            const int at = idx < n ? idx : (k < n ? k : 0);
+            cn[u] = n > 0 ? (unsigned)ld_stream(colp + at) : 0u;
+            wn[u] = (W && n > 0) ? ld_stream(wp + at) : 1.f;
+        }
+    };
+    fetch(gl);
+    for (int k = gl; k < n; k += L * UNR) {
         uint4 xv[UNR][NV];
         float wv[UNR];
 #pragma unroll
         for (int u = 0; u < UNR; ++u) {
-            const bool in = k + 32 * u < n;
-            const long long e = es + (in ? k + 32 * u : k);
-            const long long c = ld_stream(p.col + e);
-            wv[u] = p.w ? ld_stream(p.w + (p.epos ? (long long)ld_stream(p.epos + e) : e)) : 1.f;
+            const bool in = k + L * u < n;
+            wv[u] = wn[u];
+            const uint4* r = src.row(cn[u]);
 #pragma unroll
-            for (int i = 0; i < NV; ++i) xv[u][i] = in ? __ldg(xbase + c * p.nvec + i) : make_uint4(0, 0, 0, 0);
+            for (int i = 0; i < NV; ++i) xv[u][i] = in ? __ldg(r + i) : make_uint4(0, 0, 0, 0);
         }
+        if (k + L * UNR < n) fetch(k + L * UNR);
 #pragma unroll
         for (int u = 0; u < UNR; ++u) {
-            if (k + 32 * u < n) {
-                float xf[VW];
+            if (k + L * u < n) {
+                if constexpr (RED == 0 && !W) {
 #pragma unroll
-                for (int i = 0; i < NV; ++i) {
-                    XTraits<XT>::unpack(xv[u][i], xf);
+                    for (int i = 0; i < NV; ++i) XTraits<XT>::add_to(xv[u][i], &s.v[i][0]);
+                } else {
+                    float xf[VW];
 #pragma unroll
-                    for (int q = 0; q < VW; ++q) s.message(i, q, wv[u], xf[q], (int)(es + k + 32 * u));
+                    for (int i = 0; i < NV; ++i) {
+                        XTraits<XT>::unpack(xv[u][i], xf);
+#pragma unroll
+                        for (int q = 0; q < VW; ++q) s.message(i, q, wv[u], xf[q], (int)(es + k + L * u));
+                    }
                 }
             }
         }
     }
-    tree_merge<RED, NV, VW>(s);
     return s;
 }
 
-// ACC: the state is added to what the row already holds (planned apply: one segment of a row per pass)
-template <typename XT, int NV, int RED, bool ACC = false>
+template <typename XT, int NV, int RED>
 __device__ __forceinline__ void store_state(const CsrParams& p, float* out, int32_t* arg, const State<RED, NV, XTraits<XT>::VW>& s) {
     constexpr int VW = XTraits<XT>::VW;
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
 #pragma unroll
         for (int k = 0; k < VW; k += 4) {
-            float4 v = make_float4(s.v[i][k], s.v[i][k + 1], s.v[i][k + 2], s.v[i][k + 3]);
-            if constexpr (ACC) {
-                const float4 old = ld_stream(reinterpret_cast<const float4*>(out + i * VW + k));
-                v.x += old.x; v.y += old.y; v.z += old.z; v.w += old.w;
-            }
-            st_stream(reinterpret_cast<float4*>(out + i * VW + k), v);
+            st_stream(reinterpret_cast<float4*>(out + i * VW + k), make_float4(s.v[i][k], s.v[i][k + 1], s.v[i][k + 2], s.v[i][k + 3]));
             if constexpr (RED != 0)
                 st_stream(reinterpret_cast<int4*>(arg + i * VW + k), make_int4(s.a[i][k], s.a[i][k + 1], s.a[i][k + 2], s.a[i][k + 3]));
         }
     }
 }
 
-template <typename XT, int NV, int RED, typename IT, bool ACC = false>
+// combine the partial states of a group of L lanes and store the row: every lane writes its share
+template <typename XT, int NV, int RED, int L>
+__device__ __forceinline__ void reduce_and_store(State<RED, NV, XTraits<XT>::VW>& s, int gl, bool valid, float* out, int32_t* arg) {
+    constexpr int NVAL = NV * XTraits<XT>::VW;
+    constexpr int KEEP = NVAL >= L ? NVAL / L : 1;
+    float* v = &s.v[0][0];
+    int* a = &s.a[0][0];
+    Spread<RED, NVAL, 0, L>::run(v, a, gl);
+    if (valid && gl < NVAL) {
+        const int base = spread_index<NVAL, L>(gl);
+#pragma unroll
+        for (int k = 0; k < KEEP; ++k) {
+            st_stream(out + base + k, v[k]);
+            if constexpr (RED != 0) st_stream(arg + base + k, a[k]);
+        }
+    }
+}
+
+template <typename XT, int NV, int RED, typename IT, bool HOT, bool W>
 __global__ void __launch_bounds__(CSR_THREADS) csr_rows_kernel(const CsrParams p) {
     constexpr int VW = XTraits<XT>::VW;
     constexpr unsigned FULL = 0xffffffffu;
     using St = State<RED, NV, VW>;
     const IT* __restrict__ rowptr = static_cast<const IT*>(p.rowptr);
-    const uint4* __restrict__ xbase = static_cast<const uint4*>(p.x);
+    const Sources<HOT> src(p);
     const int lane = threadIdx.x & 31;
     const long long row = ((long long)blockIdx.x * CSR_THREADS + threadIdx.x);      // warp-contiguous rows
     const bool valid = row < p.n_dst;
@@ -359,66 +451,96 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_rows_kernel(const CsrParams p
     const long long ee = valid ? (long long)rowptr[row + 1] : 0;
     const long long deg = ee - es;
 
+    // queues of the CTA's longer rows: group rows fill from the front, warp rows from the back
+    __shared__ short q_row[CSR_THREADS];
+    __shared__ long long q_start[CSR_THREADS];
+    __shared__ int q_len[CSR_THREADS];
+    __shared__ int q_ng, q_nw, q_next;
+    if (threadIdx.x == 0) { q_ng = 0; q_nw = 0; q_next = 0; }
+    __syncthreads();
+    const bool is_g = valid && deg > ROW_OWN && deg <= ROW_GROUP;
+    const bool is_w = valid && deg > ROW_GROUP && deg <= ROW_HUGE;
+    {
+        const unsigned mg = __ballot_sync(FULL, is_g), mw = __ballot_sync(FULL, is_w);
+        int bg = 0, bw = 0;
+        if (lane == 0) {
+            if (mg) bg = atomicAdd(&q_ng, __popc(mg));
+            if (mw) bw = atomicAdd(&q_nw, __popc(mw));
+        }
+        bg = __shfl_sync(FULL, bg, 0); bw = __shfl_sync(FULL, bw, 0);
+        const unsigned lt = (1u << lane) - 1u;
+        if (is_g || is_w) {
+            const int slot = is_g ? bg + __popc(mg & lt) : CSR_THREADS - 1 - (bw + __popc(mw & lt));
+            q_row[slot] = (short)threadIdx.x; q_start[slot] = es; q_len[slot] = (int)deg;
+        }
+    }
+
+    // short rows: one lane each, edge order, one pass with all gathers in flight
     St st;
     st.reset();
-    // short rows: one lane each, edge order
-    if (valid && deg <= ROW_SHORT) {
+    if (valid && deg <= ROW_OWN) {
         const int n = (int)deg;
-        for (int k = 0; k < n; k += 4) {
-            uint4 xv[4][NV];
-            float wv[4];
+        uint4 xv[ROW_OWN][NV];
+        float wv[ROW_OWN];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const bool in = k + u < n;
-                const long long e = es + (in ? k + u : k);
-                const long long c = __ldg(p.col + e);
-                wv[u] = p.w ? __ldg(p.w + (p.epos ? (long long)__ldg(p.epos + e) : e)) : 1.f;
+        for (int u = 0; u < ROW_OWN; ++u) {
+            const bool in = u < n;
+            const long long e = es + (in ? u : 0);
+            const unsigned c = in ? (unsigned)__ldg(p.col + e) : 0u;
+            wv[u] = (W && in) ? __ldg(p.w + e) : 1.f;
+            const uint4* r = src.row(c);
 #pragma unroll
-                for (int i = 0; i < NV; ++i) xv[u][i] = in ? __ldg(xbase + c * p.nvec + i) : make_uint4(0, 0, 0, 0);
-            }
+            for (int i = 0; i < NV; ++i) xv[u][i] = in ? __ldg(r + i) : make_uint4(0, 0, 0, 0);
+        }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (k + u < n) {
+        for (int u = 0; u < ROW_OWN; ++u) {
+            if (u < n) {
+                if constexpr (RED == 0 && !W) {
+#pragma unroll
+                    for (int i = 0; i < NV; ++i) XTraits<XT>::add_to(xv[u][i], &st.v[i][0]);
+                } else {
                     float xf[VW];
 #pragma unroll
                     for (int i = 0; i < NV; ++i) {
                         XTraits<XT>::unpack(xv[u][i], xf);
 #pragma unroll
-                        for (int q = 0; q < VW; ++q) st.message(i, q, wv[u], xf[q], (int)(es + k + u));
+                        for (int q = 0; q < VW; ++q) st.message(i, q, wv[u], xf[q], (int)(es + u));
                     }
                 }
             }
         }
-    }
-    // longer rows go through a queue in shared memory that all warps of the CTA drain together,
-    // so one warp with several long rows does not hold the others back
-    __shared__ int q_row[CSR_THREADS];
-    __shared__ long long q_start[CSR_THREADS];
-    __shared__ int q_len[CSR_THREADS];
-    __shared__ int q_n, q_next;
-    if (threadIdx.x == 0) { q_n = 0; q_next = 0; }
-    __syncthreads();
-    const bool is_mid = valid && deg > ROW_SHORT && deg <= ROW_HUGE;
-    if (is_mid) {
-        const int slot = atomicAdd(&q_n, 1);
-        q_row[slot] = threadIdx.x; q_start[slot] = es; q_len[slot] = (int)deg;
+        store_state<XT, NV, RED>(p, p.out + row * p.F, RED ? p.arg + row * p.F : nullptr, st);
     }
     __syncthreads();
-    const int nmid = q_n;
     const long long row0 = (long long)blockIdx.x * CSR_THREADS;
+    const int ng = q_ng, nw = q_nw;
+
+    // rows for groups of eight lanes: 32 groups per CTA, four rows per warp at a time
+    {
+        const int gl = lane & (GROUP_LANES - 1);
+        const int gid = (threadIdx.x >> 5) * (32 / GROUP_LANES) + lane / GROUP_LANES;
+        constexpr int NGROUPS = CSR_THREADS / GROUP_LANES;
+        for (int it0 = 0; it0 < ng; it0 += NGROUPS) {           // uniform over the CTA
+            const int it = it0 + gid;
+            const bool have = it < ng;
+            const long long rs = have ? q_start[it] : 0;
+            const int rn = have ? q_len[it] : 0;
+            const long long r = row0 + (have ? q_row[it] : 0);
+            St part = strided_row<XT, NV, RED, GROUP_LANES, 4, HOT, W>(p, src, rs, rn, gl);
+            __syncwarp();
+            reduce_and_store<XT, NV, RED, GROUP_LANES>(part, gl, have, p.out + r * p.F, RED ? p.arg + r * p.F : nullptr);
+        }
+    }
+    // rows for whole warps, taken from the back of the queue
     for (;;) {
         int idx = 0;
         if (lane == 0) idx = atomicAdd(&q_next, 1);
         idx = __shfl_sync(FULL, idx, 0);
-        if (idx >= nmid) break;
-        const long long r = row0 + q_row[idx];
-        const long long rs = q_start[idx];
-        const int rn = q_len[idx];
-        const St tot = warp_row<XT, NV, RED>(p, rs, rn, lane);
-        if (lane == 0) {
-            const long long orow = ACC ? (long long)p.row_map[r] : r;
-            store_state<XT, NV, RED, ACC>(p, p.out + orow * p.F, RED ? p.arg + orow * p.F : nullptr, tot);
-        }
+        if (idx >= nw) break;
+        const int slot = CSR_THREADS - 1 - idx;
+        const long long r = row0 + q_row[slot];
+        St part = strided_row<XT, NV, RED, 32, 4, HOT, W>(p, src, q_start[slot], q_len[slot], lane);
+        reduce_and_store<XT, NV, RED, 32>(part, lane, true, p.out + r * p.F, RED ? p.arg + r * p.F : nullptr);
     }
     // huge rows: queue their chunks
     if (valid && deg > ROW_HUGE) {
@@ -426,16 +548,13 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_rows_kernel(const CsrParams p
         const int base = atomicAdd(p.huge_count, chunks);
         for (int c = 0; c < chunks; ++c) p.huge_list[base + c] = make_int4((int)row, c, chunks, base);
     }
-    if (valid && deg <= ROW_SHORT) {
-        const long long orow = ACC ? (long long)p.row_map[row] : row;
-        store_state<XT, NV, RED, ACC>(p, p.out + orow * p.F, RED ? p.arg + orow * p.F : nullptr, st);
-    }
 }
 
 // one warp per queued chunk of a huge row
-template <typename XT, int NV, int RED, typename IT>
+template <typename XT, int NV, int RED, typename IT, bool HOT, bool W>
 __global__ void __launch_bounds__(CSR_THREADS) csr_huge_chunks_kernel(const CsrParams p) {
     const IT* __restrict__ rowptr = static_cast<const IT*>(p.rowptr);
+    const Sources<HOT> src(p);
     const int lane = threadIdx.x & 31;
     const int nwarps = gridDim.x * (CSR_THREADS / 32);
     const int total = *p.huge_count;
@@ -444,14 +563,13 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_huge_chunks_kernel(const CsrP
         const long long es = (long long)rowptr[ent.x] + (long long)ent.y * ROW_HUGE;
         const long long ee = (long long)rowptr[ent.x + 1];
         const int n = (int)(ee - es < ROW_HUGE ? ee - es : ROW_HUGE);
-        const auto tot = warp_row<XT, NV, RED, (NV == 1 ? 8 : 4)>(p, es, n, lane);
-        if (lane == 0)
-            store_state<XT, NV, RED>(p, p.carry_val + (size_t)idx * p.F, RED ? p.carry_arg + (size_t)idx * p.F : nullptr, tot);
+        auto part = strided_row<XT, NV, RED, 32, 4, HOT, W>(p, src, es, n, lane);
+        reduce_and_store<XT, NV, RED, 32>(part, lane, true, p.carry_val + (size_t)idx * p.F, RED ? p.carry_arg + (size_t)idx * p.F : nullptr);
     }
 }
 
 // fold the chunk states of every huge row in chunk (= edge) order; one thread per (row, feature)
-template <int RED, bool ACC = false>
+template <int RED>
 __global__ void csr_huge_fold_kernel(const CsrParams p) {
     const int total = *p.huge_count;
     const long long nthreads = (long long)gridDim.x * blockDim.x;
@@ -469,10 +587,8 @@ __global__ void csr_huge_fold_kernel(const CsrParams p) {
                 if (oa >= 0 && (a < 0 || ov > v)) { v = ov; a = oa; }
             }
         }
-        const size_t orow = ACC ? (size_t)p.row_map[ent.x] : (size_t)ent.x;
-        if (ACC) v += p.out[orow * p.F + f];
-        p.out[orow * p.F + f] = v;
-        if (RED) p.arg[orow * p.F + f] = a;
+        p.out[(size_t)ent.x * p.F + f] = v;
+        if (RED) p.arg[(size_t)ent.x * p.F + f] = a;
     }
 }
 
@@ -713,21 +829,26 @@ static tiga_status launch_fwd_t(const CsrParams& p, cudaStream_t s) {
     return launch_status();
 }
 
+// rows of at most two 16-byte vectors: row-class kernels; HOT serves the hot source rows from p.x_hot
+template <typename XT, int NV, int RED, typename IT, bool HOT, bool W>
+static tiga_status launch_fwd_narrow_t(const CsrParams& p, cudaStream_t s) {
+    TIGA_CUDA_TRY(cudaMemsetAsync(p.huge_count, 0, sizeof(int), s));
+    const unsigned blocks = (unsigned)((p.n_dst + CSR_THREADS - 1) / CSR_THREADS);
+    csr_rows_kernel<XT, NV, RED, IT, HOT, W><<<counted(blocks), CSR_THREADS, 0, s>>>(p);
+    csr_huge_chunks_kernel<XT, NV, RED, IT, HOT, W><<<counted(148 * 8), CSR_THREADS, 0, s>>>(p);
+    csr_huge_fold_kernel<RED><<<counted(148 * 2), 256, 0, s>>>(p);
+    return launch_status();
+}
+
+template <typename XT, int RED, typename IT, bool HOT>
+static tiga_status launch_fwd_narrow(const CsrParams& p, cudaStream_t s) {
+    if (p.nvec == 1) return p.w ? launch_fwd_narrow_t<XT, 1, RED, IT, HOT, true>(p, s) : launch_fwd_narrow_t<XT, 1, RED, IT, HOT, false>(p, s);
+    return p.w ? launch_fwd_narrow_t<XT, 2, RED, IT, HOT, true>(p, s) : launch_fwd_narrow_t<XT, 2, RED, IT, HOT, false>(p, s);
+}
+
 template <typename XT, int RED, typename IT>
 static tiga_status launch_fwd_g(const CsrParams& p, int G, int VPL, cudaStream_t s) {
-    if (p.nvec <= 2) {
-        TIGA_CUDA_TRY(cudaMemsetAsync(p.huge_count, 0, sizeof(int), s));
-        const unsigned blocks = (unsigned)((p.n_dst + CSR_THREADS - 1) / CSR_THREADS);
-        if (p.nvec == 1) {
-            csr_rows_kernel<XT, 1, RED, IT><<<counted(blocks), CSR_THREADS, 0, s>>>(p);
-            csr_huge_chunks_kernel<XT, 1, RED, IT><<<counted(148 * 8), CSR_THREADS, 0, s>>>(p);
-        } else {
-            csr_rows_kernel<XT, 2, RED, IT><<<counted(blocks), CSR_THREADS, 0, s>>>(p);
-            csr_huge_chunks_kernel<XT, 2, RED, IT><<<counted(148 * 8), CSR_THREADS, 0, s>>>(p);
-        }
-        csr_huge_fold_kernel<RED><<<counted(148 * 2), 256, 0, s>>>(p);
-        return launch_status();
-    }
+    if (p.nvec <= 2) return launch_fwd_narrow<XT, RED, IT, false>(p, s);
     switch (G) {
         case 1: return launch_fwd_t<XT, 1, 1, RED, IT>(p, s);
         case 2: return launch_fwd_t<XT, 2, 1, RED, IT>(p, s);
@@ -905,73 +1026,61 @@ extern "C" tiga_status tiga_apply_csr_builtin_ws(const tiga_csr* g, const void* 
     return tiga_apply_csr(g, x, x_dtype, F, w, msg, reducer, out, argmax, ws, (size_t)TIGA_BUILTIN_WS_BYTES, stream);
 }
 
-// ---- planned forward (source-block passes; see csr_plan.cu) --------------------------------
-static size_t planned_chunk_capacity(const tiga_csr_plan* plan) {
-    long long huge = 0;
-    for (int b = 0; b < plan->n_blocks; ++b) huge += plan->huge_segments[b];
-    return (size_t)(plan->n_edges / ROW_HUGE + huge + 1);
+// ---- planned forward (hot-source plan; see csr_plan.cu) ------------------------------------
+extern "C" size_t tiga_csr_planned_workspace_bytes(const tiga_csr* g, const tiga_csr_plan* plan, int32_t F, tiga_dtype x_dtype,
+                                                   tiga_reducer reducer) {
+    if (!g || !plan || F <= 0) return 0;
+    const size_t row_bytes = (size_t)F * (x_dtype == TIGA_F32 ? 4 : 2);
+    return align_up((size_t)plan->n_hot * row_bytes + 256, 256) + tiga_csr_workspace_bytes(g, F, x_dtype, reducer, 0);
 }
 
-extern "C" size_t tiga_csr_planned_workspace_bytes(const tiga_csr_plan* plan, int32_t F) {
-    if (!plan || F <= 0) return 0;
-    const size_t cap = planned_chunk_capacity(plan);
-    return 256 + align_up(cap * sizeof(int4), 256) + align_up(cap * (size_t)F * sizeof(float), 256) + 256;
-}
-
-template <typename XT, int NV>
-static tiga_status launch_planned_pass(const CsrParams& p, bool huge, cudaStream_t s) {
-    const unsigned blocks = (unsigned)((p.n_dst + CSR_THREADS - 1) / CSR_THREADS);
-    if (huge) TIGA_CUDA_TRY(cudaMemsetAsync(p.huge_count, 0, sizeof(int), s));
-    csr_rows_kernel<XT, NV, 0, int32_t, true><<<counted(blocks), CSR_THREADS, 0, s>>>(p);
-    if (huge) {
-        csr_huge_chunks_kernel<XT, NV, 0, int32_t><<<counted(148 * 8), CSR_THREADS, 0, s>>>(p);
-        csr_huge_fold_kernel<0, true><<<counted(148 * 2), 256, 0, s>>>(p);
-    }
-    return launch_status();
-}
-
-extern "C" tiga_status tiga_apply_csr_planned(const tiga_csr_plan* plan, const void* plan_buf, const void* x, tiga_dtype x_dtype,
-                                              int32_t F, const float* w, const tiga_msg* msg, float* out,
+extern "C" tiga_status tiga_apply_csr_planned(const tiga_csr* g, const tiga_csr_plan* plan, const void* plan_buf,
+                                              const void* x, tiga_dtype x_dtype, int32_t F, const float* w, const tiga_msg* msg,
+                                              tiga_reducer reducer, float* out, int32_t* argmax,
                                               void* ws, size_t ws_bytes, void* stream) {
+    tiga_status st = check_csr(g);
+    if (st != TIGA_OK) return st;
     if (!plan || !plan_buf || !aligned16(plan_buf)) return TIGA_ERR_INVALID_ARG;
-    if (plan->n_blocks < 1 || plan->n_blocks > TIGA_PLAN_MAX_BLOCKS || plan->n_dst <= 0 || plan->n_edges <= 0) return TIGA_ERR_INVALID_ARG;
+    if (plan->n_dst != g->n_dst || plan->n_src != g->n_src || plan->n_edges != g->n_edges) return TIGA_ERR_INVALID_ARG;
     int nvec, G, VPL;
-    tiga_status st = check_features(F, x_dtype, &nvec, &G, &VPL);
+    st = check_features(F, x_dtype, &nvec, &G, &VPL);
     if (st != TIGA_OK) return st;
     if (nvec > 2) return TIGA_ERR_UNSUPPORTED;            // feature rows of at most 32 bytes: the case the plan exists for
+    if (reducer != TIGA_SUM && reducer != TIGA_MAX) return TIGA_ERR_INVALID_ARG;
     if (!msg) return TIGA_ERR_INVALID_ARG;
     if (msg->kind == TIGA_MSG_COPY) { if (w) return TIGA_ERR_INVALID_ARG; }
-    else if (msg->kind == TIGA_MSG_WEIGHTED) { if (!w) return TIGA_ERR_INVALID_ARG; if (!plan->has_positions) return TIGA_ERR_UNSUPPORTED; }
+    else if (msg->kind == TIGA_MSG_WEIGHTED) { if (!w) return TIGA_ERR_INVALID_ARG; }
     else return TIGA_ERR_UNSUPPORTED;
+    if (g->n_dst == 0) return TIGA_OK;
     if (!out || !aligned16(out) || !x || !aligned16(x) || (w && !aligned16(w))) return TIGA_ERR_INVALID_ARG;
-    if (!ws || !aligned16(ws) || ws_bytes < tiga_csr_planned_workspace_bytes(plan, F)) return TIGA_ERR_WORKSPACE;
+    if (reducer == TIGA_MAX && (!argmax || !aligned16(argmax))) return TIGA_ERR_INVALID_ARG;
+    if (!ws || !aligned16(ws) || ws_bytes < tiga_csr_planned_workspace_bytes(g, plan, F, x_dtype, reducer)) return TIGA_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const char* base = static_cast<const char*>(plan_buf);
-    const int32_t* pcol = reinterpret_cast<const int32_t*>(base + plan->off_col);
-    const int32_t* ppos = plan->off_pos >= 0 ? reinterpret_cast<const int32_t*>(base + plan->off_pos) : nullptr;
-    const int32_t* seg_row = reinterpret_cast<const int32_t*>(base + plan->off_seg_row);
-    const int32_t* seg_ptr = reinterpret_cast<const int32_t*>(base + plan->off_seg_ptr);
 
     CsrParams p{};
-    p.col = pcol; p.w = w; p.epos = w ? ppos : nullptr; p.x = x; p.out = out;
-    p.n_edges = plan->n_edges; p.F = F; p.nvec = nvec;
-    const size_t cap = planned_chunk_capacity(plan);
+    p.rowptr = g->rowptr; p.col = reinterpret_cast<const int32_t*>(base + plan->off_col);
+    p.w = w; p.x = x; p.out = out; p.arg = argmax;
+    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.F = F; p.nvec = nvec;
+    p.ntiles = num_tiles(g);
     Carver cv(ws);
+    const size_t row_bytes = (size_t)F * (x_dtype == TIGA_F32 ? 4 : 2);
+    void* hot = cv.take<unsigned char>((size_t)plan->n_hot * row_bytes + 256);
+    p.x_hot = hot; p.n_hot = (int)plan->n_hot;
+    p.carry_row = cv.take<int32_t>((size_t)p.ntiles + 1);
+    p.carry_val = cv.take<float>(((size_t)p.ntiles + 1) * F);
+    p.carry_arg = reducer == TIGA_MAX ? cv.take<int32_t>(((size_t)p.ntiles + 1) * F) : nullptr;
     p.huge_count = cv.take<int>(1);
-    p.huge_list = cv.take<int4>(cap);
-    p.carry_val = cv.take<float>(cap * (size_t)F);
-    // rows start from zero; every pass adds the partial sums of its block, passes run in block order
-    TIGA_CUDA_TRY(cudaMemsetAsync(out, 0, (size_t)plan->n_dst * F * sizeof(float), s));
-    for (int b = 0; b < plan->n_blocks; ++b) {
-        const long long s0 = plan->seg_begin[b], s1 = plan->seg_begin[b + 1];
-        if (s1 <= s0) continue;
-        p.rowptr = seg_ptr + s0; p.row_map = seg_row + s0; p.n_dst = s1 - s0;
-        const bool huge = plan->huge_segments[b] > 0;
-        if (x_dtype == TIGA_F32) st = nvec == 1 ? launch_planned_pass<float, 1>(p, huge, s) : launch_planned_pass<float, 2>(p, huge, s);
-        else st = nvec == 1 ? launch_planned_pass<__half, 1>(p, huge, s) : launch_planned_pass<__half, 2>(p, huge, s);
-        if (st != TIGA_OK) return st;
+    p.huge_list = cv.take<int4>((size_t)p.ntiles + 1);
+    st = launch_gather_hot(x, reinterpret_cast<const int32_t*>(base + plan->off_hot_id), plan->n_hot, nvec, hot, s);
+    if (st != TIGA_OK) return st;
+    const bool i64 = g->rowptr_type == TIGA_I64;
+    if (x_dtype == TIGA_F32) {
+        if (reducer == TIGA_SUM) return i64 ? launch_fwd_narrow<float, 0, int64_t, true>(p, s) : launch_fwd_narrow<float, 0, int32_t, true>(p, s);
+        return i64 ? launch_fwd_narrow<float, 1, int64_t, true>(p, s) : launch_fwd_narrow<float, 1, int32_t, true>(p, s);
     }
-    return TIGA_OK;
+    if (reducer == TIGA_SUM) return i64 ? launch_fwd_narrow<__half, 0, int64_t, true>(p, s) : launch_fwd_narrow<__half, 0, int32_t, true>(p, s);
+    return i64 ? launch_fwd_narrow<__half, 1, int64_t, true>(p, s) : launch_fwd_narrow<__half, 1, int32_t, true>(p, s);
 }
 
 extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,

@@ -8,11 +8,15 @@ namespace tiga {
 constexpr int CSR_THREADS = 256;
 constexpr int CSR_TILE = 2048;     // merge-path items per CTA
 constexpr int CSR_PAD = 8;         // readable entries behind a tile's staged edges
-constexpr int ROW_HUGE = 8192;     // narrow-row path: rows (segments) above this many edges are cut into chunks
 
 template <typename XT> struct XTraits;
 template <> struct XTraits<float> {
     static constexpr int VW = 4;   // floats per 16-byte vector
+    // acc[k] += x[k]  (a message with unit weight: fma(1, x, acc) rounds exactly like this sum)
+    __device__ static __forceinline__ void add_to(const uint4& v, float* acc) {
+        acc[0] += __uint_as_float(v.x); acc[1] += __uint_as_float(v.y);
+        acc[2] += __uint_as_float(v.z); acc[3] += __uint_as_float(v.w);
+    }
     __device__ static __forceinline__ void unpack(const uint4& v, float* f) {
         f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
         f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
@@ -20,6 +24,17 @@ template <> struct XTraits<float> {
 };
 template <> struct XTraits<__half> {
     static constexpr int VW = 8;
+    // acc[k] += x[k] with the mixed-precision add of sm_100 (the half is widened exactly, one rounding)
+    __device__ static __forceinline__ void add_to(const uint4& v, float* acc) {
+        const unsigned r[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            unsigned short lo, hi;
+            asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(r[k]));
+            asm("add.rn.f32.f16 %0, %1, %0;" : "+f"(acc[2 * k]) : "h"(lo));
+            asm("add.rn.f32.f16 %0, %1, %0;" : "+f"(acc[2 * k + 1]) : "h"(hi));
+        }
+    }
     __device__ static __forceinline__ void unpack(const uint4& v, float* f) {
         const __half2* h = reinterpret_cast<const __half2*>(&v);
 #pragma unroll
@@ -47,9 +62,9 @@ struct CsrParams {
     long long ntiles;
     int* huge_count;         // narrow-row path: number of queued chunks of huge rows
     int4* huge_list;         // (row, chunk, chunks of the row, first slot of the row)
-    // planned apply (csr.cu, narrow rows): the "rows" are (destination row, source block) segments
-    const int32_t* row_map;  // segment -> destination row whose output it is added to
-    const int32_t* epos;     // permuted edge -> original edge position (indexes w), or null
+    // planned apply (narrow rows): the most often gathered source rows are served from a compact copy
+    const void* x_hot;       // [n_hot rows] copy of the hot source rows, or null
+    int n_hot;               // col values below n_hot index x_hot, the others (minus n_hot) x
     // backward
     const float* gy;
     float* gx;
@@ -61,6 +76,9 @@ struct CsrParams {
     float* lse;              // [n_dst] log of the row's total mass (caller's array or workspace)
     float2* carry_ml;        // [ntiles] (running maximum, mass) of a tile's carry-out
 };
+
+// host side, defined in csr_plan.cu: compact copy of the hot source rows, hot[r, :] = x[hot_id[r], :]
+tiga_status launch_gather_hot(const void* x, const int32_t* hot_id, long long n_hot, int nvec, void* hot, cudaStream_t s);
 
 // Number of rows whose row-end item lies before merge diagonal d:
 //   #{ i : rowptr[i+1] + i + 1 <= d }   (strictly increasing in i -> 32-ary search by one warp)

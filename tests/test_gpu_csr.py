@@ -241,6 +241,12 @@ def test_cfg4_full_size(tiga):
     assert np.array_equal(host(hist), ref) and int(host(mx)[0]) == rmx
     y, A, _ = oracle.csr_forward(c["rowptr"], c["col"], c["x"], None, oracle.SUM)
     assert rel_err(out, y, A) <= SUM_TOL
+    # the same forward through the hot-source plan: bit-identical
+    plan = tiga.tiga_csr_plan_build(g, row_bytes=16)
+    assert plan.hot_edges > 0.8 * c["E"]
+    planned, _ = tiga.tiga_apply_csr_planned(plan, xd)
+    torch.cuda.synchronize()
+    assert np.array_equal(host(planned), out)
 
 
 def test_row_gather_probe_runs_and_checks_its_arguments(tiga):

@@ -243,15 +243,14 @@ def test_lennard_jones_dense_cells_span_several_stage_chunks(tiga):
     box = np.array([6.0, 6.0, 6.0], np.float32)
     pos = _separated_points(2600, box, 77, 0.25)
     assert len(pos) > 1800
-    # The pair force goes like d^-14, so a relative error e of d^2 is an error 7 e of the force, and the
-    # closest pairs dominate the sums.  A coordinate relative to the cell corner carries an fp32
-    # rounding of 2^-24 times the cell edge (3 here, against 0.25 between the closest points):
-    # e = 2 * 2^-24 * 3 / 0.25, which is added to the usual tolerance.  Counts stay exact.
-    tol = SUM_TOL + 7.0 * 2.0 * 2.0 ** -24 * 3.0 / 0.25
+    # The pair force goes like d^-14 and the closest pairs (0.25 apart in cells of edge 3) dominate the
+    # sums: a displacement formed from coordinates relative to a cell corner would carry an fp32
+    # rounding of the CELL size and miss the tolerance here.  The kernel subtracts stored original
+    # coordinates (periodic images by exact shifts), so the plain tolerance holds.
     for periodic in ([0, 0, 0], [1, 1, 1]):
         grid, _ = tiga.tiga_radius_grid(len(pos), np.float32(2.0), box, periodic)
         assert max(grid) <= 2
-        _check_lj(tiga, pos, np.float32(2.0), box, periodic, eps=0.3, s=0.3, tol=tol)
+        _check_lj(tiga, pos, np.float32(2.0), box, periodic, eps=0.3, s=0.3)
 
 
 def test_lennard_jones_rows_are_summed_by_atomics(tiga):
