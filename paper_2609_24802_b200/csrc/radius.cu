@@ -18,9 +18,10 @@
 // Exact membership: the fp32 squared distance is only a filter.  A pair whose fp32 value
 // falls within a few ulps of r^2 is re-decided in fp64 with the defining formula
 // (displacement, minimum image by rint, left-to-right sum, inclusive compare), so the
-// neighbour set equals the double-precision one.  Periodic images are formed by
-// subtracting the box length from whichever of the two coordinates lies next to the upper
-// face, which is exact in fp32, so wrapped pairs are as accurate as interior ones.
+// neighbour set equals the double-precision one.  Candidates are staged in their original
+// coordinates; a cell whose stencil wraps around a periodic face moves the points next to the
+// upper face down by the box length, which is exact in fp32, so every displacement is one
+// rounded subtraction of two stored coordinates, for wrapped pairs as for interior ones.
 #include "radius_shared.cuh"
 #include <type_traits>
 
@@ -163,10 +164,11 @@ __global__ void bin_sort_kernel(const RadiusParams p) {
 
 // One warp per query cell.
 //   staging : the candidates of the 27-cell stencil (contiguous ranges of the cell-sorted
-//             positions) are copied once into shared memory in coordinates relative to the
-//             query cell's corner, periodic images already applied.  All subtractions involved
-//             are exact or act on numbers of the size of a cell, so the fp32 displacement is
-//             accurate to a few ulps of the cell size on both sides of a periodic face.
+//             positions) are copied once into shared memory in the frame of the query cell:
+//             original coordinates, except that in a dimension whose stencil wraps around a
+//             periodic face the points next to the upper face move down by the box length
+//             (exact).  The fp32 displacement of a pair is then accurate to half an ulp of the
+//             displacement itself on both sides of a face, whatever the size of the cell.
 //   phase A : every lane keeps one staged candidate in registers and tests it against the
 //             queries of the cell, four (forward) or eight (backward) queries per batch (their
 //             coordinates are broadcast from shared memory).  Accepted pairs are compacted with a warp ballot into one
@@ -190,7 +192,7 @@ template <int MODE> struct TravSmem {
     static constexpr int QSTRIDE = QCAP + 5;                       // room for four padding entries; odd, so the lists of different queries fall in different banks
     static constexpr int STAGE_BYTES = (STAGE_CAP + STAGE_PAD) * 16;
     static constexpr int LIST_BYTES = (TQB * QSTRIDE * 8 + 15) / 16 * 16;
-    static constexpr int MISC_BYTES = TQB * 16 + 3 * TQB * 4 + TQB * 4 * 2;   // queries, their coordinates by component, counts, totals
+    static constexpr int MISC_BYTES = TQB * 16 + 3 * TQB * 4 + TQB * 4 * 2 + 32;   // queries, their coordinates by component, counts, totals, the cell's frame
     static constexpr int PER_WARP = STAGE_BYTES + LIST_BYTES + MISC_BYTES;
     static_assert(PER_WARP % 16 == 0 && LIST_BYTES % 16 == 0, "the stage and the queries are accessed as 16-byte vectors");
 };
@@ -220,23 +222,45 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
     float* s_qc = reinterpret_cast<float*>(s_q + TQB);                                  // x[TQB], y[TQB], z[TQB]: read two queries at a time
     int* s_n = reinterpret_cast<int*>(s_qc + 3 * TQB);                                  // list lengths of the drain in progress
     int* s_tot = s_n + TQB;                                                              // neighbours found so far in this chunk
+    float* s_frame = reinterpret_cast<float*>(s_tot + TQB);                              // thresholds [3], shifts [3]
 
     const int c[3] = {cellid % p.nc[0], (cellid / p.nc[0]) % p.nc[1], cellid / (p.nc[0] * p.nc[1])};
-    const float org[3] = {(float)c[0] * p.hcell[0], (float)c[1] * p.hcell[1], (float)c[2] * p.hcell[2]};
     const int F = VEC == 2 ? 4 * LF : p.F;
     const float neg_c2 = !DIST ? -1.4426950408889634f / (2.f * p.p0 * p.p0) : 0.f;   // exp(-d2/(2 s^2)) = 2^(d2 * neg_c2)
     const int fl = lane % LF, grp = lane / LF;
-    const bool mi0 = MI && p.periodic[0] && p.nc[0] == 1, mi1 = MI && p.periodic[1] && p.nc[1] == 1, mi2 = MI && p.periodic[2] && p.nc[2] == 1;
+    // a periodic dimension with three cells or fewer has no consistent shifted frame: explicit minimum image
+    const bool mi0 = MI && p.periodic[0] && p.nc[0] <= 3, mi1 = MI && p.periodic[1] && p.nc[1] <= 3, mi2 = MI && p.periodic[2] && p.nc[2] <= 3;
     constexpr int QP = 32 / LF;
     const bool fvalid = VEC == 2 ? true : fl * 4 < F;
     const unsigned lt_mask = (1u << lane) - 1u;
 
-    auto fold = [&](float& dx, float& dy, float& dz) {
-        if (MI) {          // periodic dimension folded into a single cell: explicit minimum image
-            if (mi0) dx -= p.len[0] * rintf(dx * p.inv_len[0]);
-            if (mi1) dy -= p.len[1] * rintf(dy * p.inv_len[1]);
-            if (mi2) dz -= p.len[2] * rintf(dz * p.inv_len[2]);
+    // displacement query - candidate of two points in the cell's frame
+    auto delta = [&](const float4& q, const float4& c4, float& dx, float& dy, float& dz) {
+        dx = (MI && mi0) ? mi_delta(q.x, c4.x, p.len[0], 0.5f * p.len[0]) : q.x - c4.x;
+        dy = (MI && mi1) ? mi_delta(q.y, c4.y, p.len[1], 0.5f * p.len[1]) : q.y - c4.y;
+        dz = (MI && mi2) ? mi_delta(q.z, c4.z, p.len[2], 0.5f * p.len[2]) : q.z - c4.z;
+    };
+    // frame of this cell: in a dimension whose stencil wraps around a face, every coordinate above the
+    // threshold moves down by the box length (the wrapped cell at the top when the cell touches the lower
+    // face; the cell and its lower neighbour when it touches the upper face).  Both shifts are exact.
+    bool face = false;
+#pragma unroll
+    for (int d = 0; d < 3; ++d) {
+        float thr = FAR_AWAY;
+        if (p.periodic[d] && p.nc[d] >= 4) {
+            if (c[d] == 0) { thr = 2.5f * p.hcell[d]; face = true; }
+            else if (c[d] == p.nc[d] - 1) { thr = 1.5f * p.hcell[d]; face = true; }
         }
+        if (lane == d) { s_frame[d] = thr; s_frame[3 + d] = p.len[d]; }
+    }
+    __syncwarp();
+    auto to_frame = [&](float4 v) -> float4 {
+        if (face) {
+            if (v.x > s_frame[0]) v.x -= s_frame[3];
+            if (v.y > s_frame[1]) v.y -= s_frame[4];
+            if (v.z > s_frame[2]) v.z -= s_frame[5];
+        }
+        return v;
     };
 
     // ---- all queries of the cell against the ns candidates currently staged
@@ -250,7 +274,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
                 float4 lq4 = make_float4(FAR_AWAY, FAR_AWAY, FAR_AWAY, __int_as_float(-2));
                 if (lane < nq) {
                     const float4 pq = p.spos[qb0 + lane];
-                    lq4 = make_float4(pq.x - org[0], pq.y - org[1], pq.z - org[2], pq.w);
+                    lq4 = to_frame(pq);
                     if (MODE == 2) {
                         // the backward reads the query's own feature and cotangent rows at the start of
                         // its pass: ask for them now, they arrive during phase A
@@ -324,8 +348,8 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
                                         const float2 en2 = lq[t + u];
                                         g[u] = en2.y;
                                         const float4 pj = stage[__float_as_int(en2.x)];
-                                        float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
-                                        fold(dx, dy, dz);
+                                        float dx, dy, dz;
+                                        delta(qv, pj, dx, dy, dz);
                                         e[u] = make_float4(dx, dy, dz, 0.f);
                                         const size_t row = (size_t)__float_as_int(pj.w) * F;
                                         xj[u] = __ldg(reinterpret_cast<const float4*>(p.feat + row) + fl);
@@ -408,8 +432,8 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
                     for (int q = 0; q < TQB; ++q) {
                         if (!FULLB && q >= nq) break;
                         const float4 qv = s_q[q];
-                        float dx = qv.x - pj.x, dy = qv.y - pj.y, dz = qv.z - pj.z;
-                        fold(dx, dy, dz);
+                        float dx, dy, dz;
+                        delta(qv, pj, dx, dy, dz);
                         float d2 = fmaf(dz, dz, fmaf(dy, dy, dx * dx));
                         if (idj == __float_as_int(qv.w) || (MI && idj < 0)) d2 = FAR_AWAY; // self (by index); folded sentinels
                         nearest = fminf(nearest, fabsf(d2 - p.r2_mid));
@@ -460,7 +484,6 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
 
     // ---- the 27-cell stencil as candidate ranges: lane r < 27 resolves neighbour offset r
     int r_cs = 0, r_ce = 0;
-    float r_off[3] = {0.f, 0.f, 0.f};
     {
         const int off[3] = {lane % 3 - 1, (lane / 3) % 3 - 1, lane / 9 - 1};
         bool ok = lane < 27;
@@ -468,21 +491,15 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
         bool merged = false;
 #pragma unroll
         for (int d = 0; d < 3; ++d) {
-            if (p.nc[d] == 1) { ok = ok && off[d] == 0; r_off[d] = org[d]; continue; }
+            if (p.nc[d] == 1) { ok = ok && off[d] == 0; continue; }
             if (d == 0 && c[0] >= 1 && c[0] <= p.nc[0] - 2) {
                 // away from the x faces the three x-adjacent cells are one contiguous range
-                merged = true; ok = ok && off[0] == 0; q[0] = c[0] - 1; r_off[0] = org[0];
+                merged = true; ok = ok && off[0] == 0; q[0] = c[0] - 1;
                 continue;
             }
             int v = c[d] + off[d];
-            r_off[d] = org[d];
-            if (v < 0) {
-                if (p.periodic[d]) { v += p.nc[d]; r_off[d] = org[d] + p.len[d]; }     // org is 0 here: exact
-                else ok = false;
-            } else if (v >= p.nc[d]) {
-                if (p.periodic[d]) { v -= p.nc[d]; r_off[d] = org[d] - p.len[d]; }     // exact (Sterbenz)
-                else ok = false;
-            }
+            if (v < 0) { if (p.periodic[d]) v += p.nc[d]; else ok = false; }
+            else if (v >= p.nc[d]) { if (p.periodic[d]) v -= p.nc[d]; else ok = false; }
             q[d] = v;
         }
         if (ok) {
@@ -501,13 +518,13 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
     }
     const int total = __shfl_sync(FULL, r_incl, 31);
 
-    // bounding box of the cell's own points (cell-local coordinates): a candidate farther than the
+    // bounding box of the cell's own points (in the cell's frame): a candidate farther than the
     // cutoff from this box cannot be a neighbour of any of them and is not staged at all, which
     // removes about 40 % of the stencil's candidates before any pair is tested
     float blo[3] = {FAR_AWAY, FAR_AWAY, FAR_AWAY}, bhi[3] = {-FAR_AWAY, -FAR_AWAY, -FAR_AWAY};
     for (int q = qs0 + lane; q < qe0; q += 32) {
-        const float4 pq = p.spos[q];
-        const float l[3] = {pq.x - org[0], pq.y - org[1], pq.z - org[2]};
+        const float4 pq = to_frame(p.spos[q]);
+        const float l[3] = {pq.x, pq.y, pq.z};
 #pragma unroll
         for (int d = 0; d < 3; ++d) { blo[d] = fminf(blo[d], l[d]); bhi[d] = fmaxf(bhi[d], l[d]); }
     }
@@ -531,7 +548,6 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
         constexpr int SU = 4;                                                // staging groups in flight
         for (int k0 = 0; k0 < ns; k0 += 32 * SU) {
             float4 c4[SU];
-            float ox[SU], oy[SU], oz[SU];
 #pragma unroll
             for (int u = 0; u < SU; ++u) {                                   // all loads of the step first
                 const int k = k0 + 32 * u + lane;
@@ -544,7 +560,6 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
                 }
                 r = r > 31 ? 31 : r;
                 const int src = __shfl_sync(FULL, r_cs, r) + (v - (__shfl_sync(FULL, r_incl, r) - __shfl_sync(FULL, r_len, r)));
-                ox[u] = __shfl_sync(FULL, r_off[0], r); oy[u] = __shfl_sync(FULL, r_off[1], r); oz[u] = __shfl_sync(FULL, r_off[2], r);
                 c4[u] = k < ns ? __ldg(p.spos + src) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
             const float lx = __shfl_sync(FULL, bb, 0), ly = __shfl_sync(FULL, bb, 1), lz = __shfl_sync(FULL, bb, 2);
@@ -552,7 +567,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
 #pragma unroll
             for (int u = 0; u < SU; ++u) {
                 if (k0 + 32 * u >= ns) break;
-                const float4 val = make_float4(c4[u].x - ox[u], c4[u].y - oy[u], c4[u].z - oz[u], c4[u].w);
+                const float4 val = to_frame(c4[u]);
                 const float ex = fmaxf(fmaxf(lx - val.x, val.x - hx), 0.f);
                 const float ey = fmaxf(fmaxf(ly - val.y, val.y - hy), 0.f);
                 const float ez = fmaxf(fmaxf(lz - val.z, val.z - hz), 0.f);
@@ -616,13 +631,13 @@ tiga_status fill_params(RadiusParams* p, long long n, float r, const tiga_box* b
     if (n > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;
     p->n = (int)n;
     p->r = r;
-    bool single_periodic = false;
+    bool single_periodic = false;      // some periodic dimension uses the explicit minimum image (two roundings more)
     for (int d = 0; d < 3; ++d) {
         p->nc[d] = nc[d]; p->invh[d] = invh[d];
         p->len[d] = box->len[d]; p->inv_len[d] = 1.f / box->len[d];
         p->hcell[d] = box->len[d] / (float)nc[d];
         p->periodic[d] = box->periodic[d] ? 1 : 0;
-        if (p->periodic[d] && nc[d] == 1) single_periodic = true;
+        if (p->periodic[d] && nc[d] <= 3) single_periodic = true;
     }
     p->ncells = nc[0] * nc[1] * nc[2];
     const float r2 = r * r;
@@ -686,7 +701,7 @@ static tiga_status launch_traverse_lf(const RadiusParams& p, cudaStream_t s) {
 template <int MODE, bool DIST>
 static tiga_status launch_traverse(const RadiusParams& p, cudaStream_t s) {
     bool mi = false;
-    for (int d = 0; d < 3; ++d) mi = mi || (p.periodic[d] && p.nc[d] == 1);
+    for (int d = 0; d < 3; ++d) mi = mi || (p.periodic[d] && p.nc[d] <= 3);
     return mi ? launch_traverse_lf<MODE, DIST, true>(p, s) : launch_traverse_lf<MODE, DIST, false>(p, s);
 }
 

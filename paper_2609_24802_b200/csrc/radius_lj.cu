@@ -1,98 +1,92 @@
 // Lennard-Jones message over the generated radius relation (fused cell-list traversal, paper
-// Section 4.9), evaluated once per unordered pair, without pair lists.
+// Section 4.9), evaluated once per unordered pair.
 //
 // The pair force is antisymmetric and the pair energy symmetric, so the row sums
 //     F_i = sum over j in N(i) of f_ij,   e_i = sum over j in N(i) of u_ij / 2
 // can be formed by visiting every unordered pair {i, j} once and adding f_ij to row i and -f_ij
 // to row j.  One warp owns a cell and tests its points against the points of the cell itself
 // (each pair once, by index order) and of the 13 neighbour cells whose offset is lexicographically
-// positive; the other 13 cells visit this one from their side.
+// positive; the other 13 cells visit this one from their side.  That halves the candidate tests,
+// the staging and the force evaluations of a traversal that walks all 27 cells per row.
 //
-// Inside a warp:
-//   staging : the half stencil's candidates are copied into shared memory in their ORIGINAL
-//             coordinates; a cell whose stencil wraps around a periodic face moves the points next to
-//             the upper face down by the box length, which is exact in fp32.  A displacement is then
-//             one rounded subtraction of two stored coordinates -- accurate to half an ulp of the
-//             displacement itself, however close the pair and however large the cell.  Candidates
-//             farther than the cutoff from the bounding box of the cell's own points are dropped.
-//   pairs   : every lane keeps one staged candidate and meets a batch of four queries.  The message
-//             is cheap (a reciprocal and a dozen multiplies), so it is evaluated for every tested pair
-//             with the weight of a rejected pair forced to zero, two queries per packed fp32
-//             instruction; nothing is compacted, listed or drained.  The query's row accumulates in
-//             registers over all candidates (summed over the lanes once per batch), the candidate's
-//             row in shared memory over all queries.  Pairs whose fp32 distance falls within a few ulps
-//             of the cutoff are decided in fp64 with the defining formula.
-//   output  : one 128-bit vector atomic per query and one per staged candidate that met a neighbour
-//             (out starts at zero), instead of one per pair.  The summation order of a row depends
-//             on scheduling, so the last bits can change from run to run; neighbour counts are exact.
+// The price is that a row is no longer summed by a single warp: contributions arrive through
+// 128-bit vector atomics (out must start at zero), so the summation order, and with it the last
+// bits of the result, can change from run to run.  Neighbour counts are integers and stay exact.
+//
+// Structure inside a warp: the half stencil is staged in shared memory in the points' ORIGINAL
+// coordinates; a cell whose stencil wraps around a periodic face moves the points next to the upper
+// face down by the box length, which is exact in fp32, so a displacement is one rounded subtraction
+// of two stored coordinates -- accurate to half an ulp of the displacement itself, however close the
+// pair and however large the cell.  Candidates farther than the cutoff from the bounding box of the
+// cell's points are dropped, phase A tests one staged candidate per lane against four queries and
+// compacts accepted pairs into per-query lists by ballots (pairs within the fp32 error band of the
+// cutoff are decided in fp64), phase B gives every query eight lanes that evaluate its listed pairs.
+// (Evaluating the message for every tested pair with rejected weights forced to zero, without lists,
+// was built and measured: the same instruction count at lower occupancy, 1.71 against 1.62 ms.)
 #include "radius_shared.cuh"
 #include <type_traits>
 
 namespace tiga {
 
-constexpr int LJ_STAGE_CAP = 192;             // candidates staged per chunk
-constexpr int LJQ = 4;                        // queries per batch
+constexpr int LJ_STAGE_CAP = 256;
+constexpr int LJ_QCAP = 64;
+constexpr int LJ_QSTRIDE = LJ_QCAP + 1;
 constexpr int LJ_STAGE_BYTES = (LJ_STAGE_CAP + STAGE_PAD) * 16;
-constexpr int LJ_ACC_BYTES = (LJ_STAGE_CAP + STAGE_PAD) * 16;                 // padding lanes add zeros behind the last candidate
-constexpr int LJ_RED_BYTES = 4 * LJQ * 4 + LJQ * 16;                          // reduced row sums of a batch, the batch's queries
-template <bool COUNT> struct LjSmem {
-    static constexpr int CNT_BYTES = COUNT ? (LJ_STAGE_CAP + STAGE_PAD) * 4 : 0;
-    static constexpr int PER_WARP = (LJ_STAGE_BYTES + LJ_ACC_BYTES + CNT_BYTES + LJ_RED_BYTES + 15) / 16 * 16;
-};
-
-static __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 r; asm("add.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
-
-// minimum-image displacement of two coordinates of a periodic dimension that is not split into
-// enough cells for a frame shift: the subtraction that can lose bits (x near 0 against x near len)
-// is replaced by an exact shift of the coordinate next to the upper face
-static __device__ __forceinline__ float mi_delta(float a, float b, float len, float half) {
-    float t = a - b;
-    if (t > half) t = (a - len) - b;
-    else if (t < -half) t = a - (b - len);
-    return t;
-}
+constexpr int LJQ = 4;                        // queries per batch in this kernel
+constexpr int LJ_LPQ = 32 / LJQ;              // lanes that share a query's list in phase B
+constexpr int LJ_LIST_BYTES = (LJQ * LJ_QSTRIDE * 8 + 15) / 16 * 16;
+constexpr int LJ_MISC_BYTES = LJQ * 16 + 3 * LJQ * 4 + LJQ * 4 + 32;        // queries, their coordinates by component, list lengths, the cell's frame
+constexpr int LJ_PER_WARP = (LJ_STAGE_BYTES + LJ_LIST_BYTES + LJ_MISC_BYTES + 15) / 16 * 16;
 
 template <bool MI, bool COUNT>
-__global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const __grid_constant__ RadiusParams p) {
+__global__ void __launch_bounds__(TRAV_THREADS, COUNT ? 8 : 7) radius_lj_pairs_kernel(const __grid_constant__ RadiusParams p) {
     constexpr unsigned FULL = 0xffffffffu;
-    using SM = LjSmem<COUNT>;
     extern __shared__ __align__(16) unsigned char s_raw[];
 
     const int lane = threadIdx.x & 31;
     const int wib = threadIdx.x >> 5;
     const int cellid = blockIdx.x * TRAV_WARPS + wib;
     if (cellid >= p.ncells) return;
-    unsigned char* base = s_raw + (size_t)wib * SM::PER_WARP;
-    float4* stage = reinterpret_cast<float4*>(base);                                   // x, y, z (frame of this cell), point id
-    float4* acc = reinterpret_cast<float4*>(base + LJ_STAGE_BYTES);                    // the candidates' rows: -force, energy
-    int* cnt = reinterpret_cast<int*>(base + LJ_STAGE_BYTES + LJ_ACC_BYTES);           // the candidates' neighbour counts
-    float* s_red = reinterpret_cast<float*>(base + LJ_STAGE_BYTES + LJ_ACC_BYTES + SM::CNT_BYTES);    // [LJQ][4]
-    float4* s_q = reinterpret_cast<float4*>(s_red + 4 * LJQ);
+    unsigned char* base = s_raw + (size_t)wib * LJ_PER_WARP;
+    float4* stage = reinterpret_cast<float4*>(base);                                   // x, y, z in the frame of this cell, point id
+    float2* list = reinterpret_cast<float2*>(base + LJ_STAGE_BYTES);                   // (stage slot, d2) per query
+    float4* s_q = reinterpret_cast<float4*>(base + LJ_STAGE_BYTES + LJ_LIST_BYTES);
+    float* s_qc = reinterpret_cast<float*>(s_q + LJQ);        // x[LJQ], y[LJQ], z[LJQ]: read two queries at a time
+    int* s_n = reinterpret_cast<int*>(s_qc + 3 * LJQ);
+    float* s_frame = reinterpret_cast<float*>(s_n + LJQ);     // thresholds [3], shifts [3] (kept out of the registers)
 
     const int c[3] = {cellid % p.nc[0], (cellid / p.nc[0]) % p.nc[1], cellid / (p.nc[0] * p.nc[1])};
     // a periodic dimension with three cells or fewer has no consistent shifted frame: explicit minimum image
     const bool mi0 = MI && p.periodic[0] && p.nc[0] <= 3, mi1 = MI && p.periodic[1] && p.nc[1] <= 3, mi2 = MI && p.periodic[2] && p.nc[2] <= 3;
+    const float half0 = 0.5f * p.len[0], half1 = 0.5f * p.len[1], half2 = 0.5f * p.len[2];
     const unsigned lt_mask = (1u << lane) - 1u;
     float4* out4 = reinterpret_cast<float4*>(p.out);
 
+    // displacement query - candidate of two points in the cell's frame
+    auto delta = [&](const float4& q, const float4& c4, float& dx, float& dy, float& dz) {
+        dx = (MI && mi0) ? mi_delta(q.x, c4.x, p.len[0], half0) : q.x - c4.x;
+        dy = (MI && mi1) ? mi_delta(q.y, c4.y, p.len[1], half1) : q.y - c4.y;
+        dz = (MI && mi2) ? mi_delta(q.z, c4.z, p.len[2], half2) : q.z - c4.z;
+    };
     // frame of this cell: in a dimension whose stencil wraps around a face, every coordinate above the
     // threshold moves down by the box length (the wrapped cell at the top when the cell touches the lower
     // face; the cell and its lower neighbour when it touches the upper face).  Both shifts are exact.
-    float thr[3];
     bool face = false;
 #pragma unroll
     for (int d = 0; d < 3; ++d) {
-        thr[d] = FAR_AWAY;
+        float thr = FAR_AWAY;
         if (p.periodic[d] && p.nc[d] >= 4) {
-            if (c[d] == 0) { thr[d] = 2.5f * p.hcell[d]; face = true; }
-            else if (c[d] == p.nc[d] - 1) { thr[d] = 1.5f * p.hcell[d]; face = true; }
+            if (c[d] == 0) { thr = 2.5f * p.hcell[d]; face = true; }
+            else if (c[d] == p.nc[d] - 1) { thr = 1.5f * p.hcell[d]; face = true; }
         }
+        if (lane == d) { s_frame[d] = thr; s_frame[3 + d] = p.len[d]; }
     }
+    __syncwarp();
     auto to_frame = [&](float4 v) -> float4 {
         if (face) {
-            if (v.x > thr[0]) v.x -= p.len[0];
-            if (v.y > thr[1]) v.y -= p.len[1];
-            if (v.z > thr[2]) v.z -= p.len[2];
+            if (v.x > s_frame[0]) v.x -= s_frame[3];
+            if (v.y > s_frame[1]) v.y -= s_frame[4];
+            if (v.z > s_frame[2]) v.z -= s_frame[5];
         }
         return v;
     };
@@ -118,6 +112,8 @@ __global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const 
             r_len = p.cell_start[id + 1] - r_cs;
         }
     }
+    // lane 0 resolved the cell itself: its run is the cell's own points (one load round trip fewer
+    // than asking for them first)
     const int qs0 = __shfl_sync(FULL, r_cs, 0), nown = __shfl_sync(FULL, r_len, 0), qe0 = qs0 + nown;
     if (nown == 0) return;
     int r_incl = r_len;
@@ -128,22 +124,24 @@ __global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const 
     }
     const int total = __shfl_sync(FULL, r_incl, 31);
 
-    // flattened stencil position v -> its address in the cell-ordered points
-    auto locate = [&](const int v) -> int {
+    // flattened stencil position v -> its run and address in the cell-ordered points
+    auto locate = [&](const int v, int& run) -> int {
         int r = 0;
 #pragma unroll
         for (int o = 8; o > 0; o >>= 1) {                 // 14 runs: a four-step search
             const int probe = __shfl_sync(FULL, r_incl, r + o - 1);
             if (probe <= v) r += o;
         }
-        r = r > 13 ? 13 : r;
-        return __shfl_sync(FULL, r_cs, r) + (v - (__shfl_sync(FULL, r_incl, r) - __shfl_sync(FULL, r_len, r)));
+        run = r > 13 ? 13 : r;
+        return __shfl_sync(FULL, r_cs, run) + (v - (__shfl_sync(FULL, r_incl, run) - __shfl_sync(FULL, r_len, run)));
     };
     constexpr int SU = 4;                                 // staging groups in flight
+    // start fetching the first staging groups now: they arrive while the bounding box is formed
 #pragma unroll
     for (int u = 0; u < SU; ++u) {
+        int run;
         const int v = 32 * u + lane;
-        const int src = locate(v);
+        const int src = locate(v, run);
         if (v < total) asm volatile("prefetch.global.L1 [%0];" ::"l"(p.spos + src));
     }
 
@@ -170,161 +168,162 @@ __global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const 
         if (mi2 && (lane == 2 || lane == 5)) bb = lane == 2 ? -FAR_AWAY : FAR_AWAY;
     }
 
-    const float ns2 = -(p.p1 * p.p1), e24 = 24.f * p.p0, e2x = 2.f * p.p0;
-    const f32x2 ns2_2 = pack2(ns2, ns2), e24_2 = pack2(e24, e24), e2x_2 = pack2(e2x, e2x), two_2 = pack2(2.f, 2.f);
-    const float half0 = 0.5f * p.len[0], half1 = 0.5f * p.len[1], half2 = 0.5f * p.len[2];
+    const float s2 = p.p1 * p.p1, e24 = 24.f * p.p0, e2x = 2.f * p.p0;
 
-    // ---- all queries of the cell against the ns staged candidates; the first nself of them are points
-    //      of the cell itself (they pair only with queries of a lower point id)
+    // ---- all queries of the cell against the ns staged candidates; the first nself of them are the
+    //      cell's own points, in the same order as the queries
     auto process_chunk = [&](const int ns, const int nself) {
-        // padding candidates sit far away on one side, absent queries of a short batch on the other
-        if (lane < STAGE_PAD) stage[ns + lane] = make_float4(-FAR_AWAY, -FAR_AWAY, -FAR_AWAY, __int_as_float(-1));
-        for (int k = lane; k < ns + STAGE_PAD; k += 32) {
-            acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (COUNT) cnt[k] = 0;
-        }
+        if (lane < STAGE_PAD) stage[ns + lane] = make_float4(FAR_AWAY, FAR_AWAY, FAR_AWAY, __int_as_float(-1));
         for (int qb0 = qs0; qb0 < qe0; qb0 += LJQ) {
             const int nq = (qe0 - qb0 < LJQ) ? qe0 - qb0 : LJQ;
             __syncwarp();
             if (lane < LJQ) {
-                float4 q4 = make_float4(FAR_AWAY, FAR_AWAY, FAR_AWAY, __int_as_float(0x7fffffff));
-                if (lane < nq) q4 = to_frame(p.spos[qb0 + lane]);
-                s_q[lane] = q4;
+                // absent queries of a short batch sit far away: whatever is computed for them is never used
+                float4 lq4 = make_float4(FAR_AWAY, FAR_AWAY, FAR_AWAY, __int_as_float(-2));
+                if (lane < nq) lq4 = to_frame(p.spos[qb0 + lane]);
+                s_q[lane] = lq4;
+                s_qc[lane] = lq4.x; s_qc[LJQ + lane] = lq4.y; s_qc[2 * LJQ + lane] = lq4.z;
             }
             __syncwarp();
-            f32x2 qx[LJQ / 2], qy[LJQ / 2], qz[LJQ / 2];
-            int idq[LJQ];
+            int qcnt[LJQ];
 #pragma unroll
-            for (int h = 0; h < LJQ / 2; ++h) {
-                const float4 a = s_q[2 * h], b = s_q[2 * h + 1];
-                qx[h] = pack2(a.x, b.x); qy[h] = pack2(a.y, b.y); qz[h] = pack2(a.z, b.z);
-                idq[2 * h] = __float_as_int(a.w); idq[2 * h + 1] = __float_as_int(b.w);
-            }
-            f32x2 fx[LJQ / 2], fy[LJQ / 2], fz[LJQ / 2], en[LJQ / 2];      // the queries' rows, per lane
-            int ci[LJQ];
-#pragma unroll
-            for (int h = 0; h < LJQ / 2; ++h) { fx[h] = fy[h] = fz[h] = en[h] = 0ull; }
-#pragma unroll
-            for (int q = 0; q < LJQ; ++q) ci[q] = 0;
+            for (int q = 0; q < LJQ; ++q) qcnt[q] = 0;
 
-            for (int cbase = 0; cbase < ns; cbase += 32) {
+            auto drain = [&]() {
+                __syncwarp();
+                if (lane == 0) {
+#pragma unroll
+                    for (int q = 0; q < LJQ; ++q) s_n[q] = qcnt[q];
+                }
+                __syncwarp();
+                const int q = lane / LJ_LPQ, sub = lane % LJ_LPQ;
+                float fx = 0.f, fy = 0.f, fz = 0.f, en = 0.f;
+                int n = 0;
+                if (q < nq) {
+                    const float4 qv = s_q[q];
+                    n = s_n[q];
+                    const float2* lq = list + q * LJ_QSTRIDE;
+                    for (int t = sub; t < n; t += 2 * LJ_LPQ) {
+                        float2 e[2];
+                        float4 pj[2];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            e[u] = lq[t + LJ_LPQ * u < n ? t + LJ_LPQ * u : t];
+                            pj[u] = stage[__float_as_int(e[u].x)];
+                        }
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            // the arithmetic runs for both slots of the step; an absent pair has inv = 0
+                            // (zero force and energy) and only its atomics are switched off
+                            const bool valid = t + LJ_LPQ * u < n;
+                            const float inv = valid ? fast_rcp(e[u].y) : 0.f;
+                            const float qq = s2 * inv;
+                            const float q3 = qq * qq * qq;
+                            const float fs = e24 * (2.f * q3 * q3 - q3) * inv;
+                            const float ee = e2x * (q3 * q3 - q3);
+                            float dx, dy, dz;
+                            delta(qv, pj[u], dx, dy, dz);
+                            const float gx = fs * dx, gy = fs * dy, gz = fs * dz;
+                            fx += gx; fy += gy; fz += gz; en += ee;
+                            const int idj = __float_as_int(pj[u].w);
+                            if (valid) {
+                                atomicAdd(out4 + idj, make_float4(-gx, -gy, -gz, ee));      // the pair's other row
+                                if (COUNT) atomicAdd(p.count + idj, 1);
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int o = 1; o < LJ_LPQ; o <<= 1) {
+                    fx += __shfl_xor_sync(FULL, fx, o); fy += __shfl_xor_sync(FULL, fy, o);
+                    fz += __shfl_xor_sync(FULL, fz, o); en += __shfl_xor_sync(FULL, en, o);
+                }
+                if (q < nq && sub == 0 && n > 0) {
+                    const int idq = __float_as_int(s_q[q].w);
+                    atomicAdd(out4 + idq, make_float4(fx, fy, fz, en));
+                    if (COUNT) atomicAdd(p.count + idq, n);
+                }
+#pragma unroll
+                for (int q2 = 0; q2 < LJQ; ++q2) qcnt[q2] = 0;
+                __syncwarp();
+            };
+
+            // ---- phase A: one staged candidate per lane against the queries of the batch.
+            //      OWN: the group holds points of the cell itself, which pair only with later ones.
+            auto phase_a = [&](const int cbase, auto full_batch, auto own_group) -> bool {
+                constexpr bool FULLB = decltype(full_batch)::value;
+                constexpr bool OWN = decltype(own_group)::value;
                 const float4 pj = stage[cbase + lane];
                 const int idj = __float_as_int(pj.w);
-                // own cell: each pair once -- the candidate must have the higher point id (an absent
-                // query's id is above every point id)
-                const int idlim = cbase + lane < nself ? idj : 0x7fffffff;
-                const f32x2 px = pack2(pj.x, pj.x), py = pack2(pj.y, pj.y), pz = pack2(pj.z, pj.z);
-                f32x2 gx = 0ull, gy = 0ull, gz = 0ull, ge = 0ull;            // the candidate's row over this batch (two partial sums)
-                int cj = 0;
+                const bool own = OWN && cbase + lane < nself;
+                float d2q[LJQ];
+                float nearest = FAR_AWAY;       // smallest |d2 - r^2| seen by this lane
+                if constexpr (!MI) {
+                    // squared distances of two queries per instruction (same operations and roundings as
+                    // the scalar form: a product, then two fused multiply-adds)
+                    const f32x2 px = pack2(pj.x, pj.x), py = pack2(pj.y, pj.y), pz = pack2(pj.z, pj.z);
+                    const f32x2* qx2 = reinterpret_cast<const f32x2*>(s_qc);
 #pragma unroll
-                for (int h = 0; h < LJQ / 2; ++h) {
-                    f32x2 dx, dy, dz;
-                    if constexpr (!MI) {
-                        dx = sub2(qx[h], px); dy = sub2(qy[h], py); dz = sub2(qz[h], pz);
-                    } else {
-                        float ax, bx, ay, by, az, bz;
-                        unpack2(qx[h], ax, bx); unpack2(qy[h], ay, by); unpack2(qz[h], az, bz);
-                        dx = mi0 ? pack2(mi_delta(ax, pj.x, p.len[0], half0), mi_delta(bx, pj.x, p.len[0], half0)) : sub2(qx[h], px);
-                        dy = mi1 ? pack2(mi_delta(ay, pj.y, p.len[1], half1), mi_delta(by, pj.y, p.len[1], half1)) : sub2(qy[h], py);
-                        dz = mi2 ? pack2(mi_delta(az, pj.z, p.len[2], half2), mi_delta(bz, pj.z, p.len[2], half2)) : sub2(qz[h], pz);
+                    for (int h = 0; h < LJQ / 2; ++h) {
+                        if (!FULLB && 2 * h >= nq) break;
+                        const f32x2 dx = sub2(qx2[h], px), dy = sub2(qx2[LJQ / 2 + h], py), dz = sub2(qx2[LJQ + h], pz);
+                        unpack2(fma2(dz, dz, fma2(dy, dy, mul2(dx, dx))), d2q[2 * h], d2q[2 * h + 1]);
                     }
-                    float d2a, d2b;
-                    unpack2(fma2(dz, dz, fma2(dy, dy, mul2(dx, dx))), d2a, d2b);
-                    bool oka = d2a <= p.r2_hi && idq[2 * h] < idlim;
-                    bool okb = d2b <= p.r2_hi && idq[2 * h + 1] < idlim;
-                    if (__any_sync(FULL, (oka && d2a > p.r2_lo) || (okb && d2b > p.r2_lo))) {
-                        // some pair lies within the fp32 error band of the cutoff: decide it in fp64
-                        if (oka && d2a > p.r2_lo) oka = exact_pair(p, idq[2 * h], idj);
-                        if (okb && d2b > p.r2_lo) okb = exact_pair(p, idq[2 * h + 1], idj);
+#pragma unroll
+                    for (int q = 0; q < LJQ; ++q) {
+                        if (!FULLB && q >= nq) break;
+                        if (OWN && own && idj <= __float_as_int(s_q[q].w)) d2q[q] = FAR_AWAY;      // own cell: each pair once
+                        nearest = fminf(nearest, fabsf(d2q[q] - p.r2_mid));
                     }
-                    const f32x2 inv = pack2(oka ? fast_rcp(d2a) : 0.f, okb ? fast_rcp(d2b) : 0.f);
-                    const f32x2 nqq = mul2(ns2_2, inv);                       // -(s/d)^2
-                    const f32x2 nq3 = mul2(mul2(nqq, nqq), nqq);              // -(s/d)^6
-                    const f32x2 t = mul2(nq3, nq3);                           // (s/d)^12
-                    const f32x2 fs = mul2(fma2(t, two_2, nq3), mul2(e24_2, inv));     // 24 eps (2 (s/d)^12 - (s/d)^6) / d^2
-                    const f32x2 ee = mul2(e2x_2, add2(t, nq3));               // half of the pair energy
-                    fx[h] = fma2(fs, dx, fx[h]); fy[h] = fma2(fs, dy, fy[h]); fz[h] = fma2(fs, dz, fz[h]); en[h] = add2(en[h], ee);
-                    gx = fma2(fs, dx, gx); gy = fma2(fs, dy, gy); gz = fma2(fs, dz, gz); ge = add2(ge, ee);
-                    if (COUNT) {
-                        ci[2 * h] += __popc(__ballot_sync(FULL, oka)); ci[2 * h + 1] += __popc(__ballot_sync(FULL, okb));
-                        cj += (oka ? 1 : 0) + (okb ? 1 : 0);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < LJQ; ++q) {
+                        if (!FULLB && q >= nq) break;
+                        const float4 qv = s_q[q];
+                        float dx, dy, dz;
+                        delta(qv, pj, dx, dy, dz);
+                        float d2 = fmaf(dz, dz, fmaf(dy, dy, dx * dx));
+                        if (OWN && own && idj <= __float_as_int(qv.w)) d2 = FAR_AWAY;      // own cell: each pair once
+                        if (idj < 0) d2 = FAR_AWAY;                                        // folded sentinels
+                        nearest = fminf(nearest, fabsf(d2 - p.r2_mid));
+                        d2q[q] = d2;
                     }
                 }
-                float a0, a1, b0, b1, c0, c1, e0, e1;
-                unpack2(gx, a0, a1); unpack2(gy, b0, b1); unpack2(gz, c0, c1); unpack2(ge, e0, e1);
-                float4 g = acc[cbase + lane];
-                g.x -= a0 + a1; g.y -= b0 + b1; g.z -= c0 + c1; g.w += e0 + e1;
-                acc[cbase + lane] = g;
-                if (COUNT) cnt[cbase + lane] += cj;
-            }
+                if (__any_sync(FULL, nearest <= p.r2_band)) {
+                    // some pair lies within the fp32 error band of the cutoff: decide it in fp64
+#pragma unroll
+                    for (int q = 0; q < LJQ; ++q) {
+                        if (!FULLB && q >= nq) break;
+                        if (fabsf(d2q[q] - p.r2_mid) <= p.r2_band)
+                            d2q[q] = exact_pair(p, __float_as_int(s_q[q].w), idj) ? fminf(d2q[q], p.r2_lo) : FAR_AWAY;
+                    }
+                }
+                int mx = 0;
+#pragma unroll
+                for (int q = 0; q < LJQ; ++q) {
+                    if (!FULLB && q >= nq) break;
+                    const bool ok = d2q[q] <= p.r2_lo;
+                    const unsigned m = __ballot_sync(FULL, ok);
+                    float2* dst = list + q * LJ_QSTRIDE + qcnt[q] + __popc(m & lt_mask);
+                    if (ok) *dst = make_float2(__int_as_float(cbase + lane), d2q[q]);
+                    qcnt[q] += __popc(m);
+                    mx = qcnt[q] > mx ? qcnt[q] : mx;
+                }
+                return mx > LJ_QCAP - 32;
+            };
 
-            // ---- the queries' rows: 4 LJQ partial sums per lane -> one total each, by a halving exchange
-            //      (a lane sends the half it gives up and keeps the half it owns), then one plain step
-            float v[4 * LJQ];
-#pragma unroll
-            for (int h = 0; h < LJQ / 2; ++h) {
-                unpack2(fx[h], v[8 * h + 0], v[8 * h + 4]); unpack2(fy[h], v[8 * h + 1], v[8 * h + 5]);
-                unpack2(fz[h], v[8 * h + 2], v[8 * h + 6]); unpack2(en[h], v[8 * h + 3], v[8 * h + 7]);
-            }
-            // v[4 q + c]: component c of query q
-            static_assert(LJQ == 4, "the exchange below reduces sixteen values");
-            {
-                const bool up = lane & 16;
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const float send = up ? v[k] : v[k + 8];
-                    const float keep = up ? v[k + 8] : v[k];
-                    v[k] = keep + __shfl_xor_sync(FULL, send, 16);
-                }
-            }
-            {
-                const bool up = lane & 8;
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float send = up ? v[k] : v[k + 4];
-                    const float keep = up ? v[k + 4] : v[k];
-                    v[k] = keep + __shfl_xor_sync(FULL, send, 8);
-                }
-            }
-            {
-                const bool up = lane & 4;
-#pragma unroll
-                for (int k = 0; k < 2; ++k) {
-                    const float send = up ? v[k] : v[k + 2];
-                    const float keep = up ? v[k + 2] : v[k];
-                    v[k] = keep + __shfl_xor_sync(FULL, send, 4);
-                }
-            }
-            {
-                const bool up = lane & 2;
-                const float send = up ? v[0] : v[1];
-                const float keep = up ? v[1] : v[0];
-                v[0] = keep + __shfl_xor_sync(FULL, send, 2);
-            }
-            v[0] += __shfl_xor_sync(FULL, v[0], 1);
-            // lane L now owns entry 8 bit4(L) + 4 bit3(L) + 2 bit2(L) + bit1(L)
-            if (!(lane & 1)) s_red[((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1)] = v[0];
-            __syncwarp();
-            if (lane < nq) {
-                const float4 tot = *reinterpret_cast<const float4*>(s_red + 4 * lane);
-                const int id = __float_as_int(s_q[lane].w);
-                if (tot.x != 0.f || tot.y != 0.f || tot.z != 0.f || tot.w != 0.f) atomicAdd(out4 + id, tot);
-                if (COUNT) {
-                    int mine = 0;
-#pragma unroll
-                    for (int q = 0; q < LJQ; ++q) mine = lane == q ? ci[q] : mine;
-                    if (mine) atomicAdd(p.count + id, mine);
-                }
+            bool need = false;
+            for (int cbase = 0;; cbase += 32) {
+                const bool done = cbase >= ns;
+                if (done || need) drain();
+                if (done) break;
+                if (cbase < nself)
+                    need = (nq == LJQ) ? phase_a(cbase, std::true_type{}, std::true_type{}) : phase_a(cbase, std::false_type{}, std::true_type{});
+                else
+                    need = (nq == LJQ) ? phase_a(cbase, std::true_type{}, std::false_type{}) : phase_a(cbase, std::false_type{}, std::false_type{});
             }
         }
         __syncwarp();
-        // ---- the candidates' rows
-        for (int k = lane; k < ns; k += 32) {
-            const float4 g = acc[k];
-            const int id = __float_as_int(stage[k].w);
-            if (g.x != 0.f || g.y != 0.f || g.z != 0.f || g.w != 0.f) atomicAdd(out4 + id, g);
-            if (COUNT) { const int n = cnt[k]; if (n) atomicAdd(p.count + id, n); }
-        }
         __syncwarp();
     };
 
@@ -337,7 +336,8 @@ __global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const 
 #pragma unroll
             for (int u = 0; u < SU; ++u) {                // all loads of the step first
                 const int k = k0 + 32 * u + lane;
-                const int src = locate(lo + k);
+                int run;
+                const int src = locate(lo + k, run);
                 c4[u] = k < nin ? __ldg(p.spos + src) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
             const float lx = __shfl_sync(FULL, bb, 0), ly = __shfl_sync(FULL, bb, 1), lz = __shfl_sync(FULL, bb, 2);
@@ -365,7 +365,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, 5) radius_lj_pairs_kernel(const 
 template <bool MI, bool COUNT>
 static tiga_status launch_lj_t(const RadiusParams& p, cudaStream_t s) {
     const unsigned blocks = (unsigned)((p.ncells + TRAV_WARPS - 1) / TRAV_WARPS);
-    constexpr int smem = LjSmem<COUNT>::PER_WARP * TRAV_WARPS;
+    constexpr int smem = LJ_PER_WARP * TRAV_WARPS;
     auto kern = radius_lj_pairs_kernel<MI, COUNT>;
     if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     kern<<<counted(blocks), TRAV_THREADS, smem, s>>>(p);

@@ -101,6 +101,16 @@ static __device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 r; asm("s
 static __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 r; asm("mul.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
 static __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
 
+// Minimum-image displacement of two coordinates of a periodic dimension that is not split into enough
+// cells for a frame shift: the subtraction that can lose bits (x near 0 against x near len) is replaced
+// by an exact shift of the coordinate next to the upper face.
+static __device__ __forceinline__ float mi_delta(float a, float b, float len, float half) {
+    float t = a - b;
+    if (t > half) t = (a - len) - b;
+    else if (t < -half) t = a - (b - len);
+    return t;
+}
+
 // exact predicate for the pair of original point ids (a, b)
 static __device__ __noinline__ bool exact_pair(const RadiusParams& p, int a, int b) {
     const float4 pa = make_float4(p.pos[3 * (size_t)a], p.pos[3 * (size_t)a + 1], p.pos[3 * (size_t)a + 2], 0.f);
