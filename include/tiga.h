@@ -43,7 +43,8 @@ typedef enum {
     TIGA_ERR_WORKSPACE = 3,     /* ws is NULL or smaller than *_workspace_bytes() */
     TIGA_ERR_CUDA = 4,          /* a CUDA runtime call failed */
     TIGA_ERR_INVALID_GRAPH = 5, /* tiga_validate_csr found a malformed relation */
-    TIGA_ERR_TOO_LARGE = 6      /* the problem needs more scratch than the library's built-in array holds */
+    TIGA_ERR_TOO_LARGE = 6,     /* the problem needs more scratch than the library's built-in array holds */
+    TIGA_ERR_INVALID_POINTS = 7 /* tiga_validate_points found a coordinate that is not finite or lies outside the box */
 } tiga_status;
 
 typedef enum { TIGA_F32 = 0, TIGA_F16 = 1 } tiga_dtype;   /* feature storage; accumulation is fp32 */
@@ -223,6 +224,15 @@ tiga_status tiga_csr_degree_histogram(const tiga_csr* g, int64_t* hist, int64_t 
  * A point's cell is min(ncell[d]-1, (int)floorf(p[d] * invh[d])) with one fp32 multiply;
  * linear id = (c_z ncell[1] + c_y) ncell[0] + c_x.  Either output may be NULL. */
 tiga_status tiga_radius_grid(int64_t n, float r, const tiga_box* box, int32_t ncell[3], float invh[3]);
+
+/* Validation of point coordinates (Section 6, "Validation and trust boundaries", applied to the
+ * generated relation): the apply calls trust that every coordinate is finite and lies in [0, len[d]];
+ * a point outside is binned into an edge cell and silently misses neighbours.  level 0 checks the
+ * arguments on the host only; level 1 scans the coordinates on the device and SYNCHRONISES the stream.
+ *   pos : fp32 [n, 3];  ws : at least 16 bytes of device memory (level 1).
+ * Returns TIGA_ERR_INVALID_POINTS when a coordinate fails the check. */
+tiga_status tiga_validate_points(const float* pos, int64_t n, const tiga_box* box, int level,
+                                 void* ws, size_t ws_bytes, void* stream);
 
 /* Workspace bytes for tiga_radius_bin / tiga_apply_radius / tiga_apply_radius_backward. */
 size_t tiga_radius_workspace_bytes(int64_t n, int32_t F, float r, const tiga_box* box, int backward);

@@ -17,7 +17,7 @@ __all__ = [
     "CsrRelation", "tiga_status_string", "tiga_csr_workspace_bytes", "tiga_validate_csr",
     "tiga_apply_csr", "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram",
     "CsrPlan", "tiga_csr_plan_build", "tiga_csr_planned_workspace_bytes", "tiga_apply_csr_planned",
-    "tiga_radius_grid", "tiga_radius_workspace_bytes", "tiga_radius_bin",
+    "tiga_radius_grid", "tiga_validate_points", "tiga_radius_workspace_bytes", "tiga_radius_bin",
     "tiga_apply_radius", "tiga_apply_radius_backward", "tiga_apply_radius_mlp",
     "tiga_apply_radius_mlp_backward", "tiga_knn_workspace_bytes", "tiga_apply_knn",
     "tiga_csr_attention_workspace_bytes", "tiga_apply_csr_attention", "launch_count",
@@ -33,7 +33,7 @@ EXPORTS = [
     "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram", "tiga_radius_grid",
     "tiga_csr_plan_bytes", "tiga_csr_plan_workspace_bytes", "tiga_csr_plan_build", "tiga_csr_planned_workspace_bytes",
     "tiga_apply_csr_planned",
-    "tiga_radius_workspace_bytes", "tiga_radius_bin", "tiga_apply_radius",
+    "tiga_validate_points", "tiga_radius_workspace_bytes", "tiga_radius_bin", "tiga_apply_radius",
     "tiga_apply_radius_backward", "tiga_apply_radius_mlp", "tiga_apply_radius_mlp_backward",
     "tiga_knn_workspace_bytes", "tiga_apply_knn", "tiga_csr_attention_workspace_bytes", "tiga_apply_csr_attention",
 ]
@@ -117,6 +117,8 @@ def load_library() -> ctypes.CDLL:
     lib.tiga_csr_degree_histogram.argtypes = [ctypes.POINTER(_Csr), vp, i64, vp, vp]
     lib.tiga_radius_grid.restype = ctypes.c_int
     lib.tiga_radius_grid.argtypes = [i64, f, ctypes.POINTER(_Box), ctypes.POINTER(i32), ctypes.POINTER(f)]
+    lib.tiga_validate_points.restype = ctypes.c_int
+    lib.tiga_validate_points.argtypes = [vp, i64, ctypes.POINTER(_Box), ctypes.c_int, vp, sz, vp]
     lib.tiga_radius_workspace_bytes.restype = sz
     lib.tiga_radius_workspace_bytes.argtypes = [i64, i32, f, ctypes.POINTER(_Box), ctypes.c_int]
     lib.tiga_radius_bin.restype = ctypes.c_int
@@ -346,6 +348,14 @@ def tiga_radius_grid(n: int, r: float, box, periodic):
     ih = (ctypes.c_float * 3)()
     _ok(load_library().tiga_radius_grid(n, float(r), ctypes.byref(b), nc, ih), "tiga_radius_grid")
     return list(nc), list(ih)
+
+
+def tiga_validate_points(pos, box, periodic=(0, 0, 0), level: int = 1, stream=None) -> None:
+    """Raises TigaError (status 7) when a coordinate is not finite or lies outside [0, len]."""
+    b = _box(box, periodic)
+    ws = _ws(256, pos)
+    _ok(load_library().tiga_validate_points(_ptr(pos), pos.shape[0], ctypes.byref(b), level, _ptr(ws), ws.numel(),
+                                            _stream(stream)), "tiga_validate_points")
 
 
 def tiga_radius_workspace_bytes(n: int, F: int, r: float, box, periodic, backward: bool = False) -> int:

@@ -272,7 +272,7 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
 // --------------------------------------------------------------------------------------------
 constexpr int ROW_OWN = 4;
 constexpr int ROW_GROUP = 64;
-constexpr int ROW_HUGE = 8192;
+constexpr int ROW_HUGE = 4096;
 constexpr int GROUP_LANES = 8;
 
 // Where a source row lives.  HOT (planned apply): col values below n_hot address the compact copy of the
@@ -1157,6 +1157,7 @@ extern "C" const char* tiga_status_string(tiga_status s) {
         case TIGA_ERR_CUDA: return "CUDA runtime error";
         case TIGA_ERR_INVALID_GRAPH: return "malformed CSR relation";
         case TIGA_ERR_TOO_LARGE: return "problem exceeds the library's built-in scratch capacity";
+        case TIGA_ERR_INVALID_POINTS: return "a point coordinate is not finite or lies outside the box";
     }
     return "unknown status";
 }

@@ -160,6 +160,19 @@ __global__ void bin_sort_kernel(const RadiusParams p) {
     p.spos[s + rank] = make_float4(p.pos[3 * (size_t)id], p.pos[3 * (size_t)id + 1], p.pos[3 * (size_t)id + 2], __int_as_float(id));
 }
 
+// every coordinate finite and inside [0, len]: any violation raises the flag
+__global__ void validate_points_kernel(const float* __restrict__ pos, long long n3, float lx, float ly, float lz, int* flag) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    bool bad = false;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < n3; t += stride) {
+        const float v = pos[t];
+        const int d = (int)(t % 3);
+        const float len = d == 0 ? lx : (d == 1 ? ly : lz);
+        bad = bad || !(v >= 0.f && v <= len);          // also catches NaN
+    }
+    if (bad) atomicOr(flag, 1);
+}
+
 // ------------------------------------------------------------------------------ traversal
 
 // One warp per query cell.
@@ -179,7 +192,9 @@ __global__ void bin_sort_kernel(const RadiusParams p) {
 //             four gathered rows in flight per lane.  (The Lennard-Jones message has its own
 //             kernel in radius_lj.cu, which visits every unordered pair once.)
 // Lists hold QCAP entries per query and the stage STAGE_CAP candidates; when either fills up
-// the warp drains / processes and goes on, so any density works.
+// the warp drains / processes and goes on, so any density works.  A cell with more than QDENSE
+// points is cut into slices of QSLICE queries: its warp takes the first, the others are queued and a second
+// launch of the same kernel spreads over many warps (an empty queue costs one tiny launch).
 
 template <int MODE> struct TravSmem {
     // queries per batch: the forward runs fastest with short batches and seven CTAs per SM, the
@@ -201,19 +216,13 @@ template <int MODE> struct TravSmem {
 // 2: Gaussian backward.  MI: some periodic dimension has a single cell (explicit minimum image).
 // VEC: 0 = scalar feature accesses (F % 4 != 0, forward only); 1 = 128-bit accesses, F % 4 == 0;
 // 2 = additionally F == 4 LF exactly, so the row stride is a compile-time constant.
-template <int MODE, int LF, bool DIST, bool MI, int VEC = 1>
-__global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_traverse_kernel(const __grid_constant__ RadiusParams p) {
+template <int MODE, int LF, bool DIST, bool MI, int VEC>
+__device__ __forceinline__ void traverse_slice(const RadiusParams& p, const int cellid, const int qs0, const int qe0, unsigned char* s_raw) {
     using SM = TravSmem<MODE>;
     constexpr int STAGE_CAP = SM::STAGE_CAP, QCAP = SM::QCAP, QSTRIDE = SM::QSTRIDE, TQB = SM::TQB;
     constexpr unsigned FULL = 0xffffffffu;
-    extern __shared__ __align__(16) unsigned char s_raw[];
-
     const int lane = threadIdx.x & 31;
     const int wib = threadIdx.x >> 5;
-    const int cellid = blockIdx.x * TRAV_WARPS + wib;
-    if (cellid >= p.ncells) return;
-    const int qs0 = p.cell_start[cellid], qe0 = p.cell_start[cellid + 1];
-    if (qs0 == qe0) return;
 
     unsigned char* base = s_raw + (size_t)wib * SM::PER_WARP;
     float4* stage = reinterpret_cast<float4*>(base);
@@ -583,6 +592,30 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
     }
 }
 
+// Pass 1 (q_mode 0): warp w of the grid takes cell w, its first QSLICE queries, and queues the slices it
+// leaves.  Pass 2 (q_mode 1): the warps of a small grid walk the queue.
+template <int MODE, int LF, bool DIST, bool MI, int VEC = 1>
+__global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_traverse_kernel(const __grid_constant__ RadiusParams p) {
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    const int lane = threadIdx.x & 31;
+    const int w = blockIdx.x * TRAV_WARPS + (threadIdx.x >> 5);
+    if (!p.q_mode) {
+        if (w >= p.ncells) return;
+        const int qs0 = p.cell_start[w], qe0 = p.cell_start[w + 1];
+        if (qs0 == qe0) return;
+        queue_extra_slices(p, w, qe0 - qs0, lane);
+        traverse_slice<MODE, LF, DIST, MI, VEC>(p, w, qs0, qe0 - qs0 > QDENSE ? qs0 + QSLICE : qe0, s_raw);
+    } else {
+        const int n = *p.q_count;
+        for (int it = w; it < n; it += gridDim.x * TRAV_WARPS) {
+            const int2 item = p.q_items[it];
+            const int qs0 = p.cell_start[item.x] + item.y, end = p.cell_start[item.x + 1];
+            traverse_slice<MODE, LF, DIST, MI, VEC>(p, item.x, qs0, slice_end(qs0, end), s_raw);
+            __syncwarp();
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------ host side
 static long long icbrt_floor(long long v) {
     long long c = 0;
@@ -608,6 +641,9 @@ static tiga_status make_grid(long long n, float r, const tiga_box* box, int nc[3
     return TIGA_OK;
 }
 
+// bytes of the queue of extra slices: at most n / QSLICE of them exist
+static size_t queue_items(size_t n) { return n / QSLICE + 2; }
+
 RadiusLayout carve_radius(RadiusParams* p, void* ws, int32_t** fill) {
     Carver cv(ws);
     const size_t n = (size_t)p->n, nc = (size_t)p->ncells;
@@ -620,6 +656,8 @@ RadiusLayout carve_radius(RadiusParams* p, void* ws, int32_t** fill) {
     p->order = cv.take<int32_t>(n);
     p->spos = cv.take<float4>(n);
     p->blocksum = cv.take<int32_t>((size_t)nblocks + 1);
+    p->q_count = cv.take<int>(1);
+    p->q_items = cv.take<int2>(queue_items(n));
     return RadiusLayout{cv.off, nblocks};
 }
 
@@ -677,13 +715,11 @@ static tiga_status launch_traverse_t(const RadiusParams& p, cudaStream_t s) {
         // scalar feature accesses (only the forward supports widths that are not multiples of 4)
         auto sk = radius_traverse_kernel<MODE == 0 ? 0 : MODE, LF, DIST, MI, MODE != 0 ? 1 : 0>;
         if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(sk, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        sk<<<counted(blocks), TRAV_THREADS, smem, s>>>(p);
-        return launch_status();
+        return two_passes(p, s, [&](const RadiusParams& q, unsigned grid) { sk<<<counted(grid), TRAV_THREADS, smem, s>>>(q); });
     }
     auto kern = p.F == 4 * LF ? radius_traverse_kernel<MODE, LF, DIST, MI, 2> : radius_traverse_kernel<MODE, LF, DIST, MI, 1>;
     if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    kern<<<counted(blocks), TRAV_THREADS, smem, s>>>(p);
-    return launch_status();
+    return two_passes(p, s, [&](const RadiusParams& q, unsigned grid) { kern<<<counted(grid), TRAV_THREADS, smem, s>>>(q); });
 }
 
 template <int MODE, bool DIST, bool MI>
@@ -719,6 +755,27 @@ extern "C" tiga_status tiga_radius_grid(int64_t n, float r, const tiga_box* box,
         if (invh) invh[d] = ih[d];
     }
     return TIGA_OK;
+}
+
+extern "C" tiga_status tiga_validate_points(const float* pos, int64_t n, const tiga_box* box, int level,
+                                            void* ws, size_t ws_bytes, void* stream) {
+    if (!box || n < 0) return TIGA_ERR_INVALID_ARG;
+    for (int d = 0; d < 3; ++d)
+        if (!(box->len[d] > 0.f) || !isfinite(box->len[d])) return TIGA_ERR_INVALID_ARG;
+    if (n > 0 && (!pos || !aligned16(pos))) return TIGA_ERR_INVALID_ARG;
+    if (level == 0 || n == 0) return TIGA_OK;
+    if (!ws || ws_bytes < 16) return TIGA_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int* flag = static_cast<int*>(ws);
+    TIGA_CUDA_TRY(cudaMemsetAsync(flag, 0, sizeof(int), s));
+    long long blocks = (3 * n + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    validate_points_kernel<<<counted((unsigned)blocks), 256, 0, s>>>(pos, 3 * n, box->len[0], box->len[1], box->len[2], flag);
+    if (launch_status() != TIGA_OK) return TIGA_ERR_CUDA;
+    int h = 0;
+    TIGA_CUDA_TRY(cudaMemcpyAsync(&h, flag, sizeof(int), cudaMemcpyDeviceToHost, s));
+    TIGA_CUDA_TRY(cudaStreamSynchronize(s));
+    return h ? TIGA_ERR_INVALID_POINTS : TIGA_OK;
 }
 
 extern "C" size_t tiga_radius_workspace_bytes(int64_t n, int32_t F, float r, const tiga_box* box, int backward) {

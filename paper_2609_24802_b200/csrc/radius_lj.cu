@@ -38,15 +38,13 @@ constexpr int LJ_LIST_BYTES = (LJQ * LJ_QSTRIDE * 8 + 15) / 16 * 16;
 constexpr int LJ_MISC_BYTES = LJQ * 16 + 3 * LJQ * 4 + LJQ * 4 + 32;        // queries, their coordinates by component, list lengths, the cell's frame
 constexpr int LJ_PER_WARP = (LJ_STAGE_BYTES + LJ_LIST_BYTES + LJ_MISC_BYTES + 15) / 16 * 16;
 
-template <bool MI, bool COUNT>
-__global__ void __launch_bounds__(TRAV_THREADS, COUNT ? 8 : 7) radius_lj_pairs_kernel(const __grid_constant__ RadiusParams p) {
+// One warp, one cell; of a cell with more than QDENSE points only QSLICE as queries (from `first`): what such a cell
+// leaves is queued for the second pass, as in radius_traverse_kernel.
+template <bool MI, bool COUNT, bool QUEUE>
+__device__ __forceinline__ void lj_slice(const RadiusParams& p, const int cellid, const int first, unsigned char* s_raw) {
     constexpr unsigned FULL = 0xffffffffu;
-    extern __shared__ __align__(16) unsigned char s_raw[];
-
     const int lane = threadIdx.x & 31;
     const int wib = threadIdx.x >> 5;
-    const int cellid = blockIdx.x * TRAV_WARPS + wib;
-    if (cellid >= p.ncells) return;
     unsigned char* base = s_raw + (size_t)wib * LJ_PER_WARP;
     float4* stage = reinterpret_cast<float4*>(base);                                   // x, y, z in the frame of this cell, point id
     float2* list = reinterpret_cast<float2*>(base + LJ_STAGE_BYTES);                   // (stage slot, d2) per query
@@ -114,8 +112,10 @@ __global__ void __launch_bounds__(TRAV_THREADS, COUNT ? 8 : 7) radius_lj_pairs_k
     }
     // lane 0 resolved the cell itself: its run is the cell's own points (one load round trip fewer
     // than asking for them first)
-    const int qs0 = __shfl_sync(FULL, r_cs, 0), nown = __shfl_sync(FULL, r_len, 0), qe0 = qs0 + nown;
+    const int own0 = __shfl_sync(FULL, r_cs, 0), nown = __shfl_sync(FULL, r_len, 0);
     if (nown == 0) return;
+    if (!QUEUE) queue_extra_slices(p, cellid, nown, lane);
+    const int qs0 = own0 + first, qe0 = nown > QDENSE ? slice_end(qs0, own0 + nown) : own0 + nown;     // this warp's queries
     int r_incl = r_len;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -349,7 +349,10 @@ __global__ void __launch_bounds__(TRAV_THREADS, COUNT ? 8 : 7) radius_lj_pairs_k
                 const float ex = fmaxf(fmaxf(lx - val.x, val.x - hx), 0.f);
                 const float ey = fmaxf(fmaxf(ly - val.y, val.y - hy), 0.f);
                 const float ez = fmaxf(fmaxf(lz - val.z, val.z - hz), 0.f);
-                const bool keep = k0 + 32 * u + lane < nin && fmaf(ez, ez, fmaf(ey, ey, ex * ex)) <= p.r2_hi * 1.0001f;
+                // the cell's own points are always kept (a slice's box does not cover all of them, and the
+                // own-pair rule below goes by their position at the head of the stage)
+                const int kk = k0 + 32 * u + lane;
+                const bool keep = kk < nin && (lo + kk < nown || fmaf(ez, ez, fmaf(ey, ey, ex * ex)) <= p.r2_hi * 1.0001f);
                 const unsigned m = __ballot_sync(FULL, keep);
                 if (keep) stage[nst + __popc(m & lt_mask)] = val;
                 nst += __popc(m);
@@ -362,14 +365,36 @@ __global__ void __launch_bounds__(TRAV_THREADS, COUNT ? 8 : 7) radius_lj_pairs_k
     }
 }
 
+// QUEUE = false: warp w takes cell w.  QUEUE = true: the warps of a small grid walk the queued slices.
+template <bool MI, bool COUNT, bool QUEUE>
+__global__ void __launch_bounds__(TRAV_THREADS, COUNT ? 8 : 7) radius_lj_pairs_kernel(const __grid_constant__ RadiusParams p) {
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    const int w = blockIdx.x * TRAV_WARPS + (threadIdx.x >> 5);
+    if constexpr (!QUEUE) {
+        if (w < p.ncells) lj_slice<MI, COUNT, false>(p, w, 0, s_raw);
+    } else {
+        const int n = *p.q_count;
+        for (int it = w; it < n; it += gridDim.x * TRAV_WARPS) {
+            const int2 item = p.q_items[it];
+            lj_slice<MI, COUNT, true>(p, item.x, item.y, s_raw);
+            __syncwarp();
+        }
+    }
+}
+
 template <bool MI, bool COUNT>
 static tiga_status launch_lj_t(const RadiusParams& p, cudaStream_t s) {
-    const unsigned blocks = (unsigned)((p.ncells + TRAV_WARPS - 1) / TRAV_WARPS);
     constexpr int smem = LJ_PER_WARP * TRAV_WARPS;
-    auto kern = radius_lj_pairs_kernel<MI, COUNT>;
-    if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    kern<<<counted(blocks), TRAV_THREADS, smem, s>>>(p);
-    return launch_status();
+    auto kern = radius_lj_pairs_kernel<MI, COUNT, false>;
+    auto kq = radius_lj_pairs_kernel<MI, COUNT, true>;
+    if (smem > 48 * 1024) {
+        TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        TIGA_CUDA_TRY(cudaFuncSetAttribute(kq, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    }
+    return two_passes(p, s, [&](const RadiusParams& q, unsigned grid) {
+        if (q.q_mode) kq<<<counted(grid), TRAV_THREADS, smem, s>>>(q);
+        else kern<<<counted(grid), TRAV_THREADS, smem, s>>>(q);
+    });
 }
 
 tiga_status launch_lj_pairs(const RadiusParams& p, cudaStream_t s) {

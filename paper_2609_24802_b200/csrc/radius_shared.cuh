@@ -11,6 +11,9 @@ constexpr int TRAV_THREADS = TRAV_WARPS * 32;
 constexpr int STAGE_PAD = 32;           // sentinels behind the staged candidates: no bounds checks
 constexpr int QB = 8;                   // queries per batch (kernels that run faster with four define their own width)
 constexpr float FAR_AWAY = 1.0e18f;
+constexpr int QDENSE = 64;              // a cell with more points than this is cut into slices of QSLICE queries:
+constexpr int QSLICE = 16;              // its warp takes the first slice and queues the others for the second pass
+constexpr int QUEUE_BLOCKS = 148 * 8;   // grid of the pass over the queued slices
 
 struct RadiusParams {
     const float* pos;
@@ -46,6 +49,10 @@ struct RadiusParams {
     int32_t* order;
     float4* spos;             // positions in cell order, .w = original point id (bit pattern)
     int32_t* blocksum;
+    // slices of cells with more than QDENSE points, queued by the pass over the cells for a second pass
+    int2* q_items;            // (cell, first query of the slice)
+    int* q_count;
+    int q_mode;               // 0: one warp per cell (queues what it leaves), 1: warps walk the queue
     // optional user copies of the plan
     int32_t* u_cell;
     int32_t* u_cell_start;
@@ -79,6 +86,30 @@ static __device__ __noinline__ bool exact_within(const RadiusParams& p, const fl
         d2 = (d == 0) ? sq : __dadd_rn(d2, sq);
     }
     return d2 <= p.r2_exact;
+}
+
+// A cell with more than QDENSE points: the warp that owns it keeps the first QSLICE queries and queues
+// the others, QSLICE at a time, for the pass over the queue.  (Short slices: a dense cell's queries meet
+// thousands of candidates each, and many short slices fill the machine where a few long ones leave a tail.)
+static __device__ __forceinline__ int slice_end(int qs, int cell_end) { return cell_end - qs > QSLICE ? qs + QSLICE : cell_end; }
+static __device__ __forceinline__ void queue_extra_slices(const RadiusParams& p, int cell, int count, int lane) {
+    if (count > QDENSE && lane == 0) {
+        const int extra = (count - 1) / QSLICE;
+        const int at = atomicAdd(p.q_count, extra);
+        for (int k = 0; k < extra; ++k) p.q_items[at + k] = make_int2(cell, (k + 1) * QSLICE);
+    }
+}
+
+// Runs a traversal kernel twice: over the cells, then over the queue of slices the first pass left.
+template <typename Launch>
+static inline tiga_status two_passes(const RadiusParams& p, cudaStream_t s, Launch launch) {
+    TIGA_CUDA_TRY(cudaMemsetAsync(p.q_count, 0, sizeof(int), s));
+    RadiusParams q = p;
+    q.q_mode = 0;
+    launch(q, (unsigned)((p.ncells + TRAV_WARPS - 1) / TRAV_WARPS));
+    q.q_mode = 1;
+    launch(q, (unsigned)QUEUE_BLOCKS);
+    return launch_status();
 }
 
 static __device__ __forceinline__ float fast_exp2(float x) {

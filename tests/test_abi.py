@@ -32,7 +32,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_status_strings(lib):
     assert lib.tiga_status_string(0) == "ok"
-    assert len({lib.tiga_status_string(s) for s in range(7)}) == 7
+    assert len({lib.tiga_status_string(s) for s in range(8)}) == 8
 
 
 def test_grid_matches_the_oracle_reading(lib):
@@ -58,6 +58,11 @@ def test_host_side_argument_errors(lib):
     assert cdll.tiga_radius_grid(100, ctypes.c_float(-1.0), ctypes.byref(b), nc, None) == 1
     assert cdll.tiga_radius_grid(100, ctypes.c_float(0.1), None, nc, None) == 1
     assert cdll.tiga_radius_workspace_bytes(100, 4, ctypes.c_float(0.6), ctypes.byref(b), 0) == 0
+    # point validation: host-side checks need no device
+    assert cdll.tiga_validate_points(None, 10, ctypes.byref(b), 0, None, 0, None) == 1      # no positions
+    assert cdll.tiga_validate_points(256, 10, None, 0, None, 0, None) == 1                  # no box
+    assert cdll.tiga_validate_points(256, 10, ctypes.byref(b), 0, None, 0, None) == 0       # metadata only
+    assert cdll.tiga_validate_points(256, 10, ctypes.byref(b), 1, None, 0, None) == 3       # level 1 needs scratch
     # CSR: null / misaligned pointers, negative sizes, unsupported widths
     g = _Csr(0, 0, 0, 4, 4, 0)
     msg = _Msg(0, 0.0, 0.0)

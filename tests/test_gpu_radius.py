@@ -316,3 +316,62 @@ def test_cfg3_full_size(tiga):
     assert rel_err(out, y, A) <= SUM_TOL
     assert 50 < count.mean() < 58
     assert np.max(np.abs(out[:, :3].astype(np.float64).sum(0))) < 1e-6 * A[:, :3].sum()
+
+
+# ------------------------------------------------------------------------------ validation
+def test_point_validation(tiga):
+    box = np.array([1.0, 2.0, 0.5], np.float32)
+    pos = gen.uniform_points(10_000, 3) * box[None, :]
+    pos[17] = box                                              # the upper faces belong to the box
+    tiga.tiga_validate_points(dev(pos, torch), box)            # passes
+    for bad in (np.float32(-1e-6), np.float32(np.nan), np.float32(np.inf), np.float32(0.5000001)):
+        q = pos.copy()
+        q[4321, 2] = bad
+        with pytest.raises(tiga.TigaError) as e:
+            tiga.tiga_validate_points(dev(q, torch), box)
+        assert e.value.status == 7
+        tiga.tiga_validate_points(dev(q, torch), box, level=0)     # metadata only: nothing is read
+    tiga.tiga_validate_points(dev(pos[:0], torch), box)
+
+
+# ------------------------------------------------------------------------------ uneven density
+def test_clustered_points_are_spread_over_many_warps(tiga):
+    """Most points in a dozen tight blobs: some cells hold hundreds of points (a warp takes 64 queries
+    of a cell and queues the rest for a second pass).  Parity as usual, and the call must stay within
+    5x of a uniform cloud with the same number of accepted pairs."""
+    n, F = 200_000, 8
+    pos = gen.clustered_points(n, 21)
+    x = gen.normal_features(n, F, 21, 31); gy = gen.normal_features(n, F, 21, 32)
+    ones = np.ones(3, np.float32)
+    r = np.float32(0.01)
+    grid, _ = tiga.tiga_radius_grid(n, r, ones, [0, 0, 0])
+    cell = np.minimum((pos * np.float32(grid)).astype(np.int64), np.array(grid) - 1)
+    occupancy = np.bincount((cell[:, 2] * grid[1] + cell[:, 1]) * grid[0] + cell[:, 0])
+    assert occupancy.max() > 4 * 64                                   # several slices per cell
+    out, count = _check_gauss(tiga, pos, x, gy, r, ones, [0, 0, 0], np.float32(0.005), use_cells=True)
+    pairs = int(host(count).sum())
+    # Lennard-Jones on the same cloud (scaled): the length s lies below the smallest distance of any pair, so no pair
+    # energy is a difference of two nearly equal powers (the normalisation by |contributions| would not cover that)
+    # (cutoff 0.8: a few dozen neighbours per particle as in the workload, while the cells -- their number is capped
+    # by the point count -- still hold hundreds of points; rows of a thousand atomically added terms would exceed
+    # what fp32 accumulation in arbitrary order can promise)
+    _check_lj(tiga, pos * np.float32(300.0), np.float32(0.8), np.full(3, 300.0, np.float32), [0, 0, 0], eps=1e-3, s=0.005, use_cells=True)
+
+    def timed(p, rr):
+        pd, xd = dev(p, torch), dev(x, torch)
+        o, c, ws = tiga.tiga_apply_radius(pd, xd, rr, ones, [0, 0, 0], tiga.MSG_GAUSS, p0=float(rr) / 2, want_count=True)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(5):
+            tiga.tiga_apply_radius(pd, xd, rr, ones, [0, 0, 0], tiga.MSG_GAUSS, p0=float(rr) / 2, out=o, count=c, ws=ws)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / 5, int(c.sum().item())
+
+    r_uniform = np.float32((pairs * 3.0 / (4.0 * np.pi * n * n)) ** (1.0 / 3.0))
+    t_c, p_c = timed(pos, r)
+    t_u, p_u = timed(gen.uniform_points(n, 22), r_uniform)
+    print(f"clustered: {p_c} pairs in {t_c:.3f} ms; uniform: {p_u} pairs in {t_u:.3f} ms")
+    assert 0.7 * p_c < p_u < 1.4 * p_c
+    assert t_c < 5.0 * t_u
