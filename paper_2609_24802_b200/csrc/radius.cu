@@ -127,6 +127,7 @@ __global__ void scan_apply_kernel(const RadiusParams p) {
         if (base + k < p.ncells) {
             p.cell_start[base + k] = ex;
             if (p.u_cell_start) p.u_cell_start[base + k] = ex;
+            queue_extra_slices(p, base + k, v[k]);          // a dense cell is cut into slices for the traversals
         }
         ex += v[k];
     }
@@ -603,7 +604,6 @@ __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_trav
         if (w >= p.ncells) return;
         const int qs0 = p.cell_start[w], qe0 = p.cell_start[w + 1];
         if (qs0 == qe0) return;
-        queue_extra_slices(p, w, qe0 - qs0, lane);
         traverse_slice<MODE, LF, DIST, MI, VEC>(p, w, qs0, qe0 - qs0 > QDENSE ? qs0 + QSLICE : qe0, s_raw);
     } else {
         const int n = *p.q_count;
@@ -648,7 +648,8 @@ RadiusLayout carve_radius(RadiusParams* p, void* ws, int32_t** fill) {
     Carver cv(ws);
     const size_t n = (size_t)p->n, nc = (size_t)p->ncells;
     const int nblocks = (int)((nc + SCAN_BLOCK - 1) / SCAN_BLOCK);
-    p->cnt = cv.take<int32_t>(2 * nc + 2);          // counts, then the scatter cursors
+    p->cnt = cv.take<int32_t>(2 * nc + 2 + 16);     // counts, then the scatter cursors, then the length of the slice queue
+    p->q_count = p->cnt + 2 * nc + 2;
     *fill = p->cnt + nc;
     p->cell = cv.take<int32_t>(n);
     p->cell_start = cv.take<int32_t>(nc + 1);
@@ -656,7 +657,6 @@ RadiusLayout carve_radius(RadiusParams* p, void* ws, int32_t** fill) {
     p->order = cv.take<int32_t>(n);
     p->spos = cv.take<float4>(n);
     p->blocksum = cv.take<int32_t>((size_t)nblocks + 1);
-    p->q_count = cv.take<int>(1);
     p->q_items = cv.take<int2>(queue_items(n));
     return RadiusLayout{cv.off, nblocks};
 }
@@ -690,7 +690,7 @@ tiga_status fill_params(RadiusParams* p, long long n, float r, const tiga_box* b
 
 tiga_status run_binning(RadiusParams& p, int32_t* fill, int nblocks, cudaStream_t s) {
     if (p.n == 0) return TIGA_OK;
-    TIGA_CUDA_TRY(cudaMemsetAsync(p.cnt, 0, (2 * (size_t)p.ncells + 2) * sizeof(int32_t), s));
+    TIGA_CUDA_TRY(cudaMemsetAsync(p.cnt, 0, (2 * (size_t)p.ncells + 2 + 16) * sizeof(int32_t), s));
     const unsigned pb = (unsigned)((p.n + 255) / 256);
     bin_count_kernel<<<counted(pb), 256, 0, s>>>(p);
     scan_reduce_kernel<<<counted(nblocks), RAD_THREADS, 0, s>>>(p);

@@ -114,7 +114,6 @@ __device__ __forceinline__ void lj_slice(const RadiusParams& p, const int cellid
     // than asking for them first)
     const int own0 = __shfl_sync(FULL, r_cs, 0), nown = __shfl_sync(FULL, r_len, 0);
     if (nown == 0) return;
-    if (!QUEUE) queue_extra_slices(p, cellid, nown, lane);
     const int qs0 = own0 + first, qe0 = nown > QDENSE ? slice_end(qs0, own0 + nown) : own0 + nown;     // this warp's queries
     int r_incl = r_len;
 #pragma unroll

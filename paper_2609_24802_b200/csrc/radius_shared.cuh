@@ -88,12 +88,13 @@ static __device__ __noinline__ bool exact_within(const RadiusParams& p, const fl
     return d2 <= p.r2_exact;
 }
 
-// A cell with more than QDENSE points: the warp that owns it keeps the first QSLICE queries and queues
-// the others, QSLICE at a time, for the pass over the queue.  (Short slices: a dense cell's queries meet
+// A cell with more than QDENSE points: the warp that owns it keeps the first QSLICE queries; the others
+// are queued, QSLICE at a time, for the pass over the queue.  The queue is part of the binning plan
+// (written where the cell offsets are, so the traversals carry no code for it).  (Short slices: a dense cell's queries meet
 // thousands of candidates each, and many short slices fill the machine where a few long ones leave a tail.)
 static __device__ __forceinline__ int slice_end(int qs, int cell_end) { return cell_end - qs > QSLICE ? qs + QSLICE : cell_end; }
-static __device__ __forceinline__ void queue_extra_slices(const RadiusParams& p, int cell, int count, int lane) {
-    if (count > QDENSE && lane == 0) {
+static __device__ __forceinline__ void queue_extra_slices(const RadiusParams& p, int cell, int count) {
+    if (count > QDENSE) {
         const int extra = (count - 1) / QSLICE;
         const int at = atomicAdd(p.q_count, extra);
         for (int k = 0; k < extra; ++k) p.q_items[at + k] = make_int2(cell, (k + 1) * QSLICE);
@@ -103,7 +104,6 @@ static __device__ __forceinline__ void queue_extra_slices(const RadiusParams& p,
 // Runs a traversal kernel twice: over the cells, then over the queue of slices the first pass left.
 template <typename Launch>
 static inline tiga_status two_passes(const RadiusParams& p, cudaStream_t s, Launch launch) {
-    TIGA_CUDA_TRY(cudaMemsetAsync(p.q_count, 0, sizeof(int), s));
     RadiusParams q = p;
     q.q_mode = 0;
     launch(q, (unsigned)((p.ncells + TRAV_WARPS - 1) / TRAV_WARPS));
