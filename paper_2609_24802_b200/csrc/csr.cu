@@ -37,9 +37,16 @@ struct State {
         for (int i = 0; i < VPL; ++i)
 #pragma unroll
             for (int k = 0; k < VW; ++k) {
-                v[i][k] = 0.f;
+                // max: the empty state holds NaN, which every first message replaces through the
+                // "greater or unordered" comparison below; stores turn a still-empty entry into 0
+                v[i][k] = RED != 0 ? __int_as_float(0x7fc00000) : 0.f;
                 if constexpr (RED != 0) a[i][k] = -1;
             }
+    }
+    // the value an entry is stored with (finalize: the empty state of max becomes 0)
+    __device__ __forceinline__ float out(int i, int k) const {
+        if constexpr (RED != 0) return a[i][k] < 0 ? 0.f : v[i][k];
+        else return v[i][k];
     }
     // fold a message that comes later in edge order
     __device__ __forceinline__ void message(int i, int k, float wgt, float xv, int e) {
@@ -47,7 +54,7 @@ struct State {
             v[i][k] = fmaf(wgt, xv, v[i][k]);
         } else {
             const float m = __fmul_rn(wgt, xv);        // one rounding, never contracted
-            if (a[i][k] < 0 || m > v[i][k]) { v[i][k] = m; a[i][k] = e; }
+            if (!(m <= v[i][k])) { v[i][k] = m; a[i][k] = e; }      // strictly greater, or the state is still empty
         }
     }
     // fold a partial state that comes later in edge order
@@ -55,7 +62,7 @@ struct State {
         if constexpr (RED == 0) {
             v[i][k] += ov;
         } else {
-            if (oa >= 0 && (a[i][k] < 0 || ov > v[i][k])) { v[i][k] = ov; a[i][k] = oa; }
+            if (oa >= 0 && !(ov <= v[i][k])) { v[i][k] = ov; a[i][k] = oa; }
         }
     }
 };
@@ -98,7 +105,7 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
             float* o = p.out + row * F + (size_t)(i * G + ln) * VW;
 #pragma unroll
             for (int k = 0; k < VW; k += 4)
-                st_stream(reinterpret_cast<float4*>(o + k), make_float4(s.v[i][k], s.v[i][k + 1], s.v[i][k + 2], s.v[i][k + 3]));
+                st_stream(reinterpret_cast<float4*>(o + k), make_float4(s.out(i, k), s.out(i, k + 1), s.out(i, k + 2), s.out(i, k + 3)));
             if constexpr (RED != 0) {
                 int* ao = p.arg + row * F + (size_t)(i * G + ln) * VW;
 #pragma unroll
@@ -412,7 +419,7 @@ __device__ __forceinline__ void store_state(const CsrParams& p, float* out, int3
     for (int i = 0; i < NV; ++i) {
 #pragma unroll
         for (int k = 0; k < VW; k += 4) {
-            st_stream(reinterpret_cast<float4*>(out + i * VW + k), make_float4(s.v[i][k], s.v[i][k + 1], s.v[i][k + 2], s.v[i][k + 3]));
+            st_stream(reinterpret_cast<float4*>(out + i * VW + k), make_float4(s.out(i, k), s.out(i, k + 1), s.out(i, k + 2), s.out(i, k + 3)));
             if constexpr (RED != 0)
                 st_stream(reinterpret_cast<int4*>(arg + i * VW + k), make_int4(s.a[i][k], s.a[i][k + 1], s.a[i][k + 2], s.a[i][k + 3]));
         }
