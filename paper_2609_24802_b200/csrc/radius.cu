@@ -154,11 +154,60 @@ __global__ void bin_sort_kernel(const RadiusParams p) {
     const int id = p.order_tmp[t];
     const int c = p.cell[id];
     const int s = p.cell_start[c], e = p.cell_start[c + 1];
+    if (e - s > SORT_DENSE) return;        // bin_sort_dense_kernel orders this cell
     int rank = 0;
     for (int u = s; u < e; ++u) rank += (p.order_tmp[u] < id) ? 1 : 0;
     p.order[s + rank] = id;
     if (p.u_order) p.u_order[s + rank] = id;
     p.spos[s + rank] = make_float4(p.pos[3 * (size_t)id], p.pos[3 * (size_t)id + 1], p.pos[3 * (size_t)id + 2], __int_as_float(id));
+}
+
+// Cells with more than SORT_DENSE points (rank counting is quadratic in the occupancy): one CTA per
+// queued cell sorts the cell's slots by point id with a bitonic network whose comparisons all point
+// the same way (first step of a merge mirrors, the others are half-cleaners), so slots behind the
+// segment act as +infinity without being stored; up to SORT_SMEM ids are sorted in shared memory,
+// longer segments in place in global memory.
+constexpr int SORT_THREADS = 512;
+constexpr int SORT_SMEM = 8192;
+static __device__ void sort_ids_ascending(int32_t* a, int m) {
+    int P = 1;
+    while (P < m) P <<= 1;
+    for (int k = 2; k <= P; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int t = threadIdx.x; t < (P >> 1); t += blockDim.x) {
+                const int lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+                const int hi = (j == (k >> 1)) ? (lo ^ (k - 1)) : (lo + j);       // mirror within the block of k, then strides
+                if (hi < m) {
+                    const int32_t x = a[lo], y = a[hi];
+                    if (x > y) { a[lo] = y; a[hi] = x; }
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+__global__ void __launch_bounds__(SORT_THREADS) bin_sort_dense_kernel(const RadiusParams p) {
+    __shared__ int32_t s_ids[SORT_SMEM];
+    const int items = *p.b_count;
+    for (int it = blockIdx.x; it < items; it += gridDim.x) {
+        const int c = p.b_items[it];
+        const int s = p.cell_start[c], m = p.cell_start[c + 1] - s;
+        int32_t* a = p.order_tmp + s;
+        if (m <= SORT_SMEM) {
+            for (int k = threadIdx.x; k < m; k += blockDim.x) s_ids[k] = a[k];
+            __syncthreads();
+            a = s_ids;
+        }
+        sort_ids_ascending(a, m);
+        for (int k = threadIdx.x; k < m; k += blockDim.x) {
+            const int id = a[k];
+            p.order[s + k] = id;
+            if (p.u_order) p.u_order[s + k] = id;
+            p.spos[s + k] = make_float4(p.pos[3 * (size_t)id], p.pos[3 * (size_t)id + 1], p.pos[3 * (size_t)id + 2], __int_as_float(id));
+        }
+        __syncthreads();
+    }
 }
 
 // every coordinate finite and inside [0, len]: any violation raises the flag
@@ -650,6 +699,7 @@ RadiusLayout carve_radius(RadiusParams* p, void* ws, int32_t** fill) {
     const int nblocks = (int)((nc + SCAN_BLOCK - 1) / SCAN_BLOCK);
     p->cnt = cv.take<int32_t>(2 * nc + 2 + 16);     // counts, then the scatter cursors, then the length of the slice queue
     p->q_count = p->cnt + 2 * nc + 2;
+    p->b_count = p->q_count + 1;
     *fill = p->cnt + nc;
     p->cell = cv.take<int32_t>(n);
     p->cell_start = cv.take<int32_t>(nc + 1);
@@ -658,6 +708,7 @@ RadiusLayout carve_radius(RadiusParams* p, void* ws, int32_t** fill) {
     p->spos = cv.take<float4>(n);
     p->blocksum = cv.take<int32_t>((size_t)nblocks + 1);
     p->q_items = cv.take<int2>(queue_items(n));
+    p->b_items = cv.take<int32_t>(n / SORT_DENSE + 2);
     return RadiusLayout{cv.off, nblocks};
 }
 
@@ -698,6 +749,7 @@ tiga_status run_binning(RadiusParams& p, int32_t* fill, int nblocks, cudaStream_
     scan_apply_kernel<<<counted(nblocks), RAD_THREADS, 0, s>>>(p);
     bin_scatter_kernel<<<counted(pb), 256, 0, s>>>(p, fill);
     bin_sort_kernel<<<counted(pb), 256, 0, s>>>(p);
+    bin_sort_dense_kernel<<<counted(148u), SORT_THREADS, 0, s>>>(p);
     return launch_status();
 }
 

@@ -14,6 +14,7 @@ constexpr float FAR_AWAY = 1.0e18f;
 constexpr int QDENSE = 64;              // a cell with more points than this is cut into slices of QSLICE queries:
 constexpr int QSLICE = 16;              // its warp takes the first slice and queues the others for the second pass
 constexpr int QUEUE_BLOCKS = 148 * 8;   // grid of the pass over the queued slices
+constexpr int SORT_DENSE = 256;         // a cell with more points than this is ordered by a sorting network, not by rank counting
 
 struct RadiusParams {
     const float* pos;
@@ -53,6 +54,8 @@ struct RadiusParams {
     int2* q_items;            // (cell, first query of the slice)
     int* q_count;
     int q_mode;               // 0: one warp per cell (queues what it leaves), 1: warps walk the queue
+    int32_t* b_items;         // cells with more than SORT_DENSE points (queued by the same scan), and how many
+    int* b_count;
     // optional user copies of the plan
     int32_t* u_cell;
     int32_t* u_cell_start;
@@ -99,6 +102,7 @@ static __device__ __forceinline__ void queue_extra_slices(const RadiusParams& p,
         const int at = atomicAdd(p.q_count, extra);
         for (int k = 0; k < extra; ++k) p.q_items[at + k] = make_int2(cell, (k + 1) * QSLICE);
     }
+    if (count > SORT_DENSE) p.b_items[atomicAdd(p.b_count, 1)] = cell;
 }
 
 // Runs a traversal kernel twice: over the cells, then over the queue of slices the first pass left.
