@@ -202,7 +202,8 @@ tiga_status tiga_apply_csr_planned(const tiga_csr* g, const tiga_csr_plan* plan,
  *   max : the cotangent of (i,f) flows only through edge argmax[i,f] (nothing if it is -1).
  *   grad_out : fp32 [n_dst, F];  argmax : the forward's output (TIGA_MAX only).
  *   grad_x   : fp32 [n_src, F] or NULL to skip;  grad_w : fp32 [n_edges] or NULL to skip.
- * x must be fp32.  Repeated sources accumulate with floating-point atomics, so grad_x (and
+ * x is fp32 or fp16 (the forward's feature table; F % 8 == 0 for fp16); all gradients are fp32, and the
+ * cotangent of an fp16 table is the fp32 grad_x (no rounding to fp16 is applied).  Repeated sources accumulate with floating-point atomics, so grad_x (and
  * grad_w for TIGA_MAX) may differ in the last bits between runs. */
 tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
                                     const float* w, const tiga_msg* msg, tiga_reducer reducer,

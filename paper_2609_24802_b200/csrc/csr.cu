@@ -445,7 +445,7 @@ __device__ __forceinline__ void reduce_and_store(State<RED, NV, XTraits<XT>::VW>
 }
 
 template <typename XT, int NV, int RED, typename IT, bool HOT, bool W>
-__global__ void __launch_bounds__(CSR_THREADS) csr_rows_kernel(const CsrParams p) {
+__global__ void __launch_bounds__(CSR_THREADS, 6) csr_rows_kernel(const CsrParams p) {
     constexpr int VW = XTraits<XT>::VW;
     constexpr unsigned FULL = 0xffffffffu;
     using St = State<RED, NV, VW>;
@@ -637,7 +637,20 @@ __global__ void csr_fixup_kernel(const CsrParams p) {
 //   gw[e] = x[col[e],:] . gy[row,:]            (one value per edge position, duplicates not merged)
 //   gx[col[e],:] += w[e] * gy[row,:]           (reverse incidence: vector atomics)
 // --------------------------------------------------------------------------------------------
-template <int G, int VPL, typename IT>
+// four consecutive features of a source row as fp32: one 128-bit load (fp32 rows) or one 64-bit load (fp16 rows)
+template <typename XT>
+__device__ __forceinline__ float4 load_x4(const void* x, unsigned long long vec) {
+    if constexpr (sizeof(XT) == 4) {
+        return __ldg(static_cast<const float4*>(x) + vec);
+    } else {
+        const uint2 raw = __ldg(static_cast<const uint2*>(x) + vec);
+        const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+        const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+        return make_float4(lo.x, lo.y, hi.x, hi.y);
+    }
+}
+
+template <int G, int VPL, typename IT, typename XT>
 __global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const CsrParams p) {
     constexpr int VW = 4;
     constexpr int NW = CSR_THREADS / G;
@@ -653,7 +666,6 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const Csr
     const int ln = threadIdx.x % G;
     // lanes of one worker stay converged; workers of one warp do not
     const unsigned wmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) & ~(G - 1)));
-    const float4* __restrict__ xlane = static_cast<const float4*>(p.x) + ln;
     const float4* __restrict__ gybase = reinterpret_cast<const float4*>(p.gy);
     float4* gxlane = reinterpret_cast<float4*>(p.gx) + ln;
     const unsigned nvec = (unsigned)p.nvec;
@@ -687,7 +699,7 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const Csr
                 if (p.gw) {
 #pragma unroll
                     for (int i = 0; i < VPL; ++i)
-                        xv[u][i] = act[i] ? __ldg(xlane + (unsigned long long)(unsigned)cv[u] * nvec + i * G) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        xv[u][i] = act[i] ? load_x4<XT>(p.x, (unsigned long long)(unsigned)cv[u] * nvec + i * G + ln) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
 #pragma unroll
@@ -731,6 +743,7 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const Csr
 // (two rounds, each for the edge of the lowest lane not served yet; what is left goes out one by
 // one: more rounds measured slower): one atomic per edge instead of
 // up to 32 on the same address.
+template <typename XT>
 __global__ void csr_backward_max_kernel(const CsrParams p) {
     constexpr unsigned FULL = 0xffffffffu;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -743,7 +756,12 @@ __global__ void csr_backward_max_kernel(const CsrParams p) {
         const long long j = p.col[e];
         const float g = p.gy[idx];
         if (p.gx) atomicAdd(p.gx + j * p.F + f, (p.w ? p.w[e] : 1.f) * g);
-        if (p.gw) contrib = static_cast<const float*>(p.x)[j * p.F + f] * g;
+        if (p.gw) {
+            float xv;
+            if constexpr (sizeof(XT) == 4) xv = static_cast<const float*>(p.x)[j * p.F + f];
+            else xv = __half2float(static_cast<const __half*>(p.x)[j * p.F + f]);
+            contrib = xv * g;
+        }
     }
     if (!p.gw) return;
     unsigned remaining = __ballot_sync(FULL, act);
@@ -869,9 +887,9 @@ static tiga_status launch_fwd_g(const CsrParams& p, int G, int VPL, cudaStream_t
     }
 }
 
-template <typename IT>
+template <typename IT, typename XT>
 static tiga_status launch_bwd_g(const CsrParams& p, int G, int VPL, cudaStream_t s) {
-#define TIGA_BWD(GG, VV) csr_backward_sum_kernel<GG, VV, IT><<<counted((unsigned)p.ntiles), CSR_THREADS, 0, s>>>(p); break
+#define TIGA_BWD(GG, VV) csr_backward_sum_kernel<GG, VV, IT, XT><<<counted((unsigned)p.ntiles), CSR_THREADS, 0, s>>>(p); break
     switch (G) {
         case 1: TIGA_BWD(1, 1);
         case 2: TIGA_BWD(2, 1);
@@ -1098,9 +1116,10 @@ extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x,
     (void)ws; (void)ws_bytes;
     tiga_status st = check_csr(g);
     if (st != TIGA_OK) return st;
-    if (x_dtype != TIGA_F32) return TIGA_ERR_UNSUPPORTED;
     int nvec, G, VPL;
-    st = check_features(F, x_dtype, &nvec, &G, &VPL);
+    st = check_features(F, x_dtype, &nvec, &G, &VPL);        // the feature rows must be whole 16-byte vectors
+    if (st != TIGA_OK) return st;
+    st = check_features(F, TIGA_F32, &nvec, &G, &VPL);       // lanes own four fp32 gradient values whatever x's type
     if (st != TIGA_OK) return st;
     if (reducer != TIGA_SUM && reducer != TIGA_MAX) return TIGA_ERR_INVALID_ARG;
     if (!msg) return TIGA_ERR_INVALID_ARG;
@@ -1125,10 +1144,13 @@ extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x,
     p.ntiles = num_tiles(g);
     p.gy = grad_out; p.gx = grad_x; p.gw = grad_w;
     if (reducer == TIGA_SUM) {
-        return g->rowptr_type == TIGA_I64 ? launch_bwd_g<int64_t>(p, G, VPL, s) : launch_bwd_g<int32_t>(p, G, VPL, s);
+        if (x_dtype == TIGA_F16)
+            return g->rowptr_type == TIGA_I64 ? launch_bwd_g<int64_t, __half>(p, G, VPL, s) : launch_bwd_g<int32_t, __half>(p, G, VPL, s);
+        return g->rowptr_type == TIGA_I64 ? launch_bwd_g<int64_t, float>(p, G, VPL, s) : launch_bwd_g<int32_t, float>(p, G, VPL, s);
     }
     const long long work = g->n_dst * F;
-    csr_backward_max_kernel<<<counted((unsigned)((work + 255) / 256)), 256, 0, s>>>(p);
+    if (x_dtype == TIGA_F16) csr_backward_max_kernel<__half><<<counted((unsigned)((work + 255) / 256)), 256, 0, s>>>(p);
+    else csr_backward_max_kernel<float><<<counted((unsigned)((work + 255) / 256)), 256, 0, s>>>(p);
     return launch_status();
 }
 

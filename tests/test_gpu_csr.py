@@ -146,6 +146,32 @@ def test_heavy_rows_span_many_tiles(tiga):
     _check_backward(tiga, rowptr, col, x, w, gy, g, xd, wd, res)
 
 
+def test_fp16_features_backward(tiga):
+    """Backward with an fp16 feature table: the oracle sees the same (exactly representable) values."""
+    for seed, n_dst, n_src, max_deg, F in [(31, 700, 300, 40, 8), (32, 300, 900, 70, 64), (33, 50, 20, 3000, 16)]:
+        rowptr, col, x, w, gy = _random_graph(seed, n_dst, n_src, max_deg, F)
+        x16 = x.astype(np.float16)
+        xr = x16.astype(np.float32)
+        g = _relation(tiga, rowptr, col, n_src)
+        xd, wd, gyd = dev(x16, torch), dev(w, torch), dev(gy, torch)
+        ref = oracle.csr_backward_sum(rowptr, col, xr, w, gy)
+        guard = Guard(torch)
+        gx, gw = tiga.tiga_apply_csr_backward(g, xd, wd, gyd, tiga.SUM, grad_x=guard.empty((n_src, F)), grad_w=guard.empty((g.n_edges,)))
+        guard.check()
+        assert gx.dtype == torch.float32
+        assert rel_err(host(gx), ref["gx"], ref["Ax"]) <= GRAD_TOL
+        assert rel_err(host(gw), ref["gw"], ref["Aw"]) <= GRAD_TOL
+        _, _, arg = oracle.csr_forward(rowptr, col, xr, w, oracle.MAX)
+        refm = oracle.csr_backward_max(rowptr, col, xr, w, gy, arg)
+        y, am = tiga.tiga_apply_csr(g, xd, wd, tiga.MAX)
+        assert np.array_equal(host(am), arg)
+        gx, gw = tiga.tiga_apply_csr_backward(g, xd, wd, gyd, tiga.MAX, argmax=am, grad_x=guard.empty((n_src, F)),
+                                              grad_w=guard.empty((g.n_edges,)))
+        guard.check()
+        assert rel_err(host(gx), refm["gx"], refm["Ax"]) <= GRAD_TOL
+        assert rel_err(host(gw), refm["gw"], refm["Aw"]) <= GRAD_TOL
+
+
 def test_hex_mesh_degrees(tiga):
     L = 24
     rowptr, col = gen.hex_mesh_csr(L)

@@ -325,6 +325,35 @@ def test_cfg3_full_size(tiga):
     assert np.max(np.abs(out[:, :3].astype(np.float64).sum(0))) < 1e-6 * A[:, :3].sum()
 
 
+def test_sparse_periodic_box_pairs_at_the_cutoff_across_a_face(tiga):
+    """Few points, small cutoff: the grid is capped (cells eleven times the cutoff), and pairs sit
+    within a few ulps of r on both sides of it across the lower x face and inside the box.  The
+    neighbour counts must equal the fp64 predicate's, pair by pair."""
+    r = np.float32(0.01)
+    ones = np.ones(3, np.float32)
+    rows = []
+    for k in range(24):
+        y, z = np.float32(0.04 * k + 0.013), np.float32(0.9 - 0.031 * k)
+        xa = np.float32(0.003 + 0.0001 * k)
+        xb = np.float32(1.0) - (r - xa)                      # across the face, about r away
+        xb = np.nextafter(xb, np.float32(2.0 if k % 2 else 0.0), dtype=np.float32)
+        for _ in range(k % 5):
+            xb = np.nextafter(xb, np.float32(2.0 if k % 2 else 0.0), dtype=np.float32)
+        rows += [[xa, y, z], [xb, y, z]]
+        xc = np.float32(0.4 + 0.01 * k)                      # the same inside the box
+        xd = xc + r
+        for _ in range(k % 4):
+            xd = np.nextafter(xd, np.float32(2.0 if k % 2 else 0.0), dtype=np.float32)
+        rows += [[xc, y, np.float32(z * 0.5)], [xd, y, np.float32(z * 0.5)]]
+    pos = np.array(rows, np.float32)
+    assert tiga.tiga_radius_grid(len(pos), float(r), ones, [1, 1, 1])[0][0] < 12      # capped grid
+    x = gen.normal_features(len(pos), 8, 5)
+    gy = gen.normal_features(len(pos), 8, 6)
+    _, cnt = _check_gauss(tiga, pos, x, gy, r, ones, [1, 1, 1], float(r) / 2)
+    c = host(cnt)
+    assert 0 < c.sum() < len(pos)                            # some of the pairs are inside, some outside
+
+
 # ------------------------------------------------------------------------------ validation
 def test_point_validation(tiga):
     box = np.array([1.0, 2.0, 0.5], np.float32)
