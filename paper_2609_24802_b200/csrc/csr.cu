@@ -67,6 +67,17 @@ struct State {
     }
 };
 
+// acc += w * x for two neighbouring features with one packed fused multiply-add (sm_100: one issue slot
+// for both lanes of the pair; each half rounds once, exactly like fmaf)
+__device__ __forceinline__ void fma_pair(float& a0, float& a1, float w, float x0, float x1) {
+    unsigned long long acc, xx, ww;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(acc) : "f"(a0), "f"(a1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(xx) : "f"(x0), "f"(x1));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(ww) : "f"(w));
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(ww), "l"(xx));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(acc));
+}
+
 // EXACT: the feature row fills the worker exactly (nvec == G * VPL): row stride and lane activity
 // are compile-time constants, which removes address arithmetic and predicates from the edge loop.
 template <typename XT, int G, int VPL, int RED, typename IT, bool EXACT>
@@ -185,14 +196,20 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
             }
             if (e + U <= b && e + U <= cur_end) {
                 // common case: the whole batch lies inside the current row and the span
+                constexpr bool PACKED = RED == 0 && sizeof(XT) == 4;
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     float xf[VW];
 #pragma unroll
                     for (int i = 0; i < VPL; ++i) {
                         XTraits<XT>::unpack(xv[u][i], xf);
+                        if constexpr (PACKED) {
 #pragma unroll
-                        for (int k = 0; k < VW; ++k) st.message(i, k, wv[u], xf[k], (int)(e0 + e + u));
+                            for (int k = 0; k < VW; k += 2) fma_pair(st.v[i][k], st.v[i][k + 1], wv[u], xf[k], xf[k + 1]);
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < VW; ++k) st.message(i, k, wv[u], xf[k], (int)(e0 + e + u));
+                        }
                     }
                 }
                 continue;
@@ -570,7 +587,7 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_huge_chunks_kernel(const CsrP
         const long long es = (long long)rowptr[ent.x] + (long long)ent.y * ROW_HUGE;
         const long long ee = (long long)rowptr[ent.x + 1];
         const int n = (int)(ee - es < ROW_HUGE ? ee - es : ROW_HUGE);
-        auto part = strided_row<XT, NV, RED, 32, 4, HOT, W>(p, src, es, n, lane);
+        auto part = strided_row<XT, NV, RED, 32, 8, HOT, W>(p, src, es, n, lane);
         reduce_and_store<XT, NV, RED, 32>(part, lane, true, p.carry_val + (size_t)idx * p.F, RED ? p.carry_arg + (size_t)idx * p.F : nullptr);
     }
 }
