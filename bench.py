@@ -965,7 +965,9 @@ def run_case(args):
         b_alg = E * (4 + 16) + N * (8 + 32)                       # col + one 16-byte source row per edge; rowptr + fp32 output row per row
         touched = int(torch.unique(g.col).numel()) if E <= (1 << 28) else None
         b_min = 8.0 * (N + 1) + 4.0 * E + 16.0 * (touched if touched is not None else 2.7e7) + 32.0 * N
-        b_dram = 35.5e9 * E / float(1 << 30)                      # profiles/csr_large_cfg4_dram_traffic.md, per edge
+        # profiles/csr_large_cfg4_dram_traffic.md: bytes per edge of the unplanned design (once measured at
+        # full size) or of the planned scale-24 replica (a lower bound at full size)
+        b_dram = (15.2 if args.planned else 33.1) * E
         sink = torch.zeros(1, device=dev)
         for _ in range(2):
             bench_probe.row_gather(x, g.col, sink)
@@ -979,7 +981,8 @@ def run_case(args):
                     "gather_note": "row-gather probe on the same col stream and feature table: the gathers alone, no row sums, no output",
                     "f_alg": b_alg / (ms * 1e-3) / hbm, "f_dram": b_dram / (ms * 1e-3) / hbm, "f_min": b_min / (ms * 1e-3) / hbm,
                     "bytes_alg": b_alg, "bytes_dram_ncu": b_dram, "bytes_min": b_min,
-                    "bytes_dram_note": "ncu capture at full size scaled by edges: meaningful at scale 26 only (smaller feature tables fit L2)",
+                    "bytes_dram_note": ("planned: ncu capture of the scale-24 replica scaled by edges, a lower bound at scale 26" if args.planned else
+                                        "unplanned: per-edge DRAM bytes of the full-size relation; smaller feature tables fit L2 and move less"),
                     "touched_source_rows": touched if touched is not None else "2.7e7 (analytic, R-MAT scale 26)",
                     "peak_GBps": peaks[0], "peak_source": peaks[2] if len(peaks) > 2 else "measured"})
     print(json.dumps(rec))

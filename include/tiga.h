@@ -49,7 +49,9 @@ typedef enum {
 
 typedef enum { TIGA_F32 = 0, TIGA_F16 = 1 } tiga_dtype;   /* feature storage; accumulation is fp32 */
 typedef enum { TIGA_I32 = 0, TIGA_I64 = 1 } tiga_itype;   /* rowptr storage; col is always int32 */
-typedef enum { TIGA_SUM = 0, TIGA_MAX = 1 } tiga_reducer;
+/* TIGA_MAX64: the max reducer with 64-bit edge positions in argmax (an int64 array); any relation may use
+ * it, relations of 2^31 edges or more must (TIGA_MAX keeps 32-bit positions). */
+typedef enum { TIGA_SUM = 0, TIGA_MAX = 1, TIGA_MAX64 = 2 } tiga_reducer;
 
 typedef enum {
     TIGA_MSG_COPY = 0,      /* CSR: m = x_j                         (w must be NULL)           */
@@ -109,14 +111,15 @@ tiga_status tiga_validate_csr(const tiga_csr* g, int level, void* ws, size_t ws_
  *   x      : [n_src, F], x_dtype.  F must be a multiple of 4 (fp32) or 8 (fp16).
  *   w      : fp32 [n_edges] or NULL for unit weights (msg.kind = TIGA_MSG_COPY).
  *   out    : fp32 [n_dst, F].
- *   argmax : int32 [n_dst, F]; required for TIGA_MAX (needs n_edges < 2^31), ignored for TIGA_SUM.
+ *   argmax : int32 [n_dst, F] for TIGA_MAX (needs n_edges < 2^31, else TIGA_ERR_UNSUPPORTED), int64 [n_dst, F] for
+ *            TIGA_MAX64; required for both, ignored for TIGA_SUM.
  *   ws     : tiga_csr_workspace_bytes(g, F, x_dtype, reducer, 0) bytes; contents are scratch.
  * Long rows are split and their partial states merged in a fixed order (edge order for feature
  * rows of 64 bytes and more; a fixed lane-strided tree for narrower rows), without atomics, so
  * results are reproducible from run to run. */
 tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
                            const float* w, const tiga_msg* msg, tiga_reducer reducer,
-                           float* out, int32_t* argmax, void* ws, size_t ws_bytes, void* stream);
+                           float* out, void* argmax, void* ws, size_t ws_bytes, void* stream);
 
 /* tiga_apply_csr for callers that cannot hand over a workspace.  (The paper has no counterpart;
  * this entry point exists for integration reasons only.)
@@ -133,7 +136,7 @@ tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dtype x_dtype,
  *   - Capacity: the call is refused with TIGA_ERR_TOO_LARGE, before anything is launched, when
  *     tiga_csr_workspace_bytes(g, F, x_dtype, reducer, 0) exceeds TIGA_BUILTIN_WS_BYTES
  *     (roughly (n_dst + n_edges) / 2048 * (4 F + 20) bytes plus about 1.5 KiB of padding, twice
- *     the F term for TIGA_MAX; e.g. 16.8M edges at F = 64 need 2.3 MiB).
+ *     the F term for TIGA_MAX, three times for TIGA_MAX64; e.g. 16.8M edges at F = 64 need 2.3 MiB).
  *   - It never calls cudaMalloc, cudaFree or any other allocating routine.
  *   - The first call on each device looks up the array's device address (a host-side lookup,
  *     done with that device current and cached per device).  Make that first call before any
@@ -147,7 +150,7 @@ tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dtype x_dtype,
 #define TIGA_BUILTIN_WS_BYTES (8u << 20)
 tiga_status tiga_apply_csr_builtin_ws(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
                                       const float* w, const tiga_msg* msg, tiga_reducer reducer,
-                                      float* out, int32_t* argmax, void* stream);
+                                      float* out, void* argmax, void* stream);
 
 /* Hot-source plan: one-time preprocessing of a stored relation whose feature table is far larger
  * than the L2 cache (the billion-edge relation of Section 7 held in device memory).  It depends on
@@ -193,21 +196,21 @@ size_t tiga_csr_planned_workspace_bytes(const tiga_csr* g, const tiga_csr_plan* 
                                         tiga_reducer reducer);
 tiga_status tiga_apply_csr_planned(const tiga_csr* g, const tiga_csr_plan* plan, const void* plan_buf,
                                    const void* x, tiga_dtype x_dtype, int32_t F, const float* w, const tiga_msg* msg,
-                                   tiga_reducer reducer, float* out, int32_t* argmax,
+                                   tiga_reducer reducer, float* out, void* argmax,
                                    void* ws, size_t ws_bytes, void* stream);
 
 /* Reverse mode of tiga_apply_csr for fixed relation indices (Section 5):
  *   sum : grad_w[e] = sum_f x[col[e],f] * grad_out[row(e),f]
  *         grad_x[j,:] = sum over edges e with col[e] = j of w[e] * grad_out[row(e),:]
  *   max : the cotangent of (i,f) flows only through edge argmax[i,f] (nothing if it is -1).
- *   grad_out : fp32 [n_dst, F];  argmax : the forward's output (TIGA_MAX only).
+ *   grad_out : fp32 [n_dst, F];  argmax : the forward's output (int32 for TIGA_MAX, int64 for TIGA_MAX64).
  *   grad_x   : fp32 [n_src, F] or NULL to skip;  grad_w : fp32 [n_edges] or NULL to skip.
  * x is fp32 or fp16 (the forward's feature table; F % 8 == 0 for fp16); all gradients are fp32, and the
  * cotangent of an fp16 table is the fp32 grad_x (no rounding to fp16 is applied).  Repeated sources accumulate with floating-point atomics, so grad_x (and
  * grad_w for TIGA_MAX) may differ in the last bits between runs. */
 tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
                                     const float* w, const tiga_msg* msg, tiga_reducer reducer,
-                                    const float* grad_out, const int32_t* argmax,
+                                    const float* grad_out, const void* argmax,
                                     float* grad_x, float* grad_w,
                                     void* ws, size_t ws_bytes, void* stream);
 

@@ -12,7 +12,7 @@ import os
 import torch
 
 __all__ = [
-    "TigaError", "load_library", "EXPORTS", "SUM", "MAX", "F32", "F16",
+    "TigaError", "load_library", "EXPORTS", "SUM", "MAX", "MAX64", "F32", "F16",
     "MSG_COPY", "MSG_WEIGHTED", "MSG_GAUSS", "MSG_DIST", "MSG_LJ",
     "CsrRelation", "tiga_status_string", "tiga_csr_workspace_bytes", "tiga_validate_csr",
     "tiga_apply_csr", "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram",
@@ -23,7 +23,7 @@ __all__ = [
     "tiga_csr_attention_workspace_bytes", "tiga_apply_csr_attention", "launch_count",
 ]
 
-SUM, MAX = 0, 1
+SUM, MAX, MAX64 = 0, 1, 2      # MAX64: max reducer whose argmax holds 64-bit edge positions (int64)
 F32, F16 = 0, 1
 I32, I64 = 0, 1
 MSG_COPY, MSG_WEIGHTED, MSG_GAUSS, MSG_DIST, MSG_LJ = 0, 1, 2, 3, 4
@@ -218,8 +218,8 @@ def tiga_apply_csr(g: CsrRelation, x, w=None, reducer: int = SUM, out=None, argm
     F = x.shape[1]
     if out is None:
         out = torch.empty((g.n_dst, F), dtype=torch.float32, device=x.device)
-    if reducer == MAX and argmax is None:
-        argmax = torch.empty((g.n_dst, F), dtype=torch.int32, device=x.device)
+    if reducer in (MAX, MAX64) and argmax is None:
+        argmax = torch.empty((g.n_dst, F), dtype=torch.int32 if reducer == MAX else torch.int64, device=x.device)
     if ws is None:
         ws = _ws(tiga_csr_workspace_bytes(g, F, _dt(x), reducer, False), x)
     msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)
@@ -240,8 +240,8 @@ def tiga_apply_csr_builtin_ws(g: CsrRelation, x, w=None, reducer: int = SUM, out
     F = x.shape[1]
     if out is None:
         out = torch.empty((g.n_dst, F), dtype=torch.float32, device=x.device)
-    if reducer == MAX and argmax is None:
-        argmax = torch.empty((g.n_dst, F), dtype=torch.int32, device=x.device)
+    if reducer in (MAX, MAX64) and argmax is None:
+        argmax = torch.empty((g.n_dst, F), dtype=torch.int32 if reducer == MAX else torch.int64, device=x.device)
     msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)
     _ok(load_library().tiga_apply_csr_builtin_ws(g.ref, _ptr(x), _dt(x), F, _ptr(w), ctypes.byref(msg), reducer,
                                                  _ptr(out), _ptr(argmax), _stream(stream)), "tiga_apply_csr_builtin_ws")
@@ -313,8 +313,8 @@ def tiga_apply_csr_planned(plan: CsrPlan, x, w=None, reducer: int = SUM, out=Non
     g = plan.g
     if out is None:
         out = torch.empty((g.n_dst, F), dtype=torch.float32, device=x.device)
-    if reducer == MAX and argmax is None:
-        argmax = torch.empty((g.n_dst, F), dtype=torch.int32, device=x.device)
+    if reducer in (MAX, MAX64) and argmax is None:
+        argmax = torch.empty((g.n_dst, F), dtype=torch.int32 if reducer == MAX else torch.int64, device=x.device)
     if ws is None:
         ws = _ws(tiga_csr_planned_workspace_bytes(plan, F, _dt(x), reducer), x)
     msg = _Msg(MSG_COPY if w is None else MSG_WEIGHTED, 0.0, 0.0)

@@ -26,12 +26,27 @@ static std::atomic<long long> g_kernel_launches{0};
 void note_launch() { g_kernel_launches.fetch_add(1, std::memory_order_relaxed); }
 
 // --------------------------------------------------------------------------------------------
-// Forward.  G lanes per worker, VPL 16-byte vectors per lane, RED = 0 sum / 1 max.
+// Forward.  G lanes per worker, VPL 16-byte vectors per lane, RED = 0 sum / 1 max / 2 max whose
+// edge positions are 64 bits wide (relations of 2^31 edges or more).
 // --------------------------------------------------------------------------------------------
+template <int RED> struct ArgOf { using type = int; };
+template <> struct ArgOf<2> { using type = long long; };
+template <int RED> using ArgT = typename ArgOf<RED>::type;
+
+// 16-byte (32-bit positions) or 2 x 16-byte (64-bit positions) store of four edge positions
+__device__ __forceinline__ void store_arg4(int* dst, int a0, int a1, int a2, int a3) {
+    st_stream(reinterpret_cast<int4*>(dst), make_int4(a0, a1, a2, a3));
+}
+__device__ __forceinline__ void store_arg4(long long* dst, long long a0, long long a1, long long a2, long long a3) {
+    st_stream(reinterpret_cast<longlong2*>(dst), make_longlong2(a0, a1));
+    st_stream(reinterpret_cast<longlong2*>(dst + 2), make_longlong2(a2, a3));
+}
+
 template <int RED, int VPL, int VW>
 struct State {
+    using AT = ArgT<RED>;
     float v[VPL][VW];
-    int a[RED ? VPL : 1][RED ? VW : 1];
+    AT a[RED ? VPL : 1][RED ? VW : 1];
     __device__ __forceinline__ void reset() {
 #pragma unroll
         for (int i = 0; i < VPL; ++i)
@@ -49,7 +64,7 @@ struct State {
         else return v[i][k];
     }
     // fold a message that comes later in edge order
-    __device__ __forceinline__ void message(int i, int k, float wgt, float xv, int e) {
+    __device__ __forceinline__ void message(int i, int k, float wgt, float xv, AT e) {
         if constexpr (RED == 0) {
             v[i][k] = fmaf(wgt, xv, v[i][k]);
         } else {
@@ -58,7 +73,7 @@ struct State {
         }
     }
     // fold a partial state that comes later in edge order
-    __device__ __forceinline__ void merge(int i, int k, float ov, int oa) {
+    __device__ __forceinline__ void merge(int i, int k, float ov, AT oa) {
         if constexpr (RED == 0) {
             v[i][k] += ov;
         } else {
@@ -95,7 +110,8 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
     __shared__ unsigned char s_first[NW];        // tail partial starts its chain
     extern __shared__ __align__(16) unsigned char s_dyn[];
     float* s_pv = reinterpret_cast<float*>(s_dyn);              // [2*NW][LV]
-    int* s_pa = reinterpret_cast<int*>(s_pv + 2 * NW * LV);     // [2*NW][LV] (max only)
+    using AT = ArgT<RED>;
+    AT* s_pa = reinterpret_cast<AT*>(s_pv + 2 * NW * LV);       // [2*NW][LV] (max only; 2*NW*LV floats keep it 8-byte aligned)
 
     const Tile t = stage_tile<IT>(p, s_ptr, s_col, s_w, s_coord);
     const int wk = threadIdx.x / G;
@@ -118,10 +134,9 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
             for (int k = 0; k < VW; k += 4)
                 st_stream(reinterpret_cast<float4*>(o + k), make_float4(s.out(i, k), s.out(i, k + 1), s.out(i, k + 2), s.out(i, k + 3)));
             if constexpr (RED != 0) {
-                int* ao = p.arg + row * F + (size_t)(i * G + ln) * VW;
+                AT* ao = static_cast<AT*>(p.arg) + row * F + (size_t)(i * G + ln) * VW;
 #pragma unroll
-                for (int k = 0; k < VW; k += 4)
-                    st_stream(reinterpret_cast<int4*>(ao + k), make_int4(s.a[i][k], s.a[i][k + 1], s.a[i][k + 2], s.a[i][k + 3]));
+                for (int k = 0; k < VW; k += 4) store_arg4(ao + k, s.a[i][k], s.a[i][k + 1], s.a[i][k + 2], s.a[i][k + 3]);
             }
         }
     };
@@ -140,7 +155,7 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
 #pragma unroll
             for (int k = 0; k < VW; ++k)
                 s.merge(i, k, s_pv[entry * LV + (i * G + ln) * VW + k],
-                        RED ? s_pa[entry * LV + (i * G + ln) * VW + k] : 0);
+                        RED ? s_pa[entry * LV + (i * G + ln) * VW + k] : AT(0));
     };
 
     // rows that end in this tile without an edge in it: the reducer identity (finalised to 0)
@@ -208,7 +223,7 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
                             for (int k = 0; k < VW; k += 2) fma_pair(st.v[i][k], st.v[i][k + 1], wv[u], xf[k], xf[k + 1]);
                         } else {
 #pragma unroll
-                            for (int k = 0; k < VW; ++k) st.message(i, k, wv[u], xf[k], (int)(e0 + e + u));
+                            for (int k = 0; k < VW; ++k) st.message(i, k, wv[u], xf[k], (AT)(e0 + e + u));
                         }
                     }
                 }
@@ -230,7 +245,7 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
                     for (int i = 0; i < VPL; ++i) {
                         XTraits<XT>::unpack(xv[u][i], xf);
 #pragma unroll
-                        for (int k = 0; k < VW; ++k) st.message(i, k, wv[u], xf[k], (int)(e0 + e + u));
+                        for (int k = 0; k < VW; ++k) st.message(i, k, wv[u], xf[k], (AT)(e0 + e + u));
                     }
                 }
             }
@@ -268,7 +283,7 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
 #pragma unroll
                 for (int k = 0; k < VW; ++k) {
                     p.carry_val[o + k] = st.v[i][k];
-                    if constexpr (RED != 0) p.carry_arg[o + k] = st.a[i][k];
+                    if constexpr (RED != 0) static_cast<AT*>(p.carry_arg)[o + k] = st.a[i][k];
                 }
             }
         }
@@ -325,7 +340,8 @@ struct Sources {
 // kept<C, L>() entries, the group totals of the values starting at spread_index<NVAL, L>(gl).
 template <int RED, int C, int J, int L>
 struct Spread {
-    static __device__ __forceinline__ void run(float* v, int* a, int gl) {
+    static __device__ __forceinline__ void run(float* v, ArgT<RED>* a, int gl) {
+        using AT = ArgT<RED>;
         if constexpr ((1 << J) < L) {
             constexpr int o = 1 << J;
             constexpr unsigned FULL = 0xffffffffu;
@@ -340,9 +356,9 @@ struct Spread {
                     if constexpr (RED == 0) {
                         v[k] = keep + got;
                     } else {
-                        const int sa = up ? a[k] : a[k + H];
-                        const int ka = up ? a[k + H] : a[k];
-                        const int ga = __shfl_xor_sync(FULL, sa, o);
+                        const AT sa = up ? a[k] : a[k + H];
+                        const AT ka = up ? a[k + H] : a[k];
+                        const AT ga = __shfl_xor_sync(FULL, sa, o);
                         // larger message wins; equal messages: the lower edge position
                         const bool take = ga >= 0 && (ka < 0 || got > keep || (got == keep && ga < ka));
                         v[k] = take ? got : keep;
@@ -355,7 +371,7 @@ struct Spread {
                 if constexpr (RED == 0) {
                     v[0] += got;
                 } else {
-                    const int ga = __shfl_xor_sync(FULL, a[0], o);
+                    const AT ga = __shfl_xor_sync(FULL, a[0], o);
                     const bool take = ga >= 0 && (a[0] < 0 || got > v[0] || (got == v[0] && ga < a[0]));
                     if (take) { v[0] = got; a[0] = ga; }
                 }
@@ -420,7 +436,7 @@ __device__ __forceinline__ State<RED, NV, XTraits<XT>::VW> strided_row(const Csr
                     for (int i = 0; i < NV; ++i) {
                         XTraits<XT>::unpack(xv[u][i], xf);
 #pragma unroll
-                        for (int q = 0; q < VW; ++q) s.message(i, q, wv[u], xf[q], (int)(es + k + L * u));
+                        for (int q = 0; q < VW; ++q) s.message(i, q, wv[u], xf[q], (ArgT<RED>)(es + k + L * u));
                     }
                 }
             }
@@ -430,26 +446,25 @@ __device__ __forceinline__ State<RED, NV, XTraits<XT>::VW> strided_row(const Csr
 }
 
 template <typename XT, int NV, int RED>
-__device__ __forceinline__ void store_state(const CsrParams& p, float* out, int32_t* arg, const State<RED, NV, XTraits<XT>::VW>& s) {
+__device__ __forceinline__ void store_state(const CsrParams& p, float* out, ArgT<RED>* arg, const State<RED, NV, XTraits<XT>::VW>& s) {
     constexpr int VW = XTraits<XT>::VW;
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
 #pragma unroll
         for (int k = 0; k < VW; k += 4) {
             st_stream(reinterpret_cast<float4*>(out + i * VW + k), make_float4(s.out(i, k), s.out(i, k + 1), s.out(i, k + 2), s.out(i, k + 3)));
-            if constexpr (RED != 0)
-                st_stream(reinterpret_cast<int4*>(arg + i * VW + k), make_int4(s.a[i][k], s.a[i][k + 1], s.a[i][k + 2], s.a[i][k + 3]));
+            if constexpr (RED != 0) store_arg4(arg + i * VW + k, s.a[i][k], s.a[i][k + 1], s.a[i][k + 2], s.a[i][k + 3]);
         }
     }
 }
 
 // combine the partial states of a group of L lanes and store the row: every lane writes its share
 template <typename XT, int NV, int RED, int L>
-__device__ __forceinline__ void reduce_and_store(State<RED, NV, XTraits<XT>::VW>& s, int gl, bool valid, float* out, int32_t* arg) {
+__device__ __forceinline__ void reduce_and_store(State<RED, NV, XTraits<XT>::VW>& s, int gl, bool valid, float* out, ArgT<RED>* arg) {
     constexpr int NVAL = NV * XTraits<XT>::VW;
     constexpr int KEEP = NVAL >= L ? NVAL / L : 1;
     float* v = &s.v[0][0];
-    int* a = &s.a[0][0];
+    ArgT<RED>* a = &s.a[0][0];
     Spread<RED, NVAL, 0, L>::run(v, a, gl);
     if (valid && gl < NVAL) {
         const int base = spread_index<NVAL, L>(gl);
@@ -528,12 +543,12 @@ __global__ void __launch_bounds__(CSR_THREADS, 6) csr_rows_kernel(const CsrParam
                     for (int i = 0; i < NV; ++i) {
                         XTraits<XT>::unpack(xv[u][i], xf);
 #pragma unroll
-                        for (int q = 0; q < VW; ++q) st.message(i, q, wv[u], xf[q], (int)(es + u));
+                        for (int q = 0; q < VW; ++q) st.message(i, q, wv[u], xf[q], (ArgT<RED>)(es + u));
                     }
                 }
             }
         }
-        store_state<XT, NV, RED>(p, p.out + row * p.F, RED ? p.arg + row * p.F : nullptr, st);
+        store_state<XT, NV, RED>(p, p.out + row * p.F, RED ? static_cast<ArgT<RED>*>(p.arg) + row * p.F : nullptr, st);
     }
     __syncthreads();
     const long long row0 = (long long)blockIdx.x * CSR_THREADS;
@@ -552,7 +567,7 @@ __global__ void __launch_bounds__(CSR_THREADS, 6) csr_rows_kernel(const CsrParam
             const long long r = row0 + (have ? q_row[it] : 0);
             St part = strided_row<XT, NV, RED, GROUP_LANES, 4, HOT, W>(p, src, rs, rn, gl);
             __syncwarp();
-            reduce_and_store<XT, NV, RED, GROUP_LANES>(part, gl, have, p.out + r * p.F, RED ? p.arg + r * p.F : nullptr);
+            reduce_and_store<XT, NV, RED, GROUP_LANES>(part, gl, have, p.out + r * p.F, RED ? static_cast<ArgT<RED>*>(p.arg) + r * p.F : nullptr);
         }
     }
     // rows for whole warps, taken from the back of the queue
@@ -564,7 +579,7 @@ __global__ void __launch_bounds__(CSR_THREADS, 6) csr_rows_kernel(const CsrParam
         const int slot = CSR_THREADS - 1 - idx;
         const long long r = row0 + q_row[slot];
         St part = strided_row<XT, NV, RED, 32, 4, HOT, W>(p, src, q_start[slot], q_len[slot], lane);
-        reduce_and_store<XT, NV, RED, 32>(part, lane, true, p.out + r * p.F, RED ? p.arg + r * p.F : nullptr);
+        reduce_and_store<XT, NV, RED, 32>(part, lane, true, p.out + r * p.F, RED ? static_cast<ArgT<RED>*>(p.arg) + r * p.F : nullptr);
     }
     // huge rows: queue their chunks
     if (valid && deg > ROW_HUGE) {
@@ -588,7 +603,7 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_huge_chunks_kernel(const CsrP
         const long long ee = (long long)rowptr[ent.x + 1];
         const int n = (int)(ee - es < ROW_HUGE ? ee - es : ROW_HUGE);
         auto part = strided_row<XT, NV, RED, 32, 8, HOT, W>(p, src, es, n, lane);
-        reduce_and_store<XT, NV, RED, 32>(part, lane, true, p.carry_val + (size_t)idx * p.F, RED ? p.carry_arg + (size_t)idx * p.F : nullptr);
+        reduce_and_store<XT, NV, RED, 32>(part, lane, true, p.carry_val + (size_t)idx * p.F, RED ? static_cast<ArgT<RED>*>(p.carry_arg) + (size_t)idx * p.F : nullptr);
     }
 }
 
@@ -602,17 +617,19 @@ __global__ void csr_huge_fold_kernel(const CsrParams p) {
         const int4 ent = p.huge_list[idx];
         if (ent.y != 0) continue;
         float v = p.carry_val[(size_t)idx * p.F + f];
-        int a = RED ? p.carry_arg[(size_t)idx * p.F + f] : 0;
+        using AT = ArgT<RED>;
+        const AT* carg = static_cast<const AT*>(p.carry_arg);
+        AT a = RED ? carg[(size_t)idx * p.F + f] : AT(0);
         for (int c = 1; c < ent.z; ++c) {
             const float ov = p.carry_val[(size_t)(idx + c) * p.F + f];
             if (RED == 0) v += ov;
             else {
-                const int oa = p.carry_arg[(size_t)(idx + c) * p.F + f];
+                const AT oa = carg[(size_t)(idx + c) * p.F + f];
                 if (oa >= 0 && (a < 0 || ov > v)) { v = ov; a = oa; }
             }
         }
         p.out[(size_t)ent.x * p.F + f] = v;
-        if (RED) p.arg[(size_t)ent.x * p.F + f] = a;
+        if (RED) static_cast<AT*>(p.arg)[(size_t)ent.x * p.F + f] = a;
     }
 }
 
@@ -628,12 +645,14 @@ __global__ void csr_fixup_kernel(const CsrParams p) {
     if (row < 0) return;
     if (tile > 0 && p.carry_row[tile - 1] == row) return;
     float v = p.carry_val[tile * p.F + f];
-    int a = RED ? p.carry_arg[tile * p.F + f] : 0;
+    using AT = ArgT<RED>;
+    const AT* carg = static_cast<const AT*>(p.carry_arg);
+    AT a = RED ? carg[tile * p.F + f] : AT(0);
     for (long long u = tile + 1; u < p.ntiles && p.carry_row[u] == row; ++u) {
         const float ov = p.carry_val[u * p.F + f];
         if (RED == 0) v += ov;
         else {
-            const int oa = p.carry_arg[u * p.F + f];
+            const AT oa = carg[u * p.F + f];
             if (oa >= 0 && (a < 0 || ov > v)) { v = ov; a = oa; }
         }
     }
@@ -642,10 +661,10 @@ __global__ void csr_fixup_kernel(const CsrParams p) {
         p.out[o] = v + p.out[o];
     } else {
         const float ov = p.out[o];
-        const int oa = p.arg[o];
+        const AT oa = static_cast<AT*>(p.arg)[o];
         if (oa >= 0 && (a < 0 || ov > v)) { v = ov; a = oa; }
         p.out[o] = v;
-        p.arg[o] = a;
+        static_cast<AT*>(p.arg)[o] = a;
     }
 }
 
@@ -669,7 +688,6 @@ __device__ __forceinline__ float4 load_x4(const void* x, unsigned long long vec)
 
 template <int G, int VPL, typename IT, typename XT>
 __global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const CsrParams p) {
-    constexpr int VW = 4;
     constexpr int NW = CSR_THREADS / G;
     constexpr int U = (VPL == 1) ? 4 : (VPL == 2 ? 2 : 1);
     __shared__ int s_ptr[CSR_TILE + 2];
@@ -760,12 +778,13 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const Csr
 // (two rounds, each for the edge of the lowest lane not served yet; what is left goes out one by
 // one: more rounds measured slower): one atomic per edge instead of
 // up to 32 on the same address.
-template <typename XT>
+template <typename XT, int RED>
 __global__ void csr_backward_max_kernel(const CsrParams p) {
+    using AT = ArgT<RED>;
     constexpr unsigned FULL = 0xffffffffu;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const int lane = threadIdx.x & 31;
-    const int e = idx < p.n_dst * p.F ? p.arg[idx] : -1;
+    const AT e = idx < p.n_dst * p.F ? static_cast<const AT*>(p.arg)[idx] : AT(-1);
     const bool act = e >= 0;
     float contrib = 0.f;
     if (act) {
@@ -788,7 +807,7 @@ __global__ void csr_backward_max_kernel(const CsrParams p) {
             break;
         }
         const int leader = __ffs(remaining) - 1;
-        const int el = __shfl_sync(FULL, e, leader);
+        const AT el = __shfl_sync(FULL, e, leader);
         const bool mine = act && e == el;
         float s = mine ? contrib : 0.f;
 #pragma unroll
@@ -864,7 +883,7 @@ static long long num_tiles(const tiga_csr* g) { return (g->n_dst + g->n_edges + 
 template <typename XT, int G, int VPL, int RED, typename IT>
 static tiga_status launch_fwd_t(const CsrParams& p, cudaStream_t s) {
     constexpr int NW = CSR_THREADS / G;
-    const size_t dyn = (size_t)2 * NW * G * VPL * XTraits<XT>::VW * sizeof(float) * (RED ? 2 : 1);
+    const size_t dyn = (size_t)2 * NW * G * VPL * XTraits<XT>::VW * (sizeof(float) + (RED ? sizeof(ArgT<RED>) : 0));
     auto kern = p.nvec == G * VPL ? csr_forward_kernel<XT, G, VPL, RED, IT, true> : csr_forward_kernel<XT, G, VPL, RED, IT, false>;
     if (dyn > 16 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
     kern<<<counted((unsigned)p.ntiles), CSR_THREADS, dyn, s>>>(p);
@@ -943,6 +962,15 @@ static tiga_status check_features(int32_t F, tiga_dtype dt, int* nvec, int* G, i
     return pick_shape(*nvec, G, VPL) ? TIGA_OK : TIGA_ERR_UNSUPPORTED;
 }
 
+static bool known_reducer(tiga_reducer r) { return r == TIGA_SUM || r == TIGA_MAX || r == TIGA_MAX64; }
+static bool is_max(tiga_reducer r) { return r == TIGA_MAX || r == TIGA_MAX64; }
+static size_t arg_bytes(tiga_reducer r) { return r == TIGA_MAX64 ? sizeof(int64_t) : sizeof(int32_t); }
+// workspace array of edge positions, typed by the reducer
+static void* take_args(Carver& cv, tiga_reducer r, size_t n) {
+    if (!is_max(r)) return nullptr;
+    return r == TIGA_MAX64 ? static_cast<void*>(cv.take<int64_t>(n)) : static_cast<void*>(cv.take<int32_t>(n));
+}
+
 }  // namespace tiga
 
 using namespace tiga;
@@ -952,7 +980,7 @@ extern "C" size_t tiga_csr_workspace_bytes(const tiga_csr* g, int32_t F, tiga_dt
     if (backward) return 256;
     const size_t nt = (size_t)num_tiles(g) + 1;
     size_t b = align_up(nt * sizeof(int32_t), 256) + align_up(nt * F * sizeof(float), 256);
-    if (reducer == TIGA_MAX) b += align_up(nt * F * sizeof(int32_t), 256);
+    if (is_max(reducer)) b += align_up(nt * F * arg_bytes(reducer), 256);
     b += 256 + align_up(nt * sizeof(int4), 256);      // queue of huge-row chunks (narrow-row path)
     return b + 256;
 }
@@ -982,13 +1010,13 @@ extern "C" tiga_status tiga_validate_csr(const tiga_csr* g, int level, void* ws,
 
 extern "C" tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
                                       const float* w, const tiga_msg* msg, tiga_reducer reducer,
-                                      float* out, int32_t* argmax, void* ws, size_t ws_bytes, void* stream) {
+                                      float* out, void* argmax, void* ws, size_t ws_bytes, void* stream) {
     tiga_status st = check_csr(g);
     if (st != TIGA_OK) return st;
     int nvec, G, VPL;
     st = check_features(F, x_dtype, &nvec, &G, &VPL);
     if (st != TIGA_OK) return st;
-    if (reducer != TIGA_SUM && reducer != TIGA_MAX) return TIGA_ERR_INVALID_ARG;
+    if (!known_reducer(reducer)) return TIGA_ERR_INVALID_ARG;
     if (!msg) return TIGA_ERR_INVALID_ARG;
     if (msg->kind == TIGA_MSG_COPY) { if (w) return TIGA_ERR_INVALID_ARG; }
     else if (msg->kind == TIGA_MSG_WEIGHTED) { if (!w && g->n_edges > 0) return TIGA_ERR_INVALID_ARG; }
@@ -996,9 +1024,9 @@ extern "C" tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dty
     if (g->n_dst == 0) return TIGA_OK;
     if (!out || !aligned16(out) || (g->n_src > 0 && (!x || !aligned16(x)))) return TIGA_ERR_INVALID_ARG;
     if (w && !aligned16(w)) return TIGA_ERR_INVALID_ARG;
-    if (reducer == TIGA_MAX) {
+    if (is_max(reducer)) {
         if (!argmax || !aligned16(argmax)) return TIGA_ERR_INVALID_ARG;
-        if (g->n_edges > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;
+        if (reducer == TIGA_MAX && g->n_edges > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;     // 32-bit positions: use TIGA_MAX64
     }
     if (!ws || !aligned16(ws) || ws_bytes < tiga_csr_workspace_bytes(g, F, x_dtype, reducer, 0)) return TIGA_ERR_WORKSPACE;
 
@@ -1010,12 +1038,16 @@ extern "C" tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dty
     Carver cv(ws);
     p.carry_row = cv.take<int32_t>((size_t)p.ntiles + 1);
     p.carry_val = cv.take<float>(((size_t)p.ntiles + 1) * F);
-    p.carry_arg = reducer == TIGA_MAX ? cv.take<int32_t>(((size_t)p.ntiles + 1) * F) : nullptr;
+    p.carry_arg = take_args(cv, reducer, ((size_t)p.ntiles + 1) * F);
     p.huge_count = cv.take<int>(1);
     p.huge_list = cv.take<int4>((size_t)p.ntiles + 1);      // >= 2 E / ROW_HUGE + 1 entries
 
     const bool i64 = g->rowptr_type == TIGA_I64;
-    if (x_dtype == TIGA_F32) {
+    if (reducer == TIGA_MAX64) {
+        // 64-bit positions only make sense with 64-bit row offsets; a 32-bit rowptr still works
+        if (x_dtype == TIGA_F32) st = i64 ? launch_fwd_g<float, 2, int64_t>(p, G, VPL, s) : launch_fwd_g<float, 2, int32_t>(p, G, VPL, s);
+        else st = i64 ? launch_fwd_g<__half, 2, int64_t>(p, G, VPL, s) : launch_fwd_g<__half, 2, int32_t>(p, G, VPL, s);
+    } else if (x_dtype == TIGA_F32) {
         if (reducer == TIGA_SUM) st = i64 ? launch_fwd_g<float, 0, int64_t>(p, G, VPL, s) : launch_fwd_g<float, 0, int32_t>(p, G, VPL, s);
         else st = i64 ? launch_fwd_g<float, 1, int64_t>(p, G, VPL, s) : launch_fwd_g<float, 1, int32_t>(p, G, VPL, s);
     } else {
@@ -1025,8 +1057,10 @@ extern "C" tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dty
     if (st != TIGA_OK) return st;
     if (nvec <= 2) return TIGA_OK;             // the row-class path has no tile carry-outs
     const long long work = p.ntiles * F;
-    if (reducer == TIGA_SUM) csr_fixup_kernel<0><<<counted((unsigned)((work + 255) / 256)), 256, 0, s>>>(p);
-    else csr_fixup_kernel<1><<<counted((unsigned)((work + 255) / 256)), 256, 0, s>>>(p);
+    const unsigned fix_blocks = (unsigned)((work + 255) / 256);
+    if (reducer == TIGA_SUM) csr_fixup_kernel<0><<<counted(fix_blocks), 256, 0, s>>>(p);
+    else if (reducer == TIGA_MAX) csr_fixup_kernel<1><<<counted(fix_blocks), 256, 0, s>>>(p);
+    else csr_fixup_kernel<2><<<counted(fix_blocks), 256, 0, s>>>(p);
     return launch_status();
 }
 
@@ -1055,12 +1089,12 @@ static tiga_status builtin_ws_address(void** out) {
 
 extern "C" tiga_status tiga_apply_csr_builtin_ws(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
                                                  const float* w, const tiga_msg* msg, tiga_reducer reducer,
-                                                 float* out, int32_t* argmax, void* stream) {
+                                                 float* out, void* argmax, void* stream) {
     // capacity first: a refusal touches neither the device nor the array
     tiga_status st = check_csr(g);
     if (st != TIGA_OK) return st;
     if (F <= 0) return TIGA_ERR_INVALID_ARG;
-    if (reducer != TIGA_SUM && reducer != TIGA_MAX) return TIGA_ERR_INVALID_ARG;
+    if (!known_reducer(reducer)) return TIGA_ERR_INVALID_ARG;
     if (tiga_csr_workspace_bytes(g, F, x_dtype, reducer, 0) > (size_t)TIGA_BUILTIN_WS_BYTES) return TIGA_ERR_TOO_LARGE;
     void* ws = nullptr;
     st = builtin_ws_address(&ws);
@@ -1078,7 +1112,7 @@ extern "C" size_t tiga_csr_planned_workspace_bytes(const tiga_csr* g, const tiga
 
 extern "C" tiga_status tiga_apply_csr_planned(const tiga_csr* g, const tiga_csr_plan* plan, const void* plan_buf,
                                               const void* x, tiga_dtype x_dtype, int32_t F, const float* w, const tiga_msg* msg,
-                                              tiga_reducer reducer, float* out, int32_t* argmax,
+                                              tiga_reducer reducer, float* out, void* argmax,
                                               void* ws, size_t ws_bytes, void* stream) {
     tiga_status st = check_csr(g);
     if (st != TIGA_OK) return st;
@@ -1088,14 +1122,15 @@ extern "C" tiga_status tiga_apply_csr_planned(const tiga_csr* g, const tiga_csr_
     st = check_features(F, x_dtype, &nvec, &G, &VPL);
     if (st != TIGA_OK) return st;
     if (nvec > 2) return TIGA_ERR_UNSUPPORTED;            // feature rows of at most 32 bytes: the case the plan exists for
-    if (reducer != TIGA_SUM && reducer != TIGA_MAX) return TIGA_ERR_INVALID_ARG;
+    if (!known_reducer(reducer)) return TIGA_ERR_INVALID_ARG;
+    if (reducer == TIGA_MAX && g->n_edges > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;
     if (!msg) return TIGA_ERR_INVALID_ARG;
     if (msg->kind == TIGA_MSG_COPY) { if (w) return TIGA_ERR_INVALID_ARG; }
     else if (msg->kind == TIGA_MSG_WEIGHTED) { if (!w) return TIGA_ERR_INVALID_ARG; }
     else return TIGA_ERR_UNSUPPORTED;
     if (g->n_dst == 0) return TIGA_OK;
     if (!out || !aligned16(out) || !x || !aligned16(x) || (w && !aligned16(w))) return TIGA_ERR_INVALID_ARG;
-    if (reducer == TIGA_MAX && (!argmax || !aligned16(argmax))) return TIGA_ERR_INVALID_ARG;
+    if (is_max(reducer) && (!argmax || !aligned16(argmax))) return TIGA_ERR_INVALID_ARG;
     if (!ws || !aligned16(ws) || ws_bytes < tiga_csr_planned_workspace_bytes(g, plan, F, x_dtype, reducer)) return TIGA_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const char* base = static_cast<const char*>(plan_buf);
@@ -1111,12 +1146,16 @@ extern "C" tiga_status tiga_apply_csr_planned(const tiga_csr* g, const tiga_csr_
     p.x_hot = hot; p.n_hot = (int)plan->n_hot;
     p.carry_row = cv.take<int32_t>((size_t)p.ntiles + 1);
     p.carry_val = cv.take<float>(((size_t)p.ntiles + 1) * F);
-    p.carry_arg = reducer == TIGA_MAX ? cv.take<int32_t>(((size_t)p.ntiles + 1) * F) : nullptr;
+    p.carry_arg = take_args(cv, reducer, ((size_t)p.ntiles + 1) * F);
     p.huge_count = cv.take<int>(1);
     p.huge_list = cv.take<int4>((size_t)p.ntiles + 1);
     st = launch_gather_hot(x, reinterpret_cast<const int32_t*>(base + plan->off_hot_id), plan->n_hot, nvec, hot, s);
     if (st != TIGA_OK) return st;
     const bool i64 = g->rowptr_type == TIGA_I64;
+    if (reducer == TIGA_MAX64) {
+        if (x_dtype == TIGA_F32) return i64 ? launch_fwd_narrow<float, 2, int64_t, true>(p, s) : launch_fwd_narrow<float, 2, int32_t, true>(p, s);
+        return i64 ? launch_fwd_narrow<__half, 2, int64_t, true>(p, s) : launch_fwd_narrow<__half, 2, int32_t, true>(p, s);
+    }
     if (x_dtype == TIGA_F32) {
         if (reducer == TIGA_SUM) return i64 ? launch_fwd_narrow<float, 0, int64_t, true>(p, s) : launch_fwd_narrow<float, 0, int32_t, true>(p, s);
         return i64 ? launch_fwd_narrow<float, 1, int64_t, true>(p, s) : launch_fwd_narrow<float, 1, int32_t, true>(p, s);
@@ -1127,7 +1166,7 @@ extern "C" tiga_status tiga_apply_csr_planned(const tiga_csr* g, const tiga_csr_
 
 extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x, tiga_dtype x_dtype, int32_t F,
                                                const float* w, const tiga_msg* msg, tiga_reducer reducer,
-                                               const float* grad_out, const int32_t* argmax,
+                                               const float* grad_out, const void* argmax,
                                                float* grad_x, float* grad_w,
                                                void* ws, size_t ws_bytes, void* stream) {
     (void)ws; (void)ws_bytes;
@@ -1138,7 +1177,7 @@ extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x,
     if (st != TIGA_OK) return st;
     st = check_features(F, TIGA_F32, &nvec, &G, &VPL);       // lanes own four fp32 gradient values whatever x's type
     if (st != TIGA_OK) return st;
-    if (reducer != TIGA_SUM && reducer != TIGA_MAX) return TIGA_ERR_INVALID_ARG;
+    if (!known_reducer(reducer)) return TIGA_ERR_INVALID_ARG;
     if (!msg) return TIGA_ERR_INVALID_ARG;
     if (msg->kind == TIGA_MSG_COPY) { if (w) return TIGA_ERR_INVALID_ARG; }
     else if (msg->kind == TIGA_MSG_WEIGHTED) { if (!w && g->n_edges > 0) return TIGA_ERR_INVALID_ARG; }
@@ -1146,17 +1185,17 @@ extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x,
     if (g->n_dst > 0 && (!grad_out || !aligned16(grad_out))) return TIGA_ERR_INVALID_ARG;
     if (g->n_src > 0 && (!x || !aligned16(x))) return TIGA_ERR_INVALID_ARG;
     if ((grad_x && !aligned16(grad_x)) || (grad_w && !aligned16(grad_w)) || (w && !aligned16(w))) return TIGA_ERR_INVALID_ARG;
-    if (reducer == TIGA_MAX) {
+    if (is_max(reducer)) {
         if (g->n_dst > 0 && (!argmax || !aligned16(argmax))) return TIGA_ERR_INVALID_ARG;
-        if (g->n_edges > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;
+        if (reducer == TIGA_MAX && g->n_edges > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (grad_x && g->n_src > 0) TIGA_CUDA_TRY(cudaMemsetAsync(grad_x, 0, (size_t)g->n_src * F * sizeof(float), s));
-    if (reducer == TIGA_MAX && grad_w && g->n_edges > 0) TIGA_CUDA_TRY(cudaMemsetAsync(grad_w, 0, (size_t)g->n_edges * sizeof(float), s));
+    if (is_max(reducer) && grad_w && g->n_edges > 0) TIGA_CUDA_TRY(cudaMemsetAsync(grad_w, 0, (size_t)g->n_edges * sizeof(float), s));
     if (g->n_dst == 0 || g->n_edges == 0 || (!grad_x && !grad_w)) return TIGA_OK;
 
     CsrParams p{};
-    p.rowptr = g->rowptr; p.col = g->col; p.w = w; p.x = x; p.arg = const_cast<int32_t*>(argmax);
+    p.rowptr = g->rowptr; p.col = g->col; p.w = w; p.x = x; p.arg = const_cast<void*>(argmax);
     p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.F = F; p.nvec = nvec;
     p.ntiles = num_tiles(g);
     p.gy = grad_out; p.gx = grad_x; p.gw = grad_w;
@@ -1165,9 +1204,14 @@ extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x,
             return g->rowptr_type == TIGA_I64 ? launch_bwd_g<int64_t, __half>(p, G, VPL, s) : launch_bwd_g<int32_t, __half>(p, G, VPL, s);
         return g->rowptr_type == TIGA_I64 ? launch_bwd_g<int64_t, float>(p, G, VPL, s) : launch_bwd_g<int32_t, float>(p, G, VPL, s);
     }
-    const long long work = g->n_dst * F;
-    if (x_dtype == TIGA_F16) csr_backward_max_kernel<__half><<<counted((unsigned)((work + 255) / 256)), 256, 0, s>>>(p);
-    else csr_backward_max_kernel<float><<<counted((unsigned)((work + 255) / 256)), 256, 0, s>>>(p);
+    const unsigned blocks = (unsigned)((g->n_dst * F + 255) / 256);
+    if (reducer == TIGA_MAX) {
+        if (x_dtype == TIGA_F16) csr_backward_max_kernel<__half, 1><<<counted(blocks), 256, 0, s>>>(p);
+        else csr_backward_max_kernel<float, 1><<<counted(blocks), 256, 0, s>>>(p);
+    } else {
+        if (x_dtype == TIGA_F16) csr_backward_max_kernel<__half, 2><<<counted(blocks), 256, 0, s>>>(p);
+        else csr_backward_max_kernel<float, 2><<<counted(blocks), 256, 0, s>>>(p);
+    }
     return launch_status();
 }
 

@@ -51,14 +51,14 @@ struct CsrParams {
     const float* w;          // may be null (unit weights)
     const void* x;
     float* out;
-    int32_t* arg;
+    void* arg;               // int32 [n_dst, F], or int64 for the wide-position max reducer
     long long n_dst, n_edges;
     int F;                   // features per row
     int nvec;                // 16-byte vectors per feature row
     // workspace
     int32_t* carry_row;      // [ntiles]  row of the tile's trailing partial state, or -1
     float* carry_val;        // [ntiles, F]
-    int32_t* carry_arg;      // [ntiles, F] (max only)
+    void* carry_arg;         // [ntiles, F] (max only; same element type as arg)
     long long ntiles;
     int* huge_count;         // narrow-row path: number of queued chunks of huge rows
     int4* huge_list;         // (row, chunk, chunks of the row, first slot of the row)

@@ -85,4 +85,6 @@ class Guard:
                 assert not bool(t.isnan(view).any()), "an output element was not written (still NaN)"
             elif view.element_size() == 4:
                 assert not bool((view.view(t.int32) == -1515870811).any()), "an output element was not written"
+            elif view.element_size() == 8:
+                assert not bool((view.view(t.int64) == -6510615555426900571).any()), "an output element was not written"
         self.items = []

@@ -47,6 +47,13 @@ def _check_forward(tiga, rowptr, col, x, w, index64=False, reducers=(0, 1)):
             assert np.array_equal(host(out), y.astype(np.float32)), "max outputs must be bit exact"
             assert np.array_equal(host(am).astype(np.int64), arg), "argmax must be bit exact"
             assert torch.equal(am, am2)
+            # the same reducer with 64-bit edge positions: same values, same positions, wider array
+            ws64 = guard.workspace(tiga.tiga_csr_workspace_bytes(g, F, tiga.F16 if xd.dtype == torch.float16 else tiga.F32, tiga.MAX64))
+            out64, am64 = tiga.tiga_apply_csr(g, xd, wd, tiga.MAX64, out=guard.empty((g.n_dst, F)),
+                                              argmax=guard.empty((g.n_dst, F), torch.int64), ws=ws64)
+            guard.check()
+            assert am64.dtype == torch.int64 and torch.equal(out64, out) and torch.equal(am64, am.long())
+            res["arg64"] = am64
         res[red] = (out, am)
     return g, xd, wd, res
 
@@ -67,6 +74,11 @@ def _check_backward(tiga, rowptr, col, x, w, gy, g, xd, wd, res):
         _, _, arg = oracle.csr_forward(rowptr, col, x, w, oracle.MAX)
         refm = oracle.csr_backward_max(rowptr, col, x, w, gy, arg)
         gx, gw = tiga.tiga_apply_csr_backward(g, xd, wd, gyd, tiga.MAX, argmax=am, grad_x=guard.empty((g.n_src, x.shape[1])),
+                                              grad_w=guard.empty((g.n_edges,)))
+        guard.check()
+        assert rel_err(host(gx), refm["gx"], refm["Ax"]) <= GRAD_TOL
+        assert rel_err(host(gw), refm["gw"], refm["Aw"]) <= GRAD_TOL
+        gx, gw = tiga.tiga_apply_csr_backward(g, xd, wd, gyd, tiga.MAX64, argmax=res["arg64"], grad_x=guard.empty((g.n_src, x.shape[1])),
                                               grad_w=guard.empty((g.n_edges,)))
         guard.check()
         assert rel_err(host(gx), refm["gx"], refm["Ax"]) <= GRAD_TOL
@@ -273,6 +285,89 @@ def test_cfg4_full_size(tiga):
     planned, _ = tiga.tiga_apply_csr_planned(plan, xd)
     torch.cuda.synchronize()
     assert np.array_equal(host(planned), out)
+
+
+def _sample_rows_check(tiga, rowptr_h, cold, wd, x, rows, out, arg64, gy=None, gw=None, reducer="sum"):
+    """Oracle check of a sample of rows of a relation too large for the oracle as a whole: the rows'
+    edges are copied to the host and form a small relation of their own."""
+    deg = (rowptr_h[rows + 1] - rowptr_h[rows]).astype(np.int64)
+    rp = np.concatenate([[0], np.cumsum(deg)]).astype(np.int64)
+    col = np.concatenate([host(cold[int(rowptr_h[r]):int(rowptr_h[r + 1])]) for r in rows]).astype(np.int32)
+    w = None if wd is None else np.concatenate([host(wd[int(rowptr_h[r]):int(rowptr_h[r + 1])]) for r in rows]).astype(np.float32)
+    rows_t = torch.from_numpy(rows).cuda()
+    if reducer == "sum":
+        y, A, _ = oracle.csr_forward(rp, col, x, w, oracle.SUM)
+        assert rel_err(host(out[rows_t]), y, A) <= SUM_TOL
+        if gw is not None:
+            ref = oracle.csr_backward_sum(rp, col, x, w, host(gy[rows_t]))
+            got = np.concatenate([host(gw[int(rowptr_h[r]):int(rowptr_h[r + 1])]) for r in rows])
+            assert rel_err(got, ref["gw"], ref["Aw"]) <= GRAD_TOL
+        return
+    y, _, arg = oracle.csr_forward(rp, col, x, w, oracle.MAX)
+    assert np.array_equal(host(out[rows_t]), y.astype(np.float32))
+    shift = (rowptr_h[rows] - rp[:-1])[:, None]                    # sample position -> position in the full relation
+    assert np.array_equal(host(arg64[rows_t]), np.where(arg >= 0, arg + shift, -1))
+    if gw is not None:
+        ref = oracle.csr_backward_max(rp, col, x, w, host(gy[rows_t]), arg)
+        got = np.concatenate([host(gw[int(rowptr_h[r]):int(rowptr_h[r + 1])]) for r in rows])
+        assert rel_err(got, ref["gw"], ref["Aw"]) <= GRAD_TOL
+
+
+@pytest.mark.parametrize("F", [4, 16])
+def test_relation_with_more_than_2_31_edges(tiga, F):
+    """2^31 edges and more: 64-bit row offsets, 64-bit edge positions in argmax (TIGA_MAX64; the
+    32-bit reducer refuses), narrow (F = 4) and wide (F = 16) feature rows.  Sampled rows — the first
+    and last, the rows around edge 2^31, the longest — are checked completely against the oracle."""
+    n_dst, n_src = (1 << 20) + (1 << 15), 4096
+    rs = gen.rng(41, 900)
+    deg = rs.integers(0, 4099, size=n_dst).astype(np.int64)
+    deg[rs.random(n_dst) < 0.02] = 0
+    deg[[5, 77_777, n_dst - 1]] = [20_000, 150_000, 9_000]
+    rowptr = np.concatenate([[0], np.cumsum(deg)]).astype(np.int64)
+    E = int(rowptr[-1])
+    assert E > (1 << 31) + (1 << 20)
+    gt = torch.Generator(device="cuda").manual_seed(4242)
+    cold = torch.randint(0, n_src, (E,), dtype=torch.int32, device="cuda", generator=gt)
+    wd = None
+    if F == 16:
+        wd = (torch.randint(0, (1 << 24) - 1, (E,), dtype=torch.int32, device="cuda", generator=gt) + 1).float() * 2.0 ** -24
+    x = gen.normal_features(n_src, F, 9)
+    gy_h = gen.normal_features(n_dst, F, 10)
+    xd, gy = dev(x, torch), dev(gy_h, torch)
+    g = tiga.CsrRelation(dev(rowptr, torch), cold, n_src)
+    cross = int(np.searchsorted(rowptr, 1 << 31, side="right") - 1)       # the row that holds edge 2^31
+    rows = np.unique(np.concatenate([[0, 1, 5, 77_777, n_dst - 2, n_dst - 1, cross - 1, cross, cross + 1],
+                                     rs.integers(0, n_dst, size=120), np.flatnonzero(deg == 0)[:3]])).astype(np.int64)
+
+    with pytest.raises(tiga.TigaError) as e:
+        tiga.tiga_apply_csr(g, xd, wd, tiga.MAX)
+    assert e.value.status == 2
+    y, _ = tiga.tiga_apply_csr(g, xd, wd, tiga.SUM)
+    gx, gw = tiga.tiga_apply_csr_backward(g, xd, wd, gy, tiga.SUM)
+    _sample_rows_check(tiga, rowptr, cold, wd, x, rows, y, None, gy, gw, "sum")
+    # a source's gradient row gathers over all of its edges, wherever they are
+    rp_d = g.rowptr
+    for j in (0, 1234, n_src - 1):
+        e_j = torch.nonzero(cold == j).flatten()
+        r_j = torch.searchsorted(rp_d, e_j, right=True) - 1
+        wj = torch.ones_like(e_j, dtype=torch.float64) if wd is None else wd[e_j].double()
+        ref = (wj[:, None] * gy[r_j].double()).sum(0)
+        mag = (wj[:, None] * gy[r_j].double().abs()).sum(0)
+        assert float(((gx[j].double() - ref).abs() / mag).max()) <= GRAD_TOL
+    del gw, gx, y
+    ym, am = tiga.tiga_apply_csr(g, xd, wd, tiga.MAX64)
+    assert am.dtype == torch.int64 and int(am.max()) >= (1 << 31)
+    gx, gw = tiga.tiga_apply_csr_backward(g, xd, wd, gy, tiga.MAX64, argmax=am)
+    _sample_rows_check(tiga, rowptr, cold, wd, x, rows, ym, am, gy, gw, "max")
+    # all of the max cotangents, routed through the selected edges (float64 on the device)
+    valid = am >= 0
+    e_sel = am[valid]
+    f_idx = torch.arange(F, device="cuda").expand(n_dst, F)[valid]
+    wsel = torch.ones_like(e_sel, dtype=torch.float64) if wd is None else wd[e_sel].double()
+    contrib = wsel * gy[valid].double()
+    ref = torch.zeros((n_src, F), dtype=torch.float64, device="cuda").index_put_((cold[e_sel].long(), f_idx), contrib, accumulate=True)
+    mag = torch.zeros((n_src, F), dtype=torch.float64, device="cuda").index_put_((cold[e_sel].long(), f_idx), contrib.abs(), accumulate=True)
+    assert float(((gx.double() - ref).abs() / mag.clamp_min(1e-300)).max()) <= GRAD_TOL
 
 
 def test_row_gather_probe_runs_and_checks_its_arguments(tiga):
