@@ -159,17 +159,12 @@ static __device__ __forceinline__ void emit_row(const KnnParams& P, const int i,
 }
 
 // ------------------------------------------------------------------------------ cells kernel
-__global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_constant__ KnnParams P) {
+// queries [qs0, qe0) of one cell (the whole cell, or a slice of a dense one)
+__device__ __forceinline__ void knn_cell_slice(const KnnParams& P, const int cellid, const int qs0, const int qe0, unsigned char* s_raw) {
     const RadiusParams& p = P.rp;
     constexpr unsigned FULL = 0xffffffffu;
-    extern __shared__ __align__(16) unsigned char s_raw[];
-
     const int lane = threadIdx.x & 31;
     const int wib = threadIdx.x >> 5;
-    const int cellid = blockIdx.x * TRAV_WARPS + wib;
-    if (cellid >= p.ncells) return;
-    const int qs0 = p.cell_start[cellid], qe0 = p.cell_start[cellid + 1];
-    if (qs0 == qe0) return;
 
     unsigned char* base = s_raw + (size_t)wib * KNN_PER_WARP;
     float4* stage = reinterpret_cast<float4*>(base);                                      // x, y, z, point id
@@ -343,6 +338,29 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_co
             } else {
                 emit_row(P, i, select_sorted(list + q * KNN_QSTRIDE, n, lane), k, lane);
             }
+        }
+    }
+}
+
+// CTAs [0, cell_blocks): one warp per cell; of a cell with more than QDENSE points it takes the first
+// QSLICE queries.  The CTAs behind them walk the queue of the remaining slices.
+__global__ void __launch_bounds__(TRAV_THREADS) knn_cells_kernel(const __grid_constant__ KnnParams P) {
+    const RadiusParams& p = P.rp;
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    if ((int)blockIdx.x < p.cell_blocks) {
+        const int w = blockIdx.x * TRAV_WARPS + (threadIdx.x >> 5);
+        if (w >= p.ncells) return;
+        const int qs0 = p.cell_start[w], qe0 = p.cell_start[w + 1];
+        if (qs0 == qe0) return;
+        knn_cell_slice(P, w, qs0, qe0 - qs0 > QDENSE ? qs0 + QSLICE : qe0, s_raw);
+    } else {
+        const int n = *p.q_count;
+        const int w = (blockIdx.x - p.cell_blocks) * TRAV_WARPS + (threadIdx.x >> 5);
+        for (int it = w; it < n; it += (gridDim.x - p.cell_blocks) * TRAV_WARPS) {
+            const int2 item = p.q_items[it];
+            const int qs0 = p.cell_start[item.x] + item.y, end = p.cell_start[item.x + 1];
+            knn_cell_slice(P, item.x, qs0, slice_end(qs0, end), s_raw);
+            __syncwarp();
         }
     }
 }
@@ -532,7 +550,8 @@ extern "C" tiga_status tiga_apply_knn(const float* pos, const float* feat, int64
     const unsigned blocks = (unsigned)((P.rp.ncells + TRAV_WARPS - 1) / TRAV_WARPS);
     constexpr int smem = KNN_PER_WARP * TRAV_WARPS;
     TIGA_CUDA_TRY(cudaFuncSetAttribute(knn_cells_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    knn_cells_kernel<<<counted(blocks), TRAV_THREADS, smem, s>>>(P);
+    P.rp.cell_blocks = (int)blocks;
+    knn_cells_kernel<<<counted(blocks + queue_blocks(P.rp.n)), TRAV_THREADS, smem, s>>>(P);
     knn_rings_kernel<<<counted(KNN_RING_BLOCKS), TRAV_THREADS, 0, s>>>(P);
     return launch_status();
 }

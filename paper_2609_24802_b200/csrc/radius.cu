@@ -148,13 +148,20 @@ __global__ void bin_scatter_kernel(const RadiusParams p, int32_t* fill) {
 // One thread per scattered slot: the rank of its point among the point ids of its cell gives
 // the stable order (cell, then index) and the place of the sorted copy of the position.
 // Neighbouring threads belong to the same cell and read the same few slots.
-__global__ void bin_sort_kernel(const RadiusParams p) {
+static __device__ void sort_dense_cells(const RadiusParams& p, int first, int stride);
+
+// CTAs [0, point_blocks) rank the points of ordinary cells; the CTAs behind them order the queued dense cells.
+__global__ void __launch_bounds__(256) bin_sort_kernel(const RadiusParams p, const int point_blocks) {
+    if ((int)blockIdx.x >= point_blocks) {
+        sort_dense_cells(p, blockIdx.x - point_blocks, gridDim.x - point_blocks);
+        return;
+    }
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= p.n) return;
     const int id = p.order_tmp[t];
     const int c = p.cell[id];
     const int s = p.cell_start[c], e = p.cell_start[c + 1];
-    if (e - s > SORT_DENSE) return;        // bin_sort_dense_kernel orders this cell
+    if (e - s > SORT_DENSE) return;        // sort_dense_cells orders this cell
     int rank = 0;
     for (int u = s; u < e; ++u) rank += (p.order_tmp[u] < id) ? 1 : 0;
     p.order[s + rank] = id;
@@ -167,8 +174,7 @@ __global__ void bin_sort_kernel(const RadiusParams p) {
 // the same way (first step of a merge mirrors, the others are half-cleaners), so slots behind the
 // segment act as +infinity without being stored; up to SORT_SMEM ids are sorted in shared memory,
 // longer segments in place in global memory.
-constexpr int SORT_THREADS = 512;
-constexpr int SORT_SMEM = 8192;
+constexpr int SORT_SMEM = 2048;       // 8 KB: the ranking CTAs of the same launch keep their occupancy
 static __device__ void sort_ids_ascending(int32_t* a, int m) {
     int P = 1;
     while (P < m) P <<= 1;
@@ -187,10 +193,10 @@ static __device__ void sort_ids_ascending(int32_t* a, int m) {
     }
 }
 
-__global__ void __launch_bounds__(SORT_THREADS) bin_sort_dense_kernel(const RadiusParams p) {
+static __device__ void sort_dense_cells(const RadiusParams& p, const int first, const int stride) {
     __shared__ int32_t s_ids[SORT_SMEM];
     const int items = *p.b_count;
-    for (int it = blockIdx.x; it < items; it += gridDim.x) {
+    for (int it = first; it < items; it += stride) {
         const int c = p.b_items[it];
         const int s = p.cell_start[c], m = p.cell_start[c + 1] - s;
         int32_t* a = p.order_tmp + s;
@@ -642,21 +648,21 @@ __device__ __forceinline__ void traverse_slice(const RadiusParams& p, const int 
     }
 }
 
-// Pass 1 (q_mode 0): warp w of the grid takes cell w, its first QSLICE queries, and queues the slices it
-// leaves.  Pass 2 (q_mode 1): the warps of a small grid walk the queue.
+// CTAs [0, cell_blocks): warp w takes cell w (of a cell with more than QDENSE points its first QSLICE
+// queries).  The CTAs behind them walk the queue of the remaining slices.
 template <int MODE, int LF, bool DIST, bool MI, int VEC = 1>
 __global__ void __launch_bounds__(TRAV_THREADS, (MODE == 0 ? 7 : 0)) radius_traverse_kernel(const __grid_constant__ RadiusParams p) {
     extern __shared__ __align__(16) unsigned char s_raw[];
-    const int lane = threadIdx.x & 31;
-    const int w = blockIdx.x * TRAV_WARPS + (threadIdx.x >> 5);
-    if (!p.q_mode) {
+    if ((int)blockIdx.x < p.cell_blocks) {
+        const int w = blockIdx.x * TRAV_WARPS + (threadIdx.x >> 5);
         if (w >= p.ncells) return;
         const int qs0 = p.cell_start[w], qe0 = p.cell_start[w + 1];
         if (qs0 == qe0) return;
         traverse_slice<MODE, LF, DIST, MI, VEC>(p, w, qs0, qe0 - qs0 > QDENSE ? qs0 + QSLICE : qe0, s_raw);
     } else {
         const int n = *p.q_count;
-        for (int it = w; it < n; it += gridDim.x * TRAV_WARPS) {
+        const int w = (blockIdx.x - p.cell_blocks) * TRAV_WARPS + (threadIdx.x >> 5);
+        for (int it = w; it < n; it += (gridDim.x - p.cell_blocks) * TRAV_WARPS) {
             const int2 item = p.q_items[it];
             const int qs0 = p.cell_start[item.x] + item.y, end = p.cell_start[item.x + 1];
             traverse_slice<MODE, LF, DIST, MI, VEC>(p, item.x, qs0, slice_end(qs0, end), s_raw);
@@ -748,8 +754,8 @@ tiga_status run_binning(RadiusParams& p, int32_t* fill, int nblocks, cudaStream_
     scan_blocksums_kernel<<<counted(1), 1024, 0, s>>>(p, nblocks);
     scan_apply_kernel<<<counted(nblocks), RAD_THREADS, 0, s>>>(p);
     bin_scatter_kernel<<<counted(pb), 256, 0, s>>>(p, fill);
-    bin_sort_kernel<<<counted(pb), 256, 0, s>>>(p);
-    bin_sort_dense_kernel<<<counted(148u), SORT_THREADS, 0, s>>>(p);
+    const long long dense_cells = (long long)p.n / SORT_DENSE + 1;          // at most this many cells can be dense
+    bin_sort_kernel<<<counted(pb + (unsigned)(dense_cells < 148 ? dense_cells : 148)), 256, 0, s>>>(p, (int)pb);
     return launch_status();
 }
 
@@ -767,11 +773,11 @@ static tiga_status launch_traverse_t(const RadiusParams& p, cudaStream_t s) {
         // scalar feature accesses (only the forward supports widths that are not multiples of 4)
         auto sk = radius_traverse_kernel<MODE == 0 ? 0 : MODE, LF, DIST, MI, MODE != 0 ? 1 : 0>;
         if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(sk, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        return two_passes(p, s, [&](const RadiusParams& q, unsigned grid) { sk<<<counted(grid), TRAV_THREADS, smem, s>>>(q); });
+        return cells_then_queue(p, s, [&](const RadiusParams& q, unsigned grid) { sk<<<counted(grid), TRAV_THREADS, smem, s>>>(q); });
     }
     auto kern = p.F == 4 * LF ? radius_traverse_kernel<MODE, LF, DIST, MI, 2> : radius_traverse_kernel<MODE, LF, DIST, MI, 1>;
     if (smem > 48 * 1024) TIGA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    return two_passes(p, s, [&](const RadiusParams& q, unsigned grid) { kern<<<counted(grid), TRAV_THREADS, smem, s>>>(q); });
+    return cells_then_queue(p, s, [&](const RadiusParams& q, unsigned grid) { kern<<<counted(grid), TRAV_THREADS, smem, s>>>(q); });
 }
 
 template <int MODE, bool DIST, bool MI>

@@ -147,8 +147,21 @@ __global__ void __launch_bounds__(TRAV_THREADS, mlp_ctas_per_sm<HID, BWD>()) rad
 #pragma unroll
     for (int i = 0; i < (BWD ? HID / 2 : 1); ++i) gW1acc[i] = 0.f;
 
-    for (int cellid = blockIdx.x * TRAV_WARPS + wib; cellid < p.ncells; cellid += gridDim.x * TRAV_WARPS) {
-        const int qs0 = p.cell_start[cellid], qe0 = p.cell_start[cellid + 1];
+    // work items: every cell (of a cell with more than QDENSE points only its first QSLICE queries), then
+    // the queued slices of the dense cells, so that a clustered input spreads over all warps
+    const int nitems = p.ncells + *p.q_count;
+    for (int item = blockIdx.x * TRAV_WARPS + wib; item < nitems; item += gridDim.x * TRAV_WARPS) {
+        int cellid, qs0, qe0;
+        if (item < p.ncells) {
+            cellid = item;
+            qs0 = p.cell_start[cellid]; qe0 = p.cell_start[cellid + 1];
+            if (qe0 - qs0 > QDENSE) qe0 = qs0 + QSLICE;
+        } else {
+            const int2 it = p.q_items[item - p.ncells];
+            cellid = it.x;
+            qs0 = p.cell_start[cellid] + it.y;
+            qe0 = slice_end(qs0, p.cell_start[cellid + 1]);
+        }
         if (qs0 == qe0) continue;
         const int c[3] = {cellid % p.nc[0], (cellid / p.nc[0]) % p.nc[1], cellid / (p.nc[0] * p.nc[1])};
         const float org[3] = {(float)c[0] * p.hcell[0], (float)c[1] * p.hcell[1], (float)c[2] * p.hcell[2]};

@@ -53,7 +53,8 @@ struct RadiusParams {
     // slices of cells with more than QDENSE points, queued by the pass over the cells for a second pass
     int2* q_items;            // (cell, first query of the slice)
     int* q_count;
-    int q_mode;               // 0: one warp per cell (queues what it leaves), 1: warps walk the queue
+    int q_mode;               // two-launch form: 0 = one warp per cell, 1 = warps walk the queue
+    int cell_blocks;          // one-launch form: CTAs [0, cell_blocks) take cells, the CTAs behind them walk the queue
     int32_t* b_items;         // cells with more than SORT_DENSE points (queued by the same scan), and how many
     int* b_count;
     // optional user copies of the plan
@@ -105,14 +106,31 @@ static __device__ __forceinline__ void queue_extra_slices(const RadiusParams& p,
     if (count > SORT_DENSE) p.b_items[atomicAdd(p.b_count, 1)] = cell;
 }
 
-// Runs a traversal kernel twice: over the cells, then over the queue of slices the first pass left.
+// CTAs that walk the queue: no more than the queue can have items for (at most n / QSLICE slices exist)
+static inline unsigned queue_blocks(long long n) {
+    const long long need = n / ((long long)QSLICE * TRAV_WARPS) + 1;
+    return (unsigned)(need < QUEUE_BLOCKS ? need : QUEUE_BLOCKS);
+}
+
+// One launch over the cells and, in the CTAs appended behind them, over the queue of slices (which the
+// binning filled before the launch).
+template <typename Launch>
+static inline tiga_status cells_then_queue(const RadiusParams& p, cudaStream_t s, Launch launch) {
+    RadiusParams q = p;
+    q.cell_blocks = (p.ncells + TRAV_WARPS - 1) / TRAV_WARPS;
+    launch(q, (unsigned)q.cell_blocks + queue_blocks(p.n));
+    return launch_status();
+}
+
+// Runs a traversal kernel twice: over the cells, then over the queue of slices (for kernels whose
+// register allocation suffers from carrying both loops).
 template <typename Launch>
 static inline tiga_status two_passes(const RadiusParams& p, cudaStream_t s, Launch launch) {
     RadiusParams q = p;
     q.q_mode = 0;
     launch(q, (unsigned)((p.ncells + TRAV_WARPS - 1) / TRAV_WARPS));
     q.q_mode = 1;
-    launch(q, (unsigned)QUEUE_BLOCKS);
+    launch(q, queue_blocks(p.n));
     return launch_status();
 }
 

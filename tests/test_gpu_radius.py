@@ -69,11 +69,12 @@ def test_binning_is_bit_exact(tiga):
     p[:15_000] = p[:15_000] * np.float32(0.02) + np.float32(0.5)
     _check_bin(tiga, p, np.float32(0.05), ones, [1, 1, 1])
     # cell occupancies on both sides of the limits of the dense-cell ordering (256 by rank counting,
-    # above that a sorting network: in shared memory up to 8192 ids, in place beyond), ids interleaved
+    # above that a sorting network: in shared memory up to 2048 ids, in place beyond), ids interleaved
     rng = np.random.default_rng(12)
-    parts = [gen.uniform_points(m, 13 + k) * np.float32(0.2) + np.float32([0.25 * k, 0.0, 0.0])
-             for k, m in enumerate([256, 257, 8192, 8193])]
-    p = np.concatenate(parts)[rng.permutation(256 + 257 + 8192 + 8193)]
+    sizes = [256, 257, 2048, 2049, 8193]
+    parts = [gen.uniform_points(m, 13 + k) * np.float32(0.2) + np.float32([0.25 * (k % 4), 0.25 * (k // 4), 0.0])
+             for k, m in enumerate(sizes)]
+    p = np.concatenate(parts)[rng.permutation(sum(sizes))]
     _check_bin(tiga, p, np.float32(0.25), ones, [0, 0, 0])
     # anisotropic box
     box = np.array([1.0, 2.5, 0.3], np.float32)
