@@ -821,22 +821,58 @@ __global__ void csr_backward_max_kernel(const CsrParams p) {
 // Degree histogram and validation
 // --------------------------------------------------------------------------------------------
 template <typename IT>
-__global__ void degree_hist_kernel(const IT* __restrict__ rowptr, long long n, int nbins,
-                                   unsigned long long* hist, unsigned long long* maxdeg) {
+__global__ void __launch_bounds__(1024, 1) degree_hist_kernel(const IT* __restrict__ rowptr, long long n, int nbins,
+                                                              unsigned long long* hist, unsigned long long* maxdeg) {
     extern __shared__ unsigned int s_hist[];
+    constexpr unsigned FULL = 0xffffffffu;
     for (int k = threadIdx.x; k < nbins; k += blockDim.x) s_hist[k] = 0;
     __syncthreads();
+    // Most rows of a skewed relation have a handful of edges: degrees below LOW are counted in registers
+    // (no shared-memory atomics on a few hot bins) and folded in once per warp at the end.  The eight
+    // counters are bytes of one 64-bit word (one shift and one add per row), emptied into full-width
+    // counters before a byte can overflow.
+    constexpr int LOW = 8, UNR = 8, FLUSH_STEPS = 248 / UNR;
+    const bool low_ok = nbins > LOW + 1;
+    const int lane = threadIdx.x & 31;
+    unsigned long long packed = 0ull;
+    int steps = 0;
+    auto unpack = [&]() {
+#pragma unroll
+        for (int k = 0; k < LOW; ++k) {
+            const unsigned tot = __reduce_add_sync(FULL, (unsigned)((packed >> (8 * k)) & 255ull));
+            if (lane == 0 && tot) atomicAdd(&s_hist[k], tot);
+        }
+        packed = 0ull;
+    };
     long long mx = 0;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
-        const long long d = (long long)rowptr[i + 1] - (long long)rowptr[i];
-        mx = d > mx ? d : mx;
-        atomicAdd(&s_hist[d < nbins - 1 ? (int)d : nbins - 1], 1u);
+    // A warp reads 32 consecutive row offsets with one coalesced load and forms 31 degrees from them (a lane's
+    // row ends where its neighbour's begins; the last lane only supplies that end), so consecutive chunks
+    // overlap by one offset.  All loads of a step are issued before any is used.
+    const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+    for (long long c0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; c0 * 31 < n; c0 += warps * UNR) {
+        if (++steps == FLUSH_STEPS) { unpack(); steps = 0; }
+        long long v[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const long long i = (c0 + u * warps) * 31 + lane;
+            v[u] = i <= n ? (long long)rowptr[i] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const long long i = (c0 + u * warps) * 31 + lane;
+            const long long d = __shfl_down_sync(FULL, v[u], 1) - v[u];
+            if (lane == 31 || i >= n || d < 0) continue;
+            mx = d > mx ? d : mx;
+            if (low_ok && d < LOW) packed += 1ull << (8 * (int)d);
+            else atomicAdd(&s_hist[d < nbins - 1 ? (int)d : nbins - 1], 1u);
+        }
     }
+    if (low_ok) unpack();
     for (int o = 16; o > 0; o >>= 1) {
-        const long long other = __shfl_xor_sync(0xffffffffu, mx, o);
+        const long long other = __shfl_xor_sync(FULL, mx, o);
         mx = other > mx ? other : mx;
     }
-    if ((threadIdx.x & 31) == 0 && mx > 0) atomicMax(maxdeg, (unsigned long long)mx);
+    if (lane == 0 && mx > 0) atomicMax(maxdeg, (unsigned long long)mx);
     __syncthreads();
     for (int k = threadIdx.x; k < nbins; k += blockDim.x)
         if (s_hist[k]) atomicAdd(hist + k, (unsigned long long)s_hist[k]);
@@ -1224,14 +1260,16 @@ extern "C" tiga_status tiga_csr_degree_histogram(const tiga_csr* g, int64_t* his
     TIGA_CUDA_TRY(cudaMemsetAsync(hist, 0, (size_t)nbins * sizeof(int64_t), s));
     TIGA_CUDA_TRY(cudaMemsetAsync(max_degree, 0, sizeof(int64_t), s));
     if (g->n_dst == 0) return TIGA_OK;
-    long long blocks = (g->n_dst + 1023) / 1024;
-    if (blocks > 148 * 4) blocks = 148 * 4;
+    // one CTA of 1024 threads per SM (eight row-offset loads in flight per thread): every CTA ends with one global atomic per non-empty bin, so few
+    // large CTAs keep that flush (CTAs x bins atomics on nbins addresses) short
+    long long blocks = (g->n_dst + 4095) / 4096;
+    if (blocks > 148) blocks = 148;
     const size_t sm = (size_t)nbins * sizeof(unsigned int);
     if (g->rowptr_type == TIGA_I32)
-        degree_hist_kernel<int32_t><<<counted((unsigned)blocks), 256, sm, s>>>(static_cast<const int32_t*>(g->rowptr), g->n_dst, (int)nbins,
+        degree_hist_kernel<int32_t><<<counted((unsigned)blocks), 1024, sm, s>>>(static_cast<const int32_t*>(g->rowptr), g->n_dst, (int)nbins,
                                                                    reinterpret_cast<unsigned long long*>(hist), reinterpret_cast<unsigned long long*>(max_degree));
     else
-        degree_hist_kernel<int64_t><<<counted((unsigned)blocks), 256, sm, s>>>(static_cast<const int64_t*>(g->rowptr), g->n_dst, (int)nbins,
+        degree_hist_kernel<int64_t><<<counted((unsigned)blocks), 1024, sm, s>>>(static_cast<const int64_t*>(g->rowptr), g->n_dst, (int)nbins,
                                                                    reinterpret_cast<unsigned long long*>(hist), reinterpret_cast<unsigned long long*>(max_degree));
     return launch_status();
 }
