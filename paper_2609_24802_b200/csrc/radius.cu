@@ -249,8 +249,8 @@ __global__ void validate_points_kernel(const float* __restrict__ pos, long long 
 //             kernel in radius_lj.cu, which visits every unordered pair once.)
 // Lists hold QCAP entries per query and the stage STAGE_CAP candidates; when either fills up
 // the warp drains / processes and goes on, so any density works.  A cell with more than QDENSE
-// points is cut into slices of QSLICE queries: its warp takes the first, the others are queued and a second
-// launch of the same kernel spreads over many warps (an empty queue costs one tiny launch).
+// points is cut into slices of QSLICE queries: its warp takes the first, the others wait in a queue (filled
+// by the binning) that the CTAs appended behind the cells' CTAs walk, so a dense cell spreads over many warps.
 
 template <int MODE> struct TravSmem {
     // queries per batch: the forward runs fastest with short batches and seven CTAs per SM, the

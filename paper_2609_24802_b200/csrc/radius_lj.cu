@@ -39,7 +39,7 @@ constexpr int LJ_MISC_BYTES = LJQ * 16 + 3 * LJQ * 4 + LJQ * 4 + 32;        // q
 constexpr int LJ_PER_WARP = (LJ_STAGE_BYTES + LJ_LIST_BYTES + LJ_MISC_BYTES + 15) / 16 * 16;
 
 // One warp, one cell; of a cell with more than QDENSE points only QSLICE as queries (from `first`): what such a cell
-// leaves is queued for the second pass, as in radius_traverse_kernel.
+// leaves waits in the binning's queue of slices, which a second launch walks (QUEUE = true).
 template <bool MI, bool COUNT, bool QUEUE>
 __device__ __forceinline__ void lj_slice(const RadiusParams& p, const int cellid, const int first, unsigned char* s_raw) {
     constexpr unsigned FULL = 0xffffffffu;

@@ -12,8 +12,8 @@ constexpr int STAGE_PAD = 32;           // sentinels behind the staged candidate
 constexpr int QB = 8;                   // queries per batch (kernels that run faster with four define their own width)
 constexpr float FAR_AWAY = 1.0e18f;
 constexpr int QDENSE = 64;              // a cell with more points than this is cut into slices of QSLICE queries:
-constexpr int QSLICE = 16;              // its warp takes the first slice and queues the others for the second pass
-constexpr int QUEUE_BLOCKS = 148 * 8;   // grid of the pass over the queued slices
+constexpr int QSLICE = 16;              // its warp takes the first slice, the others wait in a queue that other warps walk
+constexpr int QUEUE_BLOCKS = 148 * 8;   // most CTAs that walk the queued slices
 constexpr int SORT_DENSE = 256;         // a cell with more points than this is ordered by a sorting network, not by rank counting
 
 struct RadiusParams {
@@ -50,7 +50,7 @@ struct RadiusParams {
     int32_t* order;
     float4* spos;             // positions in cell order, .w = original point id (bit pattern)
     int32_t* blocksum;
-    // slices of cells with more than QDENSE points, queued by the pass over the cells for a second pass
+    // slices of cells with more than QDENSE points, queued by the binning scan
     int2* q_items;            // (cell, first query of the slice)
     int* q_count;
     int q_mode;               // two-launch form: 0 = one warp per cell, 1 = warps walk the queue

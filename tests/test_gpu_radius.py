@@ -373,8 +373,8 @@ def test_point_validation(tiga):
 
 # ------------------------------------------------------------------------------ uneven density
 def test_clustered_points_are_spread_over_many_warps(tiga):
-    """Most points in a dozen tight blobs: some cells hold hundreds of points (a warp takes 64 queries
-    of a cell and queues the rest for a second pass).  Parity as usual, and the call must stay within
+    """Most points in a dozen tight blobs: some cells hold hundreds of points (the cell's warp takes
+    16 queries, the other slices of 16 wait in a queue that many warps walk).  Parity as usual, and the call must stay within
     5x of a uniform cloud with the same number of accepted pairs."""
     n, F = 200_000, 8
     pos = gen.clustered_points(n, 21)
