@@ -606,45 +606,49 @@ __device__ __forceinline__ void traverse_slice(const RadiusParams& p, const int 
     if (mi0 && (lane == 0 || lane == 3)) bb = lane == 0 ? -FAR_AWAY : FAR_AWAY;   // a dimension folded by the explicit
     if (mi1 && (lane == 1 || lane == 4)) bb = lane == 1 ? -FAR_AWAY : FAR_AWAY;   // minimum image is not pruned
     if (mi2 && (lane == 2 || lane == 5)) bb = lane == 2 ? -FAR_AWAY : FAR_AWAY;
+    // The stage fills with candidates that survive the pruning and is processed when the next step's
+    // candidates might not fit, so the chunks are as full as the pruning allows (one chunk for all but dense cells).
     bool first_chunk = true;
-    for (int lo = 0; lo < total || first_chunk; lo += STAGE_CAP) {
-        const int ns = total - lo < STAGE_CAP ? total - lo : STAGE_CAP;
-        int nst = 0;                                                         // candidates kept (warp uniform)
-        constexpr int SU = 4;                                                // staging groups in flight
-        for (int k0 = 0; k0 < ns; k0 += 32 * SU) {
-            float4 c4[SU];
-#pragma unroll
-            for (int u = 0; u < SU; ++u) {                                   // all loads of the step first
-                const int k = k0 + 32 * u + lane;
-                const int v = lo + k;
-                int r = 0;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    const int probe = __shfl_sync(FULL, r_incl, r + o - 1);
-                    if (probe <= v) r += o;
-                }
-                r = r > 31 ? 31 : r;
-                const int src = __shfl_sync(FULL, r_cs, r) + (v - (__shfl_sync(FULL, r_incl, r) - __shfl_sync(FULL, r_len, r)));
-                c4[u] = k < ns ? __ldg(p.spos + src) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            const float lx = __shfl_sync(FULL, bb, 0), ly = __shfl_sync(FULL, bb, 1), lz = __shfl_sync(FULL, bb, 2);
-            const float hx = __shfl_sync(FULL, bb, 3), hy = __shfl_sync(FULL, bb, 4), hz = __shfl_sync(FULL, bb, 5);
-#pragma unroll
-            for (int u = 0; u < SU; ++u) {
-                if (k0 + 32 * u >= ns) break;
-                const float4 val = to_frame(c4[u]);
-                const float ex = fmaxf(fmaxf(lx - val.x, val.x - hx), 0.f);
-                const float ey = fmaxf(fmaxf(ly - val.y, val.y - hy), 0.f);
-                const float ez = fmaxf(fmaxf(lz - val.z, val.z - hz), 0.f);
-                const bool keep = k0 + 32 * u + lane < ns && fmaf(ez, ez, fmaf(ey, ey, ex * ex)) <= p.r2_hi * 1.0001f;
-                const unsigned m = __ballot_sync(FULL, keep);
-                if (keep) stage[nst + __popc(m & lt_mask)] = val;
-                nst += __popc(m);
-            }
+    int nst = 0;                                                             // candidates staged (warp uniform)
+    constexpr int SU = 4;                                                    // staging groups in flight
+    for (int k0 = 0;; k0 += 32 * SU) {
+        const bool done = k0 >= total;
+        const int step = done ? 0 : (total - k0 < 32 * SU ? total - k0 : 32 * SU);
+        if ((done && (nst > 0 || first_chunk)) || nst + step > STAGE_CAP) {     // the one place a chunk is processed
+            __syncwarp();
+            process_chunk(nst, first_chunk);
+            first_chunk = false;
+            nst = 0;
         }
-        __syncwarp();
-        process_chunk(nst, first_chunk);
-        first_chunk = false;
+        if (done) break;
+        float4 c4[SU];
+#pragma unroll
+        for (int u = 0; u < SU; ++u) {                                       // all loads of the step first
+            const int v = k0 + 32 * u + lane;
+            int r = 0;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const int probe = __shfl_sync(FULL, r_incl, r + o - 1);
+                if (probe <= v) r += o;
+            }
+            r = r > 31 ? 31 : r;
+            const int src = __shfl_sync(FULL, r_cs, r) + (v - (__shfl_sync(FULL, r_incl, r) - __shfl_sync(FULL, r_len, r)));
+            c4[u] = v < total ? __ldg(p.spos + src) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        const float lx = __shfl_sync(FULL, bb, 0), ly = __shfl_sync(FULL, bb, 1), lz = __shfl_sync(FULL, bb, 2);
+        const float hx = __shfl_sync(FULL, bb, 3), hy = __shfl_sync(FULL, bb, 4), hz = __shfl_sync(FULL, bb, 5);
+#pragma unroll
+        for (int u = 0; u < SU; ++u) {
+            if (32 * u >= step) break;
+            const float4 val = to_frame(c4[u]);
+            const float ex = fmaxf(fmaxf(lx - val.x, val.x - hx), 0.f);
+            const float ey = fmaxf(fmaxf(ly - val.y, val.y - hy), 0.f);
+            const float ez = fmaxf(fmaxf(lz - val.z, val.z - hz), 0.f);
+            const bool keep = k0 + 32 * u + lane < total && fmaf(ez, ez, fmaf(ey, ey, ex * ex)) <= p.r2_hi * 1.0001f;
+            const unsigned m = __ballot_sync(FULL, keep);
+            if (keep) stage[nst + __popc(m & lt_mask)] = val;
+            nst += __popc(m);
+        }
     }
 }
 
