@@ -135,8 +135,8 @@ tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dtype x_dtype,
  * Same arguments and results as tiga_apply_csr, minus ws / ws_bytes.  Differences:
  *   - Capacity: the call is refused with TIGA_ERR_TOO_LARGE, before anything is launched, when
  *     tiga_csr_workspace_bytes(g, F, x_dtype, reducer, 0) exceeds TIGA_BUILTIN_WS_BYTES
- *     (roughly (n_dst + n_edges) / 2048 * (4 F + 20) bytes plus about 1.5 KiB of padding, twice
- *     the F term for TIGA_MAX, three times for TIGA_MAX64; e.g. 16.8M edges at F = 64 need 2.3 MiB).
+ *     (roughly (n_dst + n_edges) / 1792 * (4 F + 20) bytes plus about 1.5 KiB of padding, twice
+ *     the F term for TIGA_MAX, three times for TIGA_MAX64; e.g. 16.8M edges at F = 64 need 2.7 MiB).
  *   - It never calls cudaMalloc, cudaFree or any other allocating routine.
  *   - The first call on each device looks up the array's device address (a host-side lookup,
  *     done with that device current and cached per device).  Make that first call before any

@@ -102,9 +102,10 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
     constexpr int LV = G * VPL * VW;             // floats of one partial state
     constexpr int U = (VPL == 1) ? 4 : (VPL == 2 ? 2 : 1);   // gathers in flight per lane
 
-    __shared__ int s_ptr[CSR_TILE + 2];
-    __shared__ __align__(16) int s_col[CSR_TILE + CSR_PAD];
-    __shared__ __align__(16) float s_w[CSR_TILE + CSR_PAD];
+    constexpr int TILE = RED == 0 ? CSR_TILE : CSR_TILE_MAX;
+    __shared__ int s_ptr[TILE + 2];
+    __shared__ __align__(16) int s_col[TILE + CSR_PAD];
+    __shared__ __align__(16) float s_w[TILE + CSR_PAD];
     __shared__ long long s_coord[2];
     __shared__ int s_tag[2 * NW];                // local row of head (even) / tail (odd) partial, -1 = none
     __shared__ unsigned char s_first[NW];        // tail partial starts its chain
@@ -113,7 +114,7 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
     using AT = ArgT<RED>;
     AT* s_pa = reinterpret_cast<AT*>(s_pv + 2 * NW * LV);       // [2*NW][LV] (max only; 2*NW*LV floats keep it 8-byte aligned)
 
-    const Tile t = stage_tile<IT>(p, s_ptr, s_col, s_w, s_coord);
+    const Tile t = stage_tile<IT, false, TILE>(p, s_ptr, s_col, s_w, s_coord);
     const int wk = threadIdx.x / G;
     const int ln = threadIdx.x % G;
     const uint4* __restrict__ xlane = static_cast<const uint4*>(p.x) + ln;
@@ -690,13 +691,14 @@ template <int G, int VPL, typename IT, typename XT>
 __global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const CsrParams p) {
     constexpr int NW = CSR_THREADS / G;
     constexpr int U = (VPL == 1) ? 4 : (VPL == 2 ? 2 : 1);
-    __shared__ int s_ptr[CSR_TILE + 2];
-    __shared__ int s_col[CSR_TILE + CSR_PAD];
-    __shared__ float s_w[CSR_TILE + CSR_PAD];
-    __shared__ float s_gw[CSR_TILE];
+    constexpr int TILE = CSR_TILE_BWD;
+    __shared__ int s_ptr[TILE + 2];
+    __shared__ int s_col[TILE + CSR_PAD];
+    __shared__ float s_w[TILE + CSR_PAD];
+    __shared__ float s_gw[TILE];
     __shared__ long long s_coord[2];
 
-    const Tile t = stage_tile<IT>(p, s_ptr, s_col, s_w, s_coord);
+    const Tile t = stage_tile<IT, false, TILE>(p, s_ptr, s_col, s_w, s_coord);
     const int wk = threadIdx.x / G;
     const int ln = threadIdx.x % G;
     // lanes of one worker stay converged; workers of one warp do not
@@ -914,7 +916,8 @@ static bool pick_shape(int nvec, int* G, int* VPL) {
     return true;
 }
 
-static long long num_tiles(const tiga_csr* g) { return (g->n_dst + g->n_edges + CSR_TILE - 1) / CSR_TILE; }
+// tiles of a relation for a given tile length; without one, for the shortest (sizes workspaces, bounds grids)
+static long long num_tiles(const tiga_csr* g, int tile = CSR_TILE_MIN) { return (g->n_dst + g->n_edges + tile - 1) / tile; }
 
 template <typename XT, int G, int VPL, int RED, typename IT>
 static tiga_status launch_fwd_t(const CsrParams& p, cudaStream_t s) {
@@ -1077,6 +1080,7 @@ extern "C" tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dty
     p.carry_arg = take_args(cv, reducer, ((size_t)p.ntiles + 1) * F);
     p.huge_count = cv.take<int>(1);
     p.huge_list = cv.take<int4>((size_t)p.ntiles + 1);      // >= 2 E / ROW_HUGE + 1 entries
+    p.ntiles = num_tiles(g, reducer == TIGA_SUM ? CSR_TILE : CSR_TILE_MAX);      // the launch's tiles (the arrays hold at least as many)
 
     const bool i64 = g->rowptr_type == TIGA_I64;
     if (reducer == TIGA_MAX64) {
@@ -1233,7 +1237,7 @@ extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x,
     CsrParams p{};
     p.rowptr = g->rowptr; p.col = g->col; p.w = w; p.x = x; p.arg = const_cast<void*>(argmax);
     p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.F = F; p.nvec = nvec;
-    p.ntiles = num_tiles(g);
+    p.ntiles = num_tiles(g, CSR_TILE_BWD);
     p.gy = grad_out; p.gx = grad_x; p.gw = grad_w;
     if (reducer == TIGA_SUM) {
         if (x_dtype == TIGA_F16)

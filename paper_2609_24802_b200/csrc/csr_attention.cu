@@ -53,9 +53,9 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_attention_kernel(const CsrPar
     constexpr int LV = G * 4;                    // floats of one partial accumulator
     constexpr int U = 4;                         // edges per step
 
-    __shared__ int s_ptr[CSR_TILE + 2];
-    __shared__ __align__(16) int s_col[CSR_TILE + CSR_PAD];
-    __shared__ __align__(16) float s_w[CSR_TILE + CSR_PAD];
+    __shared__ int s_ptr[CSR_TILE_ATT + 2];
+    __shared__ __align__(16) int s_col[CSR_TILE_ATT + CSR_PAD];
+    __shared__ __align__(16) float s_w[CSR_TILE_ATT + CSR_PAD];
     __shared__ long long s_coord[2];
     __shared__ int s_tag[2 * NW];                // local row of head (even) / tail (odd) partial, -1 = none
     __shared__ unsigned char s_first[NW];        // tail partial starts its chain
@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_attention_kernel(const CsrPar
     extern __shared__ __align__(16) unsigned char s_dyn[];
     float* s_pv = reinterpret_cast<float*>(s_dyn);              // [2*NW][LV]
 
-    const Tile t = stage_tile<IT>(p, s_ptr, s_col, s_w, s_coord);
+    const Tile t = stage_tile<IT, false, CSR_TILE_ATT>(p, s_ptr, s_col, s_w, s_coord);
     const int wk = threadIdx.x / G;
     const int ln = threadIdx.x % G;
     const unsigned wmask = G == 32 ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
@@ -272,7 +272,7 @@ static tiga_status attention_check(const tiga_csr* g, int32_t D) {
     if (D < 4 || (D & 3)) return TIGA_ERR_INVALID_ARG;
     if (D > 128) return TIGA_ERR_UNSUPPORTED;
     if (g->n_dst > 0x7fffffffLL || g->n_src > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;
-    if ((g->n_dst + g->n_edges + CSR_TILE - 1) / CSR_TILE > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;
+    if ((g->n_dst + g->n_edges + CSR_TILE_ATT - 1) / CSR_TILE_ATT > 0x7fffffffLL) return TIGA_ERR_UNSUPPORTED;
     return TIGA_OK;
 }
 
@@ -293,7 +293,7 @@ extern "C" size_t tiga_csr_attention_workspace_bytes(const tiga_csr* g, int32_t 
     if (attention_check(g, D) != TIGA_OK) return 0;
     CsrParams p{};
     p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.F = D;
-    p.ntiles = (g->n_dst + g->n_edges + CSR_TILE - 1) / CSR_TILE;
+    p.ntiles = (g->n_dst + g->n_edges + CSR_TILE_ATT - 1) / CSR_TILE_ATT;
     return attention_carve(&p, nullptr) + 256;
 }
 
@@ -311,7 +311,7 @@ extern "C" tiga_status tiga_apply_csr_attention(const tiga_csr* g, const float* 
     CsrParams p{};
     p.rowptr = g->rowptr; p.col = g->col; p.w = nullptr;
     p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.F = D; p.nvec = D / 4;
-    p.ntiles = (g->n_dst + g->n_edges + CSR_TILE - 1) / CSR_TILE;
+    p.ntiles = (g->n_dst + g->n_edges + CSR_TILE_ATT - 1) / CSR_TILE_ATT;
     p.q = q; p.key = key; p.x = value; p.scale = scale; p.out = out; p.lse = lse;
     attention_carve(&p, ws);
     cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -6,7 +6,11 @@
 namespace tiga {
 
 constexpr int CSR_THREADS = 256;
-constexpr int CSR_TILE = 2048;     // merge-path items per CTA
+constexpr int CSR_TILE = 2048;     // merge-path items per CTA (sum forward)
+constexpr int CSR_TILE_ATT = 2048; // online-softmax reducer
+constexpr int CSR_TILE_MAX = 1792; // max forward: a larger state per lane, more CTAs per SM with shorter tiles
+constexpr int CSR_TILE_BWD = 1792; // sum backward: a fourth staged array (edge gradients)
+constexpr int CSR_TILE_MIN = 1792; // the shortest of them: sizes the per-tile workspace arrays
 constexpr int CSR_PAD = 8;         // readable entries behind a tile's staged edges
 
 template <typename XT> struct XTraits;
@@ -111,12 +115,12 @@ struct Tile {
 // index with one pad word per 32: threads that read consecutive runs of 8 stay conflict free
 static __device__ __forceinline__ int pad32(int i) { return i + (i >> 5); }
 
-template <typename IT, bool PADDED = false>
+template <typename IT, bool PADDED = false, int TILE = CSR_TILE>
 __device__ Tile stage_tile(const CsrParams& p, int* s_ptr, int* s_col, float* s_w, long long* s_coord) {
     const IT* rowptr = static_cast<const IT*>(p.rowptr);
     const long long total = p.n_dst + p.n_edges;
-    const long long d0 = (long long)blockIdx.x * CSR_TILE;
-    const long long d1 = (d0 + CSR_TILE < total) ? d0 + CSR_TILE : total;
+    const long long d0 = (long long)blockIdx.x * TILE;
+    const long long d1 = (d0 + TILE < total) ? d0 + TILE : total;
     const int warp = threadIdx.x >> 5;
     if (warp == 0) {
         long long i = rows_done(rowptr, p.n_dst, d0);

@@ -102,7 +102,7 @@ def test_relations_beyond_the_builtin_capacity_are_refused_on_the_host():
     from paper_2609_24802_b200.api import _Csr, _Msg
     lib = T.load_library()
     msg = _Msg(0, 0.0, 0.0)
-    # (2^23 rows + 2^27 edges) / 2048 tiles * 260 bytes = 17.7 MiB > 8 MiB: refused before any device access
+    # (2^23 rows + 2^27 edges) / 1792 tiles * 276 bytes = 20.9 MiB > 8 MiB: refused before any device access
     big = _Csr(256, 0, 256, 1 << 23, 1 << 23, 1 << 27)
     assert lib.tiga_csr_workspace_bytes(ctypes.byref(big), 64, 0, 0, 0) > T.BUILTIN_WS_BYTES
     assert lib.tiga_apply_csr_builtin_ws(ctypes.byref(big), 256, 0, 64, None, ctypes.byref(msg), 0, 256, None, None) == 6
