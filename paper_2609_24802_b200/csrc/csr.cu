@@ -314,6 +314,7 @@ constexpr int ROW_OWN = 4;
 constexpr int ROW_GROUP = 64;
 constexpr int ROW_HUGE = 4096;
 constexpr int GROUP_LANES = 8;
+constexpr int ROW_THREADS = 256;     // rows (= threads) per CTA of the row-class kernel
 
 // Where a source row lives.  HOT (planned apply): col values below n_hot address the compact copy of the
 // hot source rows, the others (minus n_hot) the feature table; both bases are set up once per thread.
@@ -478,23 +479,23 @@ __device__ __forceinline__ void reduce_and_store(State<RED, NV, XTraits<XT>::VW>
 }
 
 template <typename XT, int NV, int RED, typename IT, bool HOT, bool W>
-__global__ void __launch_bounds__(CSR_THREADS, 6) csr_rows_kernel(const CsrParams p) {
+__global__ void __launch_bounds__(ROW_THREADS, 1536 / ROW_THREADS) csr_rows_kernel(const CsrParams p) {
     constexpr int VW = XTraits<XT>::VW;
     constexpr unsigned FULL = 0xffffffffu;
     using St = State<RED, NV, VW>;
     const IT* __restrict__ rowptr = static_cast<const IT*>(p.rowptr);
     const Sources<HOT> src(p);
     const int lane = threadIdx.x & 31;
-    const long long row = ((long long)blockIdx.x * CSR_THREADS + threadIdx.x);      // warp-contiguous rows
+    const long long row = ((long long)blockIdx.x * ROW_THREADS + threadIdx.x);      // warp-contiguous rows
     const bool valid = row < p.n_dst;
     const long long es = valid ? (long long)rowptr[row] : 0;
     const long long ee = valid ? (long long)rowptr[row + 1] : 0;
     const long long deg = ee - es;
 
     // queues of the CTA's longer rows: group rows fill from the front, warp rows from the back
-    __shared__ short q_row[CSR_THREADS];
-    __shared__ long long q_start[CSR_THREADS];
-    __shared__ int q_len[CSR_THREADS];
+    __shared__ short q_row[ROW_THREADS];
+    __shared__ long long q_start[ROW_THREADS];
+    __shared__ int q_len[ROW_THREADS];
     __shared__ int q_ng, q_nw, q_next;
     if (threadIdx.x == 0) { q_ng = 0; q_nw = 0; q_next = 0; }
     __syncthreads();
@@ -510,7 +511,7 @@ __global__ void __launch_bounds__(CSR_THREADS, 6) csr_rows_kernel(const CsrParam
         bg = __shfl_sync(FULL, bg, 0); bw = __shfl_sync(FULL, bw, 0);
         const unsigned lt = (1u << lane) - 1u;
         if (is_g || is_w) {
-            const int slot = is_g ? bg + __popc(mg & lt) : CSR_THREADS - 1 - (bw + __popc(mw & lt));
+            const int slot = is_g ? bg + __popc(mg & lt) : ROW_THREADS - 1 - (bw + __popc(mw & lt));
             q_row[slot] = (short)threadIdx.x; q_start[slot] = es; q_len[slot] = (int)deg;
         }
     }
@@ -552,14 +553,14 @@ __global__ void __launch_bounds__(CSR_THREADS, 6) csr_rows_kernel(const CsrParam
         store_state<XT, NV, RED>(p, p.out + row * p.F, RED ? static_cast<ArgT<RED>*>(p.arg) + row * p.F : nullptr, st);
     }
     __syncthreads();
-    const long long row0 = (long long)blockIdx.x * CSR_THREADS;
+    const long long row0 = (long long)blockIdx.x * ROW_THREADS;
     const int ng = q_ng, nw = q_nw;
 
     // rows for groups of eight lanes: 32 groups per CTA, four rows per warp at a time
     {
         const int gl = lane & (GROUP_LANES - 1);
         const int gid = (threadIdx.x >> 5) * (32 / GROUP_LANES) + lane / GROUP_LANES;
-        constexpr int NGROUPS = CSR_THREADS / GROUP_LANES;
+        constexpr int NGROUPS = ROW_THREADS / GROUP_LANES;
         for (int it0 = 0; it0 < ng; it0 += NGROUPS) {           // uniform over the CTA
             const int it = it0 + gid;
             const bool have = it < ng;
@@ -577,7 +578,7 @@ __global__ void __launch_bounds__(CSR_THREADS, 6) csr_rows_kernel(const CsrParam
         if (lane == 0) idx = atomicAdd(&q_next, 1);
         idx = __shfl_sync(FULL, idx, 0);
         if (idx >= nw) break;
-        const int slot = CSR_THREADS - 1 - idx;
+        const int slot = ROW_THREADS - 1 - idx;
         const long long r = row0 + q_row[slot];
         St part = strided_row<XT, NV, RED, 32, 4, HOT, W>(p, src, q_start[slot], q_len[slot], lane);
         reduce_and_store<XT, NV, RED, 32>(part, lane, true, p.out + r * p.F, RED ? static_cast<ArgT<RED>*>(p.arg) + r * p.F : nullptr);
@@ -933,8 +934,8 @@ static tiga_status launch_fwd_t(const CsrParams& p, cudaStream_t s) {
 template <typename XT, int NV, int RED, typename IT, bool HOT, bool W>
 static tiga_status launch_fwd_narrow_t(const CsrParams& p, cudaStream_t s) {
     TIGA_CUDA_TRY(cudaMemsetAsync(p.huge_count, 0, sizeof(int), s));
-    const unsigned blocks = (unsigned)((p.n_dst + CSR_THREADS - 1) / CSR_THREADS);
-    csr_rows_kernel<XT, NV, RED, IT, HOT, W><<<counted(blocks), CSR_THREADS, 0, s>>>(p);
+    const unsigned blocks = (unsigned)((p.n_dst + ROW_THREADS - 1) / ROW_THREADS);
+    csr_rows_kernel<XT, NV, RED, IT, HOT, W><<<counted(blocks), ROW_THREADS, 0, s>>>(p);
     csr_huge_chunks_kernel<XT, NV, RED, IT, HOT, W><<<counted(148 * 8), CSR_THREADS, 0, s>>>(p);
     csr_huge_fold_kernel<RED><<<counted(148 * 2), 256, 0, s>>>(p);
     return launch_status();
