@@ -50,6 +50,36 @@ def test_uneven_density_uses_shells_and_list_cuts(tiga):
     _check(tiga, pos, gen.normal_features(n, 4, 92, 31), 32)
 
 
+@pytest.mark.parametrize("cloud", ["uniform", "clustered"])
+def test_selection_agrees_with_exact_geometry(tiga, cloud):
+    """Independent of the oracle's fp32 key: in exact (fp64) geometry every selected neighbour is at
+    least as near as every point left out, up to the rounding of the fp32 key (relative 1e-6), for
+    every query; no self, no duplicates, keys in non-decreasing order."""
+    n, k = 6000, 16
+    pos = gen.uniform_points(n, 97) if cloud == "uniform" else gen.clustered_points(n, 98)
+    x = gen.normal_features(n, 1, 99, 31)
+    _, nbr, d2, _ = tiga.tiga_apply_knn(dev(pos, torch), dev(x, torch), k, UNIT)
+    nbr, d2 = host(nbr).astype(np.int64), host(d2)
+    p64 = pos.astype(np.float64)
+    assert np.all(np.diff(d2, axis=1) >= 0)
+    for lo in range(0, n, 1000):
+        q = p64[lo:lo + 1000]
+        D = ((q[:, None, :] - p64[None, :, :]) ** 2).sum(-1)            # exact squared distances (fp64 of fp32 inputs)
+        rows = np.arange(len(q))
+        D[rows, lo + rows] = np.inf                                       # a point is not its own neighbour
+        sel = nbr[lo:lo + 1000]
+        assert np.all(sel != (lo + rows)[:, None])
+        assert all(len(set(r)) == k for r in sel)
+        far_in = np.take_along_axis(D, sel, 1).max(1)
+        Dout = D.copy()
+        np.put_along_axis(Dout, sel, np.inf, 1)
+        near_out = Dout.min(1)
+        assert np.all(far_in <= near_out * (1 + 1e-6) + 1e-300)
+        # the reported keys are the exact squared distances rounded like an fp32 evaluation
+        exact = np.take_along_axis(D, sel, 1)
+        assert np.all(np.abs(d2[lo:lo + 1000] - exact) <= 1e-6 * exact + 1e-30)
+
+
 def test_points_on_a_surface(tiga):
     n = 35947
     _check(tiga, gen.surface_points(n, 3), gen.normal_features(n, 1, 93, 31), 16)
