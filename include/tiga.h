@@ -90,6 +90,16 @@ const char* tiga_status_string(tiga_status s);
  * a timed region to state how many of the library's kernels ran inside it. */
 int64_t tiga_kernel_launches(void);
 
+/* Checked build (libtiga_checked.so, compiled with -DTIGA_CHECKED; no counterpart in the paper): every
+ * index that is about to address a gathered source row, an edge or a point is range-checked on the device
+ * first; a violation sets a bit of a status word and the access goes to element 0 instead, so nothing
+ * faults.  tiga_checked_status synchronises the device and returns the bits seen since the last reset
+ * (1 source index, 2 edge position, 4 point id, 8 slot of the cell-ordered points; 0x80000000 if the word
+ * could not be read) and clears them when reset != 0.  The normal build checks nothing and returns 0.
+ * tiga_is_checked_build tells the two apart. */
+uint32_t tiga_checked_status(int reset);
+int tiga_is_checked_build(void);
+
 /* ------------------------------------------------------------------------------------ CSR */
 
 /* Bytes of workspace tiga_apply_csr (backward = 0) or tiga_apply_csr_backward (backward = 1)

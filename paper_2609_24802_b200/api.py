@@ -29,7 +29,7 @@ I32, I64 = 0, 1
 MSG_COPY, MSG_WEIGHTED, MSG_GAUSS, MSG_DIST, MSG_LJ = 0, 1, 2, 3, 4
 
 EXPORTS = [
-    "tiga_status_string", "tiga_kernel_launches", "tiga_csr_workspace_bytes", "tiga_validate_csr", "tiga_apply_csr",
+    "tiga_status_string", "tiga_kernel_launches", "tiga_checked_status", "tiga_is_checked_build", "tiga_csr_workspace_bytes", "tiga_validate_csr", "tiga_apply_csr",
     "tiga_apply_csr_builtin_ws", "tiga_apply_csr_backward", "tiga_csr_degree_histogram", "tiga_radius_grid",
     "tiga_csr_plan_bytes", "tiga_csr_plan_workspace_bytes", "tiga_csr_plan_build", "tiga_csr_planned_workspace_bytes",
     "tiga_apply_csr_planned",
@@ -39,7 +39,9 @@ EXPORTS = [
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libtiga.so")
+# TIGA_CHECKED=1 in the environment selects the checked build (range-checked indices, status word)
+CHECKED = os.environ.get("TIGA_CHECKED", "0") not in ("", "0")
+LIB_PATH = os.path.join(_HERE, "libtiga_checked.so" if CHECKED else "libtiga.so")
 
 
 class TigaError(RuntimeError):
@@ -89,6 +91,10 @@ def load_library() -> ctypes.CDLL:
     lib.tiga_status_string.argtypes = [ctypes.c_int]
     lib.tiga_kernel_launches.restype = i64
     lib.tiga_kernel_launches.argtypes = []
+    lib.tiga_checked_status.restype = ctypes.c_uint32
+    lib.tiga_checked_status.argtypes = [ctypes.c_int]
+    lib.tiga_is_checked_build.restype = ctypes.c_int
+    lib.tiga_is_checked_build.argtypes = []
     lib.tiga_csr_workspace_bytes.restype = sz
     lib.tiga_csr_workspace_bytes.argtypes = [ctypes.POINTER(_Csr), i32, ctypes.c_int, ctypes.c_int, ctypes.c_int]
     lib.tiga_validate_csr.restype = ctypes.c_int
@@ -146,6 +152,16 @@ def load_library() -> ctypes.CDLL:
 
 
 load_library()      # fail at import time, loudly, when the CUDA library is not there
+
+
+def checked_status(reset: bool = True) -> int:
+    """Bits of the checked build's status word (0 in the normal build): 1 source index, 2 edge position,
+    4 point id, 8 slot.  Synchronises the device."""
+    return int(load_library().tiga_checked_status(int(reset)))
+
+
+def is_checked_build() -> bool:
+    return bool(load_library().tiga_is_checked_build())
 
 
 def launch_count() -> int:

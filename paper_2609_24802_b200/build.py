@@ -11,6 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(HERE, "libtiga.so")
+LIB_CHECKED = os.path.join(HERE, "libtiga_checked.so")      # same sources with -DTIGA_CHECKED (range-checked indices)
 SOURCES = ["csr.cu", "csr_plan.cu", "csr_attention.cu", "radius.cu", "radius_lj.cu", "radius_mlp.cu", "knn.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I" + INCLUDE, "-I" + CSRC]
@@ -28,10 +29,12 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compile every CUDA source for sm_100a and link libtiga.so next to this file."""
+def build_library(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Compile every CUDA source for sm_100a and link libtiga.so (or, with checked=True, the checked
+    build libtiga_checked.so) next to this file."""
     headers = [os.path.join(INCLUDE, "tiga.h")] + [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cuh")]
-    objdir = os.path.join(HERE, "build")
+    objdir = os.path.join(HERE, "build_checked" if checked else "build")
+    lib = LIB_CHECKED if checked else LIB
     os.makedirs(objdir, exist_ok=True)
     objs = []
     jobs = []
@@ -40,7 +43,8 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         o = os.path.join(objdir, src.replace(".cu", ".o"))
         objs.append(o)
         if force or _stale(o, [s] + headers):
-            cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
+            cmd = ([_nvcc()] + NVCC_FLAGS + (["-DTIGA_CHECKED"] if checked else []) + (["-Xptxas", "-v"] if verbose else [])
+                   + ["-c", s, "-o", o])
             jobs.append(cmd)
     if jobs:
         with ThreadPoolExecutor(max_workers=len(jobs)) as ex:
@@ -49,10 +53,11 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
                     sys.stderr.write(res.stdout + res.stderr)
                 if res.returncode != 0:
                     raise RuntimeError("nvcc failed")
-    if force or jobs or _stale(LIB, objs):
-        subprocess.check_call([_nvcc(), "-shared", "-o", LIB] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
-    build_bench_probe(force)
-    return LIB
+    if force or jobs or _stale(lib, objs):
+        subprocess.check_call([_nvcc(), "-shared", "-o", lib] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
+    if not checked:
+        build_bench_probe(force)
+    return lib
 
 
 def build_bench_probe(force: bool = False) -> str:
@@ -67,3 +72,5 @@ def build_bench_probe(force: bool = False) -> str:
 
 if __name__ == "__main__":
     print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--no-checked" not in sys.argv:
+        print(build_library(force="--force" in sys.argv, checked=True))

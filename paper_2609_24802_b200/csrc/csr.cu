@@ -323,13 +323,16 @@ struct Sources {
     const uint4* cold;
     const uint4* hot;
     unsigned n_hot, nvec;
+    long long n_all;              // checked build: range of the indices
     __device__ __forceinline__ explicit Sources(const CsrParams& p) {
         nvec = (unsigned)p.nvec;
+        n_all = p.n_src;
         n_hot = HOT ? (unsigned)p.n_hot : 0u;
         cold = static_cast<const uint4*>(p.x) - (size_t)n_hot * nvec;
         hot = HOT ? static_cast<const uint4*>(p.x_hot) : cold;
     }
     __device__ __forceinline__ const uint4* row(unsigned c) const {
+        c = checked(c, n_all, CHECK_SOURCE);
         const uint4* base = (HOT && c < n_hot) ? hot : cold;
         return base + (unsigned long long)c * nvec;          // one 32 x 32 -> 64 multiply
     }
@@ -787,12 +790,13 @@ __global__ void csr_backward_max_kernel(const CsrParams p) {
     constexpr unsigned FULL = 0xffffffffu;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const int lane = threadIdx.x & 31;
-    const AT e = idx < p.n_dst * p.F ? static_cast<const AT*>(p.arg)[idx] : AT(-1);
+    AT e = idx < p.n_dst * p.F ? static_cast<const AT*>(p.arg)[idx] : AT(-1);
+    if (e >= 0) e = checked(e, p.n_edges, CHECK_EDGE);
     const bool act = e >= 0;
     float contrib = 0.f;
     if (act) {
         const int f = (int)(idx % p.F);
-        const long long j = p.col[e];
+        const long long j = checked(p.col[e], p.n_src, CHECK_SOURCE);
         const float g = p.gy[idx];
         if (p.gx) atomicAdd(p.gx + j * p.F + f, (p.w ? p.w[e] : 1.f) * g);
         if (p.gw) {
@@ -1073,7 +1077,7 @@ extern "C" tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dty
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     CsrParams p{};
     p.rowptr = g->rowptr; p.col = g->col; p.w = w; p.x = x; p.out = out; p.arg = argmax;
-    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.F = F; p.nvec = nvec;
+    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.n_src = g->n_src; p.F = F; p.nvec = nvec;
     p.ntiles = num_tiles(g);
     Carver cv(ws);
     p.carry_row = cv.take<int32_t>((size_t)p.ntiles + 1);
@@ -1179,12 +1183,13 @@ extern "C" tiga_status tiga_apply_csr_planned(const tiga_csr* g, const tiga_csr_
     CsrParams p{};
     p.rowptr = g->rowptr; p.col = reinterpret_cast<const int32_t*>(base + plan->off_col);
     p.w = w; p.x = x; p.out = out; p.arg = argmax;
-    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.F = F; p.nvec = nvec;
+    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.n_src = g->n_src; p.F = F; p.nvec = nvec;
     p.ntiles = num_tiles(g);
     Carver cv(ws);
     const size_t row_bytes = (size_t)F * (x_dtype == TIGA_F32 ? 4 : 2);
     void* hot = cv.take<unsigned char>((size_t)plan->n_hot * row_bytes + 256);
     p.x_hot = hot; p.n_hot = (int)plan->n_hot;
+    p.n_src = g->n_src + plan->n_hot;                      // range of the rewritten indices
     p.carry_row = cv.take<int32_t>((size_t)p.ntiles + 1);
     p.carry_val = cv.take<float>(((size_t)p.ntiles + 1) * F);
     p.carry_arg = take_args(cv, reducer, ((size_t)p.ntiles + 1) * F);
@@ -1237,7 +1242,7 @@ extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x,
 
     CsrParams p{};
     p.rowptr = g->rowptr; p.col = g->col; p.w = w; p.x = x; p.arg = const_cast<void*>(argmax);
-    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.F = F; p.nvec = nvec;
+    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.n_src = g->n_src; p.F = F; p.nvec = nvec;
     p.ntiles = num_tiles(g, CSR_TILE_BWD);
     p.gy = grad_out; p.gx = grad_x; p.gw = grad_w;
     if (reducer == TIGA_SUM) {
@@ -1281,6 +1286,26 @@ extern "C" tiga_status tiga_csr_degree_histogram(const tiga_csr* g, int64_t* his
 
 extern "C" int64_t tiga_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
 
+extern "C" uint32_t tiga_checked_status(int reset) {
+#ifdef TIGA_CHECKED
+    if (cudaDeviceSynchronize() != cudaSuccess) return 0x80000000u;
+    const bool r = reset != 0;
+    return check_status_csr(r) | check_status_csr_plan(r) | check_status_csr_attention(r) | check_status_radius(r) |
+           check_status_radius_lj(r) | check_status_radius_mlp(r) | check_status_knn(r);
+#else
+    (void)reset;
+    return 0u;
+#endif
+}
+
+extern "C" int tiga_is_checked_build(void) {
+#ifdef TIGA_CHECKED
+    return 1;
+#else
+    return 0;
+#endif
+}
+
 extern "C" const char* tiga_status_string(tiga_status s) {
     switch (s) {
         case TIGA_OK: return "ok";
@@ -1294,3 +1319,5 @@ extern "C" const char* tiga_status_string(tiga_status s) {
     }
     return "unknown status";
 }
+
+namespace tiga { unsigned check_status_csr(bool reset) { return read_check_status(reset); } }

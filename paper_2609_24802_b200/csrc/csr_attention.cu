@@ -292,7 +292,7 @@ using namespace tiga;
 extern "C" size_t tiga_csr_attention_workspace_bytes(const tiga_csr* g, int32_t D) {
     if (attention_check(g, D) != TIGA_OK) return 0;
     CsrParams p{};
-    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.F = D;
+    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.n_src = g->n_src; p.F = D;
     p.ntiles = (g->n_dst + g->n_edges + CSR_TILE_ATT - 1) / CSR_TILE_ATT;
     return attention_carve(&p, nullptr) + 256;
 }
@@ -310,10 +310,12 @@ extern "C" tiga_status tiga_apply_csr_attention(const tiga_csr* g, const float* 
     if (!ws || !aligned16(ws) || ws_bytes < tiga_csr_attention_workspace_bytes(g, D)) return TIGA_ERR_WORKSPACE;
     CsrParams p{};
     p.rowptr = g->rowptr; p.col = g->col; p.w = nullptr;
-    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.F = D; p.nvec = D / 4;
+    p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.n_src = g->n_src; p.F = D; p.nvec = D / 4;
     p.ntiles = (g->n_dst + g->n_edges + CSR_TILE_ATT - 1) / CSR_TILE_ATT;
     p.q = q; p.key = key; p.x = value; p.scale = scale; p.out = out; p.lse = lse;
     attention_carve(&p, ws);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     return g->rowptr_type == TIGA_I64 ? launch_attention<int64_t>(p, s) : launch_attention<int32_t>(p, s);
 }
+
+namespace tiga { unsigned check_status_csr_attention(bool reset) { return read_check_status(reset); } }

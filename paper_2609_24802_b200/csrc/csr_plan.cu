@@ -120,9 +120,10 @@ __global__ void __launch_bounds__(256) plan_number_kernel(int32_t* indeg, long l
     if (threadIdx.x == 0 && s_cov) atomicAdd(covered, s_cov);
 }
 
-__global__ void __launch_bounds__(256) plan_indegree_kernel(const int32_t* __restrict__ col, long long n_edges, int32_t* indeg) {
+__global__ void __launch_bounds__(256) plan_indegree_kernel(const int32_t* __restrict__ col, long long n_edges, long long n_src, int32_t* indeg) {
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < n_edges; e += stride) atomicAdd(indeg + ld_stream(col + e), 1);
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < n_edges; e += stride)
+        atomicAdd(indeg + checked(ld_stream(col + e), n_src, CHECK_SOURCE), 1);
 }
 
 // histogram of min(in-degree, PLAN_BINS - 1): per-CTA counts in shared memory, then global atomics
@@ -141,11 +142,11 @@ __global__ void __launch_bounds__(256) plan_degree_hist_kernel(const int32_t* __
         if (s_hist[k]) atomicAdd(hist + k, (unsigned long long)s_hist[k]);
 }
 
-__global__ void __launch_bounds__(256) plan_rewrite_kernel(const int32_t* __restrict__ col, long long n_edges,
+__global__ void __launch_bounds__(256) plan_rewrite_kernel(const int32_t* __restrict__ col, long long n_edges, long long n_src,
                                                            const int32_t* __restrict__ remap, int32_t* pcol) {
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < n_edges; e += stride)
-        st_stream(pcol + e, __ldg(remap + ld_stream(col + e)));
+        st_stream(pcol + e, __ldg(remap + checked(ld_stream(col + e), n_src, CHECK_SOURCE)));
 }
 
 // compact copy of the hot source rows (16-byte vectors): hot[r, :] = x[hot_id[r], :]
@@ -212,7 +213,7 @@ extern "C" tiga_status tiga_csr_plan_build(const tiga_csr* g, int64_t max_hot_ro
 
     TIGA_CUDA_TRY(cudaMemsetAsync(indeg, 0, (size_t)n * sizeof(int32_t), s));
     TIGA_CUDA_TRY(cudaMemsetAsync(hist, 0, (PLAN_BINS + 1) * sizeof(unsigned long long), s));
-    plan_indegree_kernel<<<counted(148 * 16), 256, 0, s>>>(g->col, E, indeg);
+    plan_indegree_kernel<<<counted(148 * 16), 256, 0, s>>>(g->col, E, n, indeg);
     plan_degree_hist_kernel<<<counted(148 * 4), 256, 0, s>>>(indeg, n, hist);
     if (launch_status() != TIGA_OK) return TIGA_ERR_CUDA;
     std::vector<unsigned long long> hh(PLAN_BINS + 1);
@@ -232,7 +233,7 @@ extern "C" tiga_status tiga_csr_plan_build(const tiga_csr* g, int64_t max_hot_ro
     plan_hot_count_kernel<<<counted((unsigned)nchunks), 256, 0, s>>>(indeg, n, thr, sums);
     plan_scan_sums_kernel<<<counted(1), 1024, 0, s>>>(sums, nchunks);
     plan_number_kernel<<<counted((unsigned)nchunks), 256, 0, s>>>(indeg, n, thr, sums, (int)n_hot, hot_id, hist + PLAN_BINS);
-    plan_rewrite_kernel<<<counted(148 * 16), 256, 0, s>>>(g->col, E, indeg, pcol);
+    plan_rewrite_kernel<<<counted(148 * 16), 256, 0, s>>>(g->col, E, n, indeg, pcol);
     if (launch_status() != TIGA_OK) return TIGA_ERR_CUDA;
     unsigned long long covered = 0;
     TIGA_CUDA_TRY(cudaMemcpyAsync(&covered, hist + PLAN_BINS, sizeof(covered), cudaMemcpyDeviceToHost, s));
@@ -242,3 +243,5 @@ extern "C" tiga_status tiga_csr_plan_build(const tiga_csr* g, int64_t max_hot_ro
     plan->n_hot = n_hot; plan->min_hot_degree = n_hot ? thr : 0; plan->hot_edges = (int64_t)covered;
     return TIGA_OK;
 }
+
+namespace tiga { unsigned check_status_csr_plan(bool reset) { return read_check_status(reset); } }

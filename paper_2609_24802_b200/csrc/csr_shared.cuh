@@ -57,6 +57,7 @@ struct CsrParams {
     float* out;
     void* arg;               // int32 [n_dst, F], or int64 for the wide-position max reducer
     long long n_dst, n_edges;
+    long long n_src;         // rows of x (checked build: bound of every gathered index; a planned relation adds n_hot)
     int F;                   // features per row
     int nvec;                // 16-byte vectors per feature row
     // workspace
@@ -148,7 +149,7 @@ __device__ Tile stage_tile(const CsrParams& p, int* s_ptr, int* s_col, float* s_
     }
     for (int k = threadIdx.x; k < t.ne; k += CSR_THREADS) {
         const int kk = PADDED ? pad32(k) : k;
-        s_col[kk] = ld_stream(p.col + t.e0 + k);
+        s_col[kk] = checked(ld_stream(p.col + t.e0 + k), p.n_src, CHECK_SOURCE);
         s_w[kk] = p.w ? ld_stream(p.w + t.e0 + k) : 1.f;
     }
     // a few valid entries behind the last edge: unrolled loops may load (never use) past their span

@@ -555,3 +555,5 @@ extern "C" tiga_status tiga_apply_knn(const float* pos, const float* feat, int64
     knn_rings_kernel<<<counted(KNN_RING_BLOCKS), TRAV_THREADS, 0, s>>>(P);
     return launch_status();
 }
+
+namespace tiga { unsigned check_status_knn(bool reset) { return read_check_status(reset); } }

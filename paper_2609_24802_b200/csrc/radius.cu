@@ -380,7 +380,7 @@ __device__ __forceinline__ void traverse_slice(const RadiusParams& p, const int 
                         int oqq = 0;
                         if (valid) {
                             const float4 qv = s_q[qq];
-                            oqq = __float_as_int(qv.w);
+                            oqq = checked(__float_as_int(qv.w), p.n, CHECK_POINT);
                             const int n = s_n[qq];
                             const float2* lq = list + qq * QSTRIDE;
                             if (MODE == 0) {
@@ -390,7 +390,7 @@ __device__ __forceinline__ void traverse_slice(const RadiusParams& p, const int 
 #pragma unroll
                                     for (int u = 0; u < 4; ++u) {      // four gathered rows in flight
                                         e[u] = lq[t + u];
-                                        const float* xr = p.feat + (size_t)__float_as_int(e[u].x) * F + fl * 4;
+                                        const float* xr = p.feat + (size_t)checked(__float_as_int(e[u].x), p.n, CHECK_POINT) * F + fl * 4;
                                         if (VEC) x[u] = __ldg(reinterpret_cast<const float4*>(xr));
                                         else x[u] = make_float4(__ldg(xr), fl * 4 + 1 < F ? __ldg(xr + 1) : 0.f,
                                                                 fl * 4 + 2 < F ? __ldg(xr + 2) : 0.f, fl * 4 + 3 < F ? __ldg(xr + 3) : 0.f);
@@ -416,7 +416,7 @@ __device__ __forceinline__ void traverse_slice(const RadiusParams& p, const int 
                                         float dx, dy, dz;
                                         delta(qv, pj, dx, dy, dz);
                                         e[u] = make_float4(dx, dy, dz, 0.f);
-                                        const size_t row = (size_t)__float_as_int(pj.w) * F;
+                                        const size_t row = (size_t)checked(__float_as_int(pj.w), p.n, CHECK_POINT) * F;
                                         xj[u] = __ldg(reinterpret_cast<const float4*>(p.feat + row) + fl);
                                         gj[u] = __ldg(reinterpret_cast<const float4*>(p.gy + row) + fl);
                                     }
@@ -633,7 +633,7 @@ __device__ __forceinline__ void traverse_slice(const RadiusParams& p, const int 
             }
             r = r > 31 ? 31 : r;
             const int src = __shfl_sync(FULL, r_cs, r) + (v - (__shfl_sync(FULL, r_incl, r) - __shfl_sync(FULL, r_len, r)));
-            c4[u] = v < total ? __ldg(p.spos + src) : make_float4(0.f, 0.f, 0.f, 0.f);
+            c4[u] = v < total ? __ldg(p.spos + checked(src, p.n, CHECK_SLOT)) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         const float lx = __shfl_sync(FULL, bb, 0), ly = __shfl_sync(FULL, bb, 1), lz = __shfl_sync(FULL, bb, 2);
         const float hx = __shfl_sync(FULL, bb, 3), hy = __shfl_sync(FULL, bb, 4), hz = __shfl_sync(FULL, bb, 5);
@@ -934,3 +934,5 @@ extern "C" tiga_status tiga_apply_radius_backward(const float* pos, const float*
     }
     return launch_traverse<2, false>(p, s);
 }
+
+namespace tiga { unsigned check_status_radius(bool reset) { return read_check_status(reset); } }

@@ -226,8 +226,9 @@ __device__ __forceinline__ void lj_slice(const RadiusParams& p, const int cellid
                             fx += gx; fy += gy; fz += gz; en += ee;
                             const int idj = __float_as_int(pj[u].w);
                             if (valid) {
-                                atomicAdd(out4 + idj, make_float4(-gx, -gy, -gz, ee));      // the pair's other row
-                                if (COUNT) atomicAdd(p.count + idj, 1);
+                                const int row_j = checked(idj, p.n, CHECK_POINT);
+                                atomicAdd(out4 + row_j, make_float4(-gx, -gy, -gz, ee));    // the pair's other row
+                                if (COUNT) atomicAdd(p.count + row_j, 1);
                             }
                         }
                     }
@@ -238,7 +239,7 @@ __device__ __forceinline__ void lj_slice(const RadiusParams& p, const int cellid
                     fz += __shfl_xor_sync(FULL, fz, o); en += __shfl_xor_sync(FULL, en, o);
                 }
                 if (q < nq && sub == 0 && n > 0) {
-                    const int idq = __float_as_int(s_q[q].w);
+                    const int idq = checked(__float_as_int(s_q[q].w), p.n, CHECK_POINT);
                     atomicAdd(out4 + idq, make_float4(fx, fy, fz, en));
                     if (COUNT) atomicAdd(p.count + idq, n);
                 }
@@ -337,7 +338,7 @@ __device__ __forceinline__ void lj_slice(const RadiusParams& p, const int cellid
                 const int k = k0 + 32 * u + lane;
                 int run;
                 const int src = locate(lo + k, run);
-                c4[u] = k < nin ? __ldg(p.spos + src) : make_float4(0.f, 0.f, 0.f, 0.f);
+                c4[u] = k < nin ? __ldg(p.spos + checked(src, p.n, CHECK_SLOT)) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
             const float lx = __shfl_sync(FULL, bb, 0), ly = __shfl_sync(FULL, bb, 1), lz = __shfl_sync(FULL, bb, 2);
             const float hx = __shfl_sync(FULL, bb, 3), hy = __shfl_sync(FULL, bb, 4), hz = __shfl_sync(FULL, bb, 5);
@@ -407,3 +408,5 @@ tiga_status launch_lj_pairs(const RadiusParams& p, cudaStream_t s) {
 }
 
 }  // namespace tiga
+
+namespace tiga { unsigned check_status_radius_lj(bool reset) { return read_check_status(reset); } }

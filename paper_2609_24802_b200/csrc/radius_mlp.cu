@@ -605,3 +605,5 @@ extern "C" tiga_status tiga_apply_radius_mlp_backward(const float* pos, const fl
     }
     return launch_mlp<true>(p, mlp->hidden, s);
 }
+
+namespace tiga { unsigned check_status_radius_mlp(bool reset) { return read_check_status(reset); } }

@@ -30,6 +30,19 @@ def test_every_declared_symbol_is_exported(lib):
         assert getattr(cdll, name) is not None
 
 
+def test_checked_build_exports_the_same_symbols(lib):
+    """libtiga_checked.so (same sources, -DTIGA_CHECKED) loads and exports every declared symbol; the two
+    builds tell themselves apart without a device."""
+    from paper_2609_24802_b200 import build
+    path = build.build_library(checked=True)
+    checked = ctypes.CDLL(path)
+    for name in lib.EXPORTS:
+        assert getattr(checked, name) is not None
+    checked.tiga_is_checked_build.restype = ctypes.c_int
+    assert checked.tiga_is_checked_build() == 1
+    assert lib.load_library().tiga_is_checked_build() == 0
+
+
 def test_status_strings(lib):
     assert lib.tiga_status_string(0) == "ok"
     assert len({lib.tiga_status_string(s) for s in range(8)}) == 8
