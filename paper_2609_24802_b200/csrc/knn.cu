@@ -143,12 +143,12 @@ static __device__ __forceinline__ void emit_row(const KnnParams& P, const int i,
             float acc = 0.f;
             for (int t = 0; t < m; ++t) {
                 const int idt = __shfl_sync(0xffffffffu, id, t);
-                if (f < F) acc += __ldg(feat + (size_t)idt * F + f);
+                if (f < F) acc += __ldg(feat + (size_t)checked(idt, P.rp.n, CHECK_POINT) * F + f);
             }
             if (f < F) P.out[(size_t)i * F + f] = acc;
         }
     } else {
-        const size_t row = v ? (size_t)id * F : 0;
+        const size_t row = v ? (size_t)checked(id, P.rp.n, CHECK_POINT) * F : 0;
         for (int f = 0; f < F; ++f) {
             float x = v ? __ldg(feat + row + f) : 0.f;
 #pragma unroll
@@ -234,7 +234,7 @@ __device__ __forceinline__ void knn_cell_slice(const KnnParams& P, const int cel
             bool keep = false;
             float4 c4 = make_float4(0.f, 0.f, 0.f, 0.f);
             if (v < total) {
-                c4 = __ldg(p.spos + src);
+                c4 = __ldg(p.spos + checked(src, p.n, CHECK_SLOT));
                 const float ex = fmaxf(fmaxf(lx - c4.x, c4.x - hx), 0.f);
                 const float ey = fmaxf(fmaxf(ly - c4.y, c4.y - hy), 0.f);
                 const float ez = fmaxf(fmaxf(lz - c4.z, c4.z - hz), 0.f);
@@ -445,7 +445,7 @@ __global__ void __launch_bounds__(TRAV_THREADS) knn_rings_kernel(const __grid_co
                     float4 c4 = make_float4(0.f, 0.f, 0.f, 0.f);
                     float d2 = 0.f;
                     if (v < total) {
-                        c4 = __ldg(p.spos + src);
+                        c4 = __ldg(p.spos + checked(src, p.n, CHECK_SLOT));
                         d2 = key_d2(qx, qy, qz, c4.x, c4.y, c4.z);
                         ok = d2 <= tau && __float_as_int(c4.w) != i;
                     }

@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, mlp_ctas_per_sm<HID, BWD>()) rad
                         for (int j = 0; j < QB; ++j) tq = (j == q) ? f - pre[j] : tq;
                         const int key = valid ? q : -1 - lane;               // idle lanes form segments of their own
                         const float4 qv = s_q[q];
-                        const int oq = __float_as_int(qv.w);
+                        const int oq = checked(__float_as_int(qv.w), p.n, CHECK_POINT);
                         float4 pj = make_float4(0.f, 0.f, 0.f, __int_as_float(0));
                         if (valid) pj = stage[list[q * MLP_QSTRIDE + tq]];
                         float dx = pj.x - qv.x, dy = pj.y - qv.y, dz = pj.z - qv.z;      // source minus destination
@@ -225,7 +225,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, mlp_ctas_per_sm<HID, BWD>()) rad
                             if (valid) {
                                 float u[KU], h[HID], m[4];
                                 u[0] = dx; u[1] = dy; u[2] = dz;
-                                const float* xr = p.feat + (size_t)__float_as_int(pj.w) * Fin;
+                                const float* xr = p.feat + (size_t)checked(__float_as_int(pj.w), p.n, CHECK_POINT) * Fin;
 #pragma unroll
                                 for (int k = 3; k < KU; ++k) u[k] = (k - 3 < Fin) ? __ldg(xr + k - 3) : 0.f;
                                 mlp_forward<HID, KQ>(sW1, sb1, sW2, sb2, u, h, m);
@@ -235,7 +235,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, mlp_ctas_per_sm<HID, BWD>()) rad
                         } else {
                             float* mine = pairbuf + lane * PS;
                             if (valid) {
-                                const int om = __float_as_int(pj.w);
+                                const int om = checked(__float_as_int(pj.w), p.n, CHECK_POINT);
                                 float gyk[4], gym[4];
 #pragma unroll
                                 for (int o = 0; o < 4; ++o) {
@@ -463,7 +463,7 @@ __global__ void __launch_bounds__(TRAV_THREADS, mlp_ctas_per_sm<HID, BWD>()) rad
                     r = r > 31 ? 31 : r;
                     const int src = __shfl_sync(FULL, r_cs, r) + (v - (__shfl_sync(FULL, r_incl, r) - __shfl_sync(FULL, r_len, r)));
                     ox[u] = __shfl_sync(FULL, r_off[0], r); oy[u] = __shfl_sync(FULL, r_off[1], r); oz[u] = __shfl_sync(FULL, r_off[2], r);
-                    c4[u] = k < ns ? __ldg(p.spos + src) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    c4[u] = k < ns ? __ldg(p.spos + checked(src, p.n, CHECK_SLOT)) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
                 const float lx = __shfl_sync(FULL, bb, 0), ly = __shfl_sync(FULL, bb, 1), lz = __shfl_sync(FULL, bb, 2);
                 const float hx = __shfl_sync(FULL, bb, 3), hy = __shfl_sync(FULL, bb, 4), hz = __shfl_sync(FULL, bb, 5);

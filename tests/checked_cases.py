@@ -97,6 +97,17 @@ def main():
     outl, countl, _ = T.tiga_apply_radius(dev(c["pos"], torch), None, c["r"], c["box"], c["periodic"], T.MSG_LJ, p0=1.0, p1=1.0,
                                           count=torch.empty(len(c["pos"]), dtype=torch.int32, device="cuda"))
     assert np.array_equal(host(countl), cl) and rel_err(host(outl), yl, Al) <= SUM_TOL
+    params = gen.mlp_params(8, 16, 4, 7)
+    xm, gm = gen.normal_features(n, 8, 62, 31), gen.normal_features(n, 4, 62, 32)
+    ym, Am, cm = oracle.radius_mlp_forward(pos, xm, r, ones, [1, 1, 1], *params, use_cells=True)
+    P = [dev(a, torch) for a in params]
+    outm, countm, wsm = T.tiga_apply_radius_mlp(dev(pos, torch), dev(xm, torch), r, ones, [1, 1, 1], *P,
+                                                count=torch.empty(n, dtype=torch.int32, device="cuda"))
+    assert np.array_equal(host(countm), cm) and rel_err(host(outm), ym, Am) <= SUM_TOL
+    T.tiga_apply_radius_mlp_backward(dev(pos, torch), dev(xm, torch), dev(gm, torch), r, ones, [1, 1, 1], *P)
+    idx, rd2, yk, Ak = oracle.knn(pos, xm, 16)
+    outk, nbr, d2, _ = T.tiga_apply_knn(dev(pos, torch), dev(xm, torch), 16, ones)
+    assert np.array_equal(host(nbr), idx) and rel_err(host(outk), yk, Ak) <= SUM_TOL
     assert T.checked_status() == 0, "well-formed inputs must not raise the status word"
 
     # ---- part 2: a few source indices just outside [0, n_src): flagged, redirected to row 0, no fault
