@@ -76,7 +76,7 @@ def test_dense_cluster_overflows_the_lists(tiga):
     gy = gen.normal_features(n, 4, 15, 32)
     # about 400 neighbours per point: many pre-activations per row, so a tighter kink margin
     _check(tiga, pos, x, gy, np.float32(0.04), np.ones(3, np.float32), [0, 0, 0], gen.mlp_params(8, 16, 4, 9),
-           kink_eps=3e-6, min_keep=0.5)
+           kink_eps=3e-6, min_keep=0.9)      # 93 % of the rows are kept with this margin
 
 
 @pytest.mark.parametrize("hidden", [8, 32])
