@@ -155,10 +155,10 @@ TRAFFIC_PER_UNIT = {
     "radius_lj_fwd": ("particle", 48.4),          # profiles/radius_lj_pairs_1M.md: 32.4 B measured + the 16-byte row that leaves L2 at full size
     "radius_gauss_fwd": ("point", 186.7),         # profiles/radius_traverse_gaussian_300k.md
     "radius_gauss_bwd": ("point", 364.6),
-    "csr_sum_fwd": ("edge", 21.1),                # profiles/csr_kernels_rmat_scale18.md
-    "csr_max_fwd": ("edge", 37.0),
-    "csr_sum_bwd": ("edge", 45.3),
-    "csr_max_bwd": ("edge", 52.1),
+    "csr_sum_fwd": ("edge", 21.3),                # profiles/csr_kernels_rmat_scale18.md
+    "csr_max_fwd": ("edge", 37.4),
+    "csr_sum_bwd": ("edge", 45.4),
+    "csr_max_bwd": ("edge", 51.9),
     "csr_large_fwd": ("edge", 33.1),              # profiles/csr_large_cfg4_dram_traffic.md (unplanned kernels)
 }
 
