@@ -164,7 +164,7 @@ TRAFFIC_PER_UNIT = {
 
 
 def work_models(snap, counts, clock_mhz):
-    """Algorithmic work per launch of every row (SURVEY-style models).
+    """Algorithmic work per launch of every row.
 
     CSR: cache-oblivious gather model, bytes = E (col + w + one source row) + N (rowptr + one output
     row); backward adds the cotangent row, the read-modify-write of the source-gradient row and the
