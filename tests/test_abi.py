@@ -90,6 +90,14 @@ def test_host_side_argument_errors(lib):
     assert cdll.tiga_apply_csr(ctypes.byref(g), 256, 0, 4, None, ctypes.byref(msg), 1, 256, None, 256, 1 << 20, None) == 1  # max needs argmax
     assert cdll.tiga_apply_csr(ctypes.byref(g), 256, 0, 4, 256, ctypes.byref(msg), 0, 256, None, 256, 1 << 20, None) == 1   # COPY with weights
     assert cdll.tiga_csr_workspace_bytes(ctypes.byref(g), 64, 0, 0, 0) >= 2 * 64 * 4
+    # the three reducers: unknown values are refused, 64-bit positions need the widest per-tile array, a relation of
+    # 2^31 edges and more is refused by the 32-bit max reducer on the host (nothing is read: the pointers are fakes)
+    assert cdll.tiga_apply_csr(ctypes.byref(g), 256, 0, 4, None, ctypes.byref(msg), 3, 256, 256, 256, 1 << 20, None) == 1
+    ws = [cdll.tiga_csr_workspace_bytes(ctypes.byref(g), 64, 0, red, 0) for red in (0, 1, 2)]
+    assert ws[0] < ws[1] < ws[2]
+    huge = _Csr(256, 1, 256, 4, 4, (1 << 31) + 5)
+    assert cdll.tiga_apply_csr(ctypes.byref(huge), 256, 0, 4, None, ctypes.byref(msg), 1, 256, 256, 256, 1 << 40, None) == 2
+    assert cdll.tiga_apply_csr_backward(ctypes.byref(huge), 256, 0, 4, None, ctypes.byref(msg), 1, 256, 256, 256, None, None, 0, None) == 2
     assert cdll.tiga_csr_degree_histogram(ctypes.byref(g), 256, 0, 256, None) == 1                          # nbins < 1
     assert cdll.tiga_validate_csr(ctypes.byref(g), 0, None, 0, None) == 0                                   # metadata only
     # radius: message descriptor, widths, message parameters (all refused before any device access)
