@@ -779,35 +779,65 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_backward_sum_kernel(const Csr
 }
 
 // Backward, max reducer: the cotangent of (i, f) goes through the selected edge only.
-// One thread per (i, f).  The features of a row often select the same edge (always, for a row with
-// one edge), so a warp first sums the edge-gradient contributions of lanes that share an edge
-// (two rounds, each for the edge of the lowest lane not served yet; what is left goes out one by
-// one: more rounds measured slower): one atomic per edge instead of
-// up to 32 on the same address.
+// One thread per four consecutive features of a row.  They often select the same edge (always, for a
+// row with one edge): then the thread gathers the source row slice with one vector load, sends the
+// feature gradient as one vector atomic and contributes one value to the edge gradient; a warp sums
+// the edge-gradient contributions of such threads that share an edge (two rounds, each for the edge of
+// the lowest lane not served yet; what is left goes out one by one: more rounds measured slower), so an
+// edge receives one atomic instead of up to 32 on the same address.  Features whose selected edges
+// differ go one by one.
 template <typename XT, int RED>
 __global__ void csr_backward_max_kernel(const CsrParams p) {
     using AT = ArgT<RED>;
     constexpr unsigned FULL = 0xffffffffu;
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long idx = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     const int lane = threadIdx.x & 31;
-    AT e = idx < p.n_dst * p.F ? static_cast<const AT*>(p.arg)[idx] : AT(-1);
-    if (e >= 0) e = checked(e, p.n_edges, CHECK_EDGE);
-    const bool act = e >= 0;
+    const bool in = idx < p.n_dst * p.F;
+    AT a[4] = {AT(-1), AT(-1), AT(-1), AT(-1)};
+    float g[4] = {0.f, 0.f, 0.f, 0.f};
+    if (in) {
+        const AT* ap = static_cast<const AT*>(p.arg) + idx;
+        if constexpr (sizeof(AT) == 4) {
+            const int4 v = *reinterpret_cast<const int4*>(ap);
+            a[0] = v.x; a[1] = v.y; a[2] = v.z; a[3] = v.w;
+        } else {
+            const longlong2 v0 = *reinterpret_cast<const longlong2*>(ap), v1 = *reinterpret_cast<const longlong2*>(ap + 2);
+            a[0] = v0.x; a[1] = v0.y; a[2] = v1.x; a[3] = v1.y;
+        }
+        const float4 gv = *reinterpret_cast<const float4*>(p.gy + idx);
+        g[0] = gv.x; g[1] = gv.y; g[2] = gv.z; g[3] = gv.w;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (a[k] >= 0) a[k] = checked(a[k], p.n_edges, CHECK_EDGE);
+    }
+    const int f0 = (int)(idx % p.F);
+    const bool uni = in && a[0] >= 0 && a[0] == a[1] && a[1] == a[2] && a[2] == a[3];
+    const AT e = uni ? a[0] : AT(-1);
     float contrib = 0.f;
-    if (act) {
-        const int f = (int)(idx % p.F);
+    if (uni) {
         const long long j = checked(p.col[e], p.n_src, CHECK_SOURCE);
-        const float g = p.gy[idx];
-        if (p.gx) atomicAdd(p.gx + j * p.F + f, (p.w ? p.w[e] : 1.f) * g);
+        const float wgt = p.w ? p.w[e] : 1.f;
+        if (p.gx) atomicAdd(reinterpret_cast<float4*>(p.gx + j * p.F + f0), make_float4(wgt * g[0], wgt * g[1], wgt * g[2], wgt * g[3]));
         if (p.gw) {
-            float xv;
-            if constexpr (sizeof(XT) == 4) xv = static_cast<const float*>(p.x)[j * p.F + f];
-            else xv = __half2float(static_cast<const __half*>(p.x)[j * p.F + f]);
-            contrib = xv * g;
+            const float4 xv = load_x4<XT>(p.x, (unsigned long long)(j * p.F + f0) >> 2);
+            contrib = fmaf(xv.w, g[3], fmaf(xv.z, g[2], fmaf(xv.y, g[1], xv.x * g[0])));
+        }
+    } else if (in) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (a[k] < 0) continue;
+            const long long j = checked(p.col[a[k]], p.n_src, CHECK_SOURCE);
+            if (p.gx) atomicAdd(p.gx + j * p.F + f0 + k, (p.w ? p.w[a[k]] : 1.f) * g[k]);
+            if (p.gw) {
+                float xv;
+                if constexpr (sizeof(XT) == 4) xv = static_cast<const float*>(p.x)[j * p.F + f0 + k];
+                else xv = __half2float(static_cast<const __half*>(p.x)[j * p.F + f0 + k]);
+                atomicAdd(p.gw + a[k], xv * g[k]);
+            }
         }
     }
     if (!p.gw) return;
-    unsigned remaining = __ballot_sync(FULL, act);
+    unsigned remaining = __ballot_sync(FULL, uni);
     for (int round = 0; remaining; ++round) {           // warp uniform
         if (round == 2) {
             if ((remaining >> lane) & 1u) atomicAdd(p.gw + e, contrib);
@@ -815,7 +845,7 @@ __global__ void csr_backward_max_kernel(const CsrParams p) {
         }
         const int leader = __ffs(remaining) - 1;
         const AT el = __shfl_sync(FULL, e, leader);
-        const bool mine = act && e == el;
+        const bool mine = uni && e == el;
         float s = mine ? contrib : 0.f;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(FULL, s, o);
@@ -1250,7 +1280,7 @@ extern "C" tiga_status tiga_apply_csr_backward(const tiga_csr* g, const void* x,
             return g->rowptr_type == TIGA_I64 ? launch_bwd_g<int64_t, __half>(p, G, VPL, s) : launch_bwd_g<int32_t, __half>(p, G, VPL, s);
         return g->rowptr_type == TIGA_I64 ? launch_bwd_g<int64_t, float>(p, G, VPL, s) : launch_bwd_g<int32_t, float>(p, G, VPL, s);
     }
-    const unsigned blocks = (unsigned)((g->n_dst * F + 255) / 256);
+    const unsigned blocks = (unsigned)((g->n_dst * F / 4 + 255) / 256);      // one thread per four features
     if (reducer == TIGA_MAX) {
         if (x_dtype == TIGA_F16) csr_backward_max_kernel<__half, 1><<<counted(blocks), 256, 0, s>>>(p);
         else csr_backward_max_kernel<float, 1><<<counted(blocks), 256, 0, s>>>(p);
