@@ -823,17 +823,27 @@ __global__ void csr_backward_max_kernel(const CsrParams p) {
             contrib = fmaf(xv.w, g[3], fmaf(xv.z, g[2], fmaf(xv.y, g[1], xv.x * g[0])));
         }
     } else if (in) {
+        // the four chains (edge -> source -> feature) are independent: all loads of a level first
+        long long j[4];
+        float wv[4], xv[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const AT ek = a[k] >= 0 ? a[k] : AT(0);
+            j[k] = checked(p.col[ek], p.n_src, CHECK_SOURCE);
+            wv[k] = p.w ? p.w[ek] : 1.f;
+        }
+        if (p.gw) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if constexpr (sizeof(XT) == 4) xv[k] = static_cast<const float*>(p.x)[j[k] * p.F + f0 + k];
+                else xv[k] = __half2float(static_cast<const __half*>(p.x)[j[k] * p.F + f0 + k]);
+            }
+        }
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             if (a[k] < 0) continue;
-            const long long j = checked(p.col[a[k]], p.n_src, CHECK_SOURCE);
-            if (p.gx) atomicAdd(p.gx + j * p.F + f0 + k, (p.w ? p.w[a[k]] : 1.f) * g[k]);
-            if (p.gw) {
-                float xv;
-                if constexpr (sizeof(XT) == 4) xv = static_cast<const float*>(p.x)[j * p.F + f0 + k];
-                else xv = __half2float(static_cast<const __half*>(p.x)[j * p.F + f0 + k]);
-                atomicAdd(p.gw + a[k], xv * g[k]);
-            }
+            if (p.gx) atomicAdd(p.gx + j[k] * p.F + f0 + k, wv[k] * g[k]);
+            if (p.gw) atomicAdd(p.gw + a[k], xv[k] * g[k]);
         }
     }
     if (!p.gw) return;
