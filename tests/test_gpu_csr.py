@@ -184,6 +184,30 @@ def test_fp16_features_backward(tiga):
         assert rel_err(host(gw), refm["gw"], refm["Aw"]) <= GRAD_TOL
 
 
+def test_max_backward_with_a_gradient_table_larger_than_l2(tiga):
+    """The max backward has two forms, picked by the size of the feature-gradient table (128 MB): this
+    relation has few edges but 600,000 sources of 64 features, so the four-features-per-thread form
+    runs, with fp32 and fp16 features, 32-bit and 64-bit edge positions."""
+    n_dst, n_src, F = 3000, 600_000, 64
+    rowptr, col, x, w, gy = _random_graph(91, n_dst, n_src, 40, F)
+    g = _relation(tiga, rowptr, col, n_src)
+    wd, gyd = dev(w, torch), dev(gy, torch)
+    for xt in (x, x.astype(np.float16)):
+        xr = xt.astype(np.float32)
+        xd = dev(xt, torch)
+        _, _, arg = oracle.csr_forward(rowptr, col, xr, w, oracle.MAX)
+        ref = oracle.csr_backward_max(rowptr, col, xr, w, gy, arg)
+        for red, dt in ((tiga.MAX, torch.int32), (tiga.MAX64, torch.int64)):
+            _, am = tiga.tiga_apply_csr(g, xd, wd, red)
+            assert am.dtype == dt and np.array_equal(host(am).astype(np.int64), arg)
+            guard = Guard(torch)
+            gx, gw = tiga.tiga_apply_csr_backward(g, xd, wd, gyd, red, argmax=am, grad_x=guard.empty((n_src, F)),
+                                                  grad_w=guard.empty((g.n_edges,)))
+            guard.check()
+            assert rel_err(host(gx), ref["gx"], ref["Ax"]) <= GRAD_TOL
+            assert rel_err(host(gw), ref["gw"], ref["Aw"]) <= GRAD_TOL
+
+
 def test_hex_mesh_degrees(tiga):
     L = 24
     rowptr, col = gen.hex_mesh_csr(L)
