@@ -312,7 +312,8 @@ __global__ void __launch_bounds__(CSR_THREADS, 5) csr_forward_kernel(const CsrPa
 // --------------------------------------------------------------------------------------------
 constexpr int ROW_OWN = 4;
 constexpr int ROW_GROUP = 64;
-constexpr int ROW_HUGE = 4096;
+constexpr int ROW_HUGE = 1024;       // longest row a single warp sums (the host lowers it for small relations: p.row_huge)
+constexpr int ROW_HUGE_SMALL = 256;
 constexpr int GROUP_LANES = 8;
 constexpr int ROW_THREADS = 256;     // rows (= threads) per CTA of the row-class kernel
 
@@ -503,7 +504,7 @@ __global__ void __launch_bounds__(ROW_THREADS, 1536 / ROW_THREADS) csr_rows_kern
     if (threadIdx.x == 0) { q_ng = 0; q_nw = 0; q_next = 0; }
     __syncthreads();
     const bool is_g = valid && deg > ROW_OWN && deg <= ROW_GROUP;
-    const bool is_w = valid && deg > ROW_GROUP && deg <= ROW_HUGE;
+    const bool is_w = valid && deg > ROW_GROUP && deg <= p.row_huge;
     {
         const unsigned mg = __ballot_sync(FULL, is_g), mw = __ballot_sync(FULL, is_w);
         int bg = 0, bw = 0;
@@ -587,8 +588,8 @@ __global__ void __launch_bounds__(ROW_THREADS, 1536 / ROW_THREADS) csr_rows_kern
         reduce_and_store<XT, NV, RED, 32>(part, lane, true, p.out + r * p.F, RED ? static_cast<ArgT<RED>*>(p.arg) + r * p.F : nullptr);
     }
     // huge rows: queue their chunks
-    if (valid && deg > ROW_HUGE) {
-        const int chunks = (int)((deg + ROW_HUGE - 1) / ROW_HUGE);
+    if (valid && deg > p.row_huge) {
+        const int chunks = (int)((deg + p.row_huge - 1) / p.row_huge);
         const int base = atomicAdd(p.huge_count, chunks);
         for (int c = 0; c < chunks; ++c) p.huge_list[base + c] = make_int4((int)row, c, chunks, base);
     }
@@ -604,9 +605,9 @@ __global__ void __launch_bounds__(CSR_THREADS) csr_huge_chunks_kernel(const CsrP
     const int total = *p.huge_count;
     for (int idx = blockIdx.x * (CSR_THREADS / 32) + (threadIdx.x >> 5); idx < total; idx += nwarps) {
         const int4 ent = p.huge_list[idx];
-        const long long es = (long long)rowptr[ent.x] + (long long)ent.y * ROW_HUGE;
+        const long long es = (long long)rowptr[ent.x] + (long long)ent.y * p.row_huge;
         const long long ee = (long long)rowptr[ent.x + 1];
-        const int n = (int)(ee - es < ROW_HUGE ? ee - es : ROW_HUGE);
+        const int n = (int)(ee - es < p.row_huge ? ee - es : p.row_huge);
         auto part = strided_row<XT, NV, RED, 32, 8, HOT, W>(p, src, es, n, lane);
         reduce_and_store<XT, NV, RED, 32>(part, lane, true, p.carry_val + (size_t)idx * p.F, RED ? static_cast<ArgT<RED>*>(p.carry_arg) + (size_t)idx * p.F : nullptr);
     }
@@ -1003,6 +1004,12 @@ static bool pick_shape(int nvec, int* G, int* VPL) {
     return true;
 }
 
+// Chunk length of the row-class path: a row is summed by one warp up to this many edges.  On a small relation
+// the longest row would otherwise be one warp's latency chain and set the time of the whole call (R-MAT,
+// F = 8 fp16: 2^20 edges 0.137 -> 0.042 ms with 256 instead of 4096; 2^26 edges 0.45 -> 0.39 ms and 2^28 edges
+// 1.61 -> 1.48 ms with 1024; 2^30 edges the same with 1024 and 4096).
+static int row_huge_of(const tiga_csr* g) { return g->n_edges >= (1LL << 25) ? ROW_HUGE : ROW_HUGE_SMALL; }
+
 // tiles of a relation for a given tile length; without one, for the shortest (sizes workspaces, bounds grids)
 static long long num_tiles(const tiga_csr* g, int tile = CSR_TILE_MIN) { return (g->n_dst + g->n_edges + tile - 1) / tile; }
 
@@ -1067,6 +1074,13 @@ static tiga_status launch_bwd_g(const CsrParams& p, int G, int VPL, cudaStream_t
     return launch_status();
 }
 
+// entries of the per-tile / per-chunk workspace arrays: tiles of the tile kernels, or chunks of the row-class path
+// (at most E / chunk full chunks plus one partial chunk per chunked row, and a chunked row has more than a chunk)
+static size_t work_slots(const tiga_csr* g, bool narrow_rows) {
+    const size_t tiles = (size_t)num_tiles(g) + 1, chunks = (size_t)(2 * g->n_edges / row_huge_of(g)) + 2;
+    return (narrow_rows && chunks > tiles) ? chunks : tiles;
+}
+
 static tiga_status check_csr(const tiga_csr* g) {
     if (!g) return TIGA_ERR_INVALID_ARG;
     if (g->n_dst < 0 || g->n_src < 0 || g->n_edges < 0) return TIGA_ERR_INVALID_ARG;
@@ -1101,10 +1115,10 @@ static void* take_args(Carver& cv, tiga_reducer r, size_t n) {
 
 using namespace tiga;
 
-extern "C" size_t tiga_csr_workspace_bytes(const tiga_csr* g, int32_t F, tiga_dtype, tiga_reducer reducer, int backward) {
+extern "C" size_t tiga_csr_workspace_bytes(const tiga_csr* g, int32_t F, tiga_dtype x_dtype, tiga_reducer reducer, int backward) {
     if (!g || F <= 0 || g->n_dst < 0 || g->n_edges < 0) return 0;
     if (backward) return 256;
-    const size_t nt = (size_t)num_tiles(g) + 1;
+    const size_t nt = work_slots(g, (size_t)F * (x_dtype == TIGA_F16 ? 2 : 4) <= 32);      // feature rows of at most 32 bytes: row-class path
     size_t b = align_up(nt * sizeof(int32_t), 256) + align_up(nt * F * sizeof(float), 256);
     if (is_max(reducer)) b += align_up(nt * F * arg_bytes(reducer), 256);
     b += 256 + align_up(nt * sizeof(int4), 256);      // queue of huge-row chunks (narrow-row path)
@@ -1162,11 +1176,13 @@ extern "C" tiga_status tiga_apply_csr(const tiga_csr* g, const void* x, tiga_dty
     p.n_dst = g->n_dst; p.n_edges = g->n_edges; p.n_src = g->n_src; p.F = F; p.nvec = nvec;
     p.ntiles = num_tiles(g);
     Carver cv(ws);
-    p.carry_row = cv.take<int32_t>((size_t)p.ntiles + 1);
-    p.carry_val = cv.take<float>(((size_t)p.ntiles + 1) * F);
-    p.carry_arg = take_args(cv, reducer, ((size_t)p.ntiles + 1) * F);
+    const size_t slots = work_slots(g, nvec <= 2);
+    p.carry_row = cv.take<int32_t>(slots);
+    p.carry_val = cv.take<float>(slots * F);
+    p.carry_arg = take_args(cv, reducer, slots * F);
     p.huge_count = cv.take<int>(1);
-    p.huge_list = cv.take<int4>((size_t)p.ntiles + 1);      // >= 2 E / ROW_HUGE + 1 entries
+    p.huge_list = cv.take<int4>(slots);
+    p.row_huge = row_huge_of(g);
     p.ntiles = num_tiles(g, reducer == TIGA_SUM ? CSR_TILE : CSR_TILE_MAX);      // the launch's tiles (the arrays hold at least as many)
 
     const bool i64 = g->rowptr_type == TIGA_I64;
@@ -1272,11 +1288,13 @@ extern "C" tiga_status tiga_apply_csr_planned(const tiga_csr* g, const tiga_csr_
     void* hot = cv.take<unsigned char>((size_t)plan->n_hot * row_bytes + 256);
     p.x_hot = hot; p.n_hot = (int)plan->n_hot;
     p.n_src = g->n_src + plan->n_hot;                      // range of the rewritten indices
-    p.carry_row = cv.take<int32_t>((size_t)p.ntiles + 1);
-    p.carry_val = cv.take<float>(((size_t)p.ntiles + 1) * F);
-    p.carry_arg = take_args(cv, reducer, ((size_t)p.ntiles + 1) * F);
+    const size_t slots = work_slots(g, nvec <= 2);
+    p.carry_row = cv.take<int32_t>(slots);
+    p.carry_val = cv.take<float>(slots * F);
+    p.carry_arg = take_args(cv, reducer, slots * F);
     p.huge_count = cv.take<int>(1);
-    p.huge_list = cv.take<int4>((size_t)p.ntiles + 1);
+    p.huge_list = cv.take<int4>(slots);
+    p.row_huge = row_huge_of(g);
     st = launch_gather_hot(x, reinterpret_cast<const int32_t*>(base + plan->off_hot_id), plan->n_hot, nvec, hot, s);
     if (st != TIGA_OK) return st;
     const bool i64 = g->rowptr_type == TIGA_I64;

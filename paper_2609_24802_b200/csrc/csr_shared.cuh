@@ -67,6 +67,7 @@ struct CsrParams {
     long long ntiles;
     int* huge_count;         // narrow-row path: number of queued chunks of huge rows
     int4* huge_list;         // (row, chunk, chunks of the row, first slot of the row)
+    int row_huge;            // rows above this many edges are cut into chunks of this length
     // planned apply (narrow rows): the most often gathered source rows are served from a compact copy
     const void* x_hot;       // [n_hot rows] copy of the hot source rows, or null
     int n_hot;               // col values below n_hot index x_hot, the others (minus n_hot) x
