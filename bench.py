@@ -967,7 +967,7 @@ def run_case(args):
         b_min = 8.0 * (N + 1) + 4.0 * E + 16.0 * (touched if touched is not None else 2.7e7) + 32.0 * N
         # profiles/csr_large_cfg4_dram_traffic.md: bytes per edge of the unplanned design (once measured at
         # full size) or of the planned scale-24 replica (a lower bound at full size)
-        b_dram = (16.0 if args.planned else 33.1) * E
+        b_dram = (15.7 if args.planned else 33.1) * E
         sink = torch.zeros(1, device=dev)
         for _ in range(2):
             bench_probe.row_gather(x, g.col, sink)
