@@ -29,6 +29,7 @@ namespace tiga {
 
 constexpr int RAD_THREADS = 256;
 constexpr int SCAN_BLOCK = 2048;   // elements per CTA in the scan passes
+constexpr int SCAN_SMALL_CHUNKS = 4;   // up to this many chunks are scanned by one CTA in one launch
 
 // ------------------------------------------------------------------------------ binning
 __global__ void bin_count_kernel(const RadiusParams p) {
@@ -108,11 +109,10 @@ __global__ void scan_blocksums_kernel(const RadiusParams p, int nblocks) {
     }
 }
 
-// pass C: exclusive scan inside every CTA's chunk plus its offset -> cell_start
-__global__ void scan_apply_kernel(const RadiusParams p) {
-    __shared__ int s_warp[33];
+// exclusive scan of one chunk of SCAN_BLOCK counts plus the chunk's offset -> cell_start; returns the chunk's total
+static __device__ int scan_chunk(const RadiusParams& p, const int chunk, const int offset, int* s_warp) {
     constexpr int PER = SCAN_BLOCK / RAD_THREADS;
-    const int base = blockIdx.x * SCAN_BLOCK + threadIdx.x * PER;
+    const int base = chunk * SCAN_BLOCK + threadIdx.x * PER;
     int v[PER];
     int sum = 0;
 #pragma unroll
@@ -121,7 +121,7 @@ __global__ void scan_apply_kernel(const RadiusParams p) {
         sum += v[k];
     }
     int total;
-    int ex = block_exclusive_scan(sum, s_warp, &total) + p.blocksum[blockIdx.x];
+    int ex = block_exclusive_scan(sum, s_warp, &total) + offset;
 #pragma unroll
     for (int k = 0; k < PER; ++k) {
         if (base + k < p.ncells) {
@@ -131,10 +131,28 @@ __global__ void scan_apply_kernel(const RadiusParams p) {
         }
         ex += v[k];
     }
-    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == blockDim.x - 1) {
-        p.cell_start[p.ncells] = p.n;
-        if (p.u_cell_start) p.u_cell_start[p.ncells] = p.n;
-    }
+    return total;
+}
+
+static __device__ void scan_finish(const RadiusParams& p) {
+    p.cell_start[p.ncells] = p.n;
+    if (p.u_cell_start) p.u_cell_start[p.ncells] = p.n;
+}
+
+// pass C: exclusive scan inside every CTA's chunk plus its offset -> cell_start
+__global__ void scan_apply_kernel(const RadiusParams p) {
+    __shared__ int s_warp[33];
+    scan_chunk(p, blockIdx.x, p.blocksum[blockIdx.x], s_warp);
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == blockDim.x - 1) scan_finish(p);
+}
+
+// Few cells (a handful of chunks): one CTA walks the chunks and carries the offset along, which replaces the
+// three scan launches of small inputs by one.
+__global__ void scan_small_kernel(const RadiusParams p, const int nblocks) {
+    __shared__ int s_warp[33];
+    int offset = 0;
+    for (int chunk = 0; chunk < nblocks; ++chunk) offset += scan_chunk(p, chunk, offset, s_warp);
+    if (threadIdx.x == 0) scan_finish(p);
 }
 
 __global__ void bin_scatter_kernel(const RadiusParams p, int32_t* fill) {
@@ -754,9 +772,13 @@ tiga_status run_binning(RadiusParams& p, int32_t* fill, int nblocks, cudaStream_
     TIGA_CUDA_TRY(cudaMemsetAsync(p.cnt, 0, (2 * (size_t)p.ncells + 2 + 16) * sizeof(int32_t), s));
     const unsigned pb = (unsigned)((p.n + 255) / 256);
     bin_count_kernel<<<counted(pb), 256, 0, s>>>(p);
-    scan_reduce_kernel<<<counted(nblocks), RAD_THREADS, 0, s>>>(p);
-    scan_blocksums_kernel<<<counted(1), 1024, 0, s>>>(p, nblocks);
-    scan_apply_kernel<<<counted(nblocks), RAD_THREADS, 0, s>>>(p);
+    if (nblocks <= SCAN_SMALL_CHUNKS) {
+        scan_small_kernel<<<counted(1), RAD_THREADS, 0, s>>>(p, nblocks);
+    } else {
+        scan_reduce_kernel<<<counted(nblocks), RAD_THREADS, 0, s>>>(p);
+        scan_blocksums_kernel<<<counted(1), 1024, 0, s>>>(p, nblocks);
+        scan_apply_kernel<<<counted(nblocks), RAD_THREADS, 0, s>>>(p);
+    }
     bin_scatter_kernel<<<counted(pb), 256, 0, s>>>(p, fill);
     const long long dense_cells = (long long)p.n / SORT_DENSE + 1;          // at most this many cells can be dense
     bin_sort_kernel<<<counted(pb + (unsigned)(dense_cells < 148 ? dense_cells : 148)), 256, 0, s>>>(p, (int)pb);
